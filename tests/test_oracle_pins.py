@@ -1,0 +1,328 @@
+"""Pins of the CPU oracle against things other than itself: a dense full-matrix numpy
+forward, invariants of paging and chunking, hand-worked integer cases, closed forms,
+and the capped-geometric acceptance expectation (paper Sec. 5)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import Oracle, verify_greedy
+from workloads import gen, rng
+from workloads.configs import CONFIGS, TINY, ModelShape
+
+from dense_ref import dense_forward, f64
+from orc_util import PIN, PIN1, model, prefill, tokens_for
+
+P = 4  # small page size so that short sequences span many pages
+
+
+def _run(shape, glob, layers, toks, ctx, page_table, n_pages, u=1, f32=False, page_size=P):
+    orc = Oracle(shape, page_size=page_size, f32=f32)
+    pools = orc.new_pool(n_pages)
+    if ctx:
+        prefill(orc, glob, layers, pools, page_table, toks[:ctx], step=5)
+    res = orc.forward_chunk(glob, lambda l: layers[l], pools, page_table, ctx, list(toks[ctx:]), u=u)
+    return res, pools
+
+
+# ---------------------------------------------------------------- P-1 dense full-matrix attention
+@pytest.mark.parametrize("shape,ctx,n", [(PIN, 13, 5), (PIN, 0, 7), (PIN1, 9, 1), (TINY, 21, 4)])
+def test_chunk_logits_equal_dense_full_matrix_forward(shape, ctx, n):
+    glob, layers = model(shape)
+    toks = tokens_for(shape, ctx + n)
+    n_pages = -(-(ctx + n) // P) + 3
+    pt = np.random.default_rng(1).permutation(n_pages).astype(np.int32)
+    res, pools = _run(shape, glob, layers, toks, ctx, pt, n_pages)
+    ref, kvs = dense_forward(shape, glob, layers, toks)
+    scale = np.abs(ref).max()
+    assert np.abs(res.logits - ref[ctx:]).max() <= 1e-11 * scale
+    assert (res.top1 == ref[ctx:].argmax(-1)).all()
+    # the cache holds exactly the dense forward's post-RoPE K and V, at the paged slots
+    for l, (k, v) in enumerate(kvs):
+        for p in range(ctx + n):
+            page, row = pt[p // P], p % P
+            assert np.abs(pools[l][page, 0, :, row, :] - k[p]).max() <= 1e-11 * max(1.0, np.abs(k).max())
+            assert np.abs(pools[l][page, 1, :, row, :] - v[p]).max() <= 1e-11 * max(1.0, np.abs(v).max())
+
+
+def test_runner_up_and_gap_match_sorted_logits():
+    glob, layers = model(PIN)
+    toks = tokens_for(PIN, 12)
+    res, _ = _run(PIN, glob, layers, toks, 8, np.arange(6, dtype=np.int32), 6)
+    srt = np.sort(res.logits, axis=-1)
+    assert np.allclose(res.gap, srt[:, -1] - srt[:, -2], rtol=0, atol=0)
+    assert (np.take_along_axis(res.logits, res.top2[:, None].astype(np.int64), -1)[:, 0] == srt[:, -2]).all()
+
+
+# ---------------------------------------------------------------- P-2 paging invariance
+def test_paged_equals_contiguous_and_any_page_permutation_bitwise():
+    glob, layers = model(PIN)
+    toks = tokens_for(PIN, 23)
+    n_pages = 9
+    ident = np.arange(n_pages, dtype=np.int32)
+    base, _ = _run(PIN, glob, layers, toks, 17, ident, n_pages)
+    for s in range(3):
+        pt = np.random.default_rng(s).permutation(n_pages).astype(np.int32)
+        r, _ = _run(PIN, glob, layers, toks, 17, pt, n_pages)
+        assert np.array_equal(r.logits, base.logits)
+    # one big page == contiguous cache
+    r, _ = _run(PIN, glob, layers, toks, 17, np.zeros(1, dtype=np.int32), 1, page_size=32)
+    assert np.array_equal(r.logits, base.logits)
+
+
+# ---------------------------------------------------------------- P-3 chunking invariance
+def test_chunk_equals_token_by_token_and_any_split():
+    glob, layers = model(PIN)
+    toks = tokens_for(PIN, 20)
+    ctx, n_pages = 11, 7
+    pt = np.random.default_rng(5).permutation(n_pages).astype(np.int32)
+    whole, _ = _run(PIN, glob, layers, toks, ctx, pt, n_pages)
+    orc = Oracle(PIN, page_size=P)
+    for split in ([1] * 9, [4, 5], [2, 3, 4], [8, 1]):
+        pools = orc.new_pool(n_pages)
+        prefill(orc, glob, layers, pools, pt, toks[:ctx], step=3)
+        p, rows = ctx, []
+        for s in split:
+            r = orc.forward_chunk(glob, lambda l: layers[l], pools, pt, p, list(toks[p:p + s]), u=s)
+            rows.append(r.logits)
+            p += s
+        assert np.array_equal(np.concatenate(rows), whole.logits)
+
+
+# ---------------------------------------------------------------- P-4 batch composition
+def test_request_result_independent_of_batch_mates_and_order():
+    glob, layers = model(PIN)
+    wl = CONFIGS[1]
+    orc = Oracle(PIN, page_size=P)
+    lens = [(6, 3), (9, 2), (0, 4)]
+    toks = [tokens_for(PIN, c + n, seed=i) for i, (c, n) in enumerate(lens)]
+    n_pages = 12
+    perm = np.random.default_rng(9).permutation(n_pages).astype(np.int32)
+    tables = [perm[0:4], perm[4:8], perm[8:12]]
+    alone = []
+    for i, (c, n) in enumerate(lens):
+        r, _ = _run(PIN, glob, layers, toks[i], c, tables[i], n_pages)
+        alone.append(r.logits)
+    for order in ([0, 1, 2], [2, 0, 1]):
+        pools = orc.new_pool(n_pages)            # one shared pool, interleaved pages
+        for i in order:
+            prefill(orc, glob, layers, pools, tables[i], toks[i][:lens[i][0]], step=4)
+        for i in order:
+            c, n = lens[i]
+            r = orc.forward_chunk(glob, lambda l: layers[l], pools, tables[i], c, list(toks[i][c:]))
+            assert np.array_equal(r.logits, alone[i])
+
+
+# ---------------------------------------------------------------- P-5 hand-worked accept cases
+@pytest.mark.parametrize("top1,chunk,u,expect", [
+    # chunk = [anchor | drafts]; the argmax at index u-1+j judges draft j
+    ([5, 6, 7, 8], [1, 5, 6, 7], 1, (3, 8)),     # all three drafts accepted -> bonus token top1[3]
+    ([9, 6, 7, 8], [1, 5, 6, 7], 1, (0, 9)),     # first draft wrong -> correction top1[0]
+    ([5, 6, 2, 8], [1, 5, 6, 7], 1, (2, 2)),     # miss at draft 2
+    ([5, 3, 7, 8], [1, 5, 6, 7], 1, (1, 3)),     # miss at draft 1; later agreement is irrelevant
+    ([4], [1], 1, (0, 4)),                        # n = 1: plain decode step
+    ([0, 0, 5, 6, 9], [1, 2, 3, 5, 6], 3, (2, 9)),   # u = 3 anchors, 2 drafts, both accepted
+    ([0, 0, 4, 6, 9], [1, 2, 3, 5, 6], 3, (0, 4)),   # u = 3, first draft rejected
+    ([7, 7, 7, 7], [7, 7, 7, 7], 1, (3, 7)),     # repeated ids
+    ([1, 2, 3], [9, 8, 7], 3, (0, 3)),           # u = n: no drafts, result is the next token
+])
+def test_greedy_verify_hand_worked(top1, chunk, u, expect):
+    assert verify_greedy(top1, chunk, u) == expect
+
+
+def test_argmax_tie_takes_lowest_id():
+    shape = PIN1
+    glob, layers = model(shape)
+    lm = glob["lm_head"].clone()
+    lm[30] = lm[11]                      # two identical vocabulary rows -> exactly equal logits
+    lm[11] *= 64
+    lm[30] *= 64                         # and by far the largest ones for some direction
+    glob = dict(glob, lm_head=lm)
+    orc = Oracle(shape, page_size=P)
+    x = f64(lm[11:12]) * 3.0
+    _, t1, t2, gap = orc.logits(glob, x.astype(np.float64))
+    assert t1[0] == 11 and t2[0] == 30 and gap[0] == 0.0
+
+
+# ---------------------------------------------------------------- P-6 losslessness (Sec. 4.2: lossless verification)
+def test_draft_verify_loop_reproduces_greedy_continuation():
+    shape = PIN
+    glob, layers = model(shape, seed=3)
+    orc = Oracle(shape, page_size=P)
+    prompt = list(tokens_for(shape, 7, seed=4))
+    n_new, n_pages = 14, 12
+    pt = np.random.default_rng(2).permutation(n_pages).astype(np.int32)
+    lw = lambda l: layers[l]
+    # plain greedy decoding
+    pools = orc.new_pool(n_pages)
+    r = prefill(orc, glob, layers, pools, pt, prompt, step=16)
+    greedy, nxt = [], int(r.top1[-1])
+    for i in range(n_new):
+        greedy.append(nxt)
+        r = orc.forward_chunk(glob, lw, pools, pt, len(prompt) + i, [nxt])
+        nxt = int(r.top1[0])
+    # draft & verify with arbitrary (mostly wrong, sometimes right) drafts
+    g = np.random.default_rng(11)
+    pools = orc.new_pool(n_pages)
+    r = prefill(orc, glob, layers, pools, pt, prompt, step=16)
+    out, anchor, ctx = [int(r.top1[-1])], int(r.top1[-1]), len(prompt)
+    while len(out) < n_new:
+        gamma = int(g.integers(0, 5))
+        drafts = [greedy[len(out) + j] if (len(out) + j < n_new and g.random() < 0.6) else int(g.integers(0, shape.vocab))
+                  for j in range(gamma)]
+        res = orc.forward_chunk(glob, lw, pools, pt, ctx, [anchor] + drafts)
+        out += drafts[:res.accept_len] + [res.correction]
+        ctx += 1 + res.accept_len        # rejected drafts' slots are simply overwritten later
+        anchor = res.correction
+    assert out[:n_new] == greedy
+
+
+# ---------------------------------------------------------------- P-7 closed forms
+def test_zero_output_projections_reduce_logits_to_normed_embedding():
+    shape = PIN
+    glob, layers = model(shape)
+    layers = [dict(w, wo=torch.zeros_like(w["wo"]), wd=torch.zeros_like(w["wd"])) for w in layers]
+    toks = tokens_for(shape, 6)
+    res, _ = _run(shape, glob, layers, toks, 2, np.arange(2, dtype=np.int32), 2)
+    e = f64(glob["embed"])[toks[2:]]
+    ref = e / np.sqrt((e * e).mean(-1, keepdims=True) + shape.rms_eps) * f64(glob["final_norm"]) @ f64(glob["lm_head"]).T
+    assert np.abs(res.logits - ref).max() <= 1e-12 * np.abs(ref).max()
+
+
+def _rand_pool(orc, n_pages, seed):
+    g = np.random.default_rng(seed)
+    return g.standard_normal(orc.new_pool(n_pages)[0].shape)
+
+
+def test_attention_zero_query_is_mean_of_visible_values():
+    orc = Oracle(PIN, page_size=P)
+    pool = _rand_pool(orc, 5, 0)
+    pt = np.array([3, 0, 4, 1, 2], dtype=np.int32)
+    ctx, n = 10, 3
+    out = orc.attention(np.zeros((n, PIN.q_dim)), pool, pt, ctx)
+    G = PIN.group
+    for j in range(n):
+        vis = np.stack([pool[pt[t // P], 1, :, t % P, :] for t in range(ctx + j + 1)])   # [len, Hkv, hd]
+        for h in range(PIN.n_q_heads):
+            assert np.allclose(out[j].reshape(PIN.n_q_heads, -1)[h], vis[:, h // G].mean(0), rtol=1e-12, atol=1e-13)
+
+
+def test_attention_equal_value_rows_return_that_row():
+    orc = Oracle(PIN, page_size=P)
+    pool = _rand_pool(orc, 4, 1)
+    row = np.random.default_rng(2).standard_normal((PIN.n_kv_heads, PIN.head_dim))
+    pool[:, 1] = row[None, :, None, :]
+    q = np.random.default_rng(3).standard_normal((2, PIN.q_dim))
+    out = orc.attention(q, pool, np.arange(4, dtype=np.int32), 9).reshape(2, PIN.n_q_heads, PIN.head_dim)
+    for h in range(PIN.n_q_heads):
+        assert np.allclose(out[:, h], row[h // PIN.group], rtol=1e-12)
+
+
+def test_attention_brute_force_single_head_and_causal_edge():
+    """softmax(q K^T / sqrt(d_k)) V over exactly positions 0..ctx+j (paper Sec. 3.2)."""
+    orc = Oracle(PIN1, page_size=P)
+    pool = _rand_pool(orc, 3, 4)
+    pt = np.array([2, 0, 1], dtype=np.int32)
+    q = np.random.default_rng(5).standard_normal((3, PIN1.q_dim))
+    ctx = 6
+    out = orc.attention(q, pool, pt, ctx).reshape(3, PIN1.n_q_heads, PIN1.head_dim)
+    for j in range(3):
+        K = np.stack([pool[pt[t // P], 0, 0, t % P] for t in range(ctx + j + 1)])
+        V = np.stack([pool[pt[t // P], 1, 0, t % P] for t in range(ctx + j + 1)])
+        for h in range(PIN1.n_q_heads):
+            s = K @ q[j].reshape(PIN1.n_q_heads, -1)[h] / math.sqrt(PIN1.head_dim)
+            w = np.exp(s - s.max())
+            w /= w.sum()
+            assert np.allclose(out[j, h], w @ V, rtol=1e-12)
+    # changing a key/value beyond the causal horizon of row 0 must not change row 0
+    pool2 = pool.copy()
+    pool2[pt[(ctx + 1) // P], :, :, (ctx + 1) % P] += 7.0
+    out2 = orc.attention(q, pool2, pt, ctx).reshape(3, PIN1.n_q_heads, PIN1.head_dim)
+    assert np.array_equal(out2[0], out[0]) and not np.array_equal(out2[1], out[1])
+
+
+def test_rope_identity_at_zero_norm_preserving_and_relative():
+    orc = Oracle(PIN, page_size=P)
+    g = np.random.default_rng(0)
+    hd = PIN.head_dim
+    a, b = g.standard_normal(hd), g.standard_normal(hd)
+    assert np.array_equal(orc.rope(a, 1, 0), a)
+    assert np.isclose(np.linalg.norm(orc.rope(a, 1, 777)), np.linalg.norm(a), rtol=1e-12)
+    d0 = orc.rope(a, 1, 5) @ orc.rope(b, 1, 2)
+    for s in (1, 40, 8000):
+        assert np.isclose(orc.rope(a, 1, 5 + s) @ orc.rope(b, 1, 2 + s), d0, rtol=1e-9, atol=1e-9)
+    # explicit 2-D rotation of the pair (i, i + hd/2) by pos * base^(-2i/hd)
+    pos, i = 3, 2
+    ang = pos * PIN.rope_base ** (-2.0 * i / hd)
+    r = orc.rope(a, 1, pos)
+    assert np.isclose(r[i], a[i] * math.cos(ang) - a[i + hd // 2] * math.sin(ang), rtol=1e-12)
+    assert np.isclose(r[i + hd // 2], a[i + hd // 2] * math.cos(ang) + a[i] * math.sin(ang), rtol=1e-12)
+
+
+def test_rmsnorm_and_linear_against_numpy():
+    orc = Oracle(PIN, page_size=P)
+    g = np.random.default_rng(1)
+    x = g.standard_normal((3, PIN.d_model))
+    w = gen.gen_weight(PIN, 0, "wg", 0)
+    gain = gen.gen_gain(PIN, 0, "norm1", 0)
+    assert np.allclose(orc.linear(x, w), x @ f64(w).T, rtol=1e-12, atol=1e-14)
+    ref = x / np.sqrt((x * x).mean(-1, keepdims=True) + PIN.rms_eps) * f64(gain)
+    assert np.allclose(orc.rmsnorm(x, gain), ref, rtol=1e-13)
+    # a transposed weight must be caught: non-square matrix, distinct rows
+    assert orc.linear(x, w).shape == (3, PIN.d_ffn)
+
+
+# ---------------------------------------------------------------- P-8 slot map, hand-written
+def test_slot_map_hand_written_page_tables():
+    orc = Oracle(PIN, page_size=16)
+    pt = [7, 2, 9, 4, 0]
+    # ctx 48, chunk 4: starts exactly on a page boundary -> logical page 3 -> physical 4
+    assert [orc.slot(pt, 48 + j) for j in range(4)] == [(4, 0), (4, 1), (4, 2), (4, 3)]
+    # ctx 60, chunk 8: crosses from logical page 3 (rows 12..15) into logical page 4 (rows 0..3)
+    assert [orc.slot(pt, 60 + j) for j in range(8)] == [(4, 12), (4, 13), (4, 14), (4, 15),
+                                                        (0, 0), (0, 1), (0, 2), (0, 3)]
+    # ctx 0
+    assert [orc.slot(pt, j) for j in range(3)] == [(7, 0), (7, 1), (7, 2)]
+
+
+# ---------------------------------------------------------------- P-9 acceptance statistics (Sec. 5)
+def test_mean_accept_len_follows_capped_geometric():
+    """With i.i.d. match probability p' per draft, E[accepted + 1] = (1 - p'^(gamma+1)) / (1 - p')."""
+    wl = CONFIGS[1]
+    V, gamma, p = wl.shape.vocab, 3, wl.p_match
+    n_req = 6000
+    total = 0
+    for r in range(n_req):
+        top1 = [(r * 31 + 7 * j) % V for j in range(gamma + 1)]
+        chunk = [0] + [gen.gen_draft(wl, r, j, top1[j]) for j in range(gamma)]
+        total += verify_greedy(top1, chunk, 1)[0]
+    pp = p + (1 - p) / V
+    expect = (1 - pp ** (gamma + 1)) / (1 - pp) - 1          # = sum_{k=1..gamma} p'^k  (1.5337 here)
+    se = 1.2 / math.sqrt(n_req)
+    assert abs(total / n_req - expect) < 4 * se
+
+
+# ---------------------------------------------------------------- the single-precision build agrees
+def test_f32_build_agrees_with_f64_far_inside_parity_tolerance():
+    shape = TINY
+    glob, layers = model(shape)
+    toks = tokens_for(shape, 40)
+    pt = np.random.default_rng(0).permutation(4).astype(np.int32)
+    a, _ = _run(shape, glob, layers, toks, 36, pt, 4, page_size=16)
+    b, _ = _run(shape, glob, layers, toks, 36, pt, 4, page_size=16, f32=True)
+    sigma = a.logits.std()
+    assert np.abs(a.logits - b.logits).max() < 1e-4 * sigma
+
+
+# ---------------------------------------------------------------- generator sanity (shared input module)
+def test_counter_rng_matches_big_int_reference_and_is_sliceable():
+    k = rng.stream_key(5, 3, 2)
+    for i in (0, 1, 7, 123456789):
+        z = (k + i * rng._GOLDEN) & rng._MASK64
+        assert (int(rng.bits64(k, i, 1)[0]) & rng._MASK64) == rng._mix_py(z)
+    a = rng.normal_f32(k, 0, 1000, 0.02)
+    b = rng.normal_f32(k, 400, 100, 0.02)
+    assert torch.equal(a[400:500], b)
+    big = rng.normal_f32(k, 0, 400000, 1.0)
+    assert abs(float(big.mean())) < 0.01 and abs(float(big.std()) - 1.0) < 0.01
