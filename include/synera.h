@@ -1,0 +1,203 @@
+/*
+ * synera.h -- C ABI of the cloud-side batched verification step of Synera
+ * (arxiv 2511.07423), implemented as hand-written CUDA for NVIDIA B200 (sm_100a).
+ *
+ * The step (paper Sec. 3.4 "partial prefill", Sec. 4.5 "flatten -> forward -> verify"):
+ * many devices offload short token chunks; each chunk is appended to that request's cached
+ * context (a paged KV cache), a decoder-only transformer is run over the ragged batch, and
+ * the LLM's greedy argmax at every chunk position is compared with the drafted tokens
+ * (Sec. 3.1, "draft & verify") to give, per request, the number of accepted drafts and the
+ * correction token.
+ *
+ * Conventions
+ *   - Every function returns an int status: SYN_OK (0) or a negative SYN_E_* code.  No
+ *     exceptions, no abort, nothing is printed.  syn_strerror() names a code.
+ *   - "HOST" / "DEVICE" beside a pointer says where the memory must live.  The caller owns
+ *     every array it passes; the library keeps no caller pointer after a call returns,
+ *     except where stated (syn_plan keeps nothing either: it copies).
+ *   - All validation of a call happens on the host before any kernel is launched; on error
+ *     nothing is written (outputs and KV cache untouched).
+ *   - One call at a time per syn_model.  The library allocates device memory with
+ *     cudaMalloc on the current device; it does not link or call PyTorch.
+ *   - Matrices are bf16, row-major [out_features][in_features] (y = x W^T); RMSNorm gains are
+ *     bf16 [d_model].  There are no biases.
+ */
+#ifndef SYNERA_H_
+#define SYNERA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    SYN_OK = 0,
+    SYN_E_INVALID_ARG = -1,    /* NULL pointer, zero size, unsupported shape                    */
+    SYN_E_CHUNK_LEN = -2,      /* a chunk length outside [1, SYN_MAX_CHUNK]                     */
+    SYN_E_UNCACHED = -3,       /* n_uncached[i] outside [1, chunk length]                       */
+    SYN_E_PAGE_OOB = -4,       /* a used page id outside [0, n_pages)                           */
+    SYN_E_CAPACITY = -5,       /* ctx + chunk exceeds max_pages * page_size                     */
+    SYN_E_TOKEN_OOB = -6,      /* a token id outside [0, vocab)                                 */
+    SYN_E_PAGE_ALIAS = -7,     /* two chunk tokens of the batch map to the same KV slot         */
+    SYN_E_OOM = -8,            /* device or host allocation failed                              */
+    SYN_E_ARCH = -9,           /* current device is not compute capability 10.x                 */
+    SYN_E_CUDA = -10,          /* a CUDA runtime/driver call failed                             */
+    SYN_E_DEVICE_TIMEOUT = -11 /* a bounded wait inside a kernel ran out; results are invalid   */
+};
+
+#define SYN_MAX_CHUNK 16
+
+typedef struct syn_model syn_model; /* packed device copy of the weights + workspaces */
+typedef struct syn_kv syn_kv;       /* paged KV pool                                   */
+typedef struct syn_plan syn_plan;   /* device-resident description of one batch        */
+
+/* Decoder shape (Llama family: RMSNorm, rotate-half RoPE, grouped-query attention, SwiGLU).
+ * Supported: head_dim 64 or 128; d_model a multiple of 128; n_q_heads a multiple of
+ * n_kv_heads with group size <= 8; (n_q_heads*head_dim) and (n_kv_heads*head_dim)
+ * multiples of 128; d_ffn a multiple of 8. */
+typedef struct {
+    uint32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    float rope_base; /* theta_i = rope_base^(-2i/head_dim) */
+    float rms_eps;
+    uint32_t flags;  /* must be 0 */
+} syn_model_desc;
+
+/* Weight pointers, all bf16.  Per-layer arrays hold n_layers pointers (the arrays themselves
+ * are HOST memory).  location: 0 = the matrices are in HOST memory, 1 = in DEVICE memory. */
+typedef struct {
+    const void *embed;      /* [vocab][d_model]   */
+    const void *lm_head;    /* [vocab][d_model]   */
+    const void *final_norm; /* [d_model]          */
+    const void *const *wq;  /* [n_q_heads*head_dim][d_model]  */
+    const void *const *wk;  /* [n_kv_heads*head_dim][d_model] */
+    const void *const *wv;  /* [n_kv_heads*head_dim][d_model] */
+    const void *const *wo;  /* [d_model][n_q_heads*head_dim]  */
+    const void *const *wg;  /* [d_ffn][d_model]  gate         */
+    const void *const *wu;  /* [d_ffn][d_model]  up           */
+    const void *const *wd;  /* [d_model][d_ffn]  down         */
+    const void *const *norm1; /* [d_model] gain before attention */
+    const void *const *norm2; /* [d_model] gain before the MLP   */
+    int32_t location;
+} syn_weights;
+
+/* The LLM that verifies (paper Sec. 3.1).  Makes the library's own packed device copy of the
+ * weights, layer by layer (q|k|v rows concatenated, gate/up rows interleaved in blocks of 64,
+ * d_ffn padded to a multiple of 64 with zeros), so the caller's copy may be freed afterwards.
+ * Errors: SYN_E_INVALID_ARG (NULL, unsupported shape, flags != 0), SYN_E_ARCH, SYN_E_OOM,
+ * SYN_E_CUDA.  *out is written only on success. */
+int syn_model_load(const syn_model_desc *desc, const syn_weights *weights, syn_model **out);
+void syn_model_free(syn_model *m);
+
+/* The cache that holds every request's prefix (paper Sec. 3.4: "an existing KV-cached
+ * prefix").  n_pages physical pages of page_size tokens for every layer, bf16, zero-filled.
+ * Position p of a request lives in page page_table[p / page_size], row p % page_size.
+ * page_size must be 16.  Errors: SYN_E_INVALID_ARG, SYN_E_OOM, SYN_E_CUDA. */
+int syn_kv_alloc(syn_model *m, uint32_t n_pages, uint32_t page_size, syn_kv **out);
+void syn_kv_free(syn_kv *kv);
+
+/* Place externally produced (already rotated) K and V of one request and one layer at logical
+ * positions pos0 .. pos0+n_pos-1, e.g. a prefix computed on another server.  k, v: DEVICE bf16
+ * [n_pos][n_kv_heads][head_dim]; page_table: HOST int32, at least ceil((pos0+n_pos)/page_size)
+ * entries.  Asynchronous on `cuda_stream` except for a small blocking metadata copy.
+ * syn_kv_export is the inverse (reads the same positions into k, v).
+ * Errors: SYN_E_INVALID_ARG, SYN_E_PAGE_OOB, SYN_E_CUDA. */
+int syn_kv_import(syn_kv *kv, uint32_t layer, const int32_t *page_table, int32_t pos0, int32_t n_pos,
+                  const void *k, const void *v, void *cuda_stream);
+int syn_kv_export(syn_kv *kv, uint32_t layer, const int32_t *page_table, int32_t pos0, int32_t n_pos,
+                  void *k, void *v, void *cuda_stream);
+
+/* One batched verification step: execute_partialprefill(B_verify, L_uncached) of the paper's
+ * scheduler (Algorithm 1) followed by the verification of Sec. 4.5.
+ *
+ * Request i contributes the chunk chunk_tokens[chunk_offsets[i] .. chunk_offsets[i+1]) of
+ * n_i tokens, 1 <= n_i <= SYN_MAX_CHUNK: first u_i = n_uncached[i] >= 1 tokens the device has
+ * already accepted but the cloud has not cached (Sec. 3.4, "device-accepted tokens"), then
+ * n_i - u_i pending-verify draft tokens.  The chunk is appended after the ctx_lens[i] cached
+ * tokens: K and V of all n_i tokens are written at positions ctx_lens[i] .. ctx_lens[i]+n_i-1
+ * through page_tables[i][.], and token j attends to positions 0 .. ctx_lens[i]+j.
+ * The argmax at chunk index u_i-1+j judges draft j (the engine outputs q(x|prefix),
+ * q(x|prefix,x~_1), ...: gamma+1 distributions for gamma drafts, Sec. 4.5).
+ *   accept_len[i]       = number of leading drafts equal to the argmax, in [0, n_i-u_i]
+ *   correction_token[i] = argmax at the first mismatch; the bonus token (argmax after the last
+ *                         draft) when every draft is accepted.  Ties: lowest token id.
+ * After the call the caller advances ctx_lens[i] by u_i + accept_len[i]; slots of rejected
+ * drafts are simply overwritten by a later call.  A prefill is this call with u_i = n_i.
+ *
+ * HOST inputs: req_ids [n_req] (opaque labels, may be NULL), chunk_tokens [T],
+ * chunk_offsets [n_req+1] (chunk_offsets[0] = 0, T = chunk_offsets[n_req]),
+ * page_tables [n_req][max_pages] (entries beyond a request's used pages are ignored),
+ * ctx_lens [n_req], n_uncached [n_req] or NULL (= 1 each).
+ * HOST outputs: accept_len [n_req], correction_token [n_req].
+ * logits_out: NULL, or DEVICE fp32 [T][vocab] receiving every chunk position's logits.
+ * The call returns after the results are in the host arrays (it synchronises cuda_stream).
+ * Errors: SYN_E_INVALID_ARG, SYN_E_CHUNK_LEN, SYN_E_UNCACHED, SYN_E_PAGE_OOB, SYN_E_CAPACITY,
+ * SYN_E_TOKEN_OOB, SYN_E_PAGE_ALIAS, SYN_E_OOM (workspace growth), SYN_E_CUDA,
+ * SYN_E_DEVICE_TIMEOUT. */
+int syn_verify_batch(syn_model *m, syn_kv *kv, int32_t n_req, const int64_t *req_ids,
+                     const int32_t *chunk_tokens, const int32_t *chunk_offsets,
+                     const int32_t *page_tables, int32_t max_pages, const int32_t *ctx_lens,
+                     const int32_t *n_uncached, int32_t *accept_len, int32_t *correction_token,
+                     float *logits_out, void *cuda_stream);
+
+/* The same step split in two, for callers that keep the batch description on the device
+ * (and for timing the kernels alone).  syn_plan_create validates exactly like
+ * syn_verify_batch, runs the host planner (token positions, KV slots, attention work list;
+ * the "flatten" of Sec. 4.5) and uploads the result.  syn_verify_run launches the step
+ * asynchronously on cuda_stream; accept_len_dev / correction_dev are DEVICE int32 [n_req];
+ * top1_dev is NULL or DEVICE int32 [T] (argmax per chunk position).  It does not synchronise:
+ * call syn_model_status after synchronising the stream to learn of a device-side timeout.
+ * A plan may be run any number of times (each run rewrites the same KV slots). */
+int syn_plan_create(syn_model *m, syn_kv *kv, int32_t n_req, const int32_t *chunk_tokens,
+                    const int32_t *chunk_offsets, const int32_t *page_tables, int32_t max_pages,
+                    const int32_t *ctx_lens, const int32_t *n_uncached, syn_plan **out);
+void syn_plan_free(syn_plan *p);
+int syn_verify_run(syn_model *m, syn_kv *kv, const syn_plan *p, int32_t *accept_len_dev,
+                   int32_t *correction_dev, int32_t *top1_dev, float *logits_out, void *cuda_stream);
+int syn_model_status(syn_model *m); /* SYN_OK or SYN_E_DEVICE_TIMEOUT / SYN_E_CUDA; blocking */
+
+/* Counters of the last planned step (algorithmic work, for roofline arithmetic). */
+typedef struct {
+    int32_t n_req, n_tokens;       /* B and T                                               */
+    int64_t ctx_tokens;            /* sum of ctx_lens                                       */
+    int64_t weight_bytes;          /* bf16 bytes of all projections streamed once per step  */
+    int64_t kv_read_bytes;         /* sum over requests of (ctx+n) * 2*Hkv*hd*2 * n_layers   */
+    int64_t kv_write_bytes;        /* T * 2*Hkv*hd*2 * n_layers                             */
+    double dense_flops;            /* 2 * T * projection parameters                         */
+    double attn_flops;             /* 4 * Hq*hd * n_layers * sum over tokens of keys seen    */
+    int32_t attn_items, attn_split_items; /* attention work items per layer / those that are partial */
+    int32_t kernel_launches;       /* kernels launched by one syn_verify_run                */
+    int64_t h2d_bytes;             /* batch description uploaded per step by syn_verify_batch */
+} syn_step_stats;
+int syn_last_step_stats(const syn_plan *p, syn_step_stats *out);
+
+/* Per-kernel-class device timing.  With profiling on, syn_verify_run / syn_verify_batch bracket
+ * every launch with CUDA events on the caller's stream.  syn_get_profile synchronises the device,
+ * adds up the elapsed time and launch count of each class since the last call, and clears them.
+ * Classes: 0 prep, 1 qkv GEMM, 2 attention, 3 attention merge, 4 o GEMM, 5 gate/up GEMM,
+ * 6 down GEMM, 7 lm_head GEMM, 8 verify.  ms, launches: HOST arrays of SYN_N_KERNEL_CLASSES. */
+#define SYN_N_KERNEL_CLASSES 9
+int syn_set_profile(syn_model *m, int on);
+int syn_get_profile(syn_model *m, double *ms, int32_t *launches);
+
+const char *syn_strerror(int code);
+
+/* ---- single operations, exported for per-kernel tests and roofline measurements ------- */
+
+/* y[T][N] (fp32, DEVICE) = x[T][K] (bf16, DEVICE) * W[N][K]^T (bf16, DEVICE): the tcgen05
+ * GEMM used by every projection, with a plain store epilogue.  K a multiple of 64 is not
+ * required (TMA zero-fills the tail) but K*2 bytes must be a multiple of 16; N arbitrary.
+ * Errors: SYN_E_INVALID_ARG, SYN_E_CUDA. */
+int syn_op_linear(const void *x, const void *w, float *y, int32_t T, int32_t N, int32_t K, void *cuda_stream);
+
+/* The ragged paged attention of the step on its own (paper Sec. 3.2 attention equation over a
+ * paged cache).  q: DEVICE bf16 [T][n_q_heads*head_dim] (rotated); out: DEVICE bf16, same
+ * shape.  The plan supplies page tables, lengths and the work list; the chunk's K/V must
+ * already be in the pool of `layer`.  Asynchronous on cuda_stream. */
+int syn_op_attention(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer, const void *q, void *out,
+                     void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SYNERA_H_ */

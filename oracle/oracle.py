@@ -98,11 +98,12 @@ class Oracle:
         """Place externally produced K/V ([npos][Hkv][hd], any float type) at logical positions pos0.."""
         k = np.asarray(k, dtype=self.real)
         v = np.asarray(v, dtype=self.real)
-        for i in range(k.shape[0]):
-            p = pos0 + i
-            page, row = int(page_table[p // self.P]), p % self.P
-            pool_layer[page, 0, :, row, :] = k[i]
-            pool_layer[page, 1, :, row, :] = v[i]
+        pos = pos0 + np.arange(k.shape[0])
+        pages = np.asarray(page_table, dtype=np.int64)[pos // self.P][:, None]
+        rows = (pos % self.P)[:, None]
+        heads = np.arange(self.shape.n_kv_heads)[None, :]
+        pool_layer[pages, 0, heads, rows, :] = k
+        pool_layer[pages, 1, heads, rows, :] = v
 
     # ------------------------------------------------------------------ single ops (exposed for pins)
     def embed(self, E, tokens) -> np.ndarray:

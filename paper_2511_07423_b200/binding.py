@@ -1,0 +1,273 @@
+"""ctypes binding of include/synera.h: argument marshalling only.
+
+PyTorch supplies device memory and streams; every pointer handed to the library is a raw
+``data_ptr()``.  There is no CPU fallback: if the library is missing or a call fails, a
+:class:`SynError` is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def lib_path() -> str:
+    return os.path.join(HERE, "libsynera.so")
+
+
+class SynError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {code} ({_strerror(code)})")
+        self.code = code
+
+
+class _Desc(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab")] \
+        + [("rope_base", C.c_float), ("rms_eps", C.c_float), ("flags", C.c_uint32)]
+
+
+class _Weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p)] \
+        + [(n, C.POINTER(C.c_void_p)) for n in ("wq", "wk", "wv", "wo", "wg", "wu", "wd", "norm1", "norm2")] \
+        + [("location", C.c_int32)]
+
+
+class StepStats(C.Structure):
+    _fields_ = [("n_req", C.c_int32), ("n_tokens", C.c_int32), ("ctx_tokens", C.c_int64),
+                ("weight_bytes", C.c_int64), ("kv_read_bytes", C.c_int64), ("kv_write_bytes", C.c_int64),
+                ("dense_flops", C.c_double), ("attn_flops", C.c_double), ("attn_items", C.c_int32),
+                ("attn_split_items", C.c_int32), ("kernel_launches", C.c_int32), ("h2d_bytes", C.c_int64)]
+
+KERNEL_CLASSES = ("prep", "qkv_gemm", "attention", "attention_merge", "o_gemm", "gate_up_gemm", "down_gemm",
+                  "lm_head_gemm", "verify")
+
+
+_LIB: Optional[C.CDLL] = None
+
+EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "syn_kv_import", "syn_kv_export",
+           "syn_verify_batch", "syn_plan_create", "syn_plan_free", "syn_verify_run", "syn_model_status",
+           "syn_last_step_stats", "syn_strerror", "syn_op_linear", "syn_op_attention", "syn_set_profile",
+           "syn_get_profile"]
+
+
+def load_library() -> C.CDLL:
+    global _LIB
+    if _LIB is None:
+        path = lib_path()
+        if not os.path.exists(path):
+            raise SynError(-1, f"{path} is missing: run `python -m paper_2511_07423_b200.build`")
+        lib = C.CDLL(path)
+        lib.syn_strerror.restype = C.c_char_p
+        lib.syn_strerror.argtypes = [C.c_int]
+        for fn in ("syn_model_free", "syn_kv_free", "syn_plan_free"):
+            getattr(lib, fn).restype = None
+            getattr(lib, fn).argtypes = [C.c_void_p]
+        _LIB = lib
+    return _LIB
+
+
+def _strerror(code: int) -> str:
+    try:
+        return load_library().syn_strerror(code).decode()
+    except Exception:  # pragma: no cover
+        return "?"
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise SynError(code, what)
+
+
+def _i32(t) -> torch.Tensor:
+    t = torch.as_tensor(t, dtype=torch.int32, device="cpu").contiguous()
+    return t
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> C.c_void_p:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+class Model:
+    """syn_model_load / syn_model_free."""
+
+    def __init__(self, shape, glob: Dict[str, torch.Tensor], layers: Sequence[Dict[str, torch.Tensor]]):
+        lib = load_library()
+        L = shape.n_layers
+        assert len(layers) == L
+        dev = glob["embed"].is_cuda
+        keep: List[torch.Tensor] = []
+
+        def ptr(t: torch.Tensor) -> int:
+            assert t.dtype == torch.bfloat16 and t.is_cuda == dev
+            t = t.contiguous()
+            keep.append(t)
+            return t.data_ptr()
+
+        w = _Weights()
+        w.embed, w.lm_head, w.final_norm = ptr(glob["embed"]), ptr(glob["lm_head"]), ptr(glob["final_norm"])
+        arrays = {}
+        for name in ("wq", "wk", "wv", "wo", "wg", "wu", "wd", "norm1", "norm2"):
+            arr = (C.c_void_p * L)(*[ptr(layers[l][name]) for l in range(L)])
+            arrays[name] = arr
+            setattr(w, name, C.cast(arr, C.POINTER(C.c_void_p)))
+        w.location = 1 if dev else 0
+        d = _Desc(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn,
+                  shape.vocab, float(shape.rope_base), float(shape.rms_eps), 0)
+        self._h = C.c_void_p()
+        _check(lib.syn_model_load(C.byref(d), C.byref(w), C.byref(self._h)), "syn_model_load")
+        self.shape = shape
+        self._lib = lib
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.syn_model_free(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def status(self) -> int:
+        return int(self._lib.syn_model_status(self._h))
+
+    def set_profile(self, on: bool) -> None:
+        _check(self._lib.syn_set_profile(self._h, C.c_int(1 if on else 0)), "syn_set_profile")
+
+    def get_profile(self):
+        """{class name: (total ms, launches)} since the last call (synchronises the device)."""
+        n = len(KERNEL_CLASSES)
+        ms, cnt = (C.c_double * n)(), (C.c_int32 * n)()
+        _check(self._lib.syn_get_profile(self._h, ms, cnt), "syn_get_profile")
+        return {KERNEL_CLASSES[i]: (ms[i], cnt[i]) for i in range(n)}
+
+
+class KVCache:
+    """syn_kv_alloc / syn_kv_import / syn_kv_export / syn_kv_free."""
+
+    def __init__(self, model: Model, n_pages: int, page_size: int = 16):
+        self._lib = load_library()
+        self.model = model
+        self.n_pages, self.page_size = n_pages, page_size
+        self._h = C.c_void_p()
+        _check(self._lib.syn_kv_alloc(model._h, C.c_uint32(n_pages), C.c_uint32(page_size), C.byref(self._h)),
+               "syn_kv_alloc")
+
+    def import_kv(self, layer: int, page_table, pos0: int, k: torch.Tensor, v: torch.Tensor, stream=None) -> None:
+        pt = _i32(page_table)
+        assert k.is_cuda and v.is_cuda and k.dtype == torch.bfloat16 and k.is_contiguous() and v.is_contiguous()
+        _check(self._lib.syn_kv_import(self._h, C.c_uint32(layer), C.c_void_p(pt.data_ptr()), C.c_int32(pos0),
+                                       C.c_int32(k.shape[0]), C.c_void_p(k.data_ptr()), C.c_void_p(v.data_ptr()),
+                                       _stream_ptr(stream)), "syn_kv_import")
+
+    def export_kv(self, layer: int, page_table, pos0: int, n_pos: int, stream=None):
+        s = self.model.shape
+        pt = _i32(page_table)
+        k = torch.empty(n_pos, s.n_kv_heads, s.head_dim, dtype=torch.bfloat16, device="cuda")
+        v = torch.empty_like(k)
+        _check(self._lib.syn_kv_export(self._h, C.c_uint32(layer), C.c_void_p(pt.data_ptr()), C.c_int32(pos0),
+                                       C.c_int32(n_pos), C.c_void_p(k.data_ptr()), C.c_void_p(v.data_ptr()),
+                                       _stream_ptr(stream)), "syn_kv_export")
+        return k, v
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.syn_kv_free(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -------------------------------------------------------------- the step
+    def verify_batch(self, chunk_tokens, chunk_offsets, page_tables, ctx_lens, n_uncached=None,
+                     want_logits: bool = False, req_ids=None, stream=None):
+        """syn_verify_batch with HOST metadata.  Returns (accept_len, correction_token[, logits])."""
+        tok, off, ctx = _i32(chunk_tokens), _i32(chunk_offsets), _i32(ctx_lens)
+        pt = _i32(page_tables)
+        assert pt.dim() == 2
+        n_req = ctx.numel()
+        unc = _i32(n_uncached) if n_uncached is not None else None
+        acc = torch.empty(n_req, dtype=torch.int32)
+        cor = torch.empty(n_req, dtype=torch.int32)
+        logits = None
+        if want_logits:
+            logits = torch.empty(int(off[-1]), self.model.shape.vocab, dtype=torch.float32, device="cuda")
+        ids = torch.as_tensor(req_ids, dtype=torch.int64).contiguous() if req_ids is not None else None
+        _check(self._lib.syn_verify_batch(
+            self.model._h, self._h, C.c_int32(n_req), C.c_void_p(ids.data_ptr()) if ids is not None else None,
+            C.c_void_p(tok.data_ptr()), C.c_void_p(off.data_ptr()), C.c_void_p(pt.data_ptr()), C.c_int32(pt.shape[1]),
+            C.c_void_p(ctx.data_ptr()), C.c_void_p(unc.data_ptr()) if unc is not None else None,
+            C.c_void_p(acc.data_ptr()), C.c_void_p(cor.data_ptr()),
+            C.c_void_p(logits.data_ptr()) if logits is not None else None, _stream_ptr(stream)), "syn_verify_batch")
+        return (acc, cor, logits) if want_logits else (acc, cor)
+
+
+class Plan:
+    """syn_plan_create / syn_verify_run / syn_op_attention / syn_last_step_stats / syn_plan_free."""
+
+    def __init__(self, kv: KVCache, chunk_tokens, chunk_offsets, page_tables, ctx_lens, n_uncached=None):
+        self._lib = load_library()
+        self.kv = kv
+        tok, off, ctx, pt = _i32(chunk_tokens), _i32(chunk_offsets), _i32(ctx_lens), _i32(page_tables)
+        unc = _i32(n_uncached) if n_uncached is not None else None
+        self.n_req, self.n_tokens = ctx.numel(), int(off[-1])
+        self._h = C.c_void_p()
+        _check(self._lib.syn_plan_create(
+            kv.model._h, kv._h, C.c_int32(self.n_req), C.c_void_p(tok.data_ptr()), C.c_void_p(off.data_ptr()),
+            C.c_void_p(pt.data_ptr()), C.c_int32(pt.shape[1]), C.c_void_p(ctx.data_ptr()),
+            C.c_void_p(unc.data_ptr()) if unc is not None else None, C.byref(self._h)), "syn_plan_create")
+
+    def stats(self) -> StepStats:
+        s = StepStats()
+        _check(self._lib.syn_last_step_stats(self._h, C.byref(s)), "syn_last_step_stats")
+        return s
+
+    def run(self, accept_len: torch.Tensor, correction: torch.Tensor, top1: Optional[torch.Tensor] = None,
+            logits: Optional[torch.Tensor] = None, stream=None) -> None:
+        """syn_verify_run: asynchronous, DEVICE int32 outputs."""
+        assert accept_len.is_cuda and correction.is_cuda and accept_len.dtype == torch.int32
+        _check(self._lib.syn_verify_run(
+            self.kv.model._h, self.kv._h, self._h, C.c_void_p(accept_len.data_ptr()), C.c_void_p(correction.data_ptr()),
+            C.c_void_p(top1.data_ptr()) if top1 is not None else None,
+            C.c_void_p(logits.data_ptr()) if logits is not None else None, _stream_ptr(stream)), "syn_verify_run")
+
+    def attention(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        if out is None:
+            out = torch.empty_like(q)
+        _check(self._lib.syn_op_attention(self.kv.model._h, self.kv._h, self._h, C.c_uint32(layer),
+                                          C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()), _stream_ptr(stream)),
+               "syn_op_attention")
+        return out
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.syn_plan_free(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def syn_op_linear(x: torch.Tensor, w: torch.Tensor, stream=None) -> torch.Tensor:
+    """y[T, N] fp32 = x[T, K] bf16 @ w[N, K]^T bf16 through the library's tcgen05 GEMM."""
+    assert x.is_cuda and w.is_cuda and x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
+    x, w = x.contiguous(), w.contiguous()
+    T, K = x.shape
+    N = w.shape[0]
+    y = torch.empty(T, N, dtype=torch.float32, device="cuda")
+    _check(load_library().syn_op_linear(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
+                                        C.c_int32(T), C.c_int32(N), C.c_int32(K), _stream_ptr(stream)), "syn_op_linear")
+    return y

@@ -1,0 +1,899 @@
+// Host side of the library: C ABI, weight packing, KV pool, step planner and the launch
+// sequence of one verification step.  See include/synera.h for the contract of every entry point.
+#include "../../include/synera.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <queue>
+#include <vector>
+
+#include "attention.cuh"
+#include "gemm.cuh"
+
+using namespace syn;
+typedef __nv_bfloat16 bf16;
+
+#define CU_OK(expr)                              \
+    do {                                         \
+        cudaError_t _e = (expr);                 \
+        if (_e != cudaSuccess) {                 \
+            (void)cudaGetLastError();            \
+            return _e == cudaErrorMemoryAllocation ? SYN_E_OOM : SYN_E_CUDA; \
+        }                                        \
+    } while (0)
+
+// ------------------------------------------------------------------------------------------ small kernels
+
+// Token embedding (paper Sec. 4.5: the flattened batch enters the transformer), first layer's
+// GEMM operand bf16(x * gain) with its sum-of-squares partials, RoPE table, argmax reset.
+__global__ void prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens,
+                            const int* __restrict__ pos, const bf16* __restrict__ gain, const double* __restrict__ inv_freq,
+                            float* __restrict__ x, bf16* __restrict__ xn, float* __restrict__ sumsq, float2* __restrict__ rope,
+                            unsigned long long* __restrict__ best, int d, int t_stride, int half) {
+    const int t = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    const bf16* e = embed + (size_t)tokens[t] * d;
+    for (int tile = warp; tile < d / 128; tile += nw) {
+        const int f = tile * 128 + lane * 4;
+        float ss = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float v = __bfloat162float(e[f + k]);
+            x[(size_t)t * d + f + k] = v;
+            xn[(size_t)t * d + f + k] = __float2bfloat16(v * __bfloat162float(gain[f + k]));
+            ss += v * v;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+        if (lane == 0) sumsq[(size_t)tile * t_stride + t] = ss;
+    }
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+        double s, c;
+        sincos((double)pos[t] * inv_freq[i], &s, &c);
+        rope[(size_t)t * half + i] = make_float2((float)c, (float)s);
+    }
+    if (threadIdx.x == 0) best[t] = 0ull;
+}
+
+// Greedy verification (paper Sec. 3.1 "draft & verify", Sec. 4.5): one thread per request.
+__global__ void verify_kernel(const unsigned long long* __restrict__ best, const int* __restrict__ tokens,
+                              const int* __restrict__ offsets, const int* __restrict__ n_uncached, int n_req,
+                              int* __restrict__ accept_len, int* __restrict__ correction, int* __restrict__ top1_out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_req) return;
+    const int b = offsets[i], n = offsets[i + 1] - b, u = n_uncached[i];
+    if (top1_out)
+        for (int j = 0; j < n; ++j) top1_out[b + j] = (int)(0xFFFFFFFFu - (uint32_t)(best[b + j] & 0xFFFFFFFFull));
+    int a = 0;
+    while (a < n - u && (int)(0xFFFFFFFFu - (uint32_t)(best[b + u - 1 + a] & 0xFFFFFFFFull)) == tokens[b + u + a]) ++a;
+    accept_len[i] = a;
+    correction[i] = (int)(0xFFFFFFFFu - (uint32_t)(best[b + u - 1 + a] & 0xFFFFFFFFull));
+}
+
+// Copy K/V of logical positions between a dense [n_pos][Hkv][hd] buffer and the paged pool.
+__global__ void kv_copy_kernel(bf16* pool_layer, const int* __restrict__ slots, bf16* k, bf16* v, int n_kv_heads, int hd,
+                               int page_size, int to_pool) {
+    const int i = blockIdx.x;
+    const int s = slots[i], page = s / page_size, row = s % page_size;
+    for (int e = threadIdx.x; e < n_kv_heads * hd; e += blockDim.x) {
+        const int h = e / hd, dd = e % hd;
+        const size_t ok = ((((size_t)page * n_kv_heads + h) * 2 + 0) * page_size + row) * hd + dd;
+        const size_t ov = ok + (size_t)page_size * hd;
+        const size_t oi = (size_t)i * n_kv_heads * hd + e;
+        if (to_pool) {
+            pool_layer[ok] = k[oi];
+            pool_layer[ov] = v[oi];
+        } else {
+            k[oi] = pool_layer[ok];
+            v[oi] = pool_layer[ov];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ objects
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+static int load_driver_entry() {
+    if (g_encode) return SYN_OK;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CU_OK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return SYN_E_CUDA;
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    return SYN_OK;
+}
+
+// 2-D bf16 row-major [rows][cols] (pitch in elements), box = box_rows x 64 columns, 128-byte swizzle.
+static int make_map_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch, uint32_t box_rows) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {pitch * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SYN_OK : SYN_E_CUDA;
+}
+
+struct syn_model {
+    syn_model_desc desc;
+    int f_pad, n_sm, gu_rows, qkv_rows, v_rows;
+    bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
+    std::vector<bf16*> wqkv, wo, wgu, wd, norm1, norm2;
+    std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wd;
+    CUtensorMap tm_lm;
+    double* inv_freq = nullptr;
+    int* status_dev = nullptr;
+    // workspace (grow-only)
+    int t_cap = 0;
+    float *x = nullptr, *sumsq = nullptr;
+    bf16 *xn = nullptr, *q = nullptr, *attn = nullptr, *act = nullptr;
+    float2* rope = nullptr;
+    unsigned long long* best = nullptr;
+    int *acc_dev = nullptr, *corr_dev = nullptr;
+    int b_cap = 0;
+    CUtensorMap tm_xn, tm_attn, tm_act, tm_q;
+    float* part_o = nullptr;
+    float2* part_ml = nullptr;
+    int part_cap = 0;
+    syn_plan* scratch_plan = nullptr;
+    int* pinned_out = nullptr;
+    int pinned_out_cap = 0;
+    // per-class event timing
+    bool profile = false;
+    struct Ev { cudaEvent_t a, b; int cls; };
+    std::vector<Ev> ev_used, ev_free;
+};
+
+// Brackets one launch with events when profiling is on.
+struct ProfScope {
+    syn_model* m; cudaStream_t st; syn_model::Ev ev; bool on;
+    ProfScope(syn_model* m_, int cls, cudaStream_t st_) : m(m_), st(st_), on(m_ && m_->profile) {
+        if (!on) return;
+        if (!m->ev_free.empty()) { ev = m->ev_free.back(); m->ev_free.pop_back(); }
+        else if (cudaEventCreate(&ev.a) != cudaSuccess || cudaEventCreate(&ev.b) != cudaSuccess) { on = false; return; }
+        ev.cls = cls;
+        cudaEventRecord(ev.a, st);
+    }
+    ~ProfScope() {
+        if (!on) return;
+        cudaEventRecord(ev.b, st);
+        m->ev_used.push_back(ev);
+    }
+};
+
+struct syn_kv {
+    syn_model* model;
+    bf16* pool = nullptr;
+    uint32_t n_pages, page_size;
+    size_t layer_elems;
+    CUtensorMap tm_kv;
+};
+
+struct syn_plan {
+    syn_step_stats stats;
+    int n_req = 0, T = 0, max_pages = 0, n_items = 0, n_cta = 0, n_groups = 0, n_parts = 0;
+    // one device buffer and its pinned host mirror
+    uint8_t *dev = nullptr, *host = nullptr;
+    size_t cap = 0, used = 0;
+    // offsets into the buffer
+    size_t o_tokens, o_pos, o_slot, o_offsets, o_uncached, o_tables, o_items, o_cta, o_groups;
+    bool uploaded_sync = false;
+    template <class Tp> Tp* d(size_t off) const { return reinterpret_cast<Tp*>(dev + off); }
+    template <class Tp> Tp* h(size_t off) const { return reinterpret_cast<Tp*>(host + off); }
+};
+
+static void free_workspace(syn_model* m) {
+    cudaFree(m->x); cudaFree(m->sumsq); cudaFree(m->xn); cudaFree(m->q); cudaFree(m->attn); cudaFree(m->act);
+    cudaFree(m->rope); cudaFree(m->best);
+    m->x = m->sumsq = nullptr; m->xn = m->q = m->attn = m->act = nullptr; m->rope = nullptr; m->best = nullptr;
+    m->t_cap = 0;
+}
+
+static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
+    const syn_model_desc& c = m->desc;
+    const int q_dim = c.n_q_heads * c.head_dim;
+    if (T > m->t_cap) {
+        free_workspace(m);
+        const int cap = (T + 255) / 256 * 256;
+        CU_OK(cudaMalloc(&m->x, (size_t)cap * c.d_model * 4));
+        CU_OK(cudaMalloc(&m->sumsq, (size_t)cap * (c.d_model / 128) * 4));
+        CU_OK(cudaMalloc(&m->xn, (size_t)cap * c.d_model * 2));
+        CU_OK(cudaMalloc(&m->q, (size_t)cap * q_dim * 2));
+        CU_OK(cudaMalloc(&m->attn, (size_t)cap * q_dim * 2));
+        CU_OK(cudaMalloc(&m->act, (size_t)cap * m->f_pad * 2));
+        CU_OK(cudaMalloc(&m->rope, (size_t)cap * (c.head_dim / 2) * 8));
+        CU_OK(cudaMalloc(&m->best, (size_t)cap * 8));
+        CU_OK(cudaMemset(m->xn, 0, (size_t)cap * c.d_model * 2));
+        CU_OK(cudaMemset(m->q, 0, (size_t)cap * q_dim * 2));
+        CU_OK(cudaMemset(m->attn, 0, (size_t)cap * q_dim * 2));
+        CU_OK(cudaMemset(m->act, 0, (size_t)cap * m->f_pad * 2));
+        m->t_cap = cap;
+        int r;
+        if ((r = make_map_2d(&m->tm_xn, m->xn, cap, c.d_model, c.d_model, GEMM_BOX_ROWS))) return r;
+        if ((r = make_map_2d(&m->tm_attn, m->attn, cap, q_dim, q_dim, GEMM_BOX_ROWS))) return r;
+        if ((r = make_map_2d(&m->tm_act, m->act, cap, m->f_pad, m->f_pad, GEMM_BOX_ROWS))) return r;
+        // Q tile of the attention kernel: [token][128-byte line][64]; box = 16 tokens x (G * hd/64) lines
+        const uint32_t G = c.n_q_heads / c.n_kv_heads, halves = c.head_dim / 64;
+        cuuint64_t dims[3] = {64, (cuuint64_t)q_dim / 64, (cuuint64_t)cap};
+        cuuint64_t strides[2] = {128, (cuuint64_t)q_dim * 2};
+        cuuint32_t box[3] = {64, G * halves, 16};
+        cuuint32_t estr[3] = {1, 1, 1};
+        if (g_encode(&m->tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, m->q, dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return SYN_E_CUDA;
+    }
+    if (B > m->b_cap) {
+        cudaFree(m->acc_dev); cudaFree(m->corr_dev);
+        m->acc_dev = m->corr_dev = nullptr; m->b_cap = 0;
+        const int cap = (B + 255) / 256 * 256;
+        CU_OK(cudaMalloc(&m->acc_dev, (size_t)cap * 4));
+        CU_OK(cudaMalloc(&m->corr_dev, (size_t)cap * 4));
+        m->b_cap = cap;
+    }
+    if (n_parts > m->part_cap) {
+        cudaFree(m->part_o); cudaFree(m->part_ml);
+        m->part_o = nullptr; m->part_ml = nullptr; m->part_cap = 0;
+        const int cap = (n_parts + 255) / 256 * 256;
+        CU_OK(cudaMalloc(&m->part_o, (size_t)cap * 64 * c.head_dim * 4));
+        CU_OK(cudaMalloc(&m->part_ml, (size_t)cap * 64 * 8));
+        m->part_cap = cap;
+    }
+    return SYN_OK;
+}
+
+// ------------------------------------------------------------------------------------------ model
+
+extern "C" void syn_model_free(syn_model* m) {
+    if (!m) return;
+    for (auto& v : {&m->wqkv, &m->wo, &m->wgu, &m->wd, &m->norm1, &m->norm2})
+        for (bf16* p : *v) cudaFree(p);
+    cudaFree(m->embed); cudaFree(m->lm_head); cudaFree(m->final_norm); cudaFree(m->inv_freq); cudaFree(m->status_dev);
+    free_workspace(m);
+    cudaFree(m->acc_dev); cudaFree(m->corr_dev); cudaFree(m->part_o); cudaFree(m->part_ml);
+    if (m->pinned_out) cudaFreeHost(m->pinned_out);
+    if (m->scratch_plan) syn_plan_free(m->scratch_plan);
+    for (auto* v : {&m->ev_used, &m->ev_free})
+        for (auto& e : *v) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+    delete m;
+}
+
+extern "C" int syn_model_load(const syn_model_desc* desc, const syn_weights* w, syn_model** out) {
+    if (!desc || !w || !out) return SYN_E_INVALID_ARG;
+    const syn_model_desc c = *desc;
+    if (c.flags != 0 || c.n_layers == 0 || c.vocab == 0 || c.d_ffn == 0) return SYN_E_INVALID_ARG;
+    if (c.head_dim != 64 && c.head_dim != 128) return SYN_E_INVALID_ARG;
+    if (c.d_model == 0 || c.d_model % 128 != 0 || c.d_ffn % 8 != 0) return SYN_E_INVALID_ARG;
+    if (c.n_kv_heads == 0 || c.n_q_heads % c.n_kv_heads != 0 || c.n_q_heads / c.n_kv_heads > 8) return SYN_E_INVALID_ARG;
+    if ((c.n_q_heads * c.head_dim) % 128 != 0 || (c.n_kv_heads * c.head_dim) % 128 != 0) return SYN_E_INVALID_ARG;
+    if (!(c.rope_base > 0.f) || !(c.rms_eps >= 0.f)) return SYN_E_INVALID_ARG;
+    if (!w->embed || !w->lm_head || !w->final_norm || !w->wq || !w->wk || !w->wv || !w->wo || !w->wg || !w->wu ||
+        !w->wd || !w->norm1 || !w->norm2 || (w->location != 0 && w->location != 1))
+        return SYN_E_INVALID_ARG;
+    for (uint32_t l = 0; l < c.n_layers; ++l)
+        if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->wg[l] || !w->wu[l] || !w->wd[l] || !w->norm1[l] ||
+            !w->norm2[l])
+            return SYN_E_INVALID_ARG;
+    int dev = 0;
+    cudaDeviceProp prop;
+    CU_OK(cudaGetDevice(&dev));
+    CU_OK(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return SYN_E_ARCH;
+    int r = load_driver_entry();
+    if (r) return r;
+
+    syn_model* m = new (std::nothrow) syn_model();
+    if (!m) return SYN_E_OOM;
+    m->desc = c;
+    m->n_sm = prop.multiProcessorCount;
+    m->f_pad = (c.d_ffn + 63) / 64 * 64;
+    const int d = c.d_model, q_dim = c.n_q_heads * c.head_dim, kv_dim = c.n_kv_heads * c.head_dim, f = c.d_ffn;
+    m->qkv_rows = q_dim + 2 * kv_dim;
+    m->gu_rows = 2 * m->f_pad;
+    m->v_rows = (c.vocab + 127) / 128 * 128;
+    const int loc = w->location;
+    const cudaMemcpyKind kind = loc ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+
+#define LOAD_FAIL(code)        \
+    do {                       \
+        syn_model_free(m);     \
+        return (code);         \
+    } while (0)
+#define CU_M(expr)                                                                        \
+    do {                                                                                  \
+        cudaError_t _e = (expr);                                                          \
+        if (_e != cudaSuccess) {                                                          \
+            (void)cudaGetLastError();                                                     \
+            LOAD_FAIL(_e == cudaErrorMemoryAllocation ? SYN_E_OOM : SYN_E_CUDA);          \
+        }                                                                                 \
+    } while (0)
+
+    CU_M(cudaMalloc(&m->embed, (size_t)c.vocab * d * 2));
+    CU_M(cudaMemcpy(m->embed, w->embed, (size_t)c.vocab * d * 2, kind));
+    CU_M(cudaMalloc(&m->lm_head, (size_t)m->v_rows * d * 2));
+    CU_M(cudaMemset(m->lm_head, 0, (size_t)m->v_rows * d * 2));
+    CU_M(cudaMemcpy(m->lm_head, w->lm_head, (size_t)c.vocab * d * 2, kind));
+    CU_M(cudaMalloc(&m->final_norm, (size_t)d * 2));
+    CU_M(cudaMemcpy(m->final_norm, w->final_norm, (size_t)d * 2, kind));
+    if ((r = make_map_2d(&m->tm_lm, m->lm_head, m->v_rows, d, d, 128))) LOAD_FAIL(r);
+    m->tm_wqkv.resize(c.n_layers); m->tm_wo.resize(c.n_layers); m->tm_wgu.resize(c.n_layers); m->tm_wd.resize(c.n_layers);
+    for (uint32_t l = 0; l < c.n_layers; ++l) {
+        bf16 *pqkv = nullptr, *po = nullptr, *pgu = nullptr, *pd = nullptr, *n1 = nullptr, *n2 = nullptr;
+        CU_M(cudaMalloc(&pqkv, (size_t)m->qkv_rows * d * 2)); m->wqkv.push_back(pqkv);
+        CU_M(cudaMalloc(&po, (size_t)d * q_dim * 2)); m->wo.push_back(po);
+        CU_M(cudaMalloc(&pgu, (size_t)m->gu_rows * d * 2)); m->wgu.push_back(pgu);
+        CU_M(cudaMalloc(&pd, (size_t)d * m->f_pad * 2)); m->wd.push_back(pd);
+        CU_M(cudaMalloc(&n1, (size_t)d * 2)); m->norm1.push_back(n1);
+        CU_M(cudaMalloc(&n2, (size_t)d * 2)); m->norm2.push_back(n2);
+        CU_M(cudaMemcpy(pqkv, w->wq[l], (size_t)q_dim * d * 2, kind));
+        CU_M(cudaMemcpy(pqkv + (size_t)q_dim * d, w->wk[l], (size_t)kv_dim * d * 2, kind));
+        CU_M(cudaMemcpy(pqkv + (size_t)(q_dim + kv_dim) * d, w->wv[l], (size_t)kv_dim * d * 2, kind));
+        CU_M(cudaMemcpy(po, w->wo[l], (size_t)d * q_dim * 2, kind));
+        // gate/up interleaved in blocks of 64 rows: packed rows [128b, 128b+64) = gate rows [64b, 64b+64),
+        // [128b+64, 128b+128) = up rows; rows of the padded tail are zero.
+        CU_M(cudaMemset(pgu, 0, (size_t)m->gu_rows * d * 2));
+        const int full = f / 64, tail = f % 64;
+        const size_t blk = (size_t)64 * d * 2;
+        if (full) {
+            CU_M(cudaMemcpy2D(pgu, 2 * blk, w->wg[l], blk, blk, full, kind));
+            CU_M(cudaMemcpy2D(reinterpret_cast<uint8_t*>(pgu) + blk, 2 * blk, w->wu[l], blk, blk, full, kind));
+        }
+        if (tail) {
+            CU_M(cudaMemcpy(reinterpret_cast<uint8_t*>(pgu) + 2 * blk * full,
+                            reinterpret_cast<const uint8_t*>(w->wg[l]) + blk * full, (size_t)tail * d * 2, kind));
+            CU_M(cudaMemcpy(reinterpret_cast<uint8_t*>(pgu) + 2 * blk * full + blk,
+                            reinterpret_cast<const uint8_t*>(w->wu[l]) + blk * full, (size_t)tail * d * 2, kind));
+        }
+        CU_M(cudaMemset(pd, 0, (size_t)d * m->f_pad * 2));
+        CU_M(cudaMemcpy2D(pd, (size_t)m->f_pad * 2, w->wd[l], (size_t)f * 2, (size_t)f * 2, d, kind));
+        CU_M(cudaMemcpy(n1, w->norm1[l], (size_t)d * 2, kind));
+        CU_M(cudaMemcpy(n2, w->norm2[l], (size_t)d * 2, kind));
+        if ((r = make_map_2d(&m->tm_wqkv[l], pqkv, m->qkv_rows, d, d, 128))) LOAD_FAIL(r);
+        if ((r = make_map_2d(&m->tm_wo[l], po, d, q_dim, q_dim, 128))) LOAD_FAIL(r);
+        if ((r = make_map_2d(&m->tm_wgu[l], pgu, m->gu_rows, d, d, 128))) LOAD_FAIL(r);
+        if ((r = make_map_2d(&m->tm_wd[l], pd, d, m->f_pad, m->f_pad, 128))) LOAD_FAIL(r);
+    }
+    std::vector<double> inv(c.head_dim / 2);
+    for (uint32_t i = 0; i < c.head_dim / 2; ++i) inv[i] = std::pow((double)c.rope_base, -2.0 * (double)i / (double)c.head_dim);
+    CU_M(cudaMalloc(&m->inv_freq, inv.size() * 8));
+    CU_M(cudaMemcpy(m->inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice));
+    CU_M(cudaMalloc(&m->status_dev, 4));
+    CU_M(cudaMemset(m->status_dev, 0, 4));
+    CU_M(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    CU_M(cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::TOTAL));
+    CU_M(cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::TOTAL));
+    CU_M(cudaDeviceSynchronize());
+    *out = m;
+    return SYN_OK;
+#undef CU_M
+#undef LOAD_FAIL
+}
+
+// ------------------------------------------------------------------------------------------ KV pool
+
+extern "C" void syn_kv_free(syn_kv* kv) {
+    if (!kv) return;
+    cudaFree(kv->pool);
+    delete kv;
+}
+
+extern "C" int syn_kv_alloc(syn_model* m, uint32_t n_pages, uint32_t page_size, syn_kv** out) {
+    if (!m || !out || n_pages == 0 || page_size != 16) return SYN_E_INVALID_ARG;
+    const syn_model_desc& c = m->desc;
+    const uint64_t blocks = (uint64_t)c.n_layers * n_pages * c.n_kv_heads * 2;
+    if (blocks > 0x7FFFFFFFull) return SYN_E_INVALID_ARG;
+    syn_kv* kv = new (std::nothrow) syn_kv();
+    if (!kv) return SYN_E_OOM;
+    kv->model = m;
+    kv->n_pages = n_pages;
+    kv->page_size = page_size;
+    kv->layer_elems = (size_t)n_pages * c.n_kv_heads * 2 * page_size * c.head_dim;
+    const size_t bytes = kv->layer_elems * c.n_layers * 2;
+    cudaError_t e = cudaMalloc(&kv->pool, bytes);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete kv;
+        return e == cudaErrorMemoryAllocation ? SYN_E_OOM : SYN_E_CUDA;
+    }
+    if (cudaMemset(kv->pool, 0, bytes) != cudaSuccess) {
+        syn_kv_free(kv);
+        return SYN_E_CUDA;
+    }
+    // pool as a 2-D tensor [blocks * 16 rows][head_dim]; a box of 32 rows x 64 columns is one
+    // 64-element half of the K rows and the V rows of one (page, kv head)
+    if (make_map_2d(&kv->tm_kv, kv->pool, blocks * page_size, c.head_dim, c.head_dim, 2 * page_size) != SYN_OK) {
+        syn_kv_free(kv);
+        return SYN_E_CUDA;
+    }
+    if (cudaDeviceSynchronize() != cudaSuccess) {
+        syn_kv_free(kv);
+        return SYN_E_CUDA;
+    }
+    *out = kv;
+    return SYN_OK;
+}
+
+static int kv_copy(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_t pos0, int32_t n_pos, void* k, void* v,
+                   void* stream, int to_pool) {
+    if (!kv || !page_table || !k || !v || pos0 < 0 || n_pos <= 0 || layer >= kv->model->desc.n_layers)
+        return SYN_E_INVALID_ARG;
+    const int P = (int)kv->page_size;
+    std::vector<int> slots(n_pos);
+    for (int i = 0; i < n_pos; ++i) {
+        const int p = pos0 + i, page = page_table[p / P];
+        if (page < 0 || (uint32_t)page >= kv->n_pages) return SYN_E_PAGE_OOB;
+        slots[i] = page * P + p % P;
+    }
+    int* d_slots = nullptr;
+    CU_OK(cudaMalloc(&d_slots, (size_t)n_pos * 4));
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(d_slots, slots.data(), (size_t)n_pos * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess) {
+        const syn_model_desc& c = kv->model->desc;
+        kv_copy_kernel<<<n_pos, 128, 0, st>>>(kv->pool + kv->layer_elems * layer, d_slots, (bf16*)k, (bf16*)v,
+                                              c.n_kv_heads, c.head_dim, P, to_pool);
+        e = cudaGetLastError();
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    }
+    cudaFree(d_slots);
+    return e == cudaSuccess ? SYN_OK : SYN_E_CUDA;
+}
+
+extern "C" int syn_kv_import(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_t pos0, int32_t n_pos,
+                             const void* k, const void* v, void* stream) {
+    return kv_copy(kv, layer, page_table, pos0, n_pos, const_cast<void*>(k), const_cast<void*>(v), stream, 1);
+}
+extern "C" int syn_kv_export(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_t pos0, int32_t n_pos, void* k,
+                             void* v, void* stream) {
+    return kv_copy(kv, layer, page_table, pos0, n_pos, k, v, stream, 0);
+}
+
+// ------------------------------------------------------------------------------------------ planner
+
+extern "C" void syn_plan_free(syn_plan* p) {
+    if (!p) return;
+    cudaFree(p->dev);
+    if (p->host) cudaFreeHost(p->host);
+    delete p;
+}
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Validate the batch, then build token positions, KV slots and the attention work list.
+static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, const int32_t* chunk_tokens,
+                      const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages, const int32_t* ctx_lens,
+                      const int32_t* n_uncached) {
+    if (!m || !kv || kv->model != m || n_req <= 0 || !chunk_tokens || !chunk_offsets || !page_tables || !ctx_lens ||
+        max_pages <= 0)
+        return SYN_E_INVALID_ARG;
+    const syn_model_desc& c = m->desc;
+    const int P = (int)kv->page_size, G = c.n_q_heads / c.n_kv_heads, Hkv = c.n_kv_heads;
+    if (chunk_offsets[0] != 0) return SYN_E_INVALID_ARG;
+    int64_t ctx_sum = 0, keys_seen = 0, kv_units = 0;
+    for (int i = 0; i < n_req; ++i) {
+        const int64_t n = (int64_t)chunk_offsets[i + 1] - chunk_offsets[i];
+        if (n < 1 || n > SYN_MAX_CHUNK) return SYN_E_CHUNK_LEN;
+        const int u = n_uncached ? n_uncached[i] : 1;
+        if (u < 1 || u > n) return SYN_E_UNCACHED;
+        if (ctx_lens[i] < 0) return SYN_E_INVALID_ARG;
+        if ((int64_t)ctx_lens[i] + n > (int64_t)max_pages * P) return SYN_E_CAPACITY;
+        const int used = (int)((ctx_lens[i] + n + P - 1) / P);
+        for (int k = 0; k < used; ++k) {
+            const int pg = page_tables[(size_t)i * max_pages + k];
+            if (pg < 0 || (uint32_t)pg >= kv->n_pages) return SYN_E_PAGE_OOB;
+        }
+        ctx_sum += ctx_lens[i];
+        kv_units += ctx_lens[i] + n;
+        keys_seen += n * (int64_t)ctx_lens[i] + n * (n + 1) / 2;
+    }
+    const int T = chunk_offsets[n_req];
+    for (int t = 0; t < T; ++t)
+        if (chunk_tokens[t] < 0 || (uint32_t)chunk_tokens[t] >= c.vocab) return SYN_E_TOKEN_OOB;
+    std::vector<int> pos(T), slot(T);
+    for (int i = 0; i < n_req; ++i)
+        for (int j = 0, b = chunk_offsets[i]; b + j < chunk_offsets[i + 1]; ++j) {
+            const int pp = ctx_lens[i] + j;
+            pos[b + j] = pp;
+            slot[b + j] = page_tables[(size_t)i * max_pages + pp / P] * P + pp % P;
+        }
+    {
+        std::vector<int> s2(slot);
+        std::sort(s2.begin(), s2.end());
+        for (int t = 1; t < T; ++t)
+            if (s2[t] == s2[t - 1]) return SYN_E_PAGE_ALIAS;
+    }
+    // attention work list: (request, kv head, token group, key range); split long key ranges
+    const int n_cta_max = m->n_sm;
+    const int tok_per_group = std::min(16, 64 / G);
+    int64_t split = (kv_units * Hkv) / ((int64_t)n_cta_max * 6);
+    split = std::max<int64_t>(512, (split + 63) / 64 * 64);
+    std::vector<AttnItem> items;
+    std::vector<MergeGroup> groups;
+    int n_parts = 0;
+    for (int i = 0; i < n_req; ++i) {
+        const int b = chunk_offsets[i], n = chunk_offsets[i + 1] - b;
+        for (int j0 = 0; j0 < n; j0 += tok_per_group) {
+            const int nj = std::min(tok_per_group, n - j0);
+            const int L = ctx_lens[i] + j0 + nj;
+            int np = (int)std::min<int64_t>(64, (L + split - 1) / split);
+            int len = ((L + np - 1) / np + 63) / 64 * 64;
+            np = (L + len - 1) / len;
+            for (int h = 0; h < Hkv; ++h) {
+                if (np > 1) {
+                    MergeGroup g = {b + j0, nj, h, n_parts, np, 0, 0, 0};
+                    groups.push_back(g);
+                }
+                for (int k = 0; k < np; ++k) {
+                    AttnItem it = {b + j0, nj, h, i, k * len, std::min(L, (k + 1) * len), ctx_lens[i] + j0,
+                                   np > 1 ? n_parts + k : -1};
+                    items.push_back(it);
+                }
+                if (np > 1) n_parts += np;
+            }
+        }
+    }
+    const int n_items = (int)items.size();
+    const int n_cta = std::min(n_cta_max, n_items);
+    std::vector<int> order(n_items), owner(n_items);
+    for (int i = 0; i < n_items; ++i) order[i] = i;
+    auto cost = [&](int i) { return items[i].kv_end - items[i].kv_begin + 48; };
+    std::stable_sort(order.begin(), order.end(), [&](int a, int bb) { return cost(a) > cost(bb); });
+    typedef std::pair<int64_t, int> Load;
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int k = 0; k < n_cta; ++k) heap.push(Load(0, k));
+    std::vector<int> count(n_cta + 1, 0);
+    for (int i : order) {
+        Load l = heap.top();
+        heap.pop();
+        owner[i] = l.second;
+        count[l.second + 1]++;
+        heap.push(Load(l.first + cost(i), l.second));
+    }
+    for (int k = 0; k < n_cta; ++k) count[k + 1] += count[k];
+    std::vector<AttnItem> sorted(n_items);
+    {
+        std::vector<int> cur(count.begin(), count.end() - 1);
+        for (int i : order) sorted[cur[owner[i]]++] = items[i];
+    }
+    // pack everything into one buffer
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    p->o_tokens = take((size_t)T * 4);
+    p->o_pos = take((size_t)T * 4);
+    p->o_slot = take((size_t)T * 4);
+    p->o_offsets = take((size_t)(n_req + 1) * 4);
+    p->o_uncached = take((size_t)n_req * 4);
+    p->o_tables = take((size_t)n_req * max_pages * 4);
+    p->o_items = take((size_t)n_items * sizeof(AttnItem));
+    p->o_cta = take((size_t)(n_cta + 1) * 4);
+    p->o_groups = take(std::max<size_t>(1, groups.size()) * sizeof(MergeGroup));
+    if (off > p->cap) {
+        cudaFree(p->dev);
+        if (p->host) cudaFreeHost(p->host);
+        p->dev = p->host = nullptr;
+        p->cap = 0;
+        const size_t cap = align_up(off + off / 2, 4096);
+        CU_OK(cudaMalloc(&p->dev, cap));
+        CU_OK(cudaMallocHost(&p->host, cap));
+        p->cap = cap;
+    }
+    p->used = off;
+    memcpy(p->h<int>(p->o_tokens), chunk_tokens, (size_t)T * 4);
+    memcpy(p->h<int>(p->o_pos), pos.data(), (size_t)T * 4);
+    memcpy(p->h<int>(p->o_slot), slot.data(), (size_t)T * 4);
+    memcpy(p->h<int>(p->o_offsets), chunk_offsets, (size_t)(n_req + 1) * 4);
+    for (int i = 0; i < n_req; ++i) p->h<int>(p->o_uncached)[i] = n_uncached ? n_uncached[i] : 1;
+    memcpy(p->h<int>(p->o_tables), page_tables, (size_t)n_req * max_pages * 4);
+    memcpy(p->h<AttnItem>(p->o_items), sorted.data(), (size_t)n_items * sizeof(AttnItem));
+    memcpy(p->h<int>(p->o_cta), count.data(), (size_t)(n_cta + 1) * 4);
+    if (!groups.empty()) memcpy(p->h<MergeGroup>(p->o_groups), groups.data(), groups.size() * sizeof(MergeGroup));
+    p->n_req = n_req; p->T = T; p->max_pages = max_pages; p->n_items = n_items; p->n_cta = n_cta;
+    p->n_groups = (int)groups.size(); p->n_parts = n_parts;
+
+    syn_step_stats& s = p->stats;
+    const double d = c.d_model, qd = (double)c.n_q_heads * c.head_dim, kd = (double)Hkv * c.head_dim;
+    const double params = c.n_layers * (d * (qd + 2 * kd) + qd * d + 3.0 * d * c.d_ffn) + d * c.vocab;
+    s.n_req = n_req; s.n_tokens = T; s.ctx_tokens = ctx_sum;
+    s.weight_bytes = (int64_t)(params * 2);
+    s.kv_read_bytes = kv_units * (int64_t)(2 * kd * 2) * c.n_layers;
+    s.kv_write_bytes = (int64_t)T * (int64_t)(2 * kd * 2) * c.n_layers;
+    s.dense_flops = 2.0 * T * params;
+    s.attn_flops = 4.0 * qd * c.n_layers * (double)keys_seen;
+    s.attn_items = n_items; s.attn_split_items = n_parts;
+    s.kernel_launches = 2 + c.n_layers * (5 + (groups.empty() ? 0 : 1)) + 1;
+    s.h2d_bytes = (int64_t)off;
+    return SYN_OK;
+}
+
+extern "C" int syn_plan_create(syn_model* m, syn_kv* kv, int32_t n_req, const int32_t* chunk_tokens,
+                               const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages,
+                               const int32_t* ctx_lens, const int32_t* n_uncached, syn_plan** out) {
+    if (!out) return SYN_E_INVALID_ARG;
+    syn_plan* p = new (std::nothrow) syn_plan();
+    if (!p) return SYN_E_OOM;
+    int r = plan_build(p, m, kv, n_req, chunk_tokens, chunk_offsets, page_tables, max_pages, ctx_lens, n_uncached);
+    if (r == SYN_OK) {
+        cudaError_t e = cudaMemcpy(p->dev, p->host, p->used, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) r = SYN_E_CUDA;
+    }
+    if (r == SYN_OK) r = ensure_workspace(m, p->T, p->n_req, p->n_parts);
+    if (r != SYN_OK) {
+        syn_plan_free(p);
+        return r;
+    }
+    *out = p;
+    return SYN_OK;
+}
+
+extern "C" int syn_last_step_stats(const syn_plan* p, syn_step_stats* out) {
+    if (!p || !out) return SYN_E_INVALID_ARG;
+    *out = p->stats;
+    return SYN_OK;
+}
+
+// ------------------------------------------------------------------------------------------ launches
+
+static int launch_gemm(syn_model* m, int cls, const CUtensorMap& tmA, const CUtensorMap& tmB, const bf16* W, const bf16* X,
+                       int ldw, int ldx, int n_rows, int K, EpiParams ep, cudaStream_t st) {
+    const int T = ep.T;
+    ProfScope prof(cls >= 0 ? m : nullptr, cls, st);
+#ifdef SYN_GEMM_LEGACY
+    dim3 grid((n_rows + 127) / 128, (T + 31) / 32);
+    gemm_legacy_kernel<<<grid, 128, 0, st>>>(W, X, K, ldw, ldx, ep);
+#else
+    (void)W; (void)X; (void)ldw; (void)ldx;
+    const int nt = (T + 255) / 256;
+    const int TN = (((T + nt - 1) / nt) + 15) / 16 * 16;
+    const int sb = gemm_stage_bytes(TN);
+    int stages = std::min(GEMM_MAX_STAGES, (232448 - 1024 - 2 * 32 * 128 * 4 - 1024 - 256 - 1024) / sb);
+    if (stages < 2) return SYN_E_INVALID_ARG;
+    dim3 grid((n_rows + 127) / 128, nt);
+    gemm_tc_kernel<<<grid, GEMM_THREADS, gemm_smem_bytes(TN, stages), st>>>(tmA, tmB, K, TN, stages, ep,
+                                                                          m ? m->status_dev : nullptr);
+#endif
+    return cudaGetLastError() == cudaSuccess ? SYN_OK : SYN_E_CUDA;
+}
+
+static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const CUtensorMap& tmQ,
+                            bf16* out, cudaStream_t st) {
+    const syn_model_desc& c = m->desc;
+    AttnParams ap;
+    ap.items = p->d<AttnItem>(p->o_items);
+    ap.cta_begin = p->d<int>(p->o_cta);
+    ap.page_tables = p->d<int>(p->o_tables);
+    ap.max_pages = p->max_pages;
+    ap.n_kv_heads = c.n_kv_heads;
+    ap.group = c.n_q_heads / c.n_kv_heads;
+    ap.q_dim = c.n_q_heads * c.head_dim;
+    ap.layer_block0 = (int)(2ull * layer * kv->n_pages * c.n_kv_heads);
+    ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
+    ap.out = out;
+    ap.part_o = m->part_o;
+    ap.part_ml = m->part_ml;
+    ap.status = m->status_dev;
+    {
+        ProfScope prof(m, 2, st);
+        if (c.head_dim == 128)
+            attn_kernel<128><<<p->n_cta, ATT_THREADS, AttnSmem<128>::TOTAL, st>>>(tmQ, kv->tm_kv, ap);
+        else
+            attn_kernel<64><<<p->n_cta, ATT_THREADS, AttnSmem<64>::TOTAL, st>>>(tmQ, kv->tm_kv, ap);
+    }
+    if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
+    if (p->n_groups) {
+        ProfScope prof(m, 3, st);
+        dim3 blk(32, 8);
+        if (c.head_dim == 128)
+            attn_merge_kernel<128><<<p->n_groups, blk, 0, st>>>(p->d<MergeGroup>(p->o_groups), m->part_o, m->part_ml, out,
+                                                                ap.group, ap.q_dim);
+        else
+            attn_merge_kernel<64><<<p->n_groups, blk, 0, st>>>(p->d<MergeGroup>(p->o_groups), m->part_o, m->part_ml, out,
+                                                               ap.group, ap.q_dim);
+        if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
+    }
+    return SYN_OK;
+}
+
+static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, int* corr_dev, int* top1_dev,
+                    float* logits_out, cudaStream_t st) {
+    const syn_model_desc& c = m->desc;
+    const int T = p->T, d = c.d_model, q_dim = c.n_q_heads * c.head_dim, kv_dim = c.n_kv_heads * c.head_dim;
+    if (T > m->t_cap || p->n_req > m->b_cap || p->n_parts > m->part_cap) return SYN_E_INVALID_ARG;
+    const int* tokens = p->d<int>(p->o_tokens);
+    {
+        ProfScope prof(m, 0, st);
+        prep_kernel<<<T, 128, 0, st>>>(m->embed, tokens, p->d<int>(p->o_pos), m->norm1[0], m->inv_freq, m->x, m->xn,
+                                       m->sumsq, m->rope, m->best, d, m->t_cap, c.head_dim / 2);
+    }
+    if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
+    EpiParams base;
+    memset(&base, 0, sizeof(base));
+    base.T = T;
+    base.sumsq_in = m->sumsq;
+    base.n_sumsq_tiles = d / 128;
+    base.t_stride = m->t_cap;
+    base.inv_d = 1.0f / (float)d;
+    base.eps = c.rms_eps;
+    int r;
+    for (uint32_t l = 0; l < c.n_layers; ++l) {
+        EpiParams e = base;
+        e.mode = EPI_QKV; e.N = m->qkv_rows;
+        e.q = m->q; e.q_dim = q_dim; e.kv_dim = kv_dim; e.hd = c.head_dim; e.n_kv_heads = c.n_kv_heads;
+        e.page_size = kv->page_size; e.rope = m->rope; e.pool = kv->pool + kv->layer_elems * l;
+        e.slot = p->d<int>(p->o_slot);
+        if ((r = launch_gemm(m, 1, m->tm_wqkv[l], m->tm_xn, m->wqkv[l], m->xn, d, d, m->qkv_rows, d, e, st))) return r;
+        if ((r = launch_attention(m, kv, p, l, m->tm_q, m->attn, st))) return r;
+        e = base;
+        e.mode = EPI_RESID; e.N = d; e.x = m->x; e.d = d; e.xn = m->xn; e.gain_next = m->norm2[l]; e.sumsq_out = m->sumsq;
+        if ((r = launch_gemm(m, 4, m->tm_wo[l], m->tm_attn, m->wo[l], m->attn, q_dim, q_dim, d, q_dim, e, st))) return r;
+        e = base;
+        e.mode = EPI_SWIGLU; e.N = m->gu_rows; e.act = m->act; e.f_pad = m->f_pad;
+        if ((r = launch_gemm(m, 5, m->tm_wgu[l], m->tm_xn, m->wgu[l], m->xn, d, d, m->gu_rows, d, e, st))) return r;
+        e = base;
+        e.mode = EPI_RESID; e.N = d; e.x = m->x; e.d = d; e.xn = m->xn;
+        e.gain_next = l + 1 < c.n_layers ? m->norm1[l + 1] : m->final_norm; e.sumsq_out = m->sumsq;
+        if ((r = launch_gemm(m, 6, m->tm_wd[l], m->tm_act, m->wd[l], m->act, m->f_pad, m->f_pad, d, m->f_pad, e, st))) return r;
+    }
+    EpiParams e = base;
+    e.mode = EPI_LMHEAD; e.N = m->v_rows; e.vocab = c.vocab; e.logits = logits_out; e.best = m->best;
+    if ((r = launch_gemm(m, 7, m->tm_lm, m->tm_xn, m->lm_head, m->xn, d, d, m->v_rows, d, e, st))) return r;
+    {
+        ProfScope prof(m, 8, st);
+        verify_kernel<<<(p->n_req + 127) / 128, 128, 0, st>>>(m->best, tokens, p->d<int>(p->o_offsets),
+                                                             p->d<int>(p->o_uncached), p->n_req, acc_dev, corr_dev, top1_dev);
+    }
+    return cudaGetLastError() == cudaSuccess ? SYN_OK : SYN_E_CUDA;
+}
+
+extern "C" int syn_verify_run(syn_model* m, syn_kv* kv, const syn_plan* p, int32_t* accept_len_dev, int32_t* correction_dev,
+                              int32_t* top1_dev, float* logits_out, void* cuda_stream) {
+    if (!m || !kv || !p || kv->model != m || !accept_len_dev || !correction_dev) return SYN_E_INVALID_ARG;
+    return run_step(m, kv, p, accept_len_dev, correction_dev, top1_dev, logits_out, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int syn_set_profile(syn_model* m, int on) {
+    if (!m) return SYN_E_INVALID_ARG;
+    m->profile = on != 0;
+    return SYN_OK;
+}
+
+extern "C" int syn_get_profile(syn_model* m, double* ms, int32_t* launches) {
+    if (!m || !ms || !launches) return SYN_E_INVALID_ARG;
+    CU_OK(cudaDeviceSynchronize());
+    for (int i = 0; i < SYN_N_KERNEL_CLASSES; ++i) { ms[i] = 0.0; launches[i] = 0; }
+    for (auto& e : m->ev_used) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, e.a, e.b) == cudaSuccess && e.cls >= 0 && e.cls < SYN_N_KERNEL_CLASSES) {
+            ms[e.cls] += t;
+            launches[e.cls] += 1;
+        }
+        m->ev_free.push_back(e);
+    }
+    m->ev_used.clear();
+    return SYN_OK;
+}
+
+extern "C" int syn_model_status(syn_model* m) {
+    if (!m) return SYN_E_INVALID_ARG;
+    int s = 0;
+    if (cudaMemcpy(&s, m->status_dev, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SYN_E_CUDA;
+    if (s) {
+        cudaMemset(m->status_dev, 0, 4);
+        return SYN_E_DEVICE_TIMEOUT;
+    }
+    return SYN_OK;
+}
+
+extern "C" int syn_verify_batch(syn_model* m, syn_kv* kv, int32_t n_req, const int64_t* req_ids, const int32_t* chunk_tokens,
+                                const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages,
+                                const int32_t* ctx_lens, const int32_t* n_uncached, int32_t* accept_len,
+                                int32_t* correction_token, float* logits_out, void* cuda_stream) {
+    (void)req_ids;
+    if (!m || !accept_len || !correction_token) return SYN_E_INVALID_ARG;
+    if (!m->scratch_plan) {
+        m->scratch_plan = new (std::nothrow) syn_plan();
+        if (!m->scratch_plan) return SYN_E_OOM;
+    }
+    syn_plan* p = m->scratch_plan;
+    int r = plan_build(p, m, kv, n_req, chunk_tokens, chunk_offsets, page_tables, max_pages, ctx_lens, n_uncached);
+    if (r) return r;
+    if ((r = ensure_workspace(m, p->T, p->n_req, p->n_parts))) return r;
+    if (n_req > m->pinned_out_cap) {
+        if (m->pinned_out) cudaFreeHost(m->pinned_out);
+        m->pinned_out = nullptr; m->pinned_out_cap = 0;
+        const int cap = (n_req + 255) / 256 * 256;
+        CU_OK(cudaMallocHost(&m->pinned_out, (size_t)cap * 12));
+        m->pinned_out_cap = cap;
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    CU_OK(cudaMemcpyAsync(p->dev, p->host, p->used, cudaMemcpyHostToDevice, st));
+    if ((r = run_step(m, kv, p, m->acc_dev, m->corr_dev, nullptr, logits_out, st))) return r;
+    int* po = m->pinned_out;
+    CU_OK(cudaMemcpyAsync(po, m->acc_dev, (size_t)n_req * 4, cudaMemcpyDeviceToHost, st));
+    CU_OK(cudaMemcpyAsync(po + m->pinned_out_cap, m->corr_dev, (size_t)n_req * 4, cudaMemcpyDeviceToHost, st));
+    CU_OK(cudaMemcpyAsync(po + 2 * m->pinned_out_cap, m->status_dev, 4, cudaMemcpyDeviceToHost, st));
+    CU_OK(cudaStreamSynchronize(st));
+    if (po[2 * m->pinned_out_cap]) {
+        cudaMemset(m->status_dev, 0, 4);
+        return SYN_E_DEVICE_TIMEOUT;
+    }
+    memcpy(accept_len, po, (size_t)n_req * 4);
+    memcpy(correction_token, po + m->pinned_out_cap, (size_t)n_req * 4);
+    return SYN_OK;
+}
+
+// ------------------------------------------------------------------------------------------ single ops
+
+extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, int32_t N, int32_t K, void* cuda_stream) {
+    if (!x || !w || !y || T <= 0 || N <= 0 || K <= 0 || K % 8 != 0) return SYN_E_INVALID_ARG;
+    int r = load_driver_entry();
+    if (r) return r;
+    static bool attr_set = false;
+    if (!attr_set) {
+        CU_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+        attr_set = true;
+    }
+    static int* status = nullptr;
+    if (!status) {
+        CU_OK(cudaMalloc(&status, 4));
+        CU_OK(cudaMemset(status, 0, 4));
+    }
+    CUtensorMap tmA, tmB;
+    if ((r = make_map_2d(&tmA, w, N, K, K, 128))) return r;
+    if ((r = make_map_2d(&tmB, x, T, K, K, GEMM_BOX_ROWS))) return r;
+    EpiParams e;
+    memset(&e, 0, sizeof(e));
+    e.mode = EPI_PLAIN; e.T = T; e.N = N; e.y = y; e.ldy = N;
+    syn_model fake;  // only status_dev is read
+    fake.status_dev = status;
+    r = launch_gemm(&fake, -1, tmA, tmB, (const bf16*)w, (const bf16*)x, K, K, N, K, e, reinterpret_cast<cudaStream_t>(cuda_stream));
+    if (r) return r;
+    CU_OK(cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(cuda_stream)));
+    int s = 0;
+    CU_OK(cudaMemcpy(&s, status, 4, cudaMemcpyDeviceToHost));
+    if (s) {
+        cudaMemset(status, 0, 4);
+        return SYN_E_DEVICE_TIMEOUT;
+    }
+    return SYN_OK;
+}
+
+extern "C" int syn_op_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const void* q, void* out,
+                                void* cuda_stream) {
+    if (!m || !kv || !p || kv->model != m || !q || !out || layer >= m->desc.n_layers) return SYN_E_INVALID_ARG;
+    const syn_model_desc& c = m->desc;
+    const int q_dim = c.n_q_heads * c.head_dim;
+    if (p->T > m->t_cap || p->n_parts > m->part_cap) return SYN_E_INVALID_ARG;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    // the Q tensor map is bound to the workspace buffer: stage the caller's q there
+    CU_OK(cudaMemcpyAsync(m->q, q, (size_t)p->T * q_dim * 2, cudaMemcpyDeviceToDevice, st));
+    return launch_attention(m, kv, p, layer, m->tm_q, (bf16*)out, st);
+}
+
+extern "C" const char* syn_strerror(int code) {
+    switch (code) {
+        case SYN_OK: return "ok";
+        case SYN_E_INVALID_ARG: return "invalid argument";
+        case SYN_E_CHUNK_LEN: return "chunk length outside [1, 16]";
+        case SYN_E_UNCACHED: return "n_uncached outside [1, chunk length]";
+        case SYN_E_PAGE_OOB: return "page id out of range";
+        case SYN_E_CAPACITY: return "context + chunk exceeds the page table";
+        case SYN_E_TOKEN_OOB: return "token id out of range";
+        case SYN_E_PAGE_ALIAS: return "two chunk tokens map to the same KV slot";
+        case SYN_E_OOM: return "out of memory";
+        case SYN_E_ARCH: return "device is not sm_100";
+        case SYN_E_CUDA: return "CUDA call failed";
+        case SYN_E_DEVICE_TIMEOUT: return "bounded device-side wait ran out";
+        default: return "unknown error";
+    }
+}

@@ -1,0 +1,124 @@
+"""Shared machinery of the GPU parity tests: build the same seeded batch on both sides,
+run the CPU oracle request by request, and judge the CUDA result by the stated rule.
+
+Rule (project brief): accept_len and correction_token bit-exact, except that a chunk
+position whose oracle top-2 logit gap is below 0.05 ("soft") may resolve to either of the
+oracle's two best ids; logits within 3e-2 x the standard deviation of the oracle's logits.
+"""
+from __future__ import annotations
+
+import itertools
+from dataclasses import dataclass
+from typing import Callable, Dict, List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from oracle import Oracle, verify_greedy
+from workloads import gen
+from workloads.configs import ModelShape, Workload
+
+SOFT_GAP = 0.05
+LOGIT_TOL = 3e-2
+
+
+@dataclass
+class OracleRequest:
+    chunk: List[int]
+    u: int
+    top1: np.ndarray
+    top2: np.ndarray
+    gap: np.ndarray
+    logits: Optional[np.ndarray]
+    accept_len: int
+    correction: int
+
+
+def oracle_teacher_forced(orc: Oracle, glob, layer_w: Callable[[int], dict], pools, page_table, ctx: int, wl: Workload,
+                          req: int, n: int, want_logits=True) -> OracleRequest:
+    """Build request `req`'s chunk by the sequential rule (anchor uniform; draft j = the oracle's
+    argmax after the actual earlier chunk tokens with probability p_match, else uniform) while
+    running the oracle token by token, which is bit-identical to its one-shot chunk forward."""
+    chunk = [gen.gen_anchor(wl, req)]
+    t1, t2, gp, lg = [], [], [], []
+    for j in range(n):
+        r = orc.forward_chunk(glob, layer_w, pools, page_table, ctx + j, [chunk[j]], u=1, want_logits=want_logits)
+        t1.append(int(r.top1[0])); t2.append(int(r.top2[0])); gp.append(float(r.gap[0]))
+        if want_logits:
+            lg.append(r.logits[0])
+        if j + 1 < n:
+            chunk.append(gen.gen_draft(wl, req, j, int(r.top1[0])))
+    a, c = verify_greedy(t1, chunk, 1)
+    return OracleRequest(chunk, 1, np.array(t1), np.array(t2), np.array(gp),
+                         np.stack(lg) if want_logits else None, a, c)
+
+
+def admissible_results(o: OracleRequest):
+    """All (accept_len, correction) pairs reachable when every soft position may take either of the
+    oracle's two best ids; and whether the request is strict (no soft position was consulted)."""
+    n = len(o.chunk)
+    soft = [j for j in range(n) if o.gap[j] < SOFT_GAP]
+    consulted = range(o.u - 1, o.u - 1 + o.accept_len + 1)
+    strict = not any(j in soft for j in consulted)
+    out = set()
+    for pick in itertools.product((0, 1), repeat=len(soft)):
+        t = o.top1.copy()
+        for j, b in zip(soft, pick):
+            if b:
+                t[j] = o.top2[j]
+        out.add(verify_greedy(t, o.chunk, o.u))
+    return out, strict
+
+
+def judge(oracle_reqs: Sequence[OracleRequest], acc, cor, logits: Optional[torch.Tensor], offsets) -> Dict[str, float]:
+    """Raises AssertionError on a parity violation; returns summary numbers."""
+    n_strict = n_soft = 0
+    for i, o in enumerate(oracle_reqs):
+        ok, strict = admissible_results(o)
+        got = (int(acc[i]), int(cor[i]))
+        if strict:
+            n_strict += 1
+            assert got == (o.accept_len, o.correction), f"request {i}: got {got}, oracle {(o.accept_len, o.correction)}"
+        else:
+            n_soft += 1
+            assert got in ok, f"request {i} (soft): got {got}, admissible {sorted(ok)}"
+    worst = 0.0
+    if logits is not None:
+        ref = np.concatenate([o.logits for o in oracle_reqs])
+        sigma = float(ref.std())
+        g = logits.detach().to("cpu", torch.float64).numpy()
+        for i, o in enumerate(oracle_reqs):
+            b = int(offsets[i])
+            worst = max(worst, float(np.abs(g[b:b + len(o.chunk)] - o.logits).max()) / sigma)
+        assert worst <= LOGIT_TOL, f"max |dlogit| / sigma = {worst:.4f} > {LOGIT_TOL}"
+    return {"strict": n_strict, "soft": n_soft, "max_dlogit_over_sigma": worst}
+
+
+# ------------------------------------------------------------------------------------------ model / cache set-up
+
+def cpu_model(shape: ModelShape, seed: int):
+    glob = gen.gen_globals(shape, seed)
+    layers = [gen.gen_layer(shape, seed, l) for l in range(shape.n_layers)]
+    return glob, layers
+
+
+def to_cuda(glob, layers):
+    return ({k: v.cuda() for k, v in glob.items()}, [{k: v.cuda() for k, v in w.items()} for w in layers])
+
+
+def fill_synthetic_kv(shape, seed, batch: gen.Batch, reqs: Sequence[int], kv=None, orc: Optional[Oracle] = None,
+                      pools=None):
+    """Cached prefix of the listed requests = seeded synthetic K/V (keyed by logical position).
+    Fills the CUDA cache (values generated on the device) and/or the oracle pools (on the CPU)."""
+    for r in reqs:
+        ctx = int(batch.ctx_lens[r])
+        if ctx == 0:
+            continue
+        pt = batch.page_tables[r]
+        for l in range(shape.n_layers):
+            if kv is not None:
+                k, v = gen.gen_kv(shape, seed, l, r, 0, ctx, device="cuda")
+                kv.import_kv(l, pt, 0, k, v)
+            if orc is not None:
+                k, v = gen.gen_kv(shape, seed, l, r, 0, ctx)
+                orc.load_kv(pools[l], pt.numpy(), 0, k.float().numpy(), v.float().numpy())

@@ -1,0 +1,72 @@
+"""Ragged paged attention kernel (C ABI: syn_op_attention) against the CPU oracle's attention,
+element by element, on random queries over a seeded synthetic cache."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import Oracle
+from workloads import gen, rng
+from workloads.configs import ModelShape, Workload
+
+from harness import cpu_model, fill_synthetic_kv, to_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+def _batch(ctx, chunk, P=16, seed=0):
+    wl = Workload("t", None, seed, len(ctx), ("list", tuple(ctx)), ("list", tuple(chunk)), 0.5)
+    return gen.gen_batch(wl)
+
+
+CASES = [
+    # head_dim, Hq, Hkv, ctx lens, chunk lens
+    (64, 4, 2, [48, 64, 96, 128], [4, 4, 4, 4]),                     # config-1 geometry
+    (128, 8, 2, [0, 5, 16, 100, 333], [1, 16, 7, 3, 12]),            # G=4: 1..4 row tiles, ctx 0, page-boundary starts
+    (128, 10, 2, [20, 700], [16, 13]),                               # G=5: token groups of 12
+    (64, 8, 8, [130, 31], [16, 2]),                                  # G=1
+    (128, 8, 2, [1500, 900, 2300], [16, 1, 9]),                      # long contexts: key ranges split over items
+    (64, 16, 2, [40], [8]),                                          # G=8
+]
+
+
+@pytest.mark.parametrize("hd,Hq,Hkv,ctx,chunk", CASES)
+def test_attention_matches_oracle(hd, Hq, Hkv, ctx, chunk):
+    import paper_2511_07423_b200 as syn
+    shape = ModelShape("att", 2, 256, Hq, Hkv, hd, 256, 512)
+    seed = 7
+    batch = _batch(ctx, chunk, seed=seed)
+    glob, layers = cpu_model(shape, seed)
+    gg, gl = to_cuda(glob, layers)
+    model = syn.Model(shape, gg, gl)
+    kv = syn.KVCache(model, batch.n_pages)
+    orc = Oracle(shape)
+    pools = orc.new_pool(batch.n_pages)
+    layer = 1
+    T = batch.n_tokens
+    q = rng.normal_f32(rng.stream_key(seed, 77), 0, T * shape.q_dim, 1.5).view(T, shape.q_dim).to(torch.bfloat16)
+    # cached prefix + the chunk's own keys/values: all positions < ctx + n come from the seeded stream
+    for r in range(batch.n_req):
+        tot = int(batch.ctx_lens[r] + batch.chunk_lens[r])
+        pt = batch.page_tables[r]
+        k, v = gen.gen_kv(shape, seed, layer, r, 0, tot)
+        kv.import_kv(layer, pt, 0, k.cuda(), v.cuda())
+        orc.load_kv(pools[layer], pt.numpy(), 0, k.float().numpy(), v.float().numpy())
+        # stale rows after the chunk (rejected drafts of an earlier step) must be ignored
+        if tot % 16:
+            junk = torch.full((16 - tot % 16, Hkv, hd), 300.0, dtype=torch.bfloat16)
+            kv.import_kv(layer, pt, tot, junk.cuda(), junk.cuda())
+    toks = torch.zeros(T, dtype=torch.int32)
+    plan = syn.Plan(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+    out = plan.attention(layer, q.cuda())
+    torch.cuda.synchronize()
+    assert model.status() == 0
+    got = out.float().cpu().numpy()
+    for r in range(batch.n_req):
+        b, n = int(batch.chunk_offsets[r]), int(batch.chunk_lens[r])
+        ref = orc.attention(q[b:b + n].double().numpy(), pools[layer], batch.page_tables[r].numpy(), int(batch.ctx_lens[r]))
+        scale = np.abs(ref).max()
+        err = np.abs(got[b:b + n] - ref).max()
+        assert err <= 0.02 * scale, (r, err, scale)   # bf16 P and bf16 output rounding
+    st = plan.stats()
+    if max(ctx) > 1000:
+        assert st.attn_split_items > 0

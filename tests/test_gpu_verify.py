@@ -1,0 +1,170 @@
+"""End-to-end parity of syn_verify_batch with the CPU oracle on seeded batches, the KV slots
+it writes, and its host-side error behaviour."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import Oracle
+from workloads import gen
+from workloads.configs import CONFIGS, MINI_1B, MINI_8B, TINY, ModelShape, Workload
+
+from harness import (cpu_model, fill_synthetic_kv, judge, oracle_teacher_forced, to_cuda)
+
+pytestmark = pytest.mark.gpu
+
+
+def _setup(shape, seed, batch):
+    import paper_2511_07423_b200 as syn
+    glob, layers = cpu_model(shape, seed)
+    gg, gl = to_cuda(glob, layers)
+    model = syn.Model(shape, gg, gl)
+    kv = syn.KVCache(model, batch.n_pages)
+    orc = Oracle(shape)
+    pools = orc.new_pool(batch.n_pages)
+    return glob, layers, model, kv, orc, pools
+
+
+def _run_and_judge(wl, shape, batch, glob, layers, kv, orc, pools, check_kv=True):
+    reqs = []
+    for r in range(batch.n_req):
+        reqs.append(oracle_teacher_forced(orc, glob, lambda l: layers[l], pools, batch.page_tables[r].numpy(),
+                                          int(batch.ctx_lens[r]), wl, r, int(batch.chunk_lens[r])))
+    tokens = torch.tensor([t for o in reqs for t in o.chunk], dtype=torch.int32)
+    acc, cor, logits = kv.verify_batch(tokens, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, want_logits=True)
+    assert kv.model.status() == 0
+    res = judge(reqs, acc, cor, logits, batch.chunk_offsets)
+    if check_kv:   # the chunk's K/V landed in exactly the slots the page table names
+        for r in range(batch.n_req):
+            ctx, n = int(batch.ctx_lens[r]), int(batch.chunk_lens[r])
+            pt = batch.page_tables[r]
+            for l in range(shape.n_layers):
+                k, v = kv.export_kv(l, pt, ctx, n)
+                for j in range(n):
+                    page, row = int(pt[(ctx + j) // 16]), (ctx + j) % 16
+                    for which, t in ((0, k), (1, v)):
+                        ref = pools[l][page, which, :, row, :]
+                        err = np.abs(t[j].float().cpu().numpy() - ref).max()
+                        assert err <= 0.02 * max(1.0, np.abs(ref).max()), (r, l, j, which, err)
+    return res
+
+
+def test_config1_tiny_real_prefill():
+    """Configuration 1: 2-layer decoder, real prefill of uniform-random context tokens on both sides
+    (the CUDA side prefills through its own u = n calls), 4-token chunks = 1 anchor + 3 drafts."""
+    wl = CONFIGS[1]
+    shape = wl.shape
+    batch = gen.gen_batch(wl)
+    glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
+    ctx_tokens = [gen.gen_context_tokens(wl, r, int(batch.ctx_lens[r])) for r in range(batch.n_req)]
+    # oracle prefill, request by request
+    for r in range(batch.n_req):
+        p = 0
+        while p < len(ctx_tokens[r]):
+            c = ctx_tokens[r][p:p + 16].tolist()
+            orc.forward_chunk(glob, lambda l: layers[l], pools, batch.page_tables[r].numpy(), p, c, u=len(c),
+                              want_logits=False)
+            p += len(c)
+    # CUDA prefill: rounds of <= 16 tokens per request, batched over the requests that still have tokens
+    done = [0] * batch.n_req
+    while True:
+        live = [r for r in range(batch.n_req) if done[r] < len(ctx_tokens[r])]
+        if not live:
+            break
+        toks, offs, ctxs = [], [0], []
+        for r in live:
+            c = ctx_tokens[r][done[r]:done[r] + 16].tolist()
+            toks += c
+            offs.append(offs[-1] + len(c))
+            ctxs.append(done[r])
+        unc = [offs[i + 1] - offs[i] for i in range(len(live))]
+        kv.verify_batch(toks, offs, batch.page_tables[live], ctxs, n_uncached=unc)
+        for i, r in enumerate(live):
+            done[r] += unc[i]
+    res = _run_and_judge(wl, shape, batch, glob, layers, kv, orc, pools)
+    print("config 1:", res)
+
+
+@pytest.mark.parametrize("shape,ctx,chunk", [
+    (MINI_1B, [0, 33, 48, 200, 515, 1030], [1, 8, 16, 5, 3, 11]),     # head_dim 64, G = 4
+    (MINI_8B, [17, 64, 300, 1200], [16, 2, 9, 13]),                    # head_dim 128, G = 4
+    (ModelShape("g5", 2, 640, 10, 2, 128, 1376, 3000), [100, 40], [16, 13]),   # G = 5, ffn and vocab with ragged tails
+])
+def test_mini_shapes_synthetic_cache(shape, ctx, chunk):
+    wl = Workload("mini", shape, 11, len(ctx), ("list", tuple(ctx)), ("list", tuple(chunk)), 0.7)
+    batch = gen.gen_batch(wl)
+    glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
+    fill_synthetic_kv(shape, wl.seed, batch, range(batch.n_req), kv=kv, orc=orc, pools=pools)
+    res = _run_and_judge(wl, shape, batch, glob, layers, kv, orc, pools)
+    print(shape.name, res)
+
+
+def test_uncached_prefix_longer_than_one_and_rerun_is_idempotent():
+    shape = MINI_1B
+    wl = Workload("u", shape, 5, 3, ("list", (20, 64, 7)), ("list", (6, 16, 1)), 0.7)
+    batch = gen.gen_batch(wl)
+    glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
+    fill_synthetic_kv(shape, wl.seed, batch, range(3), kv=kv, orc=orc, pools=pools)
+    reqs = [oracle_teacher_forced(orc, glob, lambda l: layers[l], pools, batch.page_tables[r].numpy(),
+                                  int(batch.ctx_lens[r]), wl, r, int(batch.chunk_lens[r])) for r in range(3)]
+    tokens = torch.tensor([t for o in reqs for t in o.chunk], dtype=torch.int32)
+    from oracle import verify_greedy
+    for u in ([1, 1, 1], [3, 16, 1], [6, 5, 1]):
+        acc, cor = kv.verify_batch(tokens, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, n_uncached=u)
+        for r, o in enumerate(reqs):
+            if o.gap.min() >= 0.05:
+                assert (int(acc[r]), int(cor[r])) == verify_greedy(o.top1, o.chunk, u[r])
+
+
+def test_plan_run_device_outputs_match_blocking_call():
+    import paper_2511_07423_b200 as syn
+    shape = MINI_8B
+    wl = Workload("p", shape, 3, 4, ("list", (10, 200, 64, 90)), ("list", (4, 16, 1, 8)), 0.7)
+    batch = gen.gen_batch(wl)
+    glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
+    fill_synthetic_kv(shape, wl.seed, batch, range(4), kv=kv)
+    toks = gen.gen_context_tokens(wl, 0, batch.n_tokens)
+    acc, cor, lg = kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, want_logits=True)
+    plan = syn.Plan(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+    a = torch.empty(4, dtype=torch.int32, device="cuda")
+    c = torch.empty(4, dtype=torch.int32, device="cuda")
+    t1 = torch.empty(batch.n_tokens, dtype=torch.int32, device="cuda")
+    plan.run(a, c, t1)
+    torch.cuda.synchronize()
+    assert model.status() == 0
+    assert torch.equal(a.cpu(), acc) and torch.equal(c.cpu(), cor)
+    assert torch.equal(t1.cpu().long(), lg.argmax(-1).cpu())
+    st = plan.stats()
+    assert st.n_tokens == batch.n_tokens and st.n_req == 4 and st.kernel_launches > 0
+
+
+def test_host_validation_errors_leave_outputs_untouched():
+    import paper_2511_07423_b200 as syn
+    shape = TINY
+    wl = CONFIGS[1]
+    batch = gen.gen_batch(wl)
+    glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
+    toks = torch.zeros(batch.n_tokens, dtype=torch.int32)
+
+    def code(**kw):
+        args = dict(chunk_tokens=toks, chunk_offsets=batch.chunk_offsets, page_tables=batch.page_tables,
+                    ctx_lens=batch.ctx_lens, n_uncached=None)
+        args.update(kw)
+        with pytest.raises(syn.SynError) as e:
+            kv.verify_batch(**args)
+        return e.value.code
+
+    assert code(chunk_offsets=torch.tensor([0, 4, 8, 12, 29])) == -2                      # chunk of 17
+    assert code(chunk_offsets=torch.tensor([0, 4, 4, 12, 16])) == -2                      # empty chunk
+    assert code(n_uncached=[1, 5, 1, 1]) == -3
+    assert code(n_uncached=[0, 1, 1, 1]) == -3
+    bad = batch.page_tables.clone(); bad[0, 0] = batch.n_pages
+    assert code(page_tables=bad) == -4
+    bad = batch.page_tables.clone(); bad[1, 0] = -1
+    assert code(page_tables=bad) == -4
+    assert code(ctx_lens=torch.tensor([48, 64, 96, 16 * batch.max_pages - 3])) == -5
+    t2 = toks.clone(); t2[3] = shape.vocab
+    assert code(chunk_tokens=t2) == -6
+    alias = batch.page_tables.clone(); alias[1] = alias[0]
+    assert code(page_tables=alias, ctx_lens=torch.tensor([48, 48, 96, 128])) == -7
+    with pytest.raises(syn.SynError):
+        syn.KVCache(model, 8, page_size=32)
