@@ -1,0 +1,334 @@
+#!/usr/bin/env python
+"""Benchmark of the cloud verification step: verified tokens/s on B200.
+
+One step = one pass of the whole hot path (embed, every layer's QKV / attention / O / gate-up /
+down, lm_head argmax, greedy verify) over one batch of seeded synthetic requests.
+Prints ONE JSON line.  `--impl reference` times the CPU oracle instead (a deliberately plain
+program; the ratio to it is not a figure of merit).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from workloads import gen  # noqa: E402
+from workloads.configs import CONFIGS  # noqa: E402
+
+METRIC = "verified_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "tf_burst": d["bf16_tflops"], "tf_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tf_burst": 1590.0, "tf_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            pass
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, reasons = [], set()
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                out["sm_max_mhz"] = float(r[1])
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                    if v.strip().lower() == "active":
+                        reasons.add(name)
+            except Exception:
+                continue
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle leg
+
+def oracle_sample(wl, batch, layers_cpu_fn, glob_cpu, req: int, n_tok: int, repeats: int = 1):
+    """Time the oracle, as it stands, on the chunk of one request (first n_tok tokens) against that
+    request's synthetic cached prefix.  Returns (seconds per pass, tokens, OracleResult)."""
+    from oracle import Oracle
+    shape = wl.shape
+    orc = Oracle(shape)
+    ctx = int(batch.ctx_lens[req])
+    n_pages = -(-(ctx + n_tok) // 16)
+    pt = torch.arange(n_pages, dtype=torch.int32).numpy()
+    pools = orc.new_pool(n_pages)
+    for l in range(shape.n_layers):
+        k, v = gen.gen_kv(shape, wl.seed, l, req, 0, ctx)
+        orc.load_kv(pools[l], pt, 0, k.float().numpy(), v.float().numpy())
+    return orc, pools, pt, ctx
+
+
+def run_reference(args):
+    rank, world, local = dist_env()
+    if rank != 0:
+        return
+    wl = CONFIGS[args.config]
+    shape = wl.shape
+    batch = gen.gen_batch(wl, pool_tokens=args.pool_tokens)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"   # input generation only
+    glob = {k: v.cpu() for k, v in gen.gen_globals(shape, wl.seed, device=dev).items()}
+    layers = [{k: v.cpu() for k, v in gen.gen_layer(shape, wl.seed, l, device=dev).items()} for l in range(shape.n_layers)]
+    req = 0
+    orc, pools, pt, ctx = oracle_sample(wl, batch, None, glob, req, int(batch.chunk_lens[req]))
+    n_full = int(batch.chunk_lens[req])
+    anchor = gen.gen_anchor(wl, req)
+    # size the per-step sample so that the whole run stays within a few minutes
+    t0 = time.perf_counter()
+    orc.forward_chunk(glob, lambda l: layers[l], pools, pt, ctx, [anchor], want_logits=False)
+    t_tok = time.perf_counter() - t0
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    n_tok = max(1, min(n_full, int(budget / max(t_tok, 1e-3))))
+    chunk = [anchor] + [int(x) for x in gen.gen_context_tokens(wl, req, n_tok - 1)]
+    for _ in range(args.warmup):
+        orc.forward_chunk(glob, lambda l: layers[l], pools, pt, ctx, chunk, want_logits=False)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.forward_chunk(glob, lambda l: layers[l], pools, pt, ctx, chunk, want_logits=False)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = n_tok / dt
+    cores = os.cpu_count()
+    sample = f"request {req} of {wl.name}: {n_tok} chunk tokens against its {ctx}-token synthetic prefix, one pass per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ------------------------------------------------------------------------------------------ CUDA leg
+
+def run_ours(args):
+    import paper_2511_07423_b200 as syn
+    from paper_2511_07423_b200 import synthetic
+    rank, world, local = dist_env()
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    wl = CONFIGS[args.config]
+    shape = wl.shape
+    peaks = _peaks()
+
+    via_host = shape.dense_params() * 2 > 40e9
+    model = synthetic.load_model(shape, wl.seed, via_host=via_host)
+    pool_tokens = args.pool_tokens
+    if wl.fit_to_pool and pool_tokens is None:
+        free, _ = torch.cuda.mem_get_info()
+        pool_tokens = int((free - 6e9) // shape.kv_bytes_per_token()) // 16 * 16
+    batch = gen.gen_batch(wl, pool_tokens=pool_tokens)
+    kv = syn.KVCache(model, batch.n_pages)
+    synthetic.fill_cache(kv, shape, wl.seed, batch)
+    toks = synthetic.teacher_forced_chunks(kv, wl, batch)
+    plan = syn.Plan(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+    st = plan.stats()
+    B, T = batch.n_req, batch.n_tokens
+    acc = torch.empty(B, dtype=torch.int32, device="cuda")
+    cor = torch.empty(B, dtype=torch.int32, device="cuda")
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for _ in range(max(3, args.warmup)):
+        plan.run(acc, cor)
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        plan.run(acc, cor)
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1) / args.steps
+    assert model.status() == 0
+    # ---- end to end through the blocking C-ABI call with host buffers
+    pin = lambda t: t.pin_memory()
+    h_tok, h_off, h_pt, h_ctx = pin(toks), pin(batch.chunk_offsets), pin(batch.page_tables), pin(batch.ctx_lens)
+    for _ in range(3):
+        kv.verify_batch(h_tok, h_off, h_pt, h_ctx)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        a_h, c_h = kv.verify_batch(h_tok, h_off, h_pt, h_ctx)
+    barrier()
+    ms_e2e = (time.perf_counter() - t0) * 1e3 / args.steps
+    clocks = sampler.stop() if sampler else None
+    # ---- per-kernel-class times (events around every launch), separate passes
+    model.set_profile(True)
+    for _ in range(args.steps):
+        plan.run(acc, cor)
+    prof = model.get_profile()
+    model.set_profile(False)
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = t.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    L = shape.n_layers
+    d, qd, kd, f, V = shape.d_model, shape.q_dim, shape.kv_dim, shape.d_ffn, shape.vocab
+    flops = {"qkv_gemm": 2.0 * T * d * (qd + 2 * kd), "o_gemm": 2.0 * T * qd * d, "gate_up_gemm": 2.0 * T * d * 2 * f,
+             "down_gemm": 2.0 * T * f * d, "lm_head_gemm": 2.0 * T * d * V}
+    wbytes = {"qkv_gemm": 2.0 * d * (qd + 2 * kd), "o_gemm": 2.0 * qd * d, "gate_up_gemm": 2.0 * d * 2 * f,
+              "down_gemm": 2.0 * f * d, "lm_head_gemm": 2.0 * d * V}
+    kv_bytes_layer = st.kv_read_bytes / L
+    total_ms = sum(v[0] for v in prof.values())
+    kernels = {}
+    for name, (tms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        avg = tms / cnt
+        k = {"launches_per_step": cnt // args.steps, "avg_ms": avg, "share": tms / total_ms}
+        if name in flops:
+            k["tflops"] = flops[name] / (avg * 1e-3) / 1e12
+            k["weight_gbs"] = wbytes[name] / (avg * 1e-3) / 1e9
+        if name == "attention":
+            k["kv_gbs"] = kv_bytes_layer / (avg * 1e-3) / 1e9
+        kernels[name] = k
+    top = max(kernels, key=lambda n: kernels[n]["share"])
+    if top == "attention":
+        roof = {"kernel": top, "bound": "hbm", "achieved": kernels[top]["kv_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        ridge = peaks["tf_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+        if top in flops and T >= ridge:
+            roof = {"kernel": top, "bound": "tensor", "achieved": kernels[top]["tflops"], "peak": peaks["tf_sustained"],
+                    "unit": "TFLOP/s"}
+        else:
+            roof = {"kernel": top, "bound": "hbm", "achieved": kernels[top].get("weight_gbs", 0.0), "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["peak_source"] = peaks["source"] + (" sustained" if roof["bound"] == "tensor" else "")
+    roof["traffic"] = None
+    step_bytes = st.weight_bytes + st.kv_read_bytes + st.kv_write_bytes
+    step_flops = st.dense_flops + st.attn_flops
+    t_roof = max(step_flops / (peaks["tf_sustained"] * 1e12), step_bytes / (peaks["hbm_gbs"] * 1e9))
+
+    # ---- CPU oracle on a bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(wl, batch, toks, a_h, c_h)
+
+    value = world * T / (ms * 1e-3)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "shape": shape.name, "n_req": B, "chunk_tokens": T, "ctx_tokens": int(st.ctx_tokens),
+                   "p_match": wl.p_match, "page_size": 16, "ctx_scale": batch.scale,
+                   "l2": "every step streams weights + KV far larger than L2; no flush needed",
+                   "replicas": world},
+        "e2e": {"value": world * T / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": int(st.h2d_bytes), "d2h_bytes_per_step": 8 * B + 4},
+        "gpu_launches": int(st.kernel_launches) * args.steps,
+        "clocks": clocks,
+        "roofline": roof,
+        "step_roofline": {"bytes": step_bytes, "flops": step_flops, "t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms,
+                          "peaks": peaks},
+        "kernels": kernels,
+        "committed_tokens_per_s": float((a_h.sum() + B)) / (ms * 1e-3),
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(wl, batch, toks, acc_gpu, cor_gpu):
+    """The oracle, as it stands, on one request of the same batch (its real chunk, its synthetic
+    prefix), on the host cores of this machine.  Also reports whether the CUDA result for that
+    request agrees under the parity rule's strict reading."""
+    shape = wl.shape
+    budget_flops = 6e11          # keep the leg to tens of seconds
+    per_tok = 2.0 * shape.dense_params()
+    n_req = batch.n_req
+    req = min(range(n_req), key=lambda r: abs(int(batch.chunk_lens[r]) * per_tok - budget_flops))
+    n = int(batch.chunk_lens[req])
+    b = int(batch.chunk_offsets[req])
+    chunk = toks[b:b + n].tolist()
+    glob = {k: v.cpu() for k, v in gen.gen_globals(shape, wl.seed, device="cuda").items()}
+    layers = [{k: v.cpu() for k, v in gen.gen_layer(shape, wl.seed, l, device="cuda").items()} for l in range(shape.n_layers)]
+    orc, pools, pt, ctx = oracle_sample(wl, batch, None, glob, req, n)
+    t0 = time.perf_counter()
+    res = orc.forward_chunk(glob, lambda l: layers[l], pools, pt, ctx, chunk, want_logits=False)
+    dt = time.perf_counter() - t0
+    agree = (res.accept_len, res.correction) == (int(acc_gpu[req]), int(cor_gpu[req]))
+    return {"value": n / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "seconds": dt,
+            "sample": f"request {req} of {wl.name}: its {n}-token chunk against its {ctx}-token synthetic prefix, one pass",
+            "sample_result_equal_to_cuda": bool(agree), "sample_min_top2_gap": float(res.gap.min())}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=3, help="1..5; 3 = the 8B-shape step the metric is quoted on")
+    ap.add_argument("--pool-tokens", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,99 @@
+"""Time single kernels of the step through the C ABI (CUDA events on the launching stream).
+
+    python -m paper_2511_07423_b200.opbench linear --T 544 --N 28672 --K 4096
+    python -m paper_2511_07423_b200.opbench attention --config 3
+
+`attention` builds a one-layer model with the attention geometry of the chosen configuration
+and that configuration's request mix (seeded synthetic cache), so one launch reads one layer's
+worth of the configuration's KV.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+
+import torch
+
+from workloads import gen, rng
+from workloads.configs import CONFIGS, ModelShape
+
+from . import binding as syn
+from . import synthetic
+
+
+def _time(fn, iters: int, warmup: int = 3):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    for a, b in ev:
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    ts = sorted(a.elapsed_time(b) for a, b in ev)
+    return ts[len(ts) // 2], ts[0]
+
+
+def bench_linear(a):
+    key = rng.stream_key(0, 1234)
+    x = rng.normal_f32(key, 0, a.T * a.K, 1.0, device="cuda").view(a.T, a.K).to(torch.bfloat16)
+    w = rng.normal_f32(key, a.T * a.K, a.N * a.K, 0.02, device="cuda").view(a.N, a.K).to(torch.bfloat16)
+    med, best = _time(lambda: syn.syn_op_linear(x, w), a.iters)
+    fl = 2.0 * a.T * a.N * a.K
+    print(json.dumps({"op": "linear", "T": a.T, "N": a.N, "K": a.K, "ms_median": med, "ms_best": best,
+                      "tflops": fl / med / 1e9, "weight_gbs": 2.0 * a.N * a.K / med / 1e6,
+                      "note": "includes the fp32 [T][N] store of the test epilogue and a stream sync per call"}))
+
+
+def bench_attention(a):
+    wl = CONFIGS[a.config]
+    s = wl.shape
+    shape = ModelShape(f"attn-{s.name}", 1, s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, 1024, 1024)
+    model = synthetic.load_model(shape, wl.seed)
+    batch = gen.gen_batch(wl, pool_tokens=a.pool_tokens)
+    kv = syn.KVCache(model, batch.n_pages)
+    for r in range(batch.n_req):
+        tot = int(batch.ctx_lens[r] + batch.chunk_lens[r])
+        k, v = gen.gen_kv(shape, wl.seed, 0, r, 0, tot, device="cuda")
+        kv.import_kv(0, batch.page_tables[r], 0, k, v)
+    T = batch.n_tokens
+    q = rng.normal_f32(rng.stream_key(wl.seed, 77), 0, T * shape.q_dim, 1.5, device="cuda").view(T, shape.q_dim).to(torch.bfloat16)
+    plan = syn.Plan(kv, torch.zeros(T, dtype=torch.int32), batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+    out = torch.empty_like(q)
+    model.set_profile(True)
+    for _ in range(3):
+        plan.attention(0, q, out)
+    model.get_profile()
+    for _ in range(a.iters):
+        plan.attention(0, q, out)
+    prof = model.get_profile()
+    st = plan.stats()
+    kvb = st.kv_read_bytes  # one layer
+    ms_att = prof["attention"][0] / prof["attention"][1]
+    ms_mrg = prof["attention_merge"][0] / max(1, prof["attention_merge"][1])
+    print(json.dumps({"op": "attention", "config": wl.name, "n_req": batch.n_req, "T": T, "kv_bytes": kvb,
+                      "items": st.attn_items, "split_items": st.attn_split_items, "ms_attention": ms_att,
+                      "ms_merge": ms_mrg, "kv_gbs": kvb / ms_att / 1e6, "kv_gbs_with_merge": kvb / (ms_att + ms_mrg) / 1e6,
+                      "attn_tflops": st.attn_flops / ms_att / 1e9}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    sub = ap.add_subparsers(dest="op", required=True)
+    l = sub.add_parser("linear")
+    l.add_argument("--T", type=int, default=544)
+    l.add_argument("--N", type=int, default=28672)
+    l.add_argument("--K", type=int, default=4096)
+    l.add_argument("--iters", type=int, default=10)
+    t = sub.add_parser("attention")
+    t.add_argument("--config", type=int, default=3)
+    t.add_argument("--pool-tokens", type=int, default=None)
+    t.add_argument("--iters", type=int, default=10)
+    a = ap.parse_args()
+    {"linear": bench_linear, "attention": bench_attention}[a.op](a)
+
+
+if __name__ == "__main__":
+    main()
