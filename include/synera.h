@@ -175,8 +175,9 @@ int syn_last_step_stats(const syn_plan *p, syn_step_stats *out);
  * every launch with CUDA events on the caller's stream.  syn_get_profile synchronises the device,
  * adds up the elapsed time and launch count of each class since the last call, and clears them.
  * Classes: 0 prep, 1 qkv GEMM, 2 attention, 3 attention merge, 4 o GEMM, 5 gate/up GEMM,
- * 6 down GEMM, 7 lm_head GEMM, 8 verify.  ms, launches: HOST arrays of SYN_N_KERNEL_CLASSES. */
-#define SYN_N_KERNEL_CLASSES 9
+ * 6 down GEMM, 7 lm_head GEMM, 8 verify, 9 residual + norm statistic.  ms, launches: HOST arrays
+ * of SYN_N_KERNEL_CLASSES. */
+#define SYN_N_KERNEL_CLASSES 10
 int syn_set_profile(syn_model *m, int on);
 int syn_get_profile(syn_model *m, double *ms, int32_t *launches);
 
@@ -185,7 +186,8 @@ const char *syn_strerror(int code);
 /* ---- single operations, exported for per-kernel tests and roofline measurements ------- */
 
 /* y[T][N] (fp32, DEVICE) = x[T][K] (bf16, DEVICE) * W[N][K]^T (bf16, DEVICE): the tcgen05
- * GEMM used by every projection, with a plain store epilogue.  K a multiple of 64 is not
+ * GEMM used by every projection, with a plain store epilogue.  The first call with a given w
+ * (pointer and shape) packs it into the library's tiled layout; later calls reuse the packed copy.  K a multiple of 64 is not
  * required (TMA zero-fills the tail) but K*2 bytes must be a multiple of 16; N arbitrary.
  * Errors: SYN_E_INVALID_ARG, SYN_E_CUDA. */
 int syn_op_linear(const void *x, const void *w, float *y, int32_t T, int32_t N, int32_t K, void *cuda_stream);

@@ -43,7 +43,7 @@ class StepStats(C.Structure):
                 ("attn_split_items", C.c_int32), ("kernel_launches", C.c_int32), ("h2d_bytes", C.c_int64)]
 
 KERNEL_CLASSES = ("prep", "qkv_gemm", "attention", "attention_merge", "o_gemm", "gate_up_gemm", "down_gemm",
-                  "lm_head_gemm", "verify")
+                  "lm_head_gemm", "verify", "resid_norm")
 
 
 _LIB: Optional[C.CDLL] = None

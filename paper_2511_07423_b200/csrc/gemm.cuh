@@ -1,33 +1,35 @@
 // Projection GEMM of the verification step for sm_100a, "swap-AB" orientation:
 //   D[feature][token] = sum_k W[feature][k] * X[token][k]
-// The weight matrix is the UMMA A operand (M = 128 output features per CTA, streamed from HBM
-// exactly once), the ragged token batch is the UMMA B operand (N = 16..256 tokens), so a batch of
-// T tokens pads to a multiple of 16 instead of 128.  Operands are staged by TMA (128-byte swizzle)
-// through an mbarrier ring, accumulated by tcgen05.mma in TMEM, read back with tcgen05.ld and
-// transposed through shared memory into a token-major tile that the fused epilogues consume:
+// The weight matrix is the UMMA A operand (M = 128 output features per tile; a CTA normally owns a
+// PAIR of such tiles that share one token tile), the ragged token batch is the UMMA B operand
+// (N = 16..256 tokens), so a batch of T tokens pads to a multiple of 16 instead of 128.  Weights are
+// stored pre-tiled and pre-swizzled ([feature pair][k-block][2][128 x 64] images of the
+// 128-byte-swizzled shared-memory tile), so a stage's weights are ONE contiguous bulk copy that is
+// also prefetched into L2 several k-blocks ahead; activations come through a TMA tensor map.
+// One persistent CTA per SM walks a static schedule: whole pair tiles in full waves, the remainder as
+// single 128-feature tiles; projections with few output tiles (o, down) split K over CTAs and write
+// fp32 partials that resid_norm_kernel adds to the residual stream in a fixed order.  Accumulation is
+// tcgen05.mma into TMEM, read back with tcgen05.ld and transposed through shared memory into a
+// token-major tile for the epilogues:
 //   EPI_QKV    : RMSNorm row scale, RoPE on q and k, q store, paged-KV append of k and v
-//   EPI_RESID  : residual add into the fp32 stream, next layer's bf16 operand (x * gain), sum x^2
+//   EPI_PART   : fp32 partial of a split-K projection (residual added by resid_norm_kernel)
 //   EPI_SWIGLU : RMSNorm row scale, silu(gate) * up
 //   EPI_LMHEAD : RMSNorm row scale, optional logits, vocabulary argmax (packed 64-bit atomicMax)
 //   EPI_PLAIN  : fp32 store (test hook)
-// RMSNorm is folded as rmsnorm(x) g W = rstd(x) * ((x g) W): the producer epilogue writes bf16(x g)
-// and per-128-feature partial sums of x^2; the consumer reduces them (fixed order) to rstd.
+// RMSNorm is folded as rmsnorm(x) g W = rstd(x) * ((x g) W): resid_norm_kernel writes bf16(x g) and
+// rstd per token; the consuming GEMM scales its accumulators by rstd.
 #pragma once
 #include "ptx.cuh"
 
 namespace syn {
 
-enum { EPI_PLAIN = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, EPI_LMHEAD = 4 };
+enum { EPI_PLAIN = 0, EPI_QKV = 1, EPI_PART = 2, EPI_SWIGLU = 3, EPI_LMHEAD = 4 };
 
 struct EpiParams {
     int mode;
     int T;  // valid tokens
     int N;  // valid output features (rows of W)
-    // RMSNorm statistics of the input rows (QKV, SWIGLU, LMHEAD): sumsq_in[tile * t_stride + t]
-    const float* sumsq_in;
-    int n_sumsq_tiles;
-    int t_stride;
-    float inv_d, eps;
+    const float* rstd;  // [T] 1 / sqrt(mean(x^2) + eps) of the input rows (QKV, SWIGLU, LMHEAD)
     // PLAIN
     float* y;
     int ldy;
@@ -37,12 +39,10 @@ struct EpiParams {
     const float2* rope;  // [T][hd/2] (cos, sin)
     __nv_bfloat16* pool; // this layer's pool: [page][kvh][K|V][row][hd]
     const int* slot;     // [T] page * page_size + row
-    // RESID
-    float* x;
+    // PART
+    float* part;         // [splits][part_stride] fp32, row pitch d
+    size_t part_stride;
     int d;
-    __nv_bfloat16* xn;
-    const __nv_bfloat16* gain_next;
-    float* sumsq_out;
     // SWIGLU
     __nv_bfloat16* act;
     int f_pad;
@@ -58,14 +58,13 @@ __device__ __forceinline__ unsigned long long pack_argmax(float v, int idx) {
     return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)idx);
 }
 
-// Consume one staged chunk: stage[c][f] = D[feature m0 + f][token t0 + c], c < 32, f < 128.
+// Consume one staged chunk: stage[c][f] = D[feature m0 + f][token t0 + c], c < ncols <= 32, f < 128.
 // Called by 4 warps (ew = 0..3); warp ew handles tokens c = ew, ew + 4, ...
 __device__ __forceinline__ void epi_chunk(const EpiParams& p, const float* __restrict__ stage, int m0, int t0,
-                                          int ncols, const float* __restrict__ rstd_s, int rs0, int ew, int lane) {
+                                          int ncols, int split, int ew, int lane) {
     const int f0 = m0 + 4 * lane;
     for (int c = ew; c < ncols; c += 4) {
         const int t = t0 + c;
-        if (t >= p.T) break;
         float4 v = *reinterpret_cast<const float4*>(stage + c * 128 + 4 * lane);
         float a[4] = {v.x, v.y, v.z, v.w};
         if (p.mode == EPI_PLAIN) {
@@ -73,7 +72,7 @@ __device__ __forceinline__ void epi_chunk(const EpiParams& p, const float* __res
             for (int e = 0; e < 4; ++e)
                 if (f0 + e < p.N) p.y[(size_t)t * p.ldy + f0 + e] = a[e];
         } else if (p.mode == EPI_QKV) {
-            const float r = rstd_s[rs0 + c];
+            const float r = p.rstd[t];
 #pragma unroll
             for (int e = 0; e < 4; ++e) a[e] *= r;
             const int which = f0 < p.q_dim ? 0 : (f0 < p.q_dim + p.kv_dim ? 1 : 2);
@@ -101,22 +100,10 @@ __device__ __forceinline__ void epi_chunk(const EpiParams& p, const float* __res
                 size_t off = ((((size_t)page * p.n_kv_heads + kvh) * 2 + (which - 1)) * p.page_size + row) * p.hd + dim;
                 *reinterpret_cast<uint2*>(p.pool + off) = pk;
             }
-        } else if (p.mode == EPI_RESID) {
-            float4 xo = *reinterpret_cast<const float4*>(p.x + (size_t)t * p.d + f0);
-            float xv[4] = {xo.x + a[0], xo.y + a[1], xo.z + a[2], xo.w + a[3]};
-            *reinterpret_cast<float4*>(p.x + (size_t)t * p.d + f0) = make_float4(xv[0], xv[1], xv[2], xv[3]);
-            uint2 gb = *reinterpret_cast<const uint2*>(p.gain_next + f0);
-            const __nv_bfloat162 g01 = *reinterpret_cast<__nv_bfloat162*>(&gb.x);
-            const __nv_bfloat162 g23 = *reinterpret_cast<__nv_bfloat162*>(&gb.y);
-            uint2 pk = make_uint2(pack_bf16(xv[0] * __low2float(g01), xv[1] * __high2float(g01)),
-                                  pack_bf16(xv[2] * __low2float(g23), xv[3] * __high2float(g23)));
-            *reinterpret_cast<uint2*>(p.xn + (size_t)t * p.d + f0) = pk;
-            float ss = xv[0] * xv[0] + xv[1] * xv[1] + xv[2] * xv[2] + xv[3] * xv[3];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-            if (lane == 0) p.sumsq_out[(size_t)(m0 >> 7) * p.t_stride + t] = ss;
+        } else if (p.mode == EPI_PART) {
+            *reinterpret_cast<float4*>(p.part + (size_t)split * p.part_stride + (size_t)t * p.d + f0) = v;
         } else if (p.mode == EPI_SWIGLU) {
-            const float r = rstd_s[rs0 + c];
+            const float r = p.rstd[t];
             float o[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -131,7 +118,7 @@ __device__ __forceinline__ void epi_chunk(const EpiParams& p, const float* __res
                 *reinterpret_cast<uint2*>(p.act + (size_t)t * p.f_pad + (m0 >> 1) + 4 * lane) = pk;
             }
         } else {  // EPI_LMHEAD
-            const float r = rstd_s[rs0 + c];
+            const float r = p.rstd[t];
             float bv = -INFINITY;
             int bi = 0x7FFFFFFF;
 #pragma unroll
@@ -159,65 +146,196 @@ __device__ __forceinline__ void epi_chunk(const EpiParams& p, const float* __res
     }
 }
 
-// rstd of the CTA's token tile from the per-feature-tile partial sums, in fixed order.
-__device__ __forceinline__ void epi_rstd(const EpiParams& p, float* rstd_s, int n0, int ncols, int tid, int nthr) {
-    if (p.mode == EPI_PLAIN || p.mode == EPI_RESID) return;
-    for (int i = tid; i < ncols; i += nthr) {
-        const int t = n0 + i;
-        float s = 0.f;
-        if (t < p.T)
-            for (int k = 0; k < p.n_sumsq_tiles; ++k) s += p.sumsq_in[(size_t)k * p.t_stride + t];
-        rstd_s[i] = rsqrtf(s * p.inv_d + p.eps);
+// Residual update after a split-K projection, in a fixed order: x += part[0] + part[1] + ...;
+// then the next GEMM's operand bf16(x * gain) and the row's RMSNorm statistic.  One CTA per token.
+__global__ void __launch_bounds__(256)
+resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, size_t part_stride, int splits,
+                  const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ xn, float* __restrict__ rstd,
+                  int d, float inv_d, float eps) {
+    __shared__ float red[8];
+    const int t = blockIdx.x;
+    float ss = 0.f;
+    for (int f = threadIdx.x * 4; f < d; f += blockDim.x * 4) {
+        float4 v = *reinterpret_cast<const float4*>(x + (size_t)t * d + f);
+        for (int s = 0; s < splits; ++s) {
+            const float4 q = *reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * d + f);
+            v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+        }
+        *reinterpret_cast<float4*>(x + (size_t)t * d + f) = v;
+        const uint2 gb = *reinterpret_cast<const uint2*>(gain + f);
+        const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gb.x);
+        const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gb.y);
+        *reinterpret_cast<uint2*>(xn + (size_t)t * d + f) =
+            make_uint2(pack_bf16(v.x * __low2float(g01), v.y * __high2float(g01)),
+                       pack_bf16(v.z * __low2float(g23), v.w * __high2float(g23)));
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
+        rstd[t] = rsqrtf(tot * inv_d + eps);
     }
 }
 
 // ------------------------------------------------------------------------------------------
-// tcgen05 kernel.  grid = (feature tiles of 128, token tiles of TN); 192 threads:
-// warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 = epilogue.
+// Weight packing: row-major sources -> [pair][k-block][2][128 rows x 64 cols], each 16 KB tile
+// stored as the 128-byte-swizzled shared-memory image (16-byte chunk c of row r at chunk c ^ (r & 7)).
+// mode 0: packed row pr = row pr of the concatenation of up to three matrices.
+// mode 1: gate/up interleave: packed rows [128b, 128b+64) = gate rows [64b, 64b+64), next 64 = up rows.
 // ------------------------------------------------------------------------------------------
-constexpr int GEMM_BK = 64;                       // bf16 elements per k-block = one 128-byte swizzle row
-constexpr int GEMM_A_BYTES = 128 * GEMM_BK * 2;   // 16 KB
-constexpr int GEMM_BOX_ROWS = 32;                 // token rows per B box
+struct PackSrc {
+    const __nv_bfloat16* p[3];
+    int rows[3];
+    int mode;
+    int src_k;   // valid columns of the sources (row pitch)
+};
+
+__global__ void pack_weight_kernel(PackSrc src, __nv_bfloat16* __restrict__ out, int num_kb) {
+    const int mtile = blockIdx.x, kb = blockIdx.y;
+    __nv_bfloat16* tile = out + (((size_t)(mtile >> 1) * num_kb + kb) * 2 + (mtile & 1)) * (128 * 64);
+    for (int i = threadIdx.x; i < 128 * 8; i += blockDim.x) {
+        const int r = i >> 3, c = i & 7;
+        const int pr = mtile * 128 + r;
+        const __nv_bfloat16* row = nullptr;
+        if (src.mode == 0) {
+            int q = pr;
+            for (int k = 0; k < 3 && !row; ++k) {
+                if (q < src.rows[k]) row = src.p[k] + (size_t)q * src.src_k;
+                q -= src.rows[k];
+            }
+        } else {
+            const int b = pr >> 7, w = pr & 127;
+            const int sr = b * 64 + (w & 63);
+            if (sr < src.rows[0]) row = src.p[w < 64 ? 0 : 1] + (size_t)sr * src.src_k;
+        }
+        uint4 v = make_uint4(0, 0, 0, 0);
+        const int col = kb * 64 + c * 8;
+        if (row) {
+            if (col + 8 <= src.src_k && (((uintptr_t)(row + col)) & 15) == 0) {
+                v = *reinterpret_cast<const uint4*>(row + col);
+            } else {
+                __nv_bfloat16 tmp[8];
+                for (int e = 0; e < 8; ++e) tmp[e] = col + e < src.src_k ? row[col + e] : __float2bfloat16(0.f);
+                v = *reinterpret_cast<uint4*>(tmp);
+            }
+        }
+        *reinterpret_cast<uint4*>(tile + r * 64 + ((c ^ (r & 7)) << 3)) = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// The kernel.  One persistent CTA per SM, 320 threads: warp 0 = producer (bulk copy of the weight
+// tiles + L2 prefetch + TMA boxes of the token tile), warp 1 = TMEM owner and MMA issuer,
+// warps 2..9 = epilogue (two groups of four; a group covers the four TMEM lane quarters).
+// ------------------------------------------------------------------------------------------
+constexpr int GEMM_BK = 64;                        // bf16 elements per k-block = one 128-byte swizzle row
+constexpr int GEMM_TILE_BYTES = 128 * GEMM_BK * 2; // 16 KB: one 128-feature tile of one k-block
+constexpr int GEMM_A_BYTES = 2 * GEMM_TILE_BYTES;  // stage room for a pair
+constexpr int GEMM_BOX_ROWS = 32;                  // token rows per B box
 constexpr int GEMM_BOX_BYTES = GEMM_BOX_ROWS * GEMM_BK * 2;
 constexpr int GEMM_MAX_STAGES = 8;
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 320;
+constexpr int GEMM_SMEM_MAX = 232448;
+constexpr int GEMM_PREFETCH_KB = 12;               // L2 prefetch distance in k-blocks
 
 __host__ __device__ inline int gemm_stage_bytes(int TN) { return GEMM_A_BYTES + ((TN + 31) / 32) * GEMM_BOX_BYTES; }
-__host__ inline int gemm_smem_bytes(int TN, int stages) {
-    return 1024 /*align*/ + stages * gemm_stage_bytes(TN) + 2 * 32 * 128 * 4 /*staging*/ + 256 * 4 /*rstd*/ + 256;
+__host__ inline int gemm_fixed_smem() { return 1024 /*align*/ + 2 * 32 * 128 * 4 /*staging*/ + 512; }
+__host__ inline int gemm_stages(int TN) {
+    int s = (GEMM_SMEM_MAX - gemm_fixed_smem()) / gemm_stage_bytes(TN);
+    return s > GEMM_MAX_STAGES ? GEMM_MAX_STAGES : s;
+}
+
+struct GemmParams {
+    const __nv_bfloat16* w;     // packed weights
+    int num_kb;                 // k-blocks of 64
+    int n_pairs;                // 256-feature pairs
+    int n_tt, TN;               // token tiles of TN columns (multiple of 16, <= 256)
+    int n_stages;
+    int splits, kb_per_split;   // splits > 1: every CTA owns one (pair tile, k range)
+    int pair_mode;              // 1: pair tiles in full waves + remainder as singles; 0: all singles
+    int* status;
+};
+
+struct GemmWork {
+    int pair, tt, mt_lo, mt_hi, kb0, kb1, split;
+};
+
+// Static schedule: work item i of CTA `cta`.  Returns false when the CTA is done.
+__device__ __forceinline__ bool gemm_work(const GemmParams& g, int cta, int n_cta, int i, GemmWork& w) {
+    const int n_tiles = g.n_pairs * g.n_tt;
+    w.split = 0; w.kb0 = 0; w.kb1 = g.num_kb; w.mt_lo = 0; w.mt_hi = 2;
+    if (g.splits > 1) {
+        if (i > 0 || cta >= n_tiles * g.splits) return false;
+        const int tile = cta / g.splits;
+        w.split = cta - tile * g.splits;
+        w.pair = tile / g.n_tt; w.tt = tile - w.pair * g.n_tt;
+        w.kb0 = w.split * g.kb_per_split;
+        w.kb1 = min(g.num_kb, w.kb0 + g.kb_per_split);
+        return true;
+    }
+    if (g.pair_mode) {
+        const int fw = n_tiles / n_cta;
+        if (i < fw) {
+            const int tile = i * n_cta + cta;
+            w.pair = tile / g.n_tt; w.tt = tile - w.pair * g.n_tt;
+            return true;
+        }
+        const int r = (i - fw) * n_cta + cta;
+        if (r >= (n_tiles - fw * n_cta) * 2) return false;
+        const int tile = fw * n_cta + (r >> 1);
+        w.pair = tile / g.n_tt; w.tt = tile - w.pair * g.n_tt;
+        w.mt_lo = r & 1; w.mt_hi = w.mt_lo + 1;
+        return true;
+    }
+    const int sidx = i * n_cta + cta;
+    if (sidx >= n_tiles * 2) return false;
+    const int mtile = sidx / g.n_tt;
+    w.tt = sidx - mtile * g.n_tt;
+    w.pair = mtile >> 1;
+    w.mt_lo = mtile & 1; w.mt_hi = w.mt_lo + 1;
+    return true;
+}
+
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(src)), "r"(bytes)
+                 : "memory");
 }
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, int K, int TN,
-               int n_stages, EpiParams p, int* status) {
+gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const int stage_bytes = gemm_stage_bytes(TN);
-    float* staging = reinterpret_cast<float*>(smem + n_stages * stage_bytes);
-    float* rstd_s = staging + 2 * 32 * 128;
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(rstd_s + 256);
+    const int stage_bytes = gemm_stage_bytes(g.TN);
+    float* staging = reinterpret_cast<float*>(smem + g.n_stages * stage_bytes);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(staging + 2 * 32 * 128);
     uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
-    uint64_t* accum_bar = empty_bar + GEMM_MAX_STAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_bar + 1);
+    uint64_t* accf_bar = empty_bar + GEMM_MAX_STAGES;   // accumulators complete (MMA -> epilogue)
+    uint64_t* acce_bar = accf_bar + 1;                  // accumulators drained (epilogue -> MMA)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acce_bar + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * 128;
-    const int n0 = blockIdx.y * TN;
-    const int n_valid = min(TN, p.T - n0);
-    const int nn = (n_valid + 15) & ~15;             // UMMA N
-    const int nbox = (nn + 31) >> 5;
-    const int num_kb = (K + GEMM_BK - 1) / GEMM_BK;
-    uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < TN) tmem_cols <<= 1;
+    const int n_cta = gridDim.x, cta = blockIdx.x;
+    uint32_t acc_stride = 32;
+    while ((int)acc_stride < g.TN) acc_stride <<= 1;
+    const uint32_t tmem_cols = 2 * acc_stride;
 
     if (threadIdx.x == 0) {
-        tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
-        for (int s = 0; s < n_stages; ++s) {
+        for (int s = 0; s < g.n_stages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(accum_bar, 1);
+        mbar_init(accf_bar, 1);
+        mbar_init(acce_bar, 8);
         mbar_fence_init();
     }
     if (warp == 1) {
@@ -230,58 +348,104 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
+        // ------------------------------------------------------------ producer
         if (elect_one()) {
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % n_stages;
-                if (kb >= n_stages && !mbar_wait(&empty_bar[s], ((kb / n_stages) - 1) & 1, status)) break;
-                uint8_t* a_s = smem + s * stage_bytes;
-                uint8_t* b_s = a_s + GEMM_A_BYTES;
-                mbar_expect_tx(&full_bar[s], GEMM_A_BYTES + nbox * GEMM_BOX_BYTES);
-                tma_load_2d(a_s, &tmA, &full_bar[s], kb * GEMM_BK, m0);
-                for (int i = 0; i < nbox; ++i)
-                    tma_load_2d(b_s + i * GEMM_BOX_BYTES, &tmB, &full_bar[s], kb * GEMM_BK, n0 + i * GEMM_BOX_ROWS);
+            uint32_t it = 0;
+            bool ok = true;
+            GemmWork w;
+            for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
+                const int n0 = w.tt * g.TN;
+                const int nbox = (((min(g.TN, p.T - n0) + 15) & ~15) + 31) >> 5;
+                const uint32_t a_bytes = (uint32_t)(w.mt_hi - w.mt_lo) * GEMM_TILE_BYTES;
+                const __nv_bfloat16* wsrc = g.w + ((size_t)w.pair * g.num_kb) * (2 * 128 * 64) + (size_t)w.mt_lo * (128 * 64);
+                for (int kb = w.kb0; kb < min(w.kb1, w.kb0 + GEMM_PREFETCH_KB); ++kb)
+                    bulk_prefetch_l2(wsrc + (size_t)kb * (2 * 128 * 64), a_bytes);
+                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+                    const int s = it % g.n_stages;
+                    if (it >= (uint32_t)g.n_stages && !mbar_wait(&empty_bar[s], ((it / g.n_stages) - 1) & 1, g.status)) {
+                        ok = false;
+                        break;
+                    }
+                    if (kb + GEMM_PREFETCH_KB < w.kb1)
+                        bulk_prefetch_l2(wsrc + (size_t)(kb + GEMM_PREFETCH_KB) * (2 * 128 * 64), a_bytes);
+                    uint8_t* a_s = smem + s * stage_bytes;
+                    uint8_t* b_s = a_s + GEMM_A_BYTES;
+                    mbar_expect_tx(&full_bar[s], a_bytes + nbox * GEMM_BOX_BYTES);
+                    bulk_load(a_s + w.mt_lo * GEMM_TILE_BYTES, wsrc + (size_t)kb * (2 * 128 * 64), a_bytes, &full_bar[s]);
+                    for (int b = 0; b < nbox; ++b)
+                        tma_load_2d(b_s + b * GEMM_BOX_BYTES, &tmB, &full_bar[s], kb * GEMM_BK, n0 + b * GEMM_BOX_ROWS);
+                }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
         if (elect_one()) {
-            const uint32_t idesc = umma_idesc_bf16(128, (uint32_t)nn);
+            uint32_t it = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % n_stages;
-                ok = mbar_wait(&full_bar[s], (kb / n_stages) & 1, status);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
-                const uint64_t da = umma_desc_k128(a_addr);
-                const uint64_t db = umma_desc_k128(a_addr + GEMM_A_BYTES);
+            GemmWork w;
+            for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
+                const uint32_t nn = (uint32_t)((min(g.TN, p.T - w.tt * g.TN) + 15) & ~15);
+                const uint32_t idesc = umma_idesc_bf16(128, nn);
+                if (i > 0) {   // the epilogue must have drained the previous item's accumulators
+                    ok = mbar_wait(acce_bar, (i - 1) & 1, g.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+                    const int s = it % g.n_stages;
+                    ok = mbar_wait(&full_bar[s], (it / g.n_stages) & 1, g.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
+                    const uint64_t db = umma_desc_k128(a_addr + GEMM_A_BYTES);
+                    for (int mt = w.mt_lo; mt < w.mt_hi; ++mt) {
+                        const uint64_t da = umma_desc_k128(a_addr + mt * GEMM_TILE_BYTES);
 #pragma unroll
-                for (int k = 0; k < GEMM_BK / 16; ++k)  // 16 bf16 = 32 bytes = 2 descriptor address units
-                    umma_bf16(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-                umma_commit(&empty_bar[s]);
+                        for (int k = 0; k < GEMM_BK / 16; ++k)  // 16 bf16 = 32 bytes = 2 descriptor address units
+                            umma_bf16(tmem_base + mt * acc_stride, da + 2 * k, db + 2 * k, idesc, (kb > w.kb0) || k > 0);
+                    }
+                    umma_commit(&empty_bar[s]);
+                }
+                if (ok) umma_commit(accf_bar);
             }
-            umma_commit(accum_bar);
         }
         __syncwarp();
     } else {
-        const int ew = warp - 2;           // epilogue warp 0..3 (work split)
-        const int quarter = warp & 3;      // TMEM lane quarter this warp may read
-        const int etid = threadIdx.x - 64;
-        epi_rstd(p, rstd_s, n0, n_valid, etid, 128);
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        const bool ok = mbar_wait(accum_bar, 0, status);
-        tc_fence_after();
-        if (ok) {
+        // ------------------------------------------------------------ epilogue
+        const int e = warp - 2;
+        const int grp = e >> 2, ew = e & 3;   // group 0/1 takes alternate chunks; ew splits a chunk's tokens
+        const int quarter = warp & 3;         // TMEM lane quarter this warp may read
+        float* st = staging + grp * 32 * 128;
+        bool ok = true;
+        GemmWork w;
+        for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
+            const int n0 = w.tt * g.TN;
+            const int n_valid = min(g.TN, p.T - n0);
             const int nchunks = (n_valid + 31) >> 5;
-            for (int c = 0; c < nchunks; ++c) {
+            ok = mbar_wait(accf_bar, i & 1, g.status);
+            if (!ok) break;
+            tc_fence_after();
+            const int total_chunks = (w.mt_hi - w.mt_lo) * nchunks;
+            for (int ci = grp; ci < total_chunks; ci += 2) {
+                const int mt = w.mt_lo + ci / nchunks, c = ci % nchunks;
+                const int m0 = w.pair * 256 + mt * 128;
                 uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), r);
+                tmem_ld32(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), r);
                 tmem_ld_wait();
-                float* st = staging + (c & 1) * 32 * 128;
+                if (ci + 2 >= total_chunks) {   // last TMEM read of this warp for this item
+                    tc_fence_before();
+                    if (lane == 0) mbar_arrive(acce_bar);
+                }
 #pragma unroll
                 for (int j = 0; j < 32; ++j) st[j * 128 + quarter * 32 + lane] = __uint_as_float(r[j]);
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                epi_chunk(p, st, m0, n0 + c * 32, min(32, n_valid - c * 32), rstd_s, c * 32, ew, lane);
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
+                if (m0 < p.N) epi_chunk(p, st, m0, n0 + c * 32, min(32, n_valid - c * 32), w.split, ew, lane);
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
+            }
+            if (grp >= total_chunks) {   // a group without any chunk still releases the accumulators
+                tc_fence_before();
+                if (lane == 0) mbar_arrive(acce_bar);
             }
         }
     }
@@ -291,68 +455,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
     }
-}
-
-// ------------------------------------------------------------------------------------------
-// Cross-check kernel on the legacy warp-MMA path (mma.sync m16n8k16), one 128-feature x 32-token
-// tile per CTA, same epilogues.  Kept for bring-up comparisons of the tcgen05 kernel; the step
-// does not dispatch to it unless the library is built with SYN_GEMM_LEGACY.
-// ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128)
-gemm_legacy_kernel(const __nv_bfloat16* __restrict__ W, const __nv_bfloat16* __restrict__ X, int K, int ldw, int ldx,
-                   EpiParams p) {
-    __shared__ __align__(16) __nv_bfloat16 As[128][40];
-    __shared__ __align__(16) __nv_bfloat16 Bs[32][40];
-    __shared__ __align__(16) float stage[32 * 128];
-    __shared__ float rstd_s[32];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
-    const int m0 = blockIdx.x * 128, n0 = blockIdx.y * 32;
-    const int n_valid = min(32, p.T - n0);
-    epi_rstd(p, rstd_s, n0, n_valid, threadIdx.x, 128);
-    float acc[2][4][4] = {};
-    for (int k0 = 0; k0 < K; k0 += 32) {
-        for (int i = threadIdx.x; i < 128 * 32; i += 128) {
-            int r = i >> 5, cc = i & 31;
-            As[r][cc] = (m0 + r < p.N && k0 + cc < K) ? W[(size_t)(m0 + r) * ldw + k0 + cc] : __float2bfloat16(0.f);
-        }
-        for (int i = threadIdx.x; i < 32 * 32; i += 128) {
-            int r = i >> 5, cc = i & 31;
-            Bs[r][cc] = (n0 + r < p.T && k0 + cc < K) ? X[(size_t)(n0 + r) * ldx + k0 + cc] : __float2bfloat16(0.f);
-        }
-        __syncthreads();
-#pragma unroll
-        for (int ks = 0; ks < 32; ks += 16) {
-            uint32_t a[2][4];
-#pragma unroll
-            for (int mt = 0; mt < 2; ++mt) {
-                int r = warp * 32 + mt * 16 + g;
-                a[mt][0] = *reinterpret_cast<uint32_t*>(&As[r][ks + 2 * c]);
-                a[mt][1] = *reinterpret_cast<uint32_t*>(&As[r + 8][ks + 2 * c]);
-                a[mt][2] = *reinterpret_cast<uint32_t*>(&As[r][ks + 2 * c + 8]);
-                a[mt][3] = *reinterpret_cast<uint32_t*>(&As[r + 8][ks + 2 * c + 8]);
-            }
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                uint32_t b0 = *reinterpret_cast<uint32_t*>(&Bs[nt * 8 + g][ks + 2 * c]);
-                uint32_t b1 = *reinterpret_cast<uint32_t*>(&Bs[nt * 8 + g][ks + 2 * c + 8]);
-#pragma unroll
-                for (int mt = 0; mt < 2; ++mt) mma_bf16_16816(acc[mt][nt], a[mt], b0, b1);
-            }
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
-            int f = warp * 32 + mt * 16 + g, t = nt * 8 + 2 * c;
-            stage[t * 128 + f] = acc[mt][nt][0];
-            stage[(t + 1) * 128 + f] = acc[mt][nt][1];
-            stage[t * 128 + f + 8] = acc[mt][nt][2];
-            stage[(t + 1) * 128 + f + 8] = acc[mt][nt][3];
-        }
-    __syncthreads();
-    epi_chunk(p, stage, m0, n0, n_valid, rstd_s, 0, warp, lane);
 }
 
 }  // namespace syn

@@ -17,6 +17,7 @@
 
 using namespace syn;
 typedef __nv_bfloat16 bf16;
+constexpr int GEMM_MAX_SPLITS = 4;   // split-K partial buffers of the o / down projections
 
 #define CU_OK(expr)                              \
     do {                                         \
@@ -30,34 +31,37 @@ typedef __nv_bfloat16 bf16;
 // ------------------------------------------------------------------------------------------ small kernels
 
 // Token embedding (paper Sec. 4.5: the flattened batch enters the transformer), first layer's
-// GEMM operand bf16(x * gain) with its sum-of-squares partials, RoPE table, argmax reset.
-__global__ void prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens,
-                            const int* __restrict__ pos, const bf16* __restrict__ gain, const double* __restrict__ inv_freq,
-                            float* __restrict__ x, bf16* __restrict__ xn, float* __restrict__ sumsq, float2* __restrict__ rope,
-                            unsigned long long* __restrict__ best, int d, int t_stride, int half) {
+// GEMM operand bf16(x * gain) with the row's RMSNorm statistic, RoPE table, argmax reset.
+__global__ void __launch_bounds__(256)
+prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens, const int* __restrict__ pos,
+            const bf16* __restrict__ gain, const double* __restrict__ inv_freq, float* __restrict__ x,
+            bf16* __restrict__ xn, float* __restrict__ rstd, float2* __restrict__ rope,
+            unsigned long long* __restrict__ best, int d, int half, float inv_d, float eps) {
+    __shared__ float red[8];
     const int t = blockIdx.x;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
     const bf16* e = embed + (size_t)tokens[t] * d;
-    for (int tile = warp; tile < d / 128; tile += nw) {
-        const int f = tile * 128 + lane * 4;
-        float ss = 0.f;
+    float ss = 0.f;
+    for (int f = threadIdx.x; f < d; f += blockDim.x) {
+        const float v = __bfloat162float(e[f]);
+        x[(size_t)t * d + f] = v;
+        xn[(size_t)t * d + f] = __float2bfloat16(v * __bfloat162float(gain[f]));
+        ss += v * v;
+    }
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float v = __bfloat162float(e[f + k]);
-            x[(size_t)t * d + f + k] = v;
-            xn[(size_t)t * d + f + k] = __float2bfloat16(v * __bfloat162float(gain[f + k]));
-            ss += v * v;
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-        if (lane == 0) sumsq[(size_t)tile * t_stride + t] = ss;
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
+        rstd[t] = rsqrtf(tot * inv_d + eps);
+        best[t] = 0ull;
     }
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
-        double s, c;
-        sincos((double)pos[t] * inv_freq[i], &s, &c);
-        rope[(size_t)t * half + i] = make_float2((float)c, (float)s);
+        double sn, cs;
+        sincos((double)pos[t] * inv_freq[i], &sn, &cs);
+        rope[(size_t)t * half + i] = make_float2((float)cs, (float)sn);
     }
-    if (threadIdx.x == 0) best[t] = 0ull;
 }
 
 // Greedy verification (paper Sec. 3.1 "draft & verify", Sec. 4.5): one thread per request.
@@ -128,14 +132,12 @@ struct syn_model {
     syn_model_desc desc;
     int f_pad, n_sm, gu_rows, qkv_rows, v_rows;
     bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
-    std::vector<bf16*> wqkv, wo, wgu, wd, norm1, norm2;
-    std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wd;
-    CUtensorMap tm_lm;
+    std::vector<bf16*> wqkv, wo, wgu, wd, norm1, norm2;   // projections in the packed tile layout
     double* inv_freq = nullptr;
     int* status_dev = nullptr;
     // workspace (grow-only)
     int t_cap = 0;
-    float *x = nullptr, *sumsq = nullptr;
+    float *x = nullptr, *rstd = nullptr, *part = nullptr;   // residual stream, 1/rms per token, split-K partials
     bf16 *xn = nullptr, *q = nullptr, *attn = nullptr, *act = nullptr;
     float2* rope = nullptr;
     unsigned long long* best = nullptr;
@@ -193,9 +195,9 @@ struct syn_plan {
 };
 
 static void free_workspace(syn_model* m) {
-    cudaFree(m->x); cudaFree(m->sumsq); cudaFree(m->xn); cudaFree(m->q); cudaFree(m->attn); cudaFree(m->act);
+    cudaFree(m->x); cudaFree(m->rstd); cudaFree(m->part); cudaFree(m->xn); cudaFree(m->q); cudaFree(m->attn); cudaFree(m->act);
     cudaFree(m->rope); cudaFree(m->best);
-    m->x = m->sumsq = nullptr; m->xn = m->q = m->attn = m->act = nullptr; m->rope = nullptr; m->best = nullptr;
+    m->x = m->rstd = m->part = nullptr; m->xn = m->q = m->attn = m->act = nullptr; m->rope = nullptr; m->best = nullptr;
     m->t_cap = 0;
 }
 
@@ -206,7 +208,8 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
         free_workspace(m);
         const int cap = (T + 255) / 256 * 256;
         CU_OK(cudaMalloc(&m->x, (size_t)cap * c.d_model * 4));
-        CU_OK(cudaMalloc(&m->sumsq, (size_t)cap * (c.d_model / 128) * 4));
+        CU_OK(cudaMalloc(&m->rstd, (size_t)cap * 4));
+        CU_OK(cudaMalloc(&m->part, (size_t)GEMM_MAX_SPLITS * cap * c.d_model * 4));
         CU_OK(cudaMalloc(&m->xn, (size_t)cap * c.d_model * 2));
         CU_OK(cudaMalloc(&m->q, (size_t)cap * q_dim * 2));
         CU_OK(cudaMalloc(&m->attn, (size_t)cap * q_dim * 2));
@@ -320,56 +323,106 @@ extern "C" int syn_model_load(const syn_model_desc* desc, const syn_weights* w, 
 
     CU_M(cudaMalloc(&m->embed, (size_t)c.vocab * d * 2));
     CU_M(cudaMemcpy(m->embed, w->embed, (size_t)c.vocab * d * 2, kind));
-    CU_M(cudaMalloc(&m->lm_head, (size_t)m->v_rows * d * 2));
-    CU_M(cudaMemset(m->lm_head, 0, (size_t)m->v_rows * d * 2));
-    CU_M(cudaMemcpy(m->lm_head, w->lm_head, (size_t)c.vocab * d * 2, kind));
     CU_M(cudaMalloc(&m->final_norm, (size_t)d * 2));
     CU_M(cudaMemcpy(m->final_norm, w->final_norm, (size_t)d * 2, kind));
-    if ((r = make_map_2d(&m->tm_lm, m->lm_head, m->v_rows, d, d, 128))) LOAD_FAIL(r);
-    m->tm_wqkv.resize(c.n_layers); m->tm_wo.resize(c.n_layers); m->tm_wgu.resize(c.n_layers); m->tm_wd.resize(c.n_layers);
+    // staging buffer for host-resident sources (largest single matrix)
+    bf16* stage[3] = {nullptr, nullptr, nullptr};
+    if (!loc) {
+        const size_t big = std::max((size_t)c.vocab * d, std::max((size_t)f * d, (size_t)q_dim * d));
+        for (int k = 0; k < 3; ++k) {
+            const size_t n = k == 0 ? big : (k == 1 ? std::max((size_t)f * d, (size_t)kv_dim * d) : (size_t)kv_dim * d);
+            cudaError_t e = cudaMalloc(&stage[k], n * 2);
+            if (e != cudaSuccess) {
+                (void)cudaGetLastError();
+                for (int j = 0; j < k; ++j) cudaFree(stage[j]);
+                LOAD_FAIL(SYN_E_OOM);
+            }
+        }
+    }
+    // pack `n` row-major sources (rows[i] x src_k each) into a new tile-layout buffer of `packed_rows` x K
+    auto pack = [&](const void* const* srcs, const int* rows, int n, int mode, int src_k, int packed_rows,
+                    bf16** out_ptr) -> int {
+        const int n_mt = (packed_rows + 255) / 256 * 2, nkb = (src_k + 63) / 64;
+        bf16* outp = nullptr;
+        cudaError_t e = cudaMalloc(&outp, (size_t)n_mt * nkb * 128 * 64 * 2);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return SYN_E_OOM; }
+        *out_ptr = outp;
+        PackSrc ps;
+        memset(&ps, 0, sizeof(ps));
+        ps.mode = mode; ps.src_k = src_k;
+        for (int i = 0; i < n; ++i) {
+            ps.rows[i] = rows[i];
+            if (loc) ps.p[i] = (const bf16*)srcs[i];
+            else {
+                if (cudaMemcpy(stage[i], srcs[i], (size_t)rows[i] * src_k * 2, cudaMemcpyHostToDevice) != cudaSuccess) {
+                    cudaFree(outp);
+                    *out_ptr = nullptr;
+                    return SYN_E_CUDA;
+                }
+                ps.p[i] = stage[i];
+            }
+        }
+        pack_weight_kernel<<<dim3(n_mt, nkb), 256>>>(ps, outp, nkb);
+        if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+            cudaFree(outp);
+            *out_ptr = nullptr;
+            return SYN_E_CUDA;
+        }
+        return SYN_OK;
+    };
+#define PACK_OR_FAIL(call)                                  \
+    do {                                                    \
+        int _r = (call);                                    \
+        if (_r) {                                           \
+            for (int j = 0; j < 3; ++j) cudaFree(stage[j]); \
+            LOAD_FAIL(_r);                                  \
+        }                                                   \
+    } while (0)
+    {
+        const void* srcs[1] = {w->lm_head};
+        const int rows[1] = {(int)c.vocab};
+        PACK_OR_FAIL(pack(srcs, rows, 1, 0, d, c.vocab, &m->lm_head));
+    }
     for (uint32_t l = 0; l < c.n_layers; ++l) {
-        bf16 *pqkv = nullptr, *po = nullptr, *pgu = nullptr, *pd = nullptr, *n1 = nullptr, *n2 = nullptr;
-        CU_M(cudaMalloc(&pqkv, (size_t)m->qkv_rows * d * 2)); m->wqkv.push_back(pqkv);
-        CU_M(cudaMalloc(&po, (size_t)d * q_dim * 2)); m->wo.push_back(po);
-        CU_M(cudaMalloc(&pgu, (size_t)m->gu_rows * d * 2)); m->wgu.push_back(pgu);
-        CU_M(cudaMalloc(&pd, (size_t)d * m->f_pad * 2)); m->wd.push_back(pd);
+        bf16 *n1 = nullptr, *n2 = nullptr, *pk = nullptr;
+        {
+            const void* srcs[3] = {w->wq[l], w->wk[l], w->wv[l]};
+            const int rows[3] = {q_dim, kv_dim, kv_dim};
+            PACK_OR_FAIL(pack(srcs, rows, 3, 0, d, m->qkv_rows, &pk));
+            m->wqkv.push_back(pk);
+        }
+        {
+            const void* srcs[1] = {w->wo[l]};
+            const int rows[1] = {d};
+            PACK_OR_FAIL(pack(srcs, rows, 1, 0, q_dim, d, &pk));
+            m->wo.push_back(pk);
+        }
+        {   // gate/up interleaved in blocks of 64 rows; rows of the padded tail are zero
+            const void* srcs[2] = {w->wg[l], w->wu[l]};
+            const int rows[2] = {f, f};
+            PACK_OR_FAIL(pack(srcs, rows, 2, 1, d, m->gu_rows, &pk));
+            m->wgu.push_back(pk);
+        }
+        {   // down projection: K = d_ffn, zero-padded to f_pad by the k-block tail
+            const void* srcs[1] = {w->wd[l]};
+            const int rows[1] = {d};
+            PACK_OR_FAIL(pack(srcs, rows, 1, 0, f, d, &pk));
+            m->wd.push_back(pk);
+        }
         CU_M(cudaMalloc(&n1, (size_t)d * 2)); m->norm1.push_back(n1);
         CU_M(cudaMalloc(&n2, (size_t)d * 2)); m->norm2.push_back(n2);
-        CU_M(cudaMemcpy(pqkv, w->wq[l], (size_t)q_dim * d * 2, kind));
-        CU_M(cudaMemcpy(pqkv + (size_t)q_dim * d, w->wk[l], (size_t)kv_dim * d * 2, kind));
-        CU_M(cudaMemcpy(pqkv + (size_t)(q_dim + kv_dim) * d, w->wv[l], (size_t)kv_dim * d * 2, kind));
-        CU_M(cudaMemcpy(po, w->wo[l], (size_t)d * q_dim * 2, kind));
-        // gate/up interleaved in blocks of 64 rows: packed rows [128b, 128b+64) = gate rows [64b, 64b+64),
-        // [128b+64, 128b+128) = up rows; rows of the padded tail are zero.
-        CU_M(cudaMemset(pgu, 0, (size_t)m->gu_rows * d * 2));
-        const int full = f / 64, tail = f % 64;
-        const size_t blk = (size_t)64 * d * 2;
-        if (full) {
-            CU_M(cudaMemcpy2D(pgu, 2 * blk, w->wg[l], blk, blk, full, kind));
-            CU_M(cudaMemcpy2D(reinterpret_cast<uint8_t*>(pgu) + blk, 2 * blk, w->wu[l], blk, blk, full, kind));
-        }
-        if (tail) {
-            CU_M(cudaMemcpy(reinterpret_cast<uint8_t*>(pgu) + 2 * blk * full,
-                            reinterpret_cast<const uint8_t*>(w->wg[l]) + blk * full, (size_t)tail * d * 2, kind));
-            CU_M(cudaMemcpy(reinterpret_cast<uint8_t*>(pgu) + 2 * blk * full + blk,
-                            reinterpret_cast<const uint8_t*>(w->wu[l]) + blk * full, (size_t)tail * d * 2, kind));
-        }
-        CU_M(cudaMemset(pd, 0, (size_t)d * m->f_pad * 2));
-        CU_M(cudaMemcpy2D(pd, (size_t)m->f_pad * 2, w->wd[l], (size_t)f * 2, (size_t)f * 2, d, kind));
         CU_M(cudaMemcpy(n1, w->norm1[l], (size_t)d * 2, kind));
         CU_M(cudaMemcpy(n2, w->norm2[l], (size_t)d * 2, kind));
-        if ((r = make_map_2d(&m->tm_wqkv[l], pqkv, m->qkv_rows, d, d, 128))) LOAD_FAIL(r);
-        if ((r = make_map_2d(&m->tm_wo[l], po, d, q_dim, q_dim, 128))) LOAD_FAIL(r);
-        if ((r = make_map_2d(&m->tm_wgu[l], pgu, m->gu_rows, d, d, 128))) LOAD_FAIL(r);
-        if ((r = make_map_2d(&m->tm_wd[l], pd, d, m->f_pad, m->f_pad, 128))) LOAD_FAIL(r);
     }
+    for (int j = 0; j < 3; ++j) cudaFree(stage[j]);
+#undef PACK_OR_FAIL
     std::vector<double> inv(c.head_dim / 2);
     for (uint32_t i = 0; i < c.head_dim / 2; ++i) inv[i] = std::pow((double)c.rope_base, -2.0 * (double)i / (double)c.head_dim);
     CU_M(cudaMalloc(&m->inv_freq, inv.size() * 8));
     CU_M(cudaMemcpy(m->inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice));
     CU_M(cudaMalloc(&m->status_dev, 4));
     CU_M(cudaMemset(m->status_dev, 0, 4));
-    CU_M(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    CU_M(cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_M(cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::TOTAL));
     CU_M(cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::TOTAL));
     CU_M(cudaDeviceSynchronize());
@@ -611,7 +664,7 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     s.dense_flops = 2.0 * T * params;
     s.attn_flops = 4.0 * qd * c.n_layers * (double)keys_seen;
     s.attn_items = n_items; s.attn_split_items = n_parts;
-    s.kernel_launches = 2 + c.n_layers * (5 + (groups.empty() ? 0 : 1)) + 1;
+    s.kernel_launches = 2 + c.n_layers * (7 + (groups.empty() ? 0 : 1)) + 1;
     s.h2d_bytes = (int64_t)off;
     return SYN_OK;
 }
@@ -644,24 +697,38 @@ extern "C" int syn_last_step_stats(const syn_plan* p, syn_step_stats* out) {
 
 // ------------------------------------------------------------------------------------------ launches
 
-static int launch_gemm(syn_model* m, int cls, const CUtensorMap& tmA, const CUtensorMap& tmB, const bf16* W, const bf16* X,
-                       int ldw, int ldx, int n_rows, int K, EpiParams ep, cudaStream_t st) {
+// D[rows][T] = Wpacked[rows][K] * X[T][K]^T with the epilogue `ep`.  Chooses the schedule: split-K
+// for partial-sum epilogues with few output tiles, pair tiles when they fill the SMs, else singles.
+// Returns the number of splits through *splits_out (EPI_PART only).
+static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const bf16* w_packed, int packed_rows, int K,
+                       const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, int* splits_out = nullptr) {
+    ProfScope prof(cls >= 0 ? prof_m : nullptr, cls, st);
     const int T = ep.T;
-    ProfScope prof(cls >= 0 ? m : nullptr, cls, st);
-#ifdef SYN_GEMM_LEGACY
-    dim3 grid((n_rows + 127) / 128, (T + 31) / 32);
-    gemm_legacy_kernel<<<grid, 128, 0, st>>>(W, X, K, ldw, ldx, ep);
-#else
-    (void)W; (void)X; (void)ldw; (void)ldx;
-    const int nt = (T + 255) / 256;
-    const int TN = (((T + nt - 1) / nt) + 15) / 16 * 16;
-    const int sb = gemm_stage_bytes(TN);
-    int stages = std::min(GEMM_MAX_STAGES, (232448 - 1024 - 2 * 32 * 128 * 4 - 1024 - 256 - 1024) / sb);
-    if (stages < 2) return SYN_E_INVALID_ARG;
-    dim3 grid((n_rows + 127) / 128, nt);
-    gemm_tc_kernel<<<grid, GEMM_THREADS, gemm_smem_bytes(TN, stages), st>>>(tmA, tmB, K, TN, stages, ep,
-                                                                          m ? m->status_dev : nullptr);
-#endif
+    GemmParams g;
+    g.w = w_packed;
+    g.num_kb = (K + 63) / 64;
+    g.n_pairs = (packed_rows + 255) / 256;
+    g.n_tt = (T + 255) / 256;
+    g.TN = (((T + g.n_tt - 1) / g.n_tt) + 15) / 16 * 16;
+    g.n_stages = gemm_stages(g.TN);
+    g.status = status;
+    g.splits = 1;
+    g.kb_per_split = g.num_kb;
+    if (g.n_stages < 2) return SYN_E_INVALID_ARG;
+    const int tiles = g.n_pairs * g.n_tt;
+    g.pair_mode = tiles >= n_sm;
+    int n_cta;
+    if (ep.mode == EPI_PART && tiles < n_sm) {
+        int sp = std::min(GEMM_MAX_SPLITS, std::min(n_sm / tiles, std::max(1, g.num_kb / 8)));
+        g.kb_per_split = (g.num_kb + sp - 1) / sp;
+        g.splits = (g.num_kb + g.kb_per_split - 1) / g.kb_per_split;
+        g.pair_mode = 1;
+    }
+    if (g.splits > 1) n_cta = tiles * g.splits;
+    else n_cta = std::min(n_sm, g.pair_mode ? tiles : 2 * tiles);
+    if (splits_out) *splits_out = g.splits;
+    const int smem = gemm_fixed_smem() + g.n_stages * gemm_stage_bytes(g.TN);
+    gemm_kernel<<<n_cta, GEMM_THREADS, smem, st>>>(tmB, g, ep);
     return cudaGetLastError() == cudaSuccess ? SYN_OK : SYN_E_CUDA;
 }
 
@@ -710,43 +777,47 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
     const int T = p->T, d = c.d_model, q_dim = c.n_q_heads * c.head_dim, kv_dim = c.n_kv_heads * c.head_dim;
     if (T > m->t_cap || p->n_req > m->b_cap || p->n_parts > m->part_cap) return SYN_E_INVALID_ARG;
     const int* tokens = p->d<int>(p->o_tokens);
+    const float inv_d = 1.0f / (float)d;
     {
         ProfScope prof(m, 0, st);
-        prep_kernel<<<T, 128, 0, st>>>(m->embed, tokens, p->d<int>(p->o_pos), m->norm1[0], m->inv_freq, m->x, m->xn,
-                                       m->sumsq, m->rope, m->best, d, m->t_cap, c.head_dim / 2);
+        prep_kernel<<<T, 256, 0, st>>>(m->embed, tokens, p->d<int>(p->o_pos), m->norm1[0], m->inv_freq, m->x, m->xn,
+                                       m->rstd, m->rope, m->best, d, c.head_dim / 2, inv_d, c.rms_eps);
     }
     if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
     EpiParams base;
     memset(&base, 0, sizeof(base));
     base.T = T;
-    base.sumsq_in = m->sumsq;
-    base.n_sumsq_tiles = d / 128;
-    base.t_stride = m->t_cap;
-    base.inv_d = 1.0f / (float)d;
-    base.eps = c.rms_eps;
-    int r;
+    base.rstd = m->rstd;
+    const size_t part_stride = (size_t)m->t_cap * d;
+    int r, splits = 1;
+    auto resid = [&](int cls, const bf16* gain) -> int {
+        ProfScope prof(m, cls, st);
+        resid_norm_kernel<<<T, 256, 0, st>>>(m->x, m->part, part_stride, splits, gain, m->xn, m->rstd, d, inv_d, c.rms_eps);
+        return cudaGetLastError() == cudaSuccess ? SYN_OK : SYN_E_CUDA;
+    };
     for (uint32_t l = 0; l < c.n_layers; ++l) {
         EpiParams e = base;
         e.mode = EPI_QKV; e.N = m->qkv_rows;
         e.q = m->q; e.q_dim = q_dim; e.kv_dim = kv_dim; e.hd = c.head_dim; e.n_kv_heads = c.n_kv_heads;
         e.page_size = kv->page_size; e.rope = m->rope; e.pool = kv->pool + kv->layer_elems * l;
         e.slot = p->d<int>(p->o_slot);
-        if ((r = launch_gemm(m, 1, m->tm_wqkv[l], m->tm_xn, m->wqkv[l], m->xn, d, d, m->qkv_rows, d, e, st))) return r;
+        if ((r = launch_gemm(m, 1, m->n_sm, m->status_dev, m->wqkv[l], m->qkv_rows, d, m->tm_xn, e, st))) return r;
         if ((r = launch_attention(m, kv, p, l, m->tm_q, m->attn, st))) return r;
         e = base;
-        e.mode = EPI_RESID; e.N = d; e.x = m->x; e.d = d; e.xn = m->xn; e.gain_next = m->norm2[l]; e.sumsq_out = m->sumsq;
-        if ((r = launch_gemm(m, 4, m->tm_wo[l], m->tm_attn, m->wo[l], m->attn, q_dim, q_dim, d, q_dim, e, st))) return r;
+        e.mode = EPI_PART; e.N = d; e.d = d; e.part = m->part; e.part_stride = part_stride;
+        if ((r = launch_gemm(m, 4, m->n_sm, m->status_dev, m->wo[l], d, q_dim, m->tm_attn, e, st, &splits))) return r;
+        if ((r = resid(9, m->norm2[l]))) return r;
         e = base;
         e.mode = EPI_SWIGLU; e.N = m->gu_rows; e.act = m->act; e.f_pad = m->f_pad;
-        if ((r = launch_gemm(m, 5, m->tm_wgu[l], m->tm_xn, m->wgu[l], m->xn, d, d, m->gu_rows, d, e, st))) return r;
+        if ((r = launch_gemm(m, 5, m->n_sm, m->status_dev, m->wgu[l], m->gu_rows, d, m->tm_xn, e, st))) return r;
         e = base;
-        e.mode = EPI_RESID; e.N = d; e.x = m->x; e.d = d; e.xn = m->xn;
-        e.gain_next = l + 1 < c.n_layers ? m->norm1[l + 1] : m->final_norm; e.sumsq_out = m->sumsq;
-        if ((r = launch_gemm(m, 6, m->tm_wd[l], m->tm_act, m->wd[l], m->act, m->f_pad, m->f_pad, d, m->f_pad, e, st))) return r;
+        e.mode = EPI_PART; e.N = d; e.d = d; e.part = m->part; e.part_stride = part_stride;
+        if ((r = launch_gemm(m, 6, m->n_sm, m->status_dev, m->wd[l], d, m->f_pad, m->tm_act, e, st, &splits))) return r;
+        if ((r = resid(9, l + 1 < c.n_layers ? m->norm1[l + 1] : m->final_norm))) return r;
     }
     EpiParams e = base;
     e.mode = EPI_LMHEAD; e.N = m->v_rows; e.vocab = c.vocab; e.logits = logits_out; e.best = m->best;
-    if ((r = launch_gemm(m, 7, m->tm_lm, m->tm_xn, m->lm_head, m->xn, d, d, m->v_rows, d, e, st))) return r;
+    if ((r = launch_gemm(m, 7, m->n_sm, m->status_dev, m->lm_head, m->v_rows, d, m->tm_xn, e, st))) return r;
     {
         ProfScope prof(m, 8, st);
         verify_kernel<<<(p->n_req + 127) / 128, 128, 0, st>>>(m->best, tokens, p->d<int>(p->o_offsets),
@@ -838,27 +909,46 @@ extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, 
     if (!x || !w || !y || T <= 0 || N <= 0 || K <= 0 || K % 8 != 0) return SYN_E_INVALID_ARG;
     int r = load_driver_entry();
     if (r) return r;
-    static bool attr_set = false;
-    if (!attr_set) {
-        CU_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
-        attr_set = true;
-    }
+    // process-wide context of the test hook: status word, stream-K workspace, and the packed copy of
+    // the last weight matrix seen (re-packed when the pointer or the shape changes)
+    static int n_sm = 0;
     static int* status = nullptr;
+    static bf16* packed = nullptr;
+    static const void* packed_src = nullptr;
+    static int packed_n = 0, packed_k = 0;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (!status) {
+        int dev = 0;
+        cudaDeviceProp prop;
+        CU_OK(cudaGetDevice(&dev));
+        CU_OK(cudaGetDeviceProperties(&prop, dev));
+        if (prop.major != 10) return SYN_E_ARCH;
+        n_sm = prop.multiProcessorCount;
+        CU_OK(cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
         CU_OK(cudaMalloc(&status, 4));
         CU_OK(cudaMemset(status, 0, 4));
     }
-    CUtensorMap tmA, tmB;
-    if ((r = make_map_2d(&tmA, w, N, K, K, 128))) return r;
+    const int n_mt = (N + 255) / 256 * 2, nkb = (K + 63) / 64;
+    if (packed_src != w || packed_n != N || packed_k != K) {
+        CU_OK(cudaDeviceSynchronize());
+        cudaFree(packed);
+        packed = nullptr; packed_src = nullptr;
+        CU_OK(cudaMalloc(&packed, (size_t)n_mt * nkb * 128 * 64 * 2));
+        PackSrc ps;
+        memset(&ps, 0, sizeof(ps));
+        ps.p[0] = (const bf16*)w; ps.rows[0] = N; ps.src_k = K;
+        pack_weight_kernel<<<dim3(n_mt, nkb), 256, 0, st>>>(ps, packed, nkb);
+        if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
+        packed_src = w; packed_n = N; packed_k = K;
+    }
+    CUtensorMap tmB;
     if ((r = make_map_2d(&tmB, x, T, K, K, GEMM_BOX_ROWS))) return r;
     EpiParams e;
     memset(&e, 0, sizeof(e));
     e.mode = EPI_PLAIN; e.T = T; e.N = N; e.y = y; e.ldy = N;
-    syn_model fake;  // only status_dev is read
-    fake.status_dev = status;
-    r = launch_gemm(&fake, -1, tmA, tmB, (const bf16*)w, (const bf16*)x, K, K, N, K, e, reinterpret_cast<cudaStream_t>(cuda_stream));
+    r = launch_gemm(nullptr, -1, n_sm, status, packed, n_mt * 128, K, tmB, e, st);
     if (r) return r;
-    CU_OK(cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(cuda_stream)));
+    CU_OK(cudaStreamSynchronize(st));
     int s = 0;
     CU_OK(cudaMemcpy(&s, status, 4, cudaMemcpyDeviceToHost));
     if (s) {
