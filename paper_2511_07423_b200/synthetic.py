@@ -45,7 +45,7 @@ def fill_cache(kv: KVCache, shape: ModelShape, seed: int, batch: gen.Batch, reqs
 def teacher_forced_chunks(kv: KVCache, wl: Workload, batch: gen.Batch, fixed: Optional[Dict[int, List[int]]] = None):
     """Chunk tokens of the whole batch by the sequential draft rule, with the argmax supplied by
     the library itself (one pass per chunk index).  Requests listed in `fixed` keep the given
-    tokens (e.g. chunks whose drafts were derived from the CPU oracle for a parity check)."""
+    tokens (e.g. chunks whose drafts a test derived by other means)."""
     fixed = fixed or {}
     B = batch.n_req
     offs = batch.chunk_offsets.tolist()
