@@ -115,20 +115,21 @@ def test_request_result_independent_of_batch_mates_and_order():
 
 
 # ---------------------------------------------------------------- P-5 hand-worked accept cases
-@pytest.mark.parametrize("top1,chunk,u,expect", [
-    # chunk = [anchor | drafts]; the argmax at index u-1+j judges draft j
-    ([5, 6, 7, 8], [1, 5, 6, 7], 1, (3, 8)),     # all three drafts accepted -> bonus token top1[3]
-    ([9, 6, 7, 8], [1, 5, 6, 7], 1, (0, 9)),     # first draft wrong -> correction top1[0]
-    ([5, 6, 2, 8], [1, 5, 6, 7], 1, (2, 2)),     # miss at draft 2
-    ([5, 3, 7, 8], [1, 5, 6, 7], 1, (1, 3)),     # miss at draft 1; later agreement is irrelevant
-    ([4], [1], 1, (0, 4)),                        # n = 1: plain decode step
-    ([0, 0, 5, 6, 9], [1, 2, 3, 5, 6], 3, (2, 9)),   # u = 3 anchors, 2 drafts, both accepted
-    ([0, 0, 4, 6, 9], [1, 2, 3, 5, 6], 3, (0, 4)),   # u = 3, first draft rejected
-    ([7, 7, 7, 7], [7, 7, 7, 7], 1, (3, 7)),     # repeated ids
-    ([1, 2, 3], [9, 8, 7], 3, (0, 3)),           # u = n: no drafts, result is the next token
-])
-def test_greedy_verify_hand_worked(top1, chunk, u, expect):
-    assert verify_greedy(top1, chunk, u) == expect
+def _golden(name):
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", name)
+    rows = []
+    for line in open(path):
+        line = line.split("#")[0].strip()
+        if line:
+            rows.append([c.strip() for c in line.split(";")])
+    return rows
+
+
+@pytest.mark.parametrize("row", _golden("verify_cases.txt"))
+def test_greedy_verify_hand_worked(row):
+    top1, chunk = [int(x) for x in row[0].split()], [int(x) for x in row[1].split()]
+    assert verify_greedy(top1, chunk, int(row[2])) == (int(row[3]), int(row[4]))
 
 
 def test_argmax_tie_takes_lowest_id():
@@ -301,6 +302,21 @@ def test_mean_accept_len_follows_capped_geometric():
     expect = (1 - pp ** (gamma + 1)) / (1 - pp) - 1          # = sum_{k=1..gamma} p'^k  (1.5337 here)
     se = 1.2 / math.sqrt(n_req)
     assert abs(total / n_req - expect) < 4 * se
+
+
+@pytest.mark.parametrize("row", _golden("expected_generated_tokens.txt"))
+def test_generated_tokens_per_verification_match_the_papers_expectation(row):
+    """Drafts that match the argmax independently with probability alpha: accepted drafts + the
+    correction/bonus token per verification average to the stored closed-form value (Sec. 5)."""
+    alpha, gamma, expect = float(row[0]), int(row[1]), float(row[2])
+    g = np.random.default_rng(int(alpha * 1000) + gamma)
+    n_req, total = 20000, 0
+    for _ in range(n_req):
+        top1 = g.integers(0, 1000, size=gamma + 1)
+        hit = g.random(gamma) < alpha
+        chunk = [0] + [int(top1[j]) if hit[j] else int(top1[j]) + 1000 for j in range(gamma)]
+        total += verify_greedy(top1, chunk, 1)[0] + 1
+    assert abs(total / n_req - expect) < 4 * 1.3 / math.sqrt(n_req) + 5e-4
 
 
 # ---------------------------------------------------------------- the single-precision build agrees
