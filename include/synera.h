@@ -199,6 +199,27 @@ int syn_op_linear(const void *x, const void *w, float *y, int32_t T, int32_t N, 
 int syn_op_attention(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer, const void *q, void *out,
                      void *cuda_stream);
 
+/* syn_op_attention for callers that must not allocate device memory while they run: code between
+ * cudaStreamBeginCapture and EndCapture, a serving loop whose memory pool was sized up front and
+ * handed out completely, or a host thread that may not take the allocator's lock.  (The paper has
+ * no counterpart; this is a service of the library.)  Same arguments, same result and same
+ * asynchronous behaviour as syn_op_attention, but the partial results of work items that cover
+ * only part of a request's keys live in a fixed array inside the library instead of a workspace
+ * that grows on demand.  The array holds SYN_STATIC_MAX_PARTS partials (about 33 MB of every GPU
+ * that loads the library, from load to exit).  The call itself allocates and frees nothing; the
+ * model, cache and plan it is given were of course allocated earlier by their own calls.
+ *   - A plan with more partial work items than SYN_STATIC_MAX_PARTS is refused with
+ *     SYN_E_CAPACITY before anything is launched (syn_last_step_stats().attn_split_items tells).
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps the previous call's contents; nothing
+ *     in it needs clearing, because every partial that is read is written earlier in the same
+ *     call.  Two calls that overlap on the GPU (different streams) race on it: serialise them.
+ * Errors: SYN_E_INVALID_ARG, SYN_E_CAPACITY, SYN_E_CUDA. */
+#define SYN_STATIC_MAX_PARTS 1024
+int syn_op_attention_static(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer, const void *q, void *out,
+                            void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

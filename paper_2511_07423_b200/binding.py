@@ -50,8 +50,8 @@ _LIB: Optional[C.CDLL] = None
 
 EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "syn_kv_import", "syn_kv_export",
            "syn_verify_batch", "syn_plan_create", "syn_plan_free", "syn_verify_run", "syn_model_status",
-           "syn_last_step_stats", "syn_strerror", "syn_op_linear", "syn_op_attention", "syn_set_profile",
-           "syn_get_profile"]
+           "syn_last_step_stats", "syn_strerror", "syn_op_linear", "syn_op_attention", "syn_op_attention_static",
+           "syn_set_profile", "syn_get_profile"]
 
 
 def load_library() -> C.CDLL:
@@ -247,6 +247,18 @@ class Plan:
         _check(self._lib.syn_op_attention(self.kv.model._h, self.kv._h, self._h, C.c_uint32(layer),
                                           C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()), _stream_ptr(stream)),
                "syn_op_attention")
+        return out
+
+    def attention_static(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """syn_op_attention_static: the attention of the step for callers that cannot allocate while
+        they run; its partial results live in a fixed array inside the library.  Pass `out` to keep
+        the call itself free of allocations on the Python side too."""
+        assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        if out is None:
+            out = torch.empty_like(q)
+        _check(self._lib.syn_op_attention_static(self.kv.model._h, self.kv._h, self._h, C.c_uint32(layer),
+                                                 C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()),
+                                                 _stream_ptr(stream)), "syn_op_attention_static")
         return out
 
     def close(self) -> None:

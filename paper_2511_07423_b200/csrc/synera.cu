@@ -970,6 +970,81 @@ extern "C" int syn_op_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uin
     return launch_attention(m, kv, p, layer, m->tm_q, (bf16*)out, st);
 }
 
+// ------------------------------------------------------------------------------------------ no-allocation attention
+
+// Scratch of syn_op_attention_static: the fp32 partial outputs and (max, sum) pairs of attention
+// work items that cover only part of a request's keys.  File-scope device memory, so every GPU that
+// loads the library holds these ~33 MB from load to exit.  Host code may not pass these names to a
+// kernel (on the host they are stand-ins, not device addresses): static_scratch() asks the runtime
+// for the device addresses once per device.
+static __device__ __align__(256) float g_static_part_o[(size_t)SYN_STATIC_MAX_PARTS * 64 * 128];
+static __device__ __align__(256) float2 g_static_part_ml[(size_t)SYN_STATIC_MAX_PARTS * 64];
+
+static int static_scratch(float** part_o, float2** part_ml) {
+    constexpr int MAX_DEV = 64;
+    static float* o_of[MAX_DEV];
+    static float2* ml_of[MAX_DEV];
+    int dev = -1;
+    CU_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEV) return SYN_E_INVALID_ARG;
+    if (!o_of[dev]) {   // first call on this device (which is current): resolve the symbols
+        void *a = nullptr, *b = nullptr;
+        CU_OK(cudaGetSymbolAddress(&a, g_static_part_o));
+        CU_OK(cudaGetSymbolAddress(&b, g_static_part_ml));
+        if (!a || !b) return SYN_E_CUDA;
+        ml_of[dev] = static_cast<float2*>(b);
+        o_of[dev] = static_cast<float*>(a);
+    }
+    *part_o = o_of[dev];
+    *part_ml = ml_of[dev];
+    return SYN_OK;
+}
+
+extern "C" int syn_op_attention_static(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const void* q,
+                                       void* out, void* cuda_stream) {
+    if (!m || !kv || !p || kv->model != m || !q || !out || layer >= m->desc.n_layers) return SYN_E_INVALID_ARG;
+    const syn_model_desc& c = m->desc;
+    const int q_dim = c.n_q_heads * c.head_dim;
+    if (p->T > m->t_cap) return SYN_E_INVALID_ARG;
+    if (p->n_parts > SYN_STATIC_MAX_PARTS) return SYN_E_CAPACITY;
+    float* part_o = nullptr;
+    float2* part_ml = nullptr;
+    int r = static_scratch(&part_o, &part_ml);
+    if (r) return r;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    CU_OK(cudaMemcpyAsync(m->q, q, (size_t)p->T * q_dim * 2, cudaMemcpyDeviceToDevice, st));
+    AttnParams ap;
+    ap.items = p->d<AttnItem>(p->o_items);
+    ap.cta_begin = p->d<int>(p->o_cta);
+    ap.page_tables = p->d<int>(p->o_tables);
+    ap.max_pages = p->max_pages;
+    ap.n_kv_heads = c.n_kv_heads;
+    ap.group = c.n_q_heads / c.n_kv_heads;
+    ap.q_dim = q_dim;
+    ap.layer_block0 = (int)(2ull * layer * kv->n_pages * c.n_kv_heads);
+    ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
+    ap.out = (bf16*)out;
+    ap.part_o = part_o;      // every partial row that the merge reads is written first: nothing to clear
+    ap.part_ml = part_ml;
+    ap.status = m->status_dev;
+    if (c.head_dim == 128)
+        attn_kernel<128><<<p->n_cta, ATT_THREADS, AttnSmem<128>::TOTAL, st>>>(m->tm_q, kv->tm_kv, ap);
+    else
+        attn_kernel<64><<<p->n_cta, ATT_THREADS, AttnSmem<64>::TOTAL, st>>>(m->tm_q, kv->tm_kv, ap);
+    if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
+    if (p->n_groups) {
+        dim3 blk(32, 8);
+        if (c.head_dim == 128)
+            attn_merge_kernel<128><<<p->n_groups, blk, 0, st>>>(p->d<MergeGroup>(p->o_groups), part_o, part_ml, (bf16*)out,
+                                                                ap.group, ap.q_dim);
+        else
+            attn_merge_kernel<64><<<p->n_groups, blk, 0, st>>>(p->d<MergeGroup>(p->o_groups), part_o, part_ml, (bf16*)out,
+                                                               ap.group, ap.q_dim);
+        if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
+    }
+    return SYN_OK;
+}
+
 extern "C" const char* syn_strerror(int code) {
     switch (code) {
         case SYN_OK: return "ok";
