@@ -171,6 +171,23 @@ typedef struct {
 } syn_step_stats;
 int syn_last_step_stats(const syn_plan *p, syn_step_stats *out);
 
+/* The host planner of syn_plan_create / syn_verify_batch on its own, without a device: the same
+ * validation (same error codes, same order) and the same outputs, written to caller-provided HOST
+ * arrays: pos, slot [T] (token position ctx+j and KV slot page*page_size+row; either may be NULL),
+ * items [items_cap][SYN_PLAN_ITEM_FIELDS] = the attention work list in CTA order, each row being
+ * (first query token, query tokens, kv head, request, first key, one past the last key, position of
+ * the first query token, index of its partial or -1, merge group or -1) (NULL to skip;
+ * SYN_E_CAPACITY if items_cap is too small, *n_items then holds the count needed), cta_begin
+ * [n_sm + 1] (CTA k owns items cta_begin[k] .. cta_begin[k+1]; NULL to skip), *n_cta, *stats (may be
+ * NULL; h2d_bytes is left 0).  n_sm = number of CTAs to plan for (the device's SM count). */
+#define SYN_PLAN_ITEM_FIELDS 9
+int syn_plan_host(const syn_model_desc *desc, uint32_t n_pages, uint32_t page_size, int32_t n_sm, int32_t n_req,
+                  const int32_t *chunk_tokens, const int32_t *chunk_offsets, const int32_t *page_tables,
+                  int32_t max_pages, const int32_t *ctx_lens, const int32_t *n_uncached, int32_t *pos, int32_t *slot,
+                  int32_t *items, int32_t items_cap, int32_t *n_items, int32_t *cta_begin, int32_t *n_cta,
+                  syn_step_stats *stats);
+
+
 /* Per-kernel-class device timing.  With profiling on, syn_verify_run / syn_verify_batch bracket
  * every launch with CUDA events on the caller's stream.  syn_get_profile synchronises the device,
  * adds up the elapsed time and launch count of each class since the last call, and clears them.
@@ -182,6 +199,9 @@ int syn_set_profile(syn_model *m, int on);
 int syn_get_profile(syn_model *m, double *ms, int32_t *launches);
 
 const char *syn_strerror(int code);
+/* Name of the CUDA error (e.g. "cudaErrorLaunchOutOfResources") behind the most recent SYN_E_CUDA or
+ * SYN_E_OOM returned on the calling thread; "" if there was none.  Static storage. */
+const char *syn_last_cuda_error(void);
 
 /* ---- single operations, exported for per-kernel tests and roofline measurements ------- */
 
@@ -205,7 +225,7 @@ int syn_op_attention(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer
  * no counterpart; this is a service of the library.)  Same arguments, same result and same
  * asynchronous behaviour as syn_op_attention, but the partial results of work items that cover
  * only part of a request's keys live in a fixed array inside the library instead of a workspace
- * that grows on demand.  The array holds SYN_STATIC_MAX_PARTS partials (about 33 MB of every GPU
+ * that grows on demand.  The array holds SYN_STATIC_MAX_PARTS partials (about 8.5 MB of every GPU
  * that loads the library, from load to exit).  The call itself allocates and frees nothing; the
  * model, cache and plan it is given were of course allocated earlier by their own calls.
  *   - A plan with more partial work items than SYN_STATIC_MAX_PARTS is refused with
@@ -216,7 +236,7 @@ int syn_op_attention(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer
  *     in it needs clearing, because every partial that is read is written earlier in the same
  *     call.  Two calls that overlap on the GPU (different streams) race on it: serialise them.
  * Errors: SYN_E_INVALID_ARG, SYN_E_CAPACITY, SYN_E_CUDA. */
-#define SYN_STATIC_MAX_PARTS 1024
+#define SYN_STATIC_MAX_PARTS 256
 int syn_op_attention_static(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer, const void *q, void *out,
                             void *cuda_stream);
 

@@ -21,7 +21,13 @@ def lib_path() -> str:
 
 class SynError(RuntimeError):
     def __init__(self, code: int, what: str):
-        super().__init__(f"{what}: {code} ({_strerror(code)})")
+        detail = ""
+        if code in (-8, -10):
+            try:
+                detail = " [" + load_library().syn_last_cuda_error().decode() + "]"
+            except Exception:  # pragma: no cover
+                pass
+        super().__init__(f"{what}: {code} ({_strerror(code)}){detail}")
         self.code = code
 
 
@@ -50,7 +56,7 @@ _LIB: Optional[C.CDLL] = None
 
 EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "syn_kv_import", "syn_kv_export",
            "syn_verify_batch", "syn_plan_create", "syn_plan_free", "syn_verify_run", "syn_model_status",
-           "syn_last_step_stats", "syn_strerror", "syn_op_linear", "syn_op_attention", "syn_op_attention_static",
+           "syn_last_step_stats", "syn_plan_host", "syn_strerror", "syn_last_cuda_error", "syn_op_linear", "syn_op_attention", "syn_op_attention_static",
            "syn_set_profile", "syn_get_profile"]
 
 
@@ -63,6 +69,8 @@ def load_library() -> C.CDLL:
         lib = C.CDLL(path)
         lib.syn_strerror.restype = C.c_char_p
         lib.syn_strerror.argtypes = [C.c_int]
+        lib.syn_last_cuda_error.restype = C.c_char_p
+        lib.syn_last_cuda_error.argtypes = []
         for fn in ("syn_model_free", "syn_kv_free", "syn_plan_free"):
             getattr(lib, fn).restype = None
             getattr(lib, fn).argtypes = [C.c_void_p]
@@ -271,6 +279,44 @@ class Plan:
             self.close()
         except Exception:
             pass
+
+
+PLAN_ITEM_FIELDS = ("q_tok", "nj", "kvh", "req", "kv_begin", "kv_end", "q_pos0", "part", "grp")
+
+
+def plan_host(shape, n_pages: int, chunk_tokens, chunk_offsets, page_tables, ctx_lens, n_uncached=None,
+              n_sm: int = 148, page_size: int = 16):
+    """syn_plan_host: the host planner without a device.  Returns a dict with pos, slot [T],
+    items [n_items, 9] (columns PLAN_ITEM_FIELDS), cta_begin [n_cta + 1] and stats."""
+    lib = load_library()
+    tok, off, ctx, pt = _i32(chunk_tokens), _i32(chunk_offsets), _i32(ctx_lens), _i32(page_tables)
+    assert pt.dim() == 2
+    unc = _i32(n_uncached) if n_uncached is not None else None
+    n_req = ctx.numel()
+    T = max(0, int(off[-1])) if off.numel() else 0
+    d = _Desc(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn,
+              shape.vocab, float(shape.rope_base), float(shape.rms_eps), 0)
+    pos = torch.zeros(max(T, 1), dtype=torch.int32)
+    slot = torch.zeros(max(T, 1), dtype=torch.int32)
+    cta = torch.zeros(n_sm + 1, dtype=torch.int32)
+    n_items, n_cta = C.c_int32(0), C.c_int32(0)
+    st = StepStats()
+    cap = 0
+    items = torch.zeros(1, len(PLAN_ITEM_FIELDS), dtype=torch.int32)
+    for _ in range(2):
+        code = lib.syn_plan_host(
+            C.byref(d), C.c_uint32(n_pages), C.c_uint32(page_size), C.c_int32(n_sm), C.c_int32(n_req),
+            C.c_void_p(tok.data_ptr()), C.c_void_p(off.data_ptr()), C.c_void_p(pt.data_ptr()), C.c_int32(pt.shape[1]),
+            C.c_void_p(ctx.data_ptr()), C.c_void_p(unc.data_ptr()) if unc is not None else None,
+            C.c_void_p(pos.data_ptr()), C.c_void_p(slot.data_ptr()), C.c_void_p(items.data_ptr()) if cap else None,
+            C.c_int32(cap), C.byref(n_items), C.c_void_p(cta.data_ptr()), C.byref(n_cta), C.byref(st))
+        _check(code, "syn_plan_host")
+        if cap:
+            break
+        cap = n_items.value
+        items = torch.zeros(max(cap, 1), len(PLAN_ITEM_FIELDS), dtype=torch.int32)
+    return {"pos": pos[:T], "slot": slot[:T], "items": items[:n_items.value], "cta_begin": cta[:n_cta.value + 1],
+            "n_cta": n_cta.value, "stats": st}
 
 
 def syn_op_linear(x: torch.Tensor, w: torch.Tensor, stream=None) -> torch.Tensor:

@@ -19,9 +19,18 @@ using namespace syn;
 typedef __nv_bfloat16 bf16;
 constexpr int GEMM_MAX_SPLITS = 4;   // split-K partial buffers of the o / down projections
 
+// Name of the last CUDA error a call of this library met on this thread (for syn_last_cuda_error).
+static thread_local const char* g_last_cuda_error = "";
+static inline cudaError_t note_cuda(cudaError_t e) {
+    if (e != cudaSuccess) g_last_cuda_error = cudaGetErrorName(e);
+    return e;
+}
+// cudaGetLastError after a launch, recorded like any other failing call
+static inline bool launch_ok() { return note_cuda(cudaGetLastError()) == cudaSuccess; }
+
 #define CU_OK(expr)                              \
     do {                                         \
-        cudaError_t _e = (expr);                 \
+        cudaError_t _e = note_cuda(expr);        \
         if (_e != cudaSuccess) {                 \
             (void)cudaGetLastError();            \
             return _e == cudaErrorMemoryAllocation ? SYN_E_OOM : SYN_E_CUDA; \
@@ -146,6 +155,7 @@ struct syn_model {
     CUtensorMap tm_xn, tm_attn, tm_act, tm_q;
     float* part_o = nullptr;
     float2* part_ml = nullptr;
+    int* group_count = nullptr;     // per merge group: partial items completed (zero between launches)
     int part_cap = 0;
     syn_plan* scratch_plan = nullptr;
     int* pinned_out = nullptr;
@@ -225,11 +235,12 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
         if ((r = make_map_2d(&m->tm_xn, m->xn, cap, c.d_model, c.d_model, GEMM_BOX_ROWS))) return r;
         if ((r = make_map_2d(&m->tm_attn, m->attn, cap, q_dim, q_dim, GEMM_BOX_ROWS))) return r;
         if ((r = make_map_2d(&m->tm_act, m->act, cap, m->f_pad, m->f_pad, GEMM_BOX_ROWS))) return r;
-        // Q tile of the attention kernel: [token][128-byte line][64]; box = 16 tokens x (G * hd/64) lines
+        // Q tile of the attention kernel: [token][128-byte line][64]; box = min(16, 64/G) tokens x (G * hd/64) lines
         const uint32_t G = c.n_q_heads / c.n_kv_heads, halves = c.head_dim / 64;
+        const uint32_t box_tokens = std::min(16u, 64u / G);
         cuuint64_t dims[3] = {64, (cuuint64_t)q_dim / 64, (cuuint64_t)cap};
         cuuint64_t strides[2] = {128, (cuuint64_t)q_dim * 2};
-        cuuint32_t box[3] = {64, G * halves, 16};
+        cuuint32_t box[3] = {64, G * halves, box_tokens};
         cuuint32_t estr[3] = {1, 1, 1};
         if (g_encode(&m->tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, m->q, dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -245,11 +256,13 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
         m->b_cap = cap;
     }
     if (n_parts > m->part_cap) {
-        cudaFree(m->part_o); cudaFree(m->part_ml);
-        m->part_o = nullptr; m->part_ml = nullptr; m->part_cap = 0;
+        cudaFree(m->part_o); cudaFree(m->part_ml); cudaFree(m->group_count);
+        m->part_o = nullptr; m->part_ml = nullptr; m->group_count = nullptr; m->part_cap = 0;
         const int cap = (n_parts + 255) / 256 * 256;
         CU_OK(cudaMalloc(&m->part_o, (size_t)cap * 64 * c.head_dim * 4));
         CU_OK(cudaMalloc(&m->part_ml, (size_t)cap * 64 * 8));
+        CU_OK(cudaMalloc(&m->group_count, (size_t)cap * 4));   // a group has >= 2 parts: cap/2 would do
+        CU_OK(cudaMemset(m->group_count, 0, (size_t)cap * 4));
         m->part_cap = cap;
     }
     return SYN_OK;
@@ -263,7 +276,7 @@ extern "C" void syn_model_free(syn_model* m) {
         for (bf16* p : *v) cudaFree(p);
     cudaFree(m->embed); cudaFree(m->lm_head); cudaFree(m->final_norm); cudaFree(m->inv_freq); cudaFree(m->status_dev);
     free_workspace(m);
-    cudaFree(m->acc_dev); cudaFree(m->corr_dev); cudaFree(m->part_o); cudaFree(m->part_ml);
+    cudaFree(m->acc_dev); cudaFree(m->corr_dev); cudaFree(m->part_o); cudaFree(m->part_ml); cudaFree(m->group_count);
     if (m->pinned_out) cudaFreeHost(m->pinned_out);
     if (m->scratch_plan) syn_plan_free(m->scratch_plan);
     for (auto* v : {&m->ev_used, &m->ev_free})
@@ -523,15 +536,23 @@ extern "C" void syn_plan_free(syn_plan* p) {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Validate the batch, then build token positions, KV slots and the attention work list.
-static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, const int32_t* chunk_tokens,
-                      const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages, const int32_t* ctx_lens,
-                      const int32_t* n_uncached) {
-    if (!m || !kv || kv->model != m || n_req <= 0 || !chunk_tokens || !chunk_offsets || !page_tables || !ctx_lens ||
-        max_pages <= 0)
+// Host-side result of planning one batch (no device involved).
+struct HostPlan {
+    int T = 0, n_cta = 0, n_parts = 0;
+    std::vector<int> pos, slot, cta_begin;
+    std::vector<AttnItem> items;          // sorted by CTA
+    std::vector<MergeGroup> groups;
+    syn_step_stats stats;
+};
+
+// Validate the batch, then build token positions, KV slots and the attention work list
+// (the "flatten" of paper Sec. 4.5).  Pure host code.
+static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_sm, int32_t n_req,
+                        const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables,
+                        int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, HostPlan& hp) {
+    if (n_req <= 0 || !chunk_tokens || !chunk_offsets || !page_tables || !ctx_lens || max_pages <= 0 || n_sm <= 0)
         return SYN_E_INVALID_ARG;
-    const syn_model_desc& c = m->desc;
-    const int P = (int)kv->page_size, G = c.n_q_heads / c.n_kv_heads, Hkv = c.n_kv_heads;
+    const int G = c.n_q_heads / c.n_kv_heads, Hkv = c.n_kv_heads;
     if (chunk_offsets[0] != 0) return SYN_E_INVALID_ARG;
     int64_t ctx_sum = 0, keys_seen = 0, kv_units = 0;
     for (int i = 0; i < n_req; ++i) {
@@ -544,7 +565,7 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
         const int used = (int)((ctx_lens[i] + n + P - 1) / P);
         for (int k = 0; k < used; ++k) {
             const int pg = page_tables[(size_t)i * max_pages + k];
-            if (pg < 0 || (uint32_t)pg >= kv->n_pages) return SYN_E_PAGE_OOB;
+            if (pg < 0 || (uint32_t)pg >= n_pages) return SYN_E_PAGE_OOB;
         }
         ctx_sum += ctx_lens[i];
         kv_units += ctx_lens[i] + n;
@@ -553,7 +574,10 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     const int T = chunk_offsets[n_req];
     for (int t = 0; t < T; ++t)
         if (chunk_tokens[t] < 0 || (uint32_t)chunk_tokens[t] >= c.vocab) return SYN_E_TOKEN_OOB;
-    std::vector<int> pos(T), slot(T);
+    std::vector<int>& pos = hp.pos;
+    std::vector<int>& slot = hp.slot;
+    pos.assign(T, 0);
+    slot.assign(T, 0);
     for (int i = 0; i < n_req; ++i)
         for (int j = 0, b = chunk_offsets[i]; b + j < chunk_offsets[i + 1]; ++j) {
             const int pp = ctx_lens[i] + j;
@@ -566,20 +590,35 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
         for (int t = 1; t < T; ++t)
             if (s2[t] == s2[t - 1]) return SYN_E_PAGE_ALIAS;
     }
-    // attention work list: (request, kv head, token group, key range); split long key ranges
-    const int n_cta_max = m->n_sm;
+    // Attention work list: (request, kv head, token group, key range).  Cost of an item = its 64-key
+    // stages weighted by the number of 16-row query tiles (more tiles = more tensor work per key
+    // byte) plus a fixed overhead.  A key range is split only when one unit alone would exceed a
+    // CTA's fair share: every split costs an fp32 partial and a merge.
+    const int n_cta_max = n_sm;
     const int tok_per_group = std::min(16, 64 / G);
-    int64_t split = (kv_units * Hkv) / ((int64_t)n_cta_max * 6);
-    split = std::max<int64_t>(512, (split + 63) / 64 * 64);
+    static const int STAGE_COST[5] = {0, 20, 21, 30, 31};
+    const int ITEM_COST = 60, PART_COST = 40;
+    auto unit_cost = [&](int L, int nj) { return (int64_t)((L + 63) / 64) * STAGE_COST[(nj * G + 15) / 16] + ITEM_COST; };
+    int64_t total_cost = 0;
+    for (int i = 0; i < n_req; ++i) {
+        const int b = chunk_offsets[i], n = chunk_offsets[i + 1] - b;
+        for (int j0 = 0; j0 < n; j0 += tok_per_group) {
+            const int nj = std::min(tok_per_group, n - j0);
+            total_cost += unit_cost(ctx_lens[i] + j0 + nj, nj) * Hkv;
+        }
+    }
+    const int64_t share = std::max<int64_t>(8 * 31 + ITEM_COST, (total_cost + n_cta_max - 1) / n_cta_max);
     std::vector<AttnItem> items;
-    std::vector<MergeGroup> groups;
+    std::vector<int> item_cost;
+    std::vector<MergeGroup>& groups = hp.groups;
+    groups.clear();
     int n_parts = 0;
     for (int i = 0; i < n_req; ++i) {
         const int b = chunk_offsets[i], n = chunk_offsets[i + 1] - b;
         for (int j0 = 0; j0 < n; j0 += tok_per_group) {
             const int nj = std::min(tok_per_group, n - j0);
             const int L = ctx_lens[i] + j0 + nj;
-            int np = (int)std::min<int64_t>(64, (L + split - 1) / split);
+            int np = (int)std::min<int64_t>(64, (unit_cost(L, nj) + share - 1) / share);
             int len = ((L + np - 1) / np + 63) / 64 * 64;
             np = (L + len - 1) / len;
             for (int h = 0; h < Hkv; ++h) {
@@ -589,8 +628,9 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
                 }
                 for (int k = 0; k < np; ++k) {
                     AttnItem it = {b + j0, nj, h, i, k * len, std::min(L, (k + 1) * len), ctx_lens[i] + j0,
-                                   np > 1 ? n_parts + k : -1};
+                                   np > 1 ? n_parts + k : -1, np > 1 ? (int)groups.size() - 1 : -1, 0, 0, 0};
                     items.push_back(it);
+                    item_cost.push_back((int)unit_cost(it.kv_end - it.kv_begin, nj) + (np > 1 ? PART_COST : 0));
                 }
                 if (np > 1) n_parts += np;
             }
@@ -600,12 +640,13 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     const int n_cta = std::min(n_cta_max, n_items);
     std::vector<int> order(n_items), owner(n_items);
     for (int i = 0; i < n_items; ++i) order[i] = i;
-    auto cost = [&](int i) { return items[i].kv_end - items[i].kv_begin + 48; };
+    auto cost = [&](int i) { return item_cost[i]; };
     std::stable_sort(order.begin(), order.end(), [&](int a, int bb) { return cost(a) > cost(bb); });
     typedef std::pair<int64_t, int> Load;
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
     for (int k = 0; k < n_cta; ++k) heap.push(Load(0, k));
-    std::vector<int> count(n_cta + 1, 0);
+    std::vector<int>& count = hp.cta_begin;
+    count.assign(n_cta + 1, 0);
     for (int i : order) {
         Load l = heap.top();
         heap.pop();
@@ -614,12 +655,38 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
         heap.push(Load(l.first + cost(i), l.second));
     }
     for (int k = 0; k < n_cta; ++k) count[k + 1] += count[k];
-    std::vector<AttnItem> sorted(n_items);
+    hp.items.assign(n_items, AttnItem());
     {
         std::vector<int> cur(count.begin(), count.end() - 1);
-        for (int i : order) sorted[cur[owner[i]]++] = items[i];
+        for (int i : order) hp.items[cur[owner[i]]++] = items[i];
     }
-    // pack everything into one buffer
+    hp.T = T; hp.n_cta = n_cta; hp.n_parts = n_parts;
+
+    syn_step_stats& s = hp.stats;
+    memset(&s, 0, sizeof(s));
+    const double d = c.d_model, qd = (double)c.n_q_heads * c.head_dim, kd = (double)Hkv * c.head_dim;
+    const double params = c.n_layers * (d * (qd + 2 * kd) + qd * d + 3.0 * d * c.d_ffn) + d * c.vocab;
+    s.n_req = n_req; s.n_tokens = T; s.ctx_tokens = ctx_sum;
+    s.weight_bytes = (int64_t)(params * 2);
+    s.kv_read_bytes = kv_units * (int64_t)(2 * kd * 2) * c.n_layers;
+    s.kv_write_bytes = (int64_t)T * (int64_t)(2 * kd * 2) * c.n_layers;
+    s.dense_flops = 2.0 * T * params;
+    s.attn_flops = 4.0 * qd * c.n_layers * (double)keys_seen;
+    s.attn_items = n_items; s.attn_split_items = n_parts;
+    s.kernel_launches = 2 + c.n_layers * 7 + 1;
+    return SYN_OK;
+}
+
+// plan_compute, then pack everything into the plan's pinned buffer (grown on demand).
+static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, const int32_t* chunk_tokens,
+                      const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages, const int32_t* ctx_lens,
+                      const int32_t* n_uncached) {
+    if (!m || !kv || kv->model != m) return SYN_E_INVALID_ARG;
+    HostPlan hp;
+    int r = plan_compute(m->desc, (int)kv->page_size, kv->n_pages, m->n_sm, n_req, chunk_tokens, chunk_offsets, page_tables,
+                         max_pages, ctx_lens, n_uncached, hp);
+    if (r) return r;
+    const int T = hp.T, n_items = (int)hp.items.size(), n_cta = hp.n_cta;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     p->o_tokens = take((size_t)T * 4);
@@ -630,7 +697,7 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     p->o_tables = take((size_t)n_req * max_pages * 4);
     p->o_items = take((size_t)n_items * sizeof(AttnItem));
     p->o_cta = take((size_t)(n_cta + 1) * 4);
-    p->o_groups = take(std::max<size_t>(1, groups.size()) * sizeof(MergeGroup));
+    p->o_groups = take(std::max<size_t>(1, hp.groups.size()) * sizeof(MergeGroup));
     if (off > p->cap) {
         cudaFree(p->dev);
         if (p->host) cudaFreeHost(p->host);
@@ -643,29 +710,50 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     }
     p->used = off;
     memcpy(p->h<int>(p->o_tokens), chunk_tokens, (size_t)T * 4);
-    memcpy(p->h<int>(p->o_pos), pos.data(), (size_t)T * 4);
-    memcpy(p->h<int>(p->o_slot), slot.data(), (size_t)T * 4);
+    memcpy(p->h<int>(p->o_pos), hp.pos.data(), (size_t)T * 4);
+    memcpy(p->h<int>(p->o_slot), hp.slot.data(), (size_t)T * 4);
     memcpy(p->h<int>(p->o_offsets), chunk_offsets, (size_t)(n_req + 1) * 4);
     for (int i = 0; i < n_req; ++i) p->h<int>(p->o_uncached)[i] = n_uncached ? n_uncached[i] : 1;
     memcpy(p->h<int>(p->o_tables), page_tables, (size_t)n_req * max_pages * 4);
-    memcpy(p->h<AttnItem>(p->o_items), sorted.data(), (size_t)n_items * sizeof(AttnItem));
-    memcpy(p->h<int>(p->o_cta), count.data(), (size_t)(n_cta + 1) * 4);
-    if (!groups.empty()) memcpy(p->h<MergeGroup>(p->o_groups), groups.data(), groups.size() * sizeof(MergeGroup));
+    memcpy(p->h<AttnItem>(p->o_items), hp.items.data(), (size_t)n_items * sizeof(AttnItem));
+    memcpy(p->h<int>(p->o_cta), hp.cta_begin.data(), (size_t)(n_cta + 1) * 4);
+    if (!hp.groups.empty()) memcpy(p->h<MergeGroup>(p->o_groups), hp.groups.data(), hp.groups.size() * sizeof(MergeGroup));
     p->n_req = n_req; p->T = T; p->max_pages = max_pages; p->n_items = n_items; p->n_cta = n_cta;
-    p->n_groups = (int)groups.size(); p->n_parts = n_parts;
+    p->n_groups = (int)hp.groups.size(); p->n_parts = hp.n_parts;
+    p->stats = hp.stats;
+    p->stats.h2d_bytes = (int64_t)off;
+    return SYN_OK;
+}
 
-    syn_step_stats& s = p->stats;
-    const double d = c.d_model, qd = (double)c.n_q_heads * c.head_dim, kd = (double)Hkv * c.head_dim;
-    const double params = c.n_layers * (d * (qd + 2 * kd) + qd * d + 3.0 * d * c.d_ffn) + d * c.vocab;
-    s.n_req = n_req; s.n_tokens = T; s.ctx_tokens = ctx_sum;
-    s.weight_bytes = (int64_t)(params * 2);
-    s.kv_read_bytes = kv_units * (int64_t)(2 * kd * 2) * c.n_layers;
-    s.kv_write_bytes = (int64_t)T * (int64_t)(2 * kd * 2) * c.n_layers;
-    s.dense_flops = 2.0 * T * params;
-    s.attn_flops = 4.0 * qd * c.n_layers * (double)keys_seen;
-    s.attn_items = n_items; s.attn_split_items = n_parts;
-    s.kernel_launches = 2 + c.n_layers * (7 + (groups.empty() ? 0 : 1)) + 1;
-    s.h2d_bytes = (int64_t)off;
+// The planner without a device: same validation and the same work list as syn_plan_create, returned
+// in caller-provided HOST arrays.
+extern "C" int syn_plan_host(const syn_model_desc* desc, uint32_t n_pages, uint32_t page_size, int32_t n_sm, int32_t n_req,
+                             const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables,
+                             int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, int32_t* pos,
+                             int32_t* slot, int32_t* items, int32_t items_cap, int32_t* n_items, int32_t* cta_begin,
+                             int32_t* n_cta, syn_step_stats* stats) {
+    if (!desc || page_size != 16 || !n_items || !n_cta) return SYN_E_INVALID_ARG;
+    if (desc->n_kv_heads == 0 || desc->n_q_heads % desc->n_kv_heads != 0 || desc->n_q_heads / desc->n_kv_heads > 8)
+        return SYN_E_INVALID_ARG;
+    HostPlan hp;
+    int r = plan_compute(*desc, (int)page_size, n_pages, n_sm, n_req, chunk_tokens, chunk_offsets, page_tables, max_pages,
+                         ctx_lens, n_uncached, hp);
+    if (r) return r;
+    *n_items = (int)hp.items.size();
+    *n_cta = hp.n_cta;
+    if (pos) memcpy(pos, hp.pos.data(), (size_t)hp.T * 4);
+    if (slot) memcpy(slot, hp.slot.data(), (size_t)hp.T * 4);
+    if (items) {
+        if (items_cap < *n_items) return SYN_E_CAPACITY;
+        for (int i = 0; i < *n_items; ++i) {
+            const AttnItem& it = hp.items[i];
+            const int32_t row[SYN_PLAN_ITEM_FIELDS] = {it.q_tok, it.nj, it.kvh, it.req, it.kv_begin, it.kv_end, it.q_pos0,
+                                                       it.part, it.grp};
+            memcpy(items + (size_t)i * SYN_PLAN_ITEM_FIELDS, row, sizeof(row));
+        }
+    }
+    if (cta_begin) memcpy(cta_begin, hp.cta_begin.data(), (size_t)(hp.n_cta + 1) * 4);
+    if (stats) *stats = hp.stats;
     return SYN_OK;
 }
 
@@ -729,13 +817,12 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     if (splits_out) *splits_out = g.splits;
     const int smem = gemm_fixed_smem() + g.n_stages * gemm_stage_bytes(g.TN);
     gemm_kernel<<<n_cta, GEMM_THREADS, smem, st>>>(tmB, g, ep);
-    return cudaGetLastError() == cudaSuccess ? SYN_OK : SYN_E_CUDA;
+    return launch_ok() ? SYN_OK : SYN_E_CUDA;
 }
 
-static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const CUtensorMap& tmQ,
-                            bf16* out, cudaStream_t st) {
+static void attn_params(AttnParams& ap, const syn_model* m, const syn_kv* kv, const syn_plan* p, uint32_t layer, bf16* out,
+                        float* part_o, float2* part_ml, int* group_count) {
     const syn_model_desc& c = m->desc;
-    AttnParams ap;
     ap.items = p->d<AttnItem>(p->o_items);
     ap.cta_begin = p->d<int>(p->o_cta);
     ap.page_tables = p->d<int>(p->o_tables);
@@ -743,12 +830,24 @@ static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_
     ap.n_kv_heads = c.n_kv_heads;
     ap.group = c.n_q_heads / c.n_kv_heads;
     ap.q_dim = c.n_q_heads * c.head_dim;
+    ap.q_box_tokens = std::min(16, 64 / ap.group);
     ap.layer_block0 = (int)(2ull * layer * kv->n_pages * c.n_kv_heads);
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
     ap.out = out;
-    ap.part_o = m->part_o;
-    ap.part_ml = m->part_ml;
+    ap.part_o = part_o;
+    ap.part_ml = part_ml;
+    ap.groups = p->d<MergeGroup>(p->o_groups);
+    ap.group_count = group_count;
     ap.status = m->status_dev;
+    ap.n_items = p->n_items; ap.n_req = p->n_req; ap.n_tokens = p->T; ap.n_pages = (int)kv->n_pages;
+    ap.n_parts = p->n_parts; ap.n_groups = p->n_groups;
+}
+
+static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const CUtensorMap& tmQ,
+                            bf16* out, cudaStream_t st) {
+    const syn_model_desc& c = m->desc;
+    AttnParams ap;
+    attn_params(ap, m, kv, p, layer, out, m->part_o, m->part_ml, m->group_count);
     {
         ProfScope prof(m, 2, st);
         if (c.head_dim == 128)
@@ -756,19 +855,7 @@ static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_
         else
             attn_kernel<64><<<p->n_cta, ATT_THREADS, AttnSmem<64>::TOTAL, st>>>(tmQ, kv->tm_kv, ap);
     }
-    if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
-    if (p->n_groups) {
-        ProfScope prof(m, 3, st);
-        dim3 blk(32, 8);
-        if (c.head_dim == 128)
-            attn_merge_kernel<128><<<p->n_groups, blk, 0, st>>>(p->d<MergeGroup>(p->o_groups), m->part_o, m->part_ml, out,
-                                                                ap.group, ap.q_dim);
-        else
-            attn_merge_kernel<64><<<p->n_groups, blk, 0, st>>>(p->d<MergeGroup>(p->o_groups), m->part_o, m->part_ml, out,
-                                                               ap.group, ap.q_dim);
-        if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
-    }
-    return SYN_OK;
+    return launch_ok() ? SYN_OK : SYN_E_CUDA;
 }
 
 static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, int* corr_dev, int* top1_dev,
@@ -783,7 +870,7 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
         prep_kernel<<<T, 256, 0, st>>>(m->embed, tokens, p->d<int>(p->o_pos), m->norm1[0], m->inv_freq, m->x, m->xn,
                                        m->rstd, m->rope, m->best, d, c.head_dim / 2, inv_d, c.rms_eps);
     }
-    if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
+    if (!launch_ok()) return SYN_E_CUDA;
     EpiParams base;
     memset(&base, 0, sizeof(base));
     base.T = T;
@@ -793,7 +880,7 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
     auto resid = [&](int cls, const bf16* gain) -> int {
         ProfScope prof(m, cls, st);
         resid_norm_kernel<<<T, 256, 0, st>>>(m->x, m->part, part_stride, splits, gain, m->xn, m->rstd, d, inv_d, c.rms_eps);
-        return cudaGetLastError() == cudaSuccess ? SYN_OK : SYN_E_CUDA;
+        return launch_ok() ? SYN_OK : SYN_E_CUDA;
     };
     for (uint32_t l = 0; l < c.n_layers; ++l) {
         EpiParams e = base;
@@ -823,7 +910,7 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
         verify_kernel<<<(p->n_req + 127) / 128, 128, 0, st>>>(m->best, tokens, p->d<int>(p->o_offsets),
                                                              p->d<int>(p->o_uncached), p->n_req, acc_dev, corr_dev, top1_dev);
     }
-    return cudaGetLastError() == cudaSuccess ? SYN_OK : SYN_E_CUDA;
+    return launch_ok() ? SYN_OK : SYN_E_CUDA;
 }
 
 extern "C" int syn_verify_run(syn_model* m, syn_kv* kv, const syn_plan* p, int32_t* accept_len_dev, int32_t* correction_dev,
@@ -860,6 +947,7 @@ extern "C" int syn_model_status(syn_model* m) {
     if (cudaMemcpy(&s, m->status_dev, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SYN_E_CUDA;
     if (s) {
         cudaMemset(m->status_dev, 0, 4);
+        if (m->group_count) cudaMemset(m->group_count, 0, (size_t)m->part_cap * 4);   // an aborted step may leave counts
         return SYN_E_DEVICE_TIMEOUT;
     }
     return SYN_OK;
@@ -896,6 +984,7 @@ extern "C" int syn_verify_batch(syn_model* m, syn_kv* kv, int32_t n_req, const i
     CU_OK(cudaStreamSynchronize(st));
     if (po[2 * m->pinned_out_cap]) {
         cudaMemset(m->status_dev, 0, 4);
+        if (m->group_count) cudaMemset(m->group_count, 0, (size_t)m->part_cap * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     memcpy(accept_len, po, (size_t)n_req * 4);
@@ -938,7 +1027,7 @@ extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, 
         memset(&ps, 0, sizeof(ps));
         ps.p[0] = (const bf16*)w; ps.rows[0] = N; ps.src_k = K;
         pack_weight_kernel<<<dim3(n_mt, nkb), 256, 0, st>>>(ps, packed, nkb);
-        if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
+        if (!launch_ok()) return SYN_E_CUDA;
         packed_src = w; packed_n = N; packed_k = K;
     }
     CUtensorMap tmB;
@@ -973,30 +1062,35 @@ extern "C" int syn_op_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uin
 // ------------------------------------------------------------------------------------------ no-allocation attention
 
 // Scratch of syn_op_attention_static: the fp32 partial outputs and (max, sum) pairs of attention
-// work items that cover only part of a request's keys.  File-scope device memory, so every GPU that
-// loads the library holds these ~33 MB from load to exit.  Host code may not pass these names to a
+// work items that cover only part of a request's keys, and the per-group completion counters.  File-scope device memory, so every GPU that
+// loads the library holds these ~8.5 MB from load to exit.  Host code may not pass these names to a
 // kernel (on the host they are stand-ins, not device addresses): static_scratch() asks the runtime
 // for the device addresses once per device.
 static __device__ __align__(256) float g_static_part_o[(size_t)SYN_STATIC_MAX_PARTS * 64 * 128];
 static __device__ __align__(256) float2 g_static_part_ml[(size_t)SYN_STATIC_MAX_PARTS * 64];
+static __device__ __align__(256) int g_static_group_count[SYN_STATIC_MAX_PARTS];
 
-static int static_scratch(float** part_o, float2** part_ml) {
+static int static_scratch(float** part_o, float2** part_ml, int** group_count) {
     constexpr int MAX_DEV = 64;
     static float* o_of[MAX_DEV];
     static float2* ml_of[MAX_DEV];
+    static int* cnt_of[MAX_DEV];
     int dev = -1;
     CU_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= MAX_DEV) return SYN_E_INVALID_ARG;
     if (!o_of[dev]) {   // first call on this device (which is current): resolve the symbols
-        void *a = nullptr, *b = nullptr;
+        void *a = nullptr, *b = nullptr, *cn = nullptr;
         CU_OK(cudaGetSymbolAddress(&a, g_static_part_o));
         CU_OK(cudaGetSymbolAddress(&b, g_static_part_ml));
-        if (!a || !b) return SYN_E_CUDA;
+        CU_OK(cudaGetSymbolAddress(&cn, g_static_group_count));
+        if (!a || !b || !cn) return SYN_E_CUDA;
         ml_of[dev] = static_cast<float2*>(b);
+        cnt_of[dev] = static_cast<int*>(cn);
         o_of[dev] = static_cast<float*>(a);
     }
     *part_o = o_of[dev];
     *part_ml = ml_of[dev];
+    *group_count = cnt_of[dev];
     return SYN_OK;
 }
 
@@ -1009,41 +1103,23 @@ extern "C" int syn_op_attention_static(syn_model* m, syn_kv* kv, const syn_plan*
     if (p->n_parts > SYN_STATIC_MAX_PARTS) return SYN_E_CAPACITY;
     float* part_o = nullptr;
     float2* part_ml = nullptr;
-    int r = static_scratch(&part_o, &part_ml);
+    int* group_count = nullptr;
+    int r = static_scratch(&part_o, &part_ml, &group_count);
     if (r) return r;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     CU_OK(cudaMemcpyAsync(m->q, q, (size_t)p->T * q_dim * 2, cudaMemcpyDeviceToDevice, st));
+    // the group counters must start at zero; every partial row that is read is written first
+    CU_OK(cudaMemsetAsync(group_count, 0, (size_t)SYN_STATIC_MAX_PARTS * 4, st));
     AttnParams ap;
-    ap.items = p->d<AttnItem>(p->o_items);
-    ap.cta_begin = p->d<int>(p->o_cta);
-    ap.page_tables = p->d<int>(p->o_tables);
-    ap.max_pages = p->max_pages;
-    ap.n_kv_heads = c.n_kv_heads;
-    ap.group = c.n_q_heads / c.n_kv_heads;
-    ap.q_dim = q_dim;
-    ap.layer_block0 = (int)(2ull * layer * kv->n_pages * c.n_kv_heads);
-    ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
-    ap.out = (bf16*)out;
-    ap.part_o = part_o;      // every partial row that the merge reads is written first: nothing to clear
-    ap.part_ml = part_ml;
-    ap.status = m->status_dev;
+    attn_params(ap, m, kv, p, layer, (bf16*)out, part_o, part_ml, group_count);
     if (c.head_dim == 128)
         attn_kernel<128><<<p->n_cta, ATT_THREADS, AttnSmem<128>::TOTAL, st>>>(m->tm_q, kv->tm_kv, ap);
     else
         attn_kernel<64><<<p->n_cta, ATT_THREADS, AttnSmem<64>::TOTAL, st>>>(m->tm_q, kv->tm_kv, ap);
-    if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
-    if (p->n_groups) {
-        dim3 blk(32, 8);
-        if (c.head_dim == 128)
-            attn_merge_kernel<128><<<p->n_groups, blk, 0, st>>>(p->d<MergeGroup>(p->o_groups), part_o, part_ml, (bf16*)out,
-                                                                ap.group, ap.q_dim);
-        else
-            attn_merge_kernel<64><<<p->n_groups, blk, 0, st>>>(p->d<MergeGroup>(p->o_groups), part_o, part_ml, (bf16*)out,
-                                                               ap.group, ap.q_dim);
-        if (cudaGetLastError() != cudaSuccess) return SYN_E_CUDA;
-    }
-    return SYN_OK;
+    return launch_ok() ? SYN_OK : SYN_E_CUDA;
 }
+
+extern "C" const char* syn_last_cuda_error(void) { return g_last_cuda_error; }
 
 extern "C" const char* syn_strerror(int code) {
     switch (code) {

@@ -48,9 +48,11 @@ def test_static_scratch_attention_equals_the_allocating_one_twice_in_a_row():
 
 def test_static_scratch_attention_refuses_more_partials_than_it_holds():
     import paper_2511_07423_b200 as syn
-    shape = ModelShape("att-static", 1, 256, 32, 32, 64, 256, 512)   # 32 kv heads: many split items
+    # 147 equal (request, kv head) units on 148 SMs: each is a little more than one CTA's share,
+    # so the planner splits every one in two -> 294 partial items, more than the fixed array holds
+    shape = ModelShape("att-static", 1, 256, 21, 21, 128, 256, 512)
     seed = 22
-    wl = Workload("t", None, seed, 24, ("const", 1600), ("const", 1), 0.5)
+    wl = Workload("t", None, seed, 7, ("const", 2000), ("const", 1), 0.5)
     batch = gen.gen_batch(wl)
     glob, layers = cpu_model(shape, seed)
     gg, gl = to_cuda(glob, layers)
@@ -58,7 +60,7 @@ def test_static_scratch_attention_refuses_more_partials_than_it_holds():
     kv = syn.KVCache(model, batch.n_pages)
     T = batch.n_tokens
     plan = syn.Plan(kv, torch.zeros(T, dtype=torch.int32), batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
-    assert plan.stats().attn_split_items > 1024
+    assert plan.stats().attn_split_items > 256
     q = torch.zeros(T, shape.q_dim, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(syn.SynError) as e:
         plan.attention_static(0, q)
