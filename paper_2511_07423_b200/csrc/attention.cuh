@@ -291,7 +291,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
         mbar_fence_init();
     }
+    pdl_launch_dependents();
     __syncthreads();
+    pdl_wait();   // Q and the chunk's K/V come from the preceding projection kernel
 
     if (warp == ATT_CONSUMER_WARPS) {
         // ------------------------------------------------------------ producer (whole warp)

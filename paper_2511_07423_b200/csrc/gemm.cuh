@@ -155,6 +155,8 @@ resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, size_t 
     __shared__ float red[8];
     const int t = blockIdx.x;
     float ss = 0.f;
+    pdl_launch_dependents();
+    pdl_wait();
     for (int f = threadIdx.x * 4; f < d; f += blockDim.x * 4) {
         float4 v = *reinterpret_cast<const float4*>(x + (size_t)t * d + f);
         for (int s = 0; s < splits; ++s) {
@@ -324,6 +326,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_cta = gridDim.x, cta = blockIdx.x;
+    pdl_launch_dependents();
     uint32_t acc_stride = 32;
     while ((int)acc_stride < g.TN) acc_stride <<= 1;
     const uint32_t tmem_cols = 2 * acc_stride;
@@ -360,6 +363,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                 const __nv_bfloat16* wsrc = g.w + ((size_t)w.pair * g.num_kb) * (2 * 128 * 64) + (size_t)w.mt_lo * (128 * 64);
                 for (int kb = w.kb0; kb < min(w.kb1, w.kb0 + GEMM_PREFETCH_KB); ++kb)
                     bulk_prefetch_l2(wsrc + (size_t)kb * (2 * 128 * 64), a_bytes);
+                if (i == 0) pdl_wait();   // weights are constant; the token operand is the predecessor's output
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const int s = it % g.n_stages;
                     if (it >= (uint32_t)g.n_stages && !mbar_wait(&empty_bar[s], ((it / g.n_stages) - 1) & 1, g.status)) {
@@ -419,6 +423,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
         float* st = staging + grp * 32 * 128;
         bool ok = true;
         GemmWork w;
+        pdl_wait();   // the epilogues read per-token statistics and write buffers of earlier kernels
         for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
             const int n0 = w.tt * g.TN;
             const int n_valid = min(g.TN, p.T - n0);

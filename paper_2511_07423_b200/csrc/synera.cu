@@ -37,6 +37,23 @@ static inline bool launch_ok() { return note_cuda(cudaGetLastError()) == cudaSuc
         }                                        \
     } while (0)
 
+// Launch with programmatic stream serialization: the kernel may start while its predecessor in the
+// stream still runs; every kernel of the step calls pdl_wait() before it touches anything an earlier
+// kernel produces or still reads.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr;
+    memset(&attr, 0, sizeof(attr));
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return note_cuda(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+}
+
 // ------------------------------------------------------------------------------------------ small kernels
 
 // Token embedding (paper Sec. 4.5: the flattened batch enters the transformer), first layer's
@@ -48,6 +65,8 @@ prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens, cons
             unsigned long long* __restrict__ best, int d, int half, float inv_d, float eps) {
     __shared__ float red[8];
     const int t = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     const bf16* e = embed + (size_t)tokens[t] * d;
     float ss = 0.f;
     for (int f = threadIdx.x; f < d; f += blockDim.x) {
@@ -78,6 +97,7 @@ __global__ void verify_kernel(const unsigned long long* __restrict__ best, const
                               const int* __restrict__ offsets, const int* __restrict__ n_uncached, int n_req,
                               int* __restrict__ accept_len, int* __restrict__ correction, int* __restrict__ top1_out) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait();
     if (i >= n_req) return;
     const int b = offsets[i], n = offsets[i + 1] - b, u = n_uncached[i];
     if (top1_out)
@@ -816,8 +836,7 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     else n_cta = std::min(n_sm, g.pair_mode ? tiles : 2 * tiles);
     if (splits_out) *splits_out = g.splits;
     const int smem = gemm_fixed_smem() + g.n_stages * gemm_stage_bytes(g.TN);
-    gemm_kernel<<<n_cta, GEMM_THREADS, smem, st>>>(tmB, g, ep);
-    return launch_ok() ? SYN_OK : SYN_E_CUDA;
+    return launch_pdl(gemm_kernel, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep) == cudaSuccess ? SYN_OK : SYN_E_CUDA;
 }
 
 static void attn_params(AttnParams& ap, const syn_model* m, const syn_kv* kv, const syn_plan* p, uint32_t layer, bf16* out,
@@ -850,12 +869,14 @@ static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_
     attn_params(ap, m, kv, p, layer, out, m->part_o, m->part_ml, m->group_count);
     {
         ProfScope prof(m, 2, st);
+        cudaError_t e;
         if (c.head_dim == 128)
-            attn_kernel<128><<<p->n_cta, ATT_THREADS, AttnSmem<128>::TOTAL, st>>>(tmQ, kv->tm_kv, ap);
+            e = launch_pdl(attn_kernel<128>, dim3(p->n_cta), dim3(ATT_THREADS), AttnSmem<128>::TOTAL, st, tmQ, kv->tm_kv, ap);
         else
-            attn_kernel<64><<<p->n_cta, ATT_THREADS, AttnSmem<64>::TOTAL, st>>>(tmQ, kv->tm_kv, ap);
+            e = launch_pdl(attn_kernel<64>, dim3(p->n_cta), dim3(ATT_THREADS), AttnSmem<64>::TOTAL, st, tmQ, kv->tm_kv, ap);
+        if (e != cudaSuccess) return SYN_E_CUDA;
     }
-    return launch_ok() ? SYN_OK : SYN_E_CUDA;
+    return SYN_OK;
 }
 
 static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, int* corr_dev, int* top1_dev,
@@ -867,10 +888,10 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
     const float inv_d = 1.0f / (float)d;
     {
         ProfScope prof(m, 0, st);
-        prep_kernel<<<T, 256, 0, st>>>(m->embed, tokens, p->d<int>(p->o_pos), m->norm1[0], m->inv_freq, m->x, m->xn,
-                                       m->rstd, m->rope, m->best, d, c.head_dim / 2, inv_d, c.rms_eps);
+        if (launch_pdl(prep_kernel, dim3(T), dim3(256), 0, st, m->embed, tokens, p->d<int>(p->o_pos), m->norm1[0], m->inv_freq,
+                       m->x, m->xn, m->rstd, m->rope, m->best, d, (int)(c.head_dim / 2), inv_d, c.rms_eps) != cudaSuccess)
+            return SYN_E_CUDA;
     }
-    if (!launch_ok()) return SYN_E_CUDA;
     EpiParams base;
     memset(&base, 0, sizeof(base));
     base.T = T;
@@ -879,8 +900,8 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
     int r, splits = 1;
     auto resid = [&](int cls, const bf16* gain) -> int {
         ProfScope prof(m, cls, st);
-        resid_norm_kernel<<<T, 256, 0, st>>>(m->x, m->part, part_stride, splits, gain, m->xn, m->rstd, d, inv_d, c.rms_eps);
-        return launch_ok() ? SYN_OK : SYN_E_CUDA;
+        return launch_pdl(resid_norm_kernel, dim3(T), dim3(256), 0, st, m->x, m->part, part_stride, splits, gain, m->xn, m->rstd, d,
+                          inv_d, c.rms_eps) == cudaSuccess ? SYN_OK : SYN_E_CUDA;
     };
     for (uint32_t l = 0; l < c.n_layers; ++l) {
         EpiParams e = base;
@@ -907,10 +928,11 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
     if ((r = launch_gemm(m, 7, m->n_sm, m->status_dev, m->lm_head, m->v_rows, d, m->tm_xn, e, st))) return r;
     {
         ProfScope prof(m, 8, st);
-        verify_kernel<<<(p->n_req + 127) / 128, 128, 0, st>>>(m->best, tokens, p->d<int>(p->o_offsets),
-                                                             p->d<int>(p->o_uncached), p->n_req, acc_dev, corr_dev, top1_dev);
+        if (launch_pdl(verify_kernel, dim3((p->n_req + 127) / 128), dim3(128), 0, st, m->best, tokens, p->d<int>(p->o_offsets),
+                       p->d<int>(p->o_uncached), p->n_req, acc_dev, corr_dev, top1_dev) != cudaSuccess)
+            return SYN_E_CUDA;
     }
-    return launch_ok() ? SYN_OK : SYN_E_CUDA;
+    return SYN_OK;
 }
 
 extern "C" int syn_verify_run(syn_model* m, syn_kv* kv, const syn_plan* p, int32_t* accept_len_dev, int32_t* correction_dev,
