@@ -52,96 +52,115 @@ struct EpiParams {
     unsigned long long* best;
 };
 
-__device__ __forceinline__ unsigned long long pack_argmax(float v, int idx) {
+__device__ __forceinline__ uint32_t orderable_f32(float v) {   // monotone map of a float to unsigned
     uint32_t u = __float_as_uint(v);
-    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-    return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)idx);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ unsigned long long pack_argmax_key(uint32_t key, int idx) {
+    return ((unsigned long long)key << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)idx);
 }
 
-// Consume one staged chunk: stage[c][f] = D[feature m0 + f][token t0 + c], c < ncols <= 32, f < 128.
-// Called by 4 warps (ew = 0..3); warp ew handles tokens c = ew, ew + 4, ...
-__device__ __forceinline__ void epi_chunk(const EpiParams& p, const float* __restrict__ stage, int m0, int t0,
-                                          int ncols, int split, int ew, int lane) {
-    const int f0 = m0 + 4 * lane;
-    for (int c = ew; c < ncols; c += 4) {
-        const int t = t0 + c;
-        float4 v = *reinterpret_cast<const float4*>(stage + c * 128 + 4 * lane);
-        float a[4] = {v.x, v.y, v.z, v.w};
-        if (p.mode == EPI_PLAIN) {
+// Row order inside one packed 128-feature tile.  TMEM lane l of the tile belongs to warp quarter
+// q = l / 32; partners that an epilogue combines (the two RoPE halves of a head dimension, a gate
+// feature and its up feature) sit 16 lanes apart in the same warp, so they meet by one shuffle.
+//   rope tiles (q and k rows): quarter q covers head q / (hd/32) of the tile, dims
+//     [16 s, 16 s + 16) for lanes 0..15 and the same dims + hd/2 for lanes 16..31, s = q % (hd/32)
+//   gate/up tiles: quarter q lanes 0..15 = gate features 64 b + 16 q + lane, lanes 16..31 = the up
+//     features of the same indices (b = tile index)
+//   every other tile: feature = tile base + lane
+__host__ __device__ __forceinline__ int rope_tile_feature(int l, int hd) {   // offset inside the tile's 128 features
+    const int half = hd >> 1, groups = half >> 4, q = l >> 5, ll = l & 31;
+    return (q / groups) * hd + 16 * (q % groups) + (ll & 15) + ((ll & 16) ? half : 0);
+}
+
+// Epilogue of one chunk straight from registers: r[j] = D[feature of this thread][token t0 + j],
+// j < 32; tokens j >= ncols are padding.  `m0` = first packed row of the tile, `quarter` = warp's
+// TMEM lane quarter.  comb: shared scratch of the warp's group for the vocabulary argmax
+// ([2][4][32] keys), ci = chunk counter of the group (buffer parity).
+template <int MODE>
+__device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&r)[32], int m0, int t0, int ncols,
+                                           int split, int quarter, int lane, unsigned long long* comb, int ci, int grp) {
+    const int l = quarter * 32 + lane;
+    if (MODE == EPI_PLAIN || MODE == EPI_PART) {
+        const int f = m0 + l;
+        float* base = MODE == EPI_PLAIN ? p.y + f : p.part + (size_t)split * p.part_stride + f;
+        const size_t ld = MODE == EPI_PLAIN ? (size_t)p.ldy : (size_t)p.d;
+        if (f < p.N) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (f0 + e < p.N) p.y[(size_t)t * p.ldy + f0 + e] = a[e];
-        } else if (p.mode == EPI_QKV) {
-            const float r = p.rstd[t];
+            for (int j = 0; j < 32; ++j)
+                if (j < ncols) base[(size_t)(t0 + j) * ld] = __uint_as_float(r[j]);
+        }
+    } else if (MODE == EPI_QKV) {
+        const int which = m0 < p.q_dim ? 0 : (m0 < p.q_dim + p.kv_dim ? 1 : 2);
+        const int region0 = which == 0 ? 0 : (which == 1 ? p.q_dim : p.q_dim + p.kv_dim);
+        const int fr = m0 - region0 + (which < 2 ? rope_tile_feature(l, p.hd) : l);   // feature inside q, k or v
+        const int half = p.hd >> 1;
+        const int dim = fr & (p.hd - 1);
+        const bool lo = dim < half;
+        const float2* cs = p.rope + (lo ? dim : dim - half);
+        const int kvh = fr / p.hd;
+        // per-token values of the chunk: lane j fetches those of token j, a shuffle hands them round
+        const float rs_mine = lane < ncols ? __ldg(p.rstd + t0 + lane) : 0.f;
+        const int slot_mine = (which > 0 && lane < ncols) ? __ldg(p.slot + t0 + lane) : 0;
+        __nv_bfloat16* const qdst = p.q + fr;
+        __nv_bfloat16* const kvdst = p.pool + ((size_t)kvh * 2 + (which > 0 ? which - 1 : 0)) * 16 * p.hd + dim;
+        const size_t page_stride = (size_t)p.n_kv_heads * 2 * 16 * p.hd;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) a[e] *= r;
-            const int which = f0 < p.q_dim ? 0 : (f0 < p.q_dim + p.kv_dim ? 1 : 2);
-            if (which < 2) {  // rotate-half RoPE: pair (i, i + hd/2) inside each head
-                const int half = p.hd >> 1;
-                const int xl = half >> 2;  // partner lane distance (16 for hd 128, 8 for hd 64)
-                const int i = (4 * lane) & (p.hd - 1);
-                const bool lo = i < half;
-                const float2* cs = p.rope + (size_t)t * half + (lo ? i : i - half);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float o = __shfl_xor_sync(0xFFFFFFFFu, a[e], xl);
-                    float2 w = cs[e];
-                    a[e] = lo ? (a[e] * w.x - o * w.y) : (a[e] * w.x + o * w.y);
-                }
+        for (int j = 0; j < 32; ++j) {
+            const int t = t0 + j;
+            const bool live = j < ncols;
+            float a = __uint_as_float(r[j]) * __shfl_sync(0xFFFFFFFFu, rs_mine, j);
+            if (which < 2) {   // rotate-half RoPE: the partner dimension is 16 lanes away
+                const float o = __shfl_xor_sync(0xFFFFFFFFu, a, 16);
+                const float2 w = live ? __ldg(cs + (size_t)t * half) : make_float2(0.f, 0.f);
+                a = lo ? (a * w.x - o * w.y) : (a * w.x + o * w.y);
             }
-            uint2 pk = make_uint2(pack_bf16(a[0], a[1]), pack_bf16(a[2], a[3]));
-            if (which == 0) {
-                *reinterpret_cast<uint2*>(p.q + (size_t)t * p.q_dim + f0) = pk;
-            } else {
-                const int fk = f0 - p.q_dim - (which == 2 ? p.kv_dim : 0);
-                const int kvh = fk / p.hd, dim = fk - kvh * p.hd;
-                const int s = p.slot[t];
-                const int page = s / p.page_size, row = s - page * p.page_size;
-                size_t off = ((((size_t)page * p.n_kv_heads + kvh) * 2 + (which - 1)) * p.page_size + row) * p.hd + dim;
-                *reinterpret_cast<uint2*>(p.pool + off) = pk;
+            const int s = __shfl_sync(0xFFFFFFFFu, slot_mine, j);   // page * 16 + row (pages hold 16 tokens)
+            if (live) {
+                if (which == 0) qdst[(size_t)t * p.q_dim] = __float2bfloat16(a);
+                else kvdst[(size_t)(s >> 4) * page_stride + (size_t)(s & 15) * p.hd] = __float2bfloat16(a);
             }
-        } else if (p.mode == EPI_PART) {
-            *reinterpret_cast<float4*>(p.part + (size_t)split * p.part_stride + (size_t)t * p.d + f0) = v;
-        } else if (p.mode == EPI_SWIGLU) {
-            const float r = p.rstd[t];
-            float o[4];
+        }
+    } else if (MODE == EPI_SWIGLU) {
+        const int f = (m0 >> 1) + 16 * quarter + (lane & 15);   // gate/up feature of this lane pair
+        const float rs_mine = lane < ncols ? __ldg(p.rstd + t0 + lane) : 0.f;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                a[e] *= r;
-                o[e] = __shfl_xor_sync(0xFFFFFFFFu, a[e], 16);  // lanes 0-15: gate, lanes 16-31: up
-            }
-            if (lane < 16) {
-                float h[4];
+        for (int j = 0; j < 32; ++j) {
+            const int t = t0 + j;
+            const bool live = j < ncols;
+            const float a = __uint_as_float(r[j]) * __shfl_sync(0xFFFFFFFFu, rs_mine, j);
+            const float u = __shfl_xor_sync(0xFFFFFFFFu, a, 16);   // lanes 0..15 receive "up"
+            if (live && lane < 16) p.act[(size_t)t * p.f_pad + f] = __float2bfloat16(__fdividef(a, 1.0f + __expf(-a)) * u);
+        }
+    } else {  // EPI_LMHEAD
+        const int f = m0 + l;
+        const bool valid = f < p.vocab;
+        unsigned long long mine = 0ull;   // lane j keeps the warp's best of token j
+        const float rs_mine = lane < ncols ? __ldg(p.rstd + t0 + lane) : 0.f;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) h[e] = a[e] / (1.0f + __expf(-a[e])) * o[e];
-                uint2 pk = make_uint2(pack_bf16(h[0], h[1]), pack_bf16(h[2], h[3]));
-                *reinterpret_cast<uint2*>(p.act + (size_t)t * p.f_pad + (m0 >> 1) + 4 * lane) = pk;
-            }
-        } else {  // EPI_LMHEAD
-            const float r = p.rstd[t];
-            float bv = -INFINITY;
-            int bi = 0x7FFFFFFF;
+        for (int j = 0; j < 32; ++j) {
+            const int t = t0 + j;
+            const bool live = j < ncols;
+            const float a = __uint_as_float(r[j]) * __shfl_sync(0xFFFFFFFFu, rs_mine, j);
+            if (p.logits && live && valid) p.logits[(size_t)t * p.vocab + f] = a;
+            const uint32_t key = valid ? orderable_f32(a) : 0u;
+            const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
+            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, key == mx && valid);
+            if (lane == j) mine = hit ? pack_argmax_key(mx, m0 + quarter * 32 + (__ffs(hit) - 1)) : 0ull;
+        }
+        // combine the four quarter-warps of the tile, then one atomic per token
+        unsigned long long* buf = comb + (ci & 1) * 128;
+        buf[quarter * 32 + lane] = mine;
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
+        if (lane < 8) {
+            const int j = quarter * 8 + lane;
+            unsigned long long b = buf[j];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                a[e] *= r;
-                if (f0 + e < p.vocab && a[e] > bv) { bv = a[e]; bi = f0 + e; }
+            for (int q2 = 1; q2 < 4; ++q2) {
+                const unsigned long long o = buf[q2 * 32 + j];
+                b = o > b ? o : b;
             }
-            if (p.logits) {
-                if (f0 + 3 < p.vocab && (((size_t)t * p.vocab + f0) & 3) == 0) {
-                    *reinterpret_cast<float4*>(p.logits + (size_t)t * p.vocab + f0) = make_float4(a[0], a[1], a[2], a[3]);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (f0 + e < p.vocab) p.logits[(size_t)t * p.vocab + f0 + e] = a[e];
-                }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
-                int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
-                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-            }
-            if (lane == 0 && bi != 0x7FFFFFFF) atomicMax(p.best + t, pack_argmax(bv, bi));
+            if (j < ncols && b) atomicMax(p.best + t0 + j, b);
         }
     }
 }
@@ -187,13 +206,16 @@ resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, size_t 
 // Weight packing: row-major sources -> [pair][k-block][2][128 rows x 64 cols], each 16 KB tile
 // stored as the 128-byte-swizzled shared-memory image (16-byte chunk c of row r at chunk c ^ (r & 7)).
 // mode 0: packed row pr = row pr of the concatenation of up to three matrices.
-// mode 1: gate/up interleave: packed rows [128b, 128b+64) = gate rows [64b, 64b+64), next 64 = up rows.
+// mode 1: gate/up: tile b holds gate and up features [64 b, 64 b + 64) in the lane order of
+//         epi_direct (quarter q: lanes 0..15 gate 64 b + 16 q + lane, lanes 16..31 the same up rows).
+// mode 2: q | k | v concatenation; q and k tiles in the RoPE lane order (rope_tile_feature), v plain.
 // ------------------------------------------------------------------------------------------
 struct PackSrc {
     const __nv_bfloat16* p[3];
     int rows[3];
     int mode;
     int src_k;   // valid columns of the sources (row pitch)
+    int hd;      // mode 2: head dimension
 };
 
 __global__ void pack_weight_kernel(PackSrc src, __nv_bfloat16* __restrict__ out, int num_kb) {
@@ -201,18 +223,21 @@ __global__ void pack_weight_kernel(PackSrc src, __nv_bfloat16* __restrict__ out,
     __nv_bfloat16* tile = out + (((size_t)(mtile >> 1) * num_kb + kb) * 2 + (mtile & 1)) * (128 * 64);
     for (int i = threadIdx.x; i < 128 * 8; i += blockDim.x) {
         const int r = i >> 3, c = i & 7;
-        const int pr = mtile * 128 + r;
         const __nv_bfloat16* row = nullptr;
         if (src.mode == 0) {
-            int q = pr;
+            int q = mtile * 128 + r;
             for (int k = 0; k < 3 && !row; ++k) {
                 if (q < src.rows[k]) row = src.p[k] + (size_t)q * src.src_k;
                 q -= src.rows[k];
             }
+        } else if (src.mode == 1) {
+            const int sr = mtile * 64 + 16 * (r >> 5) + (r & 15);
+            if (sr < src.rows[0]) row = src.p[(r & 16) ? 1 : 0] + (size_t)sr * src.src_k;
         } else {
-            const int b = pr >> 7, w = pr & 127;
-            const int sr = b * 64 + (w & 63);
-            if (sr < src.rows[0]) row = src.p[w < 64 ? 0 : 1] + (size_t)sr * src.src_k;
+            int base = mtile * 128, k = 0;   // region of this tile (regions are multiples of 128 rows)
+            while (k < 2 && base >= src.rows[k]) base -= src.rows[k++];
+            const int q = base + (k < 2 ? rope_tile_feature(r, src.hd) : r);
+            if (q < src.rows[k]) row = src.p[k] + (size_t)q * src.src_k;
         }
         uint4 v = make_uint4(0, 0, 0, 0);
         const int col = kb * 64 + c * 8;
@@ -245,7 +270,7 @@ constexpr int GEMM_SMEM_MAX = 232448;
 constexpr int GEMM_PREFETCH_KB = 12;               // L2 prefetch distance in k-blocks
 
 __host__ __device__ inline int gemm_stage_bytes(int TN) { return GEMM_A_BYTES + ((TN + 31) / 32) * GEMM_BOX_BYTES; }
-__host__ inline int gemm_fixed_smem() { return 1024 /*align*/ + 2 * 32 * 128 * 4 /*staging*/ + 512; }
+__host__ inline int gemm_fixed_smem() { return 1024 /*align*/ + 2 * 2 * 128 * 8 /*argmax scratch*/ + 512; }
 __host__ inline int gemm_stages(int TN) {
     int s = (GEMM_SMEM_MAX - gemm_fixed_smem()) / gemm_stage_bytes(TN);
     return s > GEMM_MAX_STAGES ? GEMM_MAX_STAGES : s;
@@ -302,6 +327,13 @@ __device__ __forceinline__ bool gemm_work(const GemmParams& g, int cta, int n_ct
     return true;
 }
 
+// Every CTA walks its k-blocks from a different starting point (and wraps): at any moment the CTAs
+// that share a token tile then ask L2 for different lines of it instead of all for the same ones.
+// The schedule is static, so the summation order of a given output is the same in every run.
+__device__ __forceinline__ int gemm_k_rotation(int cta, int n_cta, int nk) {
+    return (int)(((long long)cta * nk) / n_cta);
+}
+
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
@@ -317,8 +349,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int stage_bytes = gemm_stage_bytes(g.TN);
-    float* staging = reinterpret_cast<float*>(smem + g.n_stages * stage_bytes);
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(staging + 2 * 32 * 128);
+    unsigned long long* comb = reinterpret_cast<unsigned long long*>(smem + g.n_stages * stage_bytes);   // [2 groups][2][128]
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(comb + 2 * 2 * 128);
     uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
     uint64_t* accf_bar = empty_bar + GEMM_MAX_STAGES;   // accumulators complete (MMA -> epilogue)
     uint64_t* acce_bar = accf_bar + 1;                  // accumulators drained (epilogue -> MMA)
@@ -361,17 +393,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                 const int nbox = (((min(g.TN, p.T - n0) + 15) & ~15) + 31) >> 5;
                 const uint32_t a_bytes = (uint32_t)(w.mt_hi - w.mt_lo) * GEMM_TILE_BYTES;
                 const __nv_bfloat16* wsrc = g.w + ((size_t)w.pair * g.num_kb) * (2 * 128 * 64) + (size_t)w.mt_lo * (128 * 64);
-                for (int kb = w.kb0; kb < min(w.kb1, w.kb0 + GEMM_PREFETCH_KB); ++kb)
-                    bulk_prefetch_l2(wsrc + (size_t)kb * (2 * 128 * 64), a_bytes);
-                if (i == 0) pdl_wait();   // weights are constant; the token operand is the predecessor's output
-                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+                if (i == 0) pdl_wait();   // the token operand is the predecessor's output
+                const int nk = w.kb1 - w.kb0, rot = gemm_k_rotation(cta, n_cta, nk);
+                for (int j = 0; j < nk; ++j, ++it) {
+                    const int kb = w.kb0 + (j + rot) % nk;
                     const int s = it % g.n_stages;
                     if (it >= (uint32_t)g.n_stages && !mbar_wait(&empty_bar[s], ((it / g.n_stages) - 1) & 1, g.status)) {
                         ok = false;
                         break;
                     }
-                    if (kb + GEMM_PREFETCH_KB < w.kb1)
-                        bulk_prefetch_l2(wsrc + (size_t)(kb + GEMM_PREFETCH_KB) * (2 * 128 * 64), a_bytes);
                     uint8_t* a_s = smem + s * stage_bytes;
                     uint8_t* b_s = a_s + GEMM_A_BYTES;
                     mbar_expect_tx(&full_bar[s], a_bytes + nbox * GEMM_BOX_BYTES);
@@ -396,19 +426,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                     if (!ok) break;
                     tc_fence_after();
                 }
-                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+                const int nk = w.kb1 - w.kb0;
+                for (int j = 0; j < nk; ++j, ++it) {
                     const int s = it % g.n_stages;
                     ok = mbar_wait(&full_bar[s], (it / g.n_stages) & 1, g.status);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
                     const uint64_t db = umma_desc_k128(a_addr + GEMM_A_BYTES);
-                    for (int mt = w.mt_lo; mt < w.mt_hi; ++mt) {
-                        const uint64_t da = umma_desc_k128(a_addr + mt * GEMM_TILE_BYTES);
+                    // consecutive MMAs alternate between the two accumulators: back-to-back MMAs into
+                    // one accumulator wait for each other
 #pragma unroll
-                        for (int k = 0; k < GEMM_BK / 16; ++k)  // 16 bf16 = 32 bytes = 2 descriptor address units
-                            umma_bf16(tmem_base + mt * acc_stride, da + 2 * k, db + 2 * k, idesc, (kb > w.kb0) || k > 0);
-                    }
+                    for (int k = 0; k < GEMM_BK / 16; ++k)  // 16 bf16 = 32 bytes = 2 descriptor address units
+                        for (int mt = w.mt_lo; mt < w.mt_hi; ++mt) {
+                            const uint64_t da = umma_desc_k128(a_addr + mt * GEMM_TILE_BYTES);
+                            umma_bf16(tmem_base + mt * acc_stride, da + 2 * k, db + 2 * k, idesc, j > 0 || k > 0);
+                        }
                     umma_commit(&empty_bar[s]);
                 }
                 if (ok) umma_commit(accf_bar);
@@ -418,11 +451,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
     } else {
         // ------------------------------------------------------------ epilogue
         const int e = warp - 2;
-        const int grp = e >> 2, ew = e & 3;   // group 0/1 takes alternate chunks; ew splits a chunk's tokens
+        const int grp = e >> 2;               // group 0/1 takes alternate 32-token chunks
         const int quarter = warp & 3;         // TMEM lane quarter this warp may read
-        float* st = staging + grp * 32 * 128;
+        unsigned long long* cbuf = comb + grp * 2 * 128;
         bool ok = true;
         GemmWork w;
+        int nci = 0;                          // chunks this group has handled (argmax scratch parity)
         pdl_wait();   // the epilogues read per-token statistics and write buffers of earlier kernels
         for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
             const int n0 = w.tt * g.TN;
@@ -432,7 +466,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
             if (!ok) break;
             tc_fence_after();
             const int total_chunks = (w.mt_hi - w.mt_lo) * nchunks;
-            for (int ci = grp; ci < total_chunks; ci += 2) {
+            for (int ci = grp; ci < total_chunks; ci += 2, ++nci) {
                 const int mt = w.mt_lo + ci / nchunks, c = ci % nchunks;
                 const int m0 = w.pair * 256 + mt * 128;
                 uint32_t r[32];
@@ -442,11 +476,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                     tc_fence_before();
                     if (lane == 0) mbar_arrive(acce_bar);
                 }
-#pragma unroll
-                for (int j = 0; j < 32; ++j) st[j * 128 + quarter * 32 + lane] = __uint_as_float(r[j]);
-                asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
-                if (m0 < p.N) epi_chunk(p, st, m0, n0 + c * 32, min(32, n_valid - c * 32), w.split, ew, lane);
-                asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
+                const int t0 = n0 + c * 32, ncols = min(32, n_valid - c * 32);
+                if (m0 < p.N) {   // uniform over the group: the vocabulary argmax meets at a named barrier
+                    switch (p.mode) {
+                        case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
+                        case EPI_QKV: epi_direct<EPI_QKV>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
+                        case EPI_PART: epi_direct<EPI_PART>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
+                        case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
+                        default: epi_direct<EPI_LMHEAD>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
+                    }
+                }
             }
             if (grp >= total_chunks) {   // a group without any chunk still releases the accumulators
                 tc_fence_before();

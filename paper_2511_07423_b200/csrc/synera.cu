@@ -382,7 +382,7 @@ extern "C" int syn_model_load(const syn_model_desc* desc, const syn_weights* w, 
         *out_ptr = outp;
         PackSrc ps;
         memset(&ps, 0, sizeof(ps));
-        ps.mode = mode; ps.src_k = src_k;
+        ps.mode = mode; ps.src_k = src_k; ps.hd = (int)c.head_dim;
         for (int i = 0; i < n; ++i) {
             ps.rows[i] = rows[i];
             if (loc) ps.p[i] = (const bf16*)srcs[i];
@@ -421,7 +421,7 @@ extern "C" int syn_model_load(const syn_model_desc* desc, const syn_weights* w, 
         {
             const void* srcs[3] = {w->wq[l], w->wk[l], w->wv[l]};
             const int rows[3] = {q_dim, kv_dim, kv_dim};
-            PACK_OR_FAIL(pack(srcs, rows, 3, 0, d, m->qkv_rows, &pk));
+            PACK_OR_FAIL(pack(srcs, rows, 3, 2, d, m->qkv_rows, &pk));
             m->wqkv.push_back(pk);
         }
         {
