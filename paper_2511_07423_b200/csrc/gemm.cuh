@@ -16,8 +16,8 @@
 //   EPI_SWIGLU : RMSNorm row scale, silu(gate) * up
 //   EPI_LMHEAD : RMSNorm row scale, optional logits, vocabulary argmax (packed 64-bit atomicMax)
 //   EPI_PLAIN  : fp32 store (test hook)
-// RMSNorm is folded as rmsnorm(x) g W = rstd(x) * ((x g) W): resid_norm_kernel writes bf16(x g) and
-// rstd per token; the consuming GEMM scales its accumulators by rstd.
+// The token operand of the QKV, gate/up and lm_head projections is the RMSNorm of the residual stream,
+// bf16(x * rstd * gain), written by resid_norm_kernel (prep_kernel for the first layer).
 #pragma once
 #include "ptx.cuh"
 
@@ -29,7 +29,6 @@ struct EpiParams {
     int mode;
     int T;  // valid tokens
     int N;  // valid output features (rows of W)
-    const float* rstd;  // [T] 1 / sqrt(mean(x^2) + eps) of the input rows (QKV, SWIGLU, LMHEAD)
     // PLAIN
     float* y;
     int ldy;
@@ -73,22 +72,24 @@ __host__ __device__ __forceinline__ int rope_tile_feature(int l, int hd) {   // 
     return (q / groups) * hd + 16 * (q % groups) + (ll & 15) + ((ll & 16) ? half : 0);
 }
 
-// Epilogue of one chunk straight from registers: r[j] = D[feature of this thread][token t0 + j],
-// j < 32; tokens j >= ncols are padding.  `m0` = first packed row of the tile, `quarter` = warp's
-// TMEM lane quarter.  comb: shared scratch of the warp's group for the vocabulary argmax
-// ([2][4][32] keys), ci = chunk counter of the group (buffer parity).
+// Epilogue of one 32-token chunk straight from registers: r[j] = D[feature of this thread][token
+// t0 + j]; tokens j >= ncols are padding.  `m0` = first packed row of the tile, `quarter` = warp's TMEM
+// lane quarter.  Warp shuffles, votes and reductions are never moved across stores by the compiler,
+// so every mode first runs all its warp-wide exchanges back to back (their latencies overlap) and
+// only then does the arithmetic and the stores.
 template <int MODE>
 __device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&r)[32], int m0, int t0, int ncols,
-                                           int split, int quarter, int lane, unsigned long long* comb, int ci, int grp) {
+                                           int split, int quarter, int lane) {
     const int l = quarter * 32 + lane;
     if (MODE == EPI_PLAIN || MODE == EPI_PART) {
         const int f = m0 + l;
-        float* base = MODE == EPI_PLAIN ? p.y + f : p.part + (size_t)split * p.part_stride + f;
+        float* base = (MODE == EPI_PLAIN ? p.y + f : p.part + (size_t)split * p.part_stride + f) +
+                      (size_t)t0 * (MODE == EPI_PLAIN ? (size_t)p.ldy : (size_t)p.d);
         const size_t ld = MODE == EPI_PLAIN ? (size_t)p.ldy : (size_t)p.d;
         if (f < p.N) {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-                if (j < ncols) base[(size_t)(t0 + j) * ld] = __uint_as_float(r[j]);
+                if (j < ncols) base[(size_t)j * ld] = __uint_as_float(r[j]);
         }
     } else if (MODE == EPI_QKV) {
         const int which = m0 < p.q_dim ? 0 : (m0 < p.q_dim + p.kv_dim ? 1 : 2);
@@ -97,81 +98,83 @@ __device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&
         const int half = p.hd >> 1;
         const int dim = fr & (p.hd - 1);
         const bool lo = dim < half;
-        const float2* cs = p.rope + (lo ? dim : dim - half);
-        const int kvh = fr / p.hd;
-        // per-token values of the chunk: lane j fetches those of token j, a shuffle hands them round
-        const float rs_mine = lane < ncols ? __ldg(p.rstd + t0 + lane) : 0.f;
-        const int slot_mine = (which > 0 && lane < ncols) ? __ldg(p.slot + t0 + lane) : 0;
-        __nv_bfloat16* const qdst = p.q + fr;
-        __nv_bfloat16* const kvdst = p.pool + ((size_t)kvh * 2 + (which > 0 ? which - 1 : 0)) * 16 * p.hd + dim;
+        float o[32];   // rotate-half RoPE: the partner dimension is 16 lanes away
+        if (which < 2) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __shfl_xor_sync(0xFFFFFFFFu, __uint_as_float(r[j]), 16);
+        }
+        const float2* cs = p.rope + (size_t)t0 * half + (lo ? dim : dim - half);
+        const int* slot = p.slot + t0;
+        __nv_bfloat16* const qdst = p.q + (size_t)t0 * p.q_dim + fr;
+        __nv_bfloat16* const kvdst = p.pool + ((size_t)(fr / p.hd) * 2 + (which > 0 ? which - 1 : 0)) * 16 * p.hd + dim;
         const size_t page_stride = (size_t)p.n_kv_heads * 2 * 16 * p.hd;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const int t = t0 + j;
-            const bool live = j < ncols;
-            float a = __uint_as_float(r[j]) * __shfl_sync(0xFFFFFFFFu, rs_mine, j);
-            if (which < 2) {   // rotate-half RoPE: the partner dimension is 16 lanes away
-                const float o = __shfl_xor_sync(0xFFFFFFFFu, a, 16);
-                const float2 w = live ? __ldg(cs + (size_t)t * half) : make_float2(0.f, 0.f);
-                a = lo ? (a * w.x - o * w.y) : (a * w.x + o * w.y);
+        for (int j0 = 0; j0 < 32; j0 += 16) {
+            // the table entries and slots of sixteen tokens are fetched together, ahead of any store
+            // (loads are not moved above stores that might alias them)
+            float2 w[16];
+            int sl[16];
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) {
+                w[jj] = (which < 2 && j0 + jj < ncols) ? __ldg(cs + (size_t)(j0 + jj) * half) : make_float2(1.f, 0.f);
+                sl[jj] = (which > 0 && j0 + jj < ncols) ? __ldg(slot + j0 + jj) : 0;   // page * 16 + row; same address in all lanes
             }
-            const int s = __shfl_sync(0xFFFFFFFFu, slot_mine, j);   // page * 16 + row (pages hold 16 tokens)
-            if (live) {
-                if (which == 0) qdst[(size_t)t * p.q_dim] = __float2bfloat16(a);
-                else kvdst[(size_t)(s >> 4) * page_stride + (size_t)(s & 15) * p.hd] = __float2bfloat16(a);
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) {
+                const int j = j0 + jj;
+                if (j < ncols) {
+                    float a = __uint_as_float(r[j]);
+                    if (which < 2) a = lo ? (a * w[jj].x - o[j] * w[jj].y) : (a * w[jj].x + o[j] * w[jj].y);
+                    if (which == 0) qdst[(size_t)j * p.q_dim] = __float2bfloat16(a);
+                    else kvdst[(size_t)(sl[jj] >> 4) * page_stride + (size_t)(sl[jj] & 15) * p.hd] = __float2bfloat16(a);
+                }
             }
         }
     } else if (MODE == EPI_SWIGLU) {
-        const int f = (m0 >> 1) + 16 * quarter + (lane & 15);   // gate/up feature of this lane pair
-        const float rs_mine = lane < ncols ? __ldg(p.rstd + t0 + lane) : 0.f;
+        // Two tokens per step: the lower half-warp finishes token j, the upper one token j + 1, so all
+        // lanes evaluate silu and one store covers two rows of 16 features.
+        // Lanes 0..15 hold gate, lanes 16..31 the matching up features.
+        const bool up_half = lane >= 16;
+        float got[16];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const int t = t0 + j;
-            const bool live = j < ncols;
-            const float a = __uint_as_float(r[j]) * __shfl_sync(0xFFFFFFFFu, rs_mine, j);
-            const float u = __shfl_xor_sync(0xFFFFFFFFu, a, 16);   // lanes 0..15 receive "up"
-            if (live && lane < 16) p.act[(size_t)t * p.f_pad + f] = __float2bfloat16(__fdividef(a, 1.0f + __expf(-a)) * u);
+        for (int k = 0; k < 16; ++k)   // each half-warp sends what the other one needs
+            got[k] = __shfl_xor_sync(0xFFFFFFFFu, __uint_as_float(up_half ? r[2 * k] : r[2 * k + 1]), 16);
+        __nv_bfloat16* const dst = p.act + (size_t)(t0 + (up_half ? 1 : 0)) * p.f_pad + (m0 >> 1) + 16 * quarter + (lane & 15);
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const float gate = up_half ? got[k] : __uint_as_float(r[2 * k]);       // upper half: gate of token 2k + 1
+            const float upv = up_half ? __uint_as_float(r[2 * k + 1]) : got[k];    // lower half: up of token 2k
+            const float h = __fdividef(gate, 1.0f + __expf(-gate)) * upv;
+            if (2 * k + (up_half ? 1 : 0) < ncols) dst[(size_t)(2 * k) * p.f_pad] = __float2bfloat16(h);
         }
-    } else {  // EPI_LMHEAD
+    } else {  // EPI_LMHEAD: the norm scale is positive, so the argmax needs nothing but the accumulators
         const int f = m0 + l;
         const bool valid = f < p.vocab;
+        if (p.logits && valid) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (j < ncols) p.logits[(size_t)(t0 + j) * p.vocab + f] = __uint_as_float(r[j]);
+        }
+        uint32_t mx[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) mx[j] = __reduce_max_sync(0xFFFFFFFFu, valid ? orderable_f32(__uint_as_float(r[j])) : 0u);
         unsigned long long mine = 0ull;   // lane j keeps the warp's best of token j
-        const float rs_mine = lane < ncols ? __ldg(p.rstd + t0 + lane) : 0.f;
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-            const int t = t0 + j;
-            const bool live = j < ncols;
-            const float a = __uint_as_float(r[j]) * __shfl_sync(0xFFFFFFFFu, rs_mine, j);
-            if (p.logits && live && valid) p.logits[(size_t)t * p.vocab + f] = a;
-            const uint32_t key = valid ? orderable_f32(a) : 0u;
-            const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
-            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, key == mx && valid);
-            if (lane == j) mine = hit ? pack_argmax_key(mx, m0 + quarter * 32 + (__ffs(hit) - 1)) : 0ull;
+            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, valid && orderable_f32(__uint_as_float(r[j])) == mx[j]);
+            if (lane == j && hit) mine = pack_argmax_key(mx[j], m0 + quarter * 32 + (__ffs(hit) - 1));
         }
-        // combine the four quarter-warps of the tile, then one atomic per token
-        unsigned long long* buf = comb + (ci & 1) * 128;
-        buf[quarter * 32 + lane] = mine;
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
-        if (lane < 8) {
-            const int j = quarter * 8 + lane;
-            unsigned long long b = buf[j];
-#pragma unroll
-            for (int q2 = 1; q2 < 4; ++q2) {
-                const unsigned long long o = buf[q2 * 32 + j];
-                b = o > b ? o : b;
-            }
-            if (j < ncols && b) atomicMax(p.best + t0 + j, b);
-        }
+        if (lane < ncols && mine) atomicMax(p.best + t0 + lane, mine);
     }
 }
 
 // Residual update after a split-K projection, in a fixed order: x += part[0] + part[1] + ...;
-// then the next GEMM's operand bf16(x * gain) and the row's RMSNorm statistic.  One CTA per token.
+// then the next GEMM's operand, the RMSNorm of the row: bf16(x * rstd * gain).  One CTA per token.
 __global__ void __launch_bounds__(256)
 resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, size_t part_stride, int splits,
-                  const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ xn, float* __restrict__ rstd,
-                  int d, float inv_d, float eps) {
+                  const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ xn, int d, float inv_d, float eps) {
     __shared__ float red[8];
+    __shared__ float rstd_s;
     const int t = blockIdx.x;
     float ss = 0.f;
     pdl_launch_dependents();
@@ -183,12 +186,6 @@ resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, size_t 
             v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
         }
         *reinterpret_cast<float4*>(x + (size_t)t * d + f) = v;
-        const uint2 gb = *reinterpret_cast<const uint2*>(gain + f);
-        const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gb.x);
-        const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gb.y);
-        *reinterpret_cast<uint2*>(xn + (size_t)t * d + f) =
-            make_uint2(pack_bf16(v.x * __low2float(g01), v.y * __high2float(g01)),
-                       pack_bf16(v.z * __low2float(g23), v.w * __high2float(g23)));
         ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
 #pragma unroll
@@ -198,7 +195,18 @@ resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, size_t 
     if (threadIdx.x == 0) {
         float tot = 0.f;
         for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
-        rstd[t] = rsqrtf(tot * inv_d + eps);
+        rstd_s = rsqrtf(tot * inv_d + eps);
+    }
+    __syncthreads();
+    const float rs = rstd_s;
+    for (int f = threadIdx.x * 4; f < d; f += blockDim.x * 4) {   // each thread re-reads what it wrote
+        const float4 v = *reinterpret_cast<const float4*>(x + (size_t)t * d + f);
+        const uint2 gb = *reinterpret_cast<const uint2*>(gain + f);
+        const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gb.x);
+        const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gb.y);
+        *reinterpret_cast<uint2*>(xn + (size_t)t * d + f) =
+            make_uint2(pack_bf16(v.x * rs * __low2float(g01), v.y * rs * __high2float(g01)),
+                       pack_bf16(v.z * rs * __low2float(g23), v.w * rs * __high2float(g23)));
     }
 }
 
@@ -453,10 +461,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
         const int e = warp - 2;
         const int grp = e >> 2;               // group 0/1 takes alternate 32-token chunks
         const int quarter = warp & 3;         // TMEM lane quarter this warp may read
-        unsigned long long* cbuf = comb + grp * 2 * 128;
         bool ok = true;
         GemmWork w;
-        int nci = 0;                          // chunks this group has handled (argmax scratch parity)
         pdl_wait();   // the epilogues read per-token statistics and write buffers of earlier kernels
         for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
             const int n0 = w.tt * g.TN;
@@ -466,7 +472,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
             if (!ok) break;
             tc_fence_after();
             const int total_chunks = (w.mt_hi - w.mt_lo) * nchunks;
-            for (int ci = grp; ci < total_chunks; ci += 2, ++nci) {
+            for (int ci = grp; ci < total_chunks; ci += 2) {
                 const int mt = w.mt_lo + ci / nchunks, c = ci % nchunks;
                 const int m0 = w.pair * 256 + mt * 128;
                 uint32_t r[32];
@@ -476,14 +482,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                     tc_fence_before();
                     if (lane == 0) mbar_arrive(acce_bar);
                 }
-                const int t0 = n0 + c * 32, ncols = min(32, n_valid - c * 32);
-                if (m0 < p.N) {   // uniform over the group: the vocabulary argmax meets at a named barrier
+                const int tc0 = n0 + c * 32, ncols = min(32, n_valid - c * 32);
+                if (m0 < p.N) {
                     switch (p.mode) {
-                        case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
-                        case EPI_QKV: epi_direct<EPI_QKV>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
-                        case EPI_PART: epi_direct<EPI_PART>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
-                        case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
-                        default: epi_direct<EPI_LMHEAD>(p, r, m0, t0, ncols, w.split, quarter, lane, cbuf, nci, grp); break;
+                        case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                        case EPI_QKV: epi_direct<EPI_QKV>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                        case EPI_PART: epi_direct<EPI_PART>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                        case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                        default: epi_direct<EPI_LMHEAD>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
                     }
                 }
             }

@@ -56,14 +56,15 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 
 // ------------------------------------------------------------------------------------------ small kernels
 
-// Token embedding (paper Sec. 4.5: the flattened batch enters the transformer), first layer's
-// GEMM operand bf16(x * gain) with the row's RMSNorm statistic, RoPE table, argmax reset.
+// Token embedding (paper Sec. 4.5: the flattened batch enters the transformer), the first layer's
+// GEMM operand bf16(rmsnorm(x) * gain), RoPE table, argmax reset.
 __global__ void __launch_bounds__(256)
 prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens, const int* __restrict__ pos,
             const bf16* __restrict__ gain, const double* __restrict__ inv_freq, float* __restrict__ x,
-            bf16* __restrict__ xn, float* __restrict__ rstd, float2* __restrict__ rope,
-            unsigned long long* __restrict__ best, int d, int half, float inv_d, float eps) {
+            bf16* __restrict__ xn, float2* __restrict__ rope, unsigned long long* __restrict__ best, int d, int half,
+            float inv_d, float eps) {
     __shared__ float red[8];
+    __shared__ float rstd_s;
     const int t = blockIdx.x;
     pdl_launch_dependents();
     pdl_wait();
@@ -72,7 +73,6 @@ prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens, cons
     for (int f = threadIdx.x; f < d; f += blockDim.x) {
         const float v = __bfloat162float(e[f]);
         x[(size_t)t * d + f] = v;
-        xn[(size_t)t * d + f] = __float2bfloat16(v * __bfloat162float(gain[f]));
         ss += v * v;
     }
 #pragma unroll
@@ -82,9 +82,13 @@ prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens, cons
     if (threadIdx.x == 0) {
         float tot = 0.f;
         for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
-        rstd[t] = rsqrtf(tot * inv_d + eps);
+        rstd_s = rsqrtf(tot * inv_d + eps);
         best[t] = 0ull;
     }
+    __syncthreads();
+    const float rs = rstd_s;
+    for (int f = threadIdx.x; f < d; f += blockDim.x)
+        xn[(size_t)t * d + f] = __float2bfloat16(__bfloat162float(e[f]) * rs * __bfloat162float(gain[f]));
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
         double sn, cs;
         sincos((double)pos[t] * inv_freq[i], &sn, &cs);
@@ -166,7 +170,7 @@ struct syn_model {
     int* status_dev = nullptr;
     // workspace (grow-only)
     int t_cap = 0;
-    float *x = nullptr, *rstd = nullptr, *part = nullptr;   // residual stream, 1/rms per token, split-K partials
+    float *x = nullptr, *part = nullptr;   // residual stream, split-K partials
     bf16 *xn = nullptr, *q = nullptr, *attn = nullptr, *act = nullptr;
     float2* rope = nullptr;
     unsigned long long* best = nullptr;
@@ -225,9 +229,9 @@ struct syn_plan {
 };
 
 static void free_workspace(syn_model* m) {
-    cudaFree(m->x); cudaFree(m->rstd); cudaFree(m->part); cudaFree(m->xn); cudaFree(m->q); cudaFree(m->attn); cudaFree(m->act);
+    cudaFree(m->x); cudaFree(m->part); cudaFree(m->xn); cudaFree(m->q); cudaFree(m->attn); cudaFree(m->act);
     cudaFree(m->rope); cudaFree(m->best);
-    m->x = m->rstd = m->part = nullptr; m->xn = m->q = m->attn = m->act = nullptr; m->rope = nullptr; m->best = nullptr;
+    m->x = m->part = nullptr; m->xn = m->q = m->attn = m->act = nullptr; m->rope = nullptr; m->best = nullptr;
     m->t_cap = 0;
 }
 
@@ -238,7 +242,6 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
         free_workspace(m);
         const int cap = (T + 255) / 256 * 256;
         CU_OK(cudaMalloc(&m->x, (size_t)cap * c.d_model * 4));
-        CU_OK(cudaMalloc(&m->rstd, (size_t)cap * 4));
         CU_OK(cudaMalloc(&m->part, (size_t)GEMM_MAX_SPLITS * cap * c.d_model * 4));
         CU_OK(cudaMalloc(&m->xn, (size_t)cap * c.d_model * 2));
         CU_OK(cudaMalloc(&m->q, (size_t)cap * q_dim * 2));
@@ -889,18 +892,17 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
     {
         ProfScope prof(m, 0, st);
         if (launch_pdl(prep_kernel, dim3(T), dim3(256), 0, st, m->embed, tokens, p->d<int>(p->o_pos), m->norm1[0], m->inv_freq,
-                       m->x, m->xn, m->rstd, m->rope, m->best, d, (int)(c.head_dim / 2), inv_d, c.rms_eps) != cudaSuccess)
+                       m->x, m->xn, m->rope, m->best, d, (int)(c.head_dim / 2), inv_d, c.rms_eps) != cudaSuccess)
             return SYN_E_CUDA;
     }
     EpiParams base;
     memset(&base, 0, sizeof(base));
     base.T = T;
-    base.rstd = m->rstd;
     const size_t part_stride = (size_t)m->t_cap * d;
     int r, splits = 1;
     auto resid = [&](int cls, const bf16* gain) -> int {
         ProfScope prof(m, cls, st);
-        return launch_pdl(resid_norm_kernel, dim3(T), dim3(256), 0, st, m->x, m->part, part_stride, splits, gain, m->xn, m->rstd, d,
+        return launch_pdl(resid_norm_kernel, dim3(T), dim3(256), 0, st, m->x, m->part, part_stride, splits, gain, m->xn, d,
                           inv_d, c.rms_eps) == cudaSuccess ? SYN_OK : SYN_E_CUDA;
     };
     for (uint32_t l = 0; l < c.n_layers; ++l) {
