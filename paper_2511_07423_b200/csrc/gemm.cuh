@@ -72,23 +72,23 @@ __host__ __device__ __forceinline__ int rope_tile_feature(int l, int hd) {   // 
     return (q / groups) * hd + 16 * (q % groups) + (ll & 15) + ((ll & 16) ? half : 0);
 }
 
-// Epilogue of one 32-token chunk straight from registers: r[j] = D[feature of this thread][token
+// Epilogue of one 16-token chunk straight from registers: r[j] = D[feature of this thread][token
 // t0 + j]; tokens j >= ncols are padding.  `m0` = first packed row of the tile, `quarter` = warp's TMEM
-// lane quarter.  Warp shuffles, votes and reductions are never moved across stores by the compiler,
-// so every mode first runs all its warp-wide exchanges back to back (their latencies overlap) and
-// only then does the arithmetic and the stores.
+// lane quarter.  Warp shuffles, votes and reductions are never moved across stores by the compiler, and
+// loads not above stores that might alias them, so every mode first runs all its warp-wide exchanges
+// and loads back to back (their latencies overlap) and only then does the arithmetic and the stores.
+constexpr int EPI_COLS = 16;
 template <int MODE>
-__device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&r)[32], int m0, int t0, int ncols,
+__device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&r)[EPI_COLS], int m0, int t0, int ncols,
                                            int split, int quarter, int lane) {
     const int l = quarter * 32 + lane;
     if (MODE == EPI_PLAIN || MODE == EPI_PART) {
         const int f = m0 + l;
-        float* base = (MODE == EPI_PLAIN ? p.y + f : p.part + (size_t)split * p.part_stride + f) +
-                      (size_t)t0 * (MODE == EPI_PLAIN ? (size_t)p.ldy : (size_t)p.d);
         const size_t ld = MODE == EPI_PLAIN ? (size_t)p.ldy : (size_t)p.d;
+        float* base = (MODE == EPI_PLAIN ? p.y + f : p.part + (size_t)split * p.part_stride + f) + (size_t)t0 * ld;
         if (f < p.N) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
+            for (int j = 0; j < EPI_COLS; ++j)
                 if (j < ncols) base[(size_t)j * ld] = __uint_as_float(r[j]);
         }
     } else if (MODE == EPI_QKV) {
@@ -98,36 +98,27 @@ __device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&
         const int half = p.hd >> 1;
         const int dim = fr & (p.hd - 1);
         const bool lo = dim < half;
-        float o[32];   // rotate-half RoPE: the partner dimension is 16 lanes away
-        if (which < 2) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = __shfl_xor_sync(0xFFFFFFFFu, __uint_as_float(r[j]), 16);
-        }
         const float2* cs = p.rope + (size_t)t0 * half + (lo ? dim : dim - half);
         const int* slot = p.slot + t0;
+        float o[EPI_COLS];   // rotate-half RoPE: the partner dimension is 16 lanes away
+        float2 w[EPI_COLS];
+        int sl[EPI_COLS];
+#pragma unroll
+        for (int j = 0; j < EPI_COLS; ++j) {
+            o[j] = which < 2 ? __shfl_xor_sync(0xFFFFFFFFu, __uint_as_float(r[j]), 16) : 0.f;
+            w[j] = (which < 2 && j < ncols) ? __ldg(cs + (size_t)j * half) : make_float2(1.f, 0.f);
+            sl[j] = (which > 0 && j < ncols) ? __ldg(slot + j) : 0;   // page * 16 + row; same address in all lanes
+        }
         __nv_bfloat16* const qdst = p.q + (size_t)t0 * p.q_dim + fr;
         __nv_bfloat16* const kvdst = p.pool + ((size_t)(fr / p.hd) * 2 + (which > 0 ? which - 1 : 0)) * 16 * p.hd + dim;
         const size_t page_stride = (size_t)p.n_kv_heads * 2 * 16 * p.hd;
 #pragma unroll
-        for (int j0 = 0; j0 < 32; j0 += 16) {
-            // the table entries and slots of sixteen tokens are fetched together, ahead of any store
-            // (loads are not moved above stores that might alias them)
-            float2 w[16];
-            int sl[16];
-#pragma unroll
-            for (int jj = 0; jj < 16; ++jj) {
-                w[jj] = (which < 2 && j0 + jj < ncols) ? __ldg(cs + (size_t)(j0 + jj) * half) : make_float2(1.f, 0.f);
-                sl[jj] = (which > 0 && j0 + jj < ncols) ? __ldg(slot + j0 + jj) : 0;   // page * 16 + row; same address in all lanes
-            }
-#pragma unroll
-            for (int jj = 0; jj < 16; ++jj) {
-                const int j = j0 + jj;
-                if (j < ncols) {
-                    float a = __uint_as_float(r[j]);
-                    if (which < 2) a = lo ? (a * w[jj].x - o[j] * w[jj].y) : (a * w[jj].x + o[j] * w[jj].y);
-                    if (which == 0) qdst[(size_t)j * p.q_dim] = __float2bfloat16(a);
-                    else kvdst[(size_t)(sl[jj] >> 4) * page_stride + (size_t)(sl[jj] & 15) * p.hd] = __float2bfloat16(a);
-                }
+        for (int j = 0; j < EPI_COLS; ++j) {
+            if (j < ncols) {
+                float a = __uint_as_float(r[j]);
+                if (which < 2) a = lo ? (a * w[j].x - o[j] * w[j].y) : (a * w[j].x + o[j] * w[j].y);
+                if (which == 0) qdst[(size_t)j * p.q_dim] = __float2bfloat16(a);
+                else kvdst[(size_t)(sl[j] >> 4) * page_stride + (size_t)(sl[j] & 15) * p.hd] = __float2bfloat16(a);
             }
         }
     } else if (MODE == EPI_SWIGLU) {
@@ -135,13 +126,13 @@ __device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&
         // lanes evaluate silu and one store covers two rows of 16 features.
         // Lanes 0..15 hold gate, lanes 16..31 the matching up features.
         const bool up_half = lane >= 16;
-        float got[16];
+        float got[EPI_COLS / 2];
 #pragma unroll
-        for (int k = 0; k < 16; ++k)   // each half-warp sends what the other one needs
+        for (int k = 0; k < EPI_COLS / 2; ++k)   // each half-warp sends what the other one needs
             got[k] = __shfl_xor_sync(0xFFFFFFFFu, __uint_as_float(up_half ? r[2 * k] : r[2 * k + 1]), 16);
         __nv_bfloat16* const dst = p.act + (size_t)(t0 + (up_half ? 1 : 0)) * p.f_pad + (m0 >> 1) + 16 * quarter + (lane & 15);
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
+        for (int k = 0; k < EPI_COLS / 2; ++k) {
             const float gate = up_half ? got[k] : __uint_as_float(r[2 * k]);       // upper half: gate of token 2k + 1
             const float upv = up_half ? __uint_as_float(r[2 * k + 1]) : got[k];    // lower half: up of token 2k
             const float h = __fdividef(gate, 1.0f + __expf(-gate)) * upv;
@@ -152,15 +143,16 @@ __device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&
         const bool valid = f < p.vocab;
         if (p.logits && valid) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
+            for (int j = 0; j < EPI_COLS; ++j)
                 if (j < ncols) p.logits[(size_t)(t0 + j) * p.vocab + f] = __uint_as_float(r[j]);
         }
-        uint32_t mx[32];
+        uint32_t mx[EPI_COLS];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) mx[j] = __reduce_max_sync(0xFFFFFFFFu, valid ? orderable_f32(__uint_as_float(r[j])) : 0u);
+        for (int j = 0; j < EPI_COLS; ++j)
+            mx[j] = __reduce_max_sync(0xFFFFFFFFu, valid ? orderable_f32(__uint_as_float(r[j])) : 0u);
         unsigned long long mine = 0ull;   // lane j keeps the warp's best of token j
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
+        for (int j = 0; j < EPI_COLS; ++j) {
             const uint32_t hit = __ballot_sync(0xFFFFFFFFu, valid && orderable_f32(__uint_as_float(r[j])) == mx[j]);
             if (lane == j && hit) mine = pack_argmax_key(mx[j], m0 + quarter * 32 + (__ffs(hit) - 1));
         }
@@ -263,9 +255,10 @@ __global__ void pack_weight_kernel(PackSrc src, __nv_bfloat16* __restrict__ out,
 }
 
 // ------------------------------------------------------------------------------------------
-// The kernel.  One persistent CTA per SM, 320 threads: warp 0 = producer (bulk copy of the weight
-// tiles + L2 prefetch + TMA boxes of the token tile), warp 1 = TMEM owner and MMA issuer,
-// warps 2..9 = epilogue (two groups of four; a group covers the four TMEM lane quarters).
+// The kernel.  One persistent CTA per SM, 576 threads: warp 0 = producer (bulk copy of the weight
+// tiles + TMA boxes of the token tile), warp 1 = TMEM owner and MMA issuer, warps 2..17 = epilogue
+// (four groups of four; a group covers the four TMEM lane quarters; draining TMEM is limited per
+// warp, so many warps share it).
 // ------------------------------------------------------------------------------------------
 constexpr int GEMM_BK = 64;                        // bf16 elements per k-block = one 128-byte swizzle row
 constexpr int GEMM_TILE_BYTES = 128 * GEMM_BK * 2; // 16 KB: one 128-feature tile of one k-block
@@ -273,7 +266,8 @@ constexpr int GEMM_A_BYTES = 2 * GEMM_TILE_BYTES;  // stage room for a pair
 constexpr int GEMM_BOX_ROWS = 32;                  // token rows per B box
 constexpr int GEMM_BOX_BYTES = GEMM_BOX_ROWS * GEMM_BK * 2;
 constexpr int GEMM_MAX_STAGES = 8;
-constexpr int GEMM_THREADS = 320;
+constexpr int GEMM_EPI_WARPS = 16;               // four groups of four (one warp per TMEM lane quarter)
+constexpr int GEMM_THREADS = (2 + GEMM_EPI_WARPS) * 32;
 constexpr int GEMM_SMEM_MAX = 232448;
 constexpr int GEMM_PREFETCH_KB = 12;               // L2 prefetch distance in k-blocks
 
@@ -378,7 +372,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
             mbar_init(&empty_bar[s], 1);
         }
         mbar_init(accf_bar, 1);
-        mbar_init(acce_bar, 8);
+        mbar_init(acce_bar, GEMM_EPI_WARPS);
         mbar_fence_init();
     }
     if (warp == 1) {
@@ -459,30 +453,31 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
     } else {
         // ------------------------------------------------------------ epilogue
         const int e = warp - 2;
-        const int grp = e >> 2;               // group 0/1 takes alternate 32-token chunks
+        const int grp = e >> 2;               // the groups take the 16-token chunks round robin
+        constexpr int NGRP = GEMM_EPI_WARPS / 4;
         const int quarter = warp & 3;         // TMEM lane quarter this warp may read
         bool ok = true;
         GemmWork w;
-        pdl_wait();   // the epilogues read per-token statistics and write buffers of earlier kernels
+        pdl_wait();   // the epilogues write buffers that earlier kernels may still read
         for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
             const int n0 = w.tt * g.TN;
             const int n_valid = min(g.TN, p.T - n0);
-            const int nchunks = (n_valid + 31) >> 5;
+            const int nchunks = (n_valid + EPI_COLS - 1) / EPI_COLS;
             ok = mbar_wait(accf_bar, i & 1, g.status);
             if (!ok) break;
             tc_fence_after();
             const int total_chunks = (w.mt_hi - w.mt_lo) * nchunks;
-            for (int ci = grp; ci < total_chunks; ci += 2) {
+            for (int ci = grp; ci < total_chunks; ci += NGRP) {
                 const int mt = w.mt_lo + ci / nchunks, c = ci % nchunks;
                 const int m0 = w.pair * 256 + mt * 128;
-                uint32_t r[32];
-                tmem_ld32(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), r);
+                uint32_t r[EPI_COLS];
+                tmem_ld16(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * EPI_COLS), r);
                 tmem_ld_wait();
-                if (ci + 2 >= total_chunks) {   // last TMEM read of this warp for this item
+                if (ci + NGRP >= total_chunks) {   // last TMEM read of this warp for this item
                     tc_fence_before();
                     if (lane == 0) mbar_arrive(acce_bar);
                 }
-                const int tc0 = n0 + c * 32, ncols = min(32, n_valid - c * 32);
+                const int tc0 = n0 + c * EPI_COLS, ncols = min(EPI_COLS, n_valid - c * EPI_COLS);
                 if (m0 < p.N) {
                     switch (p.mode) {
                         case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
