@@ -19,7 +19,8 @@ from . import build as _build
 class _Desc(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("d_ffn", C.c_int32),
-                ("vocab", C.c_int32), ("rope_base", C.c_double), ("rms_eps", C.c_double)]
+                ("vocab", C.c_int32), ("rope_base", C.c_double), ("rms_eps", C.c_double),
+                ("bf16_operands", C.c_int32)]
 
 
 class _LayerW(C.Structure):
@@ -72,20 +73,24 @@ class Oracle:
             _build.build()
             lib = C.CDLL(_build.lib_path(f32))
             lib.orc_real_bytes.restype = C.c_int
-            for fn in ("orc_embed", "orc_rmsnorm", "orc_linear", "orc_rope", "orc_kv_write", "orc_attention",
+            for fn in ("orc_bf16_round_array", "orc_embed", "orc_rmsnorm", "orc_linear", "orc_rope", "orc_kv_write", "orc_attention",
                        "orc_layer", "orc_logits", "orc_verify", "orc_slot"):
                 getattr(lib, fn).restype = None
             cls._libs[f32] = lib
         return cls._libs[f32]
 
-    def __init__(self, shape, page_size: int = 16, f32: bool = False):
+    def __init__(self, shape, page_size: int = 16, f32: bool = False, bf16_operands: bool = False):
+        """bf16_operands: model the network as a bf16 model (bf16 weights and activations, wide
+        accumulation): every activation entering a matrix product or the KV cache is rounded to bf16.
+        False keeps every intermediate in double (or float): the plain mathematical definition."""
         self.lib = self._load(f32)
         self.real = np.float32 if f32 else np.float64
         assert self.lib.orc_real_bytes() == np.dtype(self.real).itemsize
         self.shape = shape
         self.P = page_size
         self.desc = _Desc(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
-                          shape.d_ffn, shape.vocab, float(shape.rope_base), float(shape.rms_eps))
+                          shape.d_ffn, shape.vocab, float(shape.rope_base), float(shape.rms_eps),
+                          1 if bf16_operands else 0)
 
     # ------------------------------------------------------------------ storage
     def new_pool(self, n_pages: int) -> List[np.ndarray]:
@@ -106,6 +111,12 @@ class Oracle:
         pool_layer[pages, 1, heads, rows, :] = v
 
     # ------------------------------------------------------------------ single ops (exposed for pins)
+    def bf16_round(self, a) -> np.ndarray:
+        a = np.ascontiguousarray(a, dtype=self.real).ravel()
+        out = np.empty_like(a)
+        self.lib.orc_bf16_round_array(_p(a), _p(out), C.c_int(a.size))
+        return out
+
     def embed(self, E, tokens) -> np.ndarray:
         tok = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
         x = np.empty((len(tok), self.shape.d_model), dtype=self.real)

@@ -54,6 +54,11 @@ typedef double real;
 typedef struct {
     int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
     double rope_base, rms_eps;
+    int32_t bf16_operands; /* 0: every intermediate stays in `real`.  1: the model as a bf16 model
+                              ("bf16 weights and activations, fp32 accumulation"): every activation
+                              that enters a matrix product or the KV cache is first rounded to bf16
+                              (normalised hidden states, rotated q and k, v, the attention output,
+                              the SwiGLU output); sums, softmax and the residual stream stay wide. */
 } orc_desc;
 
 int orc_real_bytes(void) { return ORC_REAL_BYTES; }
@@ -63,6 +68,24 @@ static inline real bf16_widen(uint16_t b) {
     float f;
     memcpy(&f, &u, 4);
     return (real)f;
+}
+
+/* round to the nearest bf16 (ties to even), returned in `real` */
+static inline real bf16_round(real v) {
+    float f = (float)v;
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7F800000u) != 0x7F800000u) u += 0x7FFFu + ((u >> 16) & 1u);
+    u &= 0xFFFF0000u;
+    memcpy(&f, &u, 4);
+    return (real)f;
+}
+static void round_all(real *a, size_t n) {
+    for (size_t i = 0; i < n; ++i) a[i] = bf16_round(a[i]);
+}
+
+void orc_bf16_round_array(const real *in, real *out, int n) {
+    for (int i = 0; i < n; ++i) out[i] = bf16_round(in[i]);
 }
 
 /* x_j = E[c_j]  (token embedding lookup) */
@@ -191,26 +214,36 @@ void orc_layer(const orc_desc *m, const orc_layer_weights *w, real *x, real *poo
     real *g = (real *)malloc(sizeof(real) * (size_t)n * f);
     real *u = (real *)malloc(sizeof(real) * (size_t)n * f);
 
+    const int rb = m->bf16_operands;
     orc_rmsnorm(x, w->norm1, n, d, m->rms_eps, h);
+    if (rb) round_all(h, (size_t)n * d);
     orc_linear(h, w->wq, n, d, qd, q);
     orc_linear(h, w->wk, n, d, kd, k);
     orc_linear(h, w->wv, n, d, kd, v);
     for (int j = 0; j < n; ++j) {
         orc_rope(q + (size_t)j * qd, m->n_q_heads, m->head_dim, ctx + j, m->rope_base);
         orc_rope(k + (size_t)j * kd, m->n_kv_heads, m->head_dim, ctx + j, m->rope_base);
+        if (rb) {
+            round_all(q + (size_t)j * qd, (size_t)qd);
+            round_all(k + (size_t)j * kd, (size_t)kd);
+            round_all(v + (size_t)j * kd, (size_t)kd);
+        }
         orc_kv_write(m, pool, page_table, P, ctx + j, k + (size_t)j * kd, v + (size_t)j * kd);
     }
     orc_attention(m, q, pool, page_table, P, ctx, n, a);
+    if (rb) round_all(a, (size_t)n * qd);
     orc_linear(a, w->wo, n, qd, d, o);
     for (size_t i = 0; i < (size_t)n * d; ++i) x[i] += o[i];
 
     orc_rmsnorm(x, w->norm2, n, d, m->rms_eps, h);
+    if (rb) round_all(h, (size_t)n * d);
     orc_linear(h, w->wg, n, d, f, g);
     orc_linear(h, w->wu, n, d, f, u);
     for (size_t i = 0; i < (size_t)n * f; ++i) {
         real z = g[i];
         g[i] = z / ((real)1 + (real)exp((double)-z)) * u[i]; /* silu(gate) * up */
     }
+    if (rb) round_all(g, (size_t)n * f);
     orc_linear(g, w->wd, n, f, d, o);
     for (size_t i = 0; i < (size_t)n * d; ++i) x[i] += o[i];
 
@@ -225,6 +258,7 @@ void orc_logits(const orc_desc *m, const uint16_t *final_norm, const uint16_t *l
     real *h = (real *)malloc(sizeof(real) * (size_t)n * d);
     real *l = logits ? logits : (real *)malloc(sizeof(real) * (size_t)n * V);
     orc_rmsnorm(x, final_norm, n, d, m->rms_eps, h);
+    if (m->bf16_operands) round_all(h, (size_t)n * d);
     orc_linear(h, lm_head, n, d, V, l);
     for (int j = 0; j < n; ++j) {
         const real *r = l + (size_t)j * V;

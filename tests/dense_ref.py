@@ -29,28 +29,36 @@ def rope_all(v, base):
     return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
 
 
-def dense_forward(shape, glob, layers, tokens):
-    """Returns logits [S, V] and the per-layer post-RoPE K and V ([S, Hkv, hd])."""
+def _bf16(a):
+    """Round a float64 array to bf16 (nearest even) with torch's conversion, back to float64."""
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def dense_forward(shape, glob, layers, tokens, bf16_operands=False):
+    """Returns logits [S, V] and the per-layer post-RoPE K and V ([S, Hkv, hd]).
+    bf16_operands: round every activation that enters a matrix product (or would be cached) to bf16."""
+    rnd = _bf16 if bf16_operands else (lambda a: a)
     S = len(tokens)
     Hq, Hkv, hd = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
     x = f64(glob["embed"])[np.asarray(tokens)]
     mask = np.tril(np.ones((S, S), dtype=bool))
     kvs = []
     for w in layers:
-        h = rms(x, f64(w["norm1"]), shape.rms_eps)
-        q = rope_all((h @ f64(w["wq"]).T).reshape(S, Hq, hd), shape.rope_base)
-        k = rope_all((h @ f64(w["wk"]).T).reshape(S, Hkv, hd), shape.rope_base)
-        v = (h @ f64(w["wv"]).T).reshape(S, Hkv, hd)
+        h = rnd(rms(x, f64(w["norm1"]), shape.rms_eps))
+        q = rnd(rope_all((h @ f64(w["wq"]).T).reshape(S, Hq, hd), shape.rope_base))
+        k = rnd(rope_all((h @ f64(w["wk"]).T).reshape(S, Hkv, hd), shape.rope_base))
+        v = rnd((h @ f64(w["wv"]).T).reshape(S, Hkv, hd))
         kvs.append((k, v))
         kr, vr = np.repeat(k, Hq // Hkv, axis=1), np.repeat(v, Hq // Hkv, axis=1)
         sc = np.einsum("shd,thd->hst", q, kr) / np.sqrt(hd)
         sc = np.where(mask[None], sc, -np.inf)
         sc = np.exp(sc - sc.max(axis=-1, keepdims=True))
         pr = sc / sc.sum(axis=-1, keepdims=True)
-        att = np.einsum("hst,thd->shd", pr, vr).reshape(S, Hq * hd)
+        att = rnd(np.einsum("hst,thd->shd", pr, vr).reshape(S, Hq * hd))
         x = x + att @ f64(w["wo"]).T
-        h2 = rms(x, f64(w["norm2"]), shape.rms_eps)
+        h2 = rnd(rms(x, f64(w["norm2"]), shape.rms_eps))
         g, u = h2 @ f64(w["wg"]).T, h2 @ f64(w["wu"]).T
-        x = x + (g / (1.0 + np.exp(-g)) * u) @ f64(w["wd"]).T
-    logits = rms(x, f64(glob["final_norm"]), shape.rms_eps) @ f64(glob["lm_head"]).T
+        x = x + rnd(g / (1.0 + np.exp(-g)) * u) @ f64(w["wd"]).T
+    logits = rnd(rms(x, f64(glob["final_norm"]), shape.rms_eps)) @ f64(glob["lm_head"]).T
     return logits, kvs

@@ -17,8 +17,8 @@ from orc_util import PIN, PIN1, model, prefill, tokens_for
 P = 4  # small page size so that short sequences span many pages
 
 
-def _run(shape, glob, layers, toks, ctx, page_table, n_pages, u=1, f32=False, page_size=P):
-    orc = Oracle(shape, page_size=page_size, f32=f32)
+def _run(shape, glob, layers, toks, ctx, page_table, n_pages, u=1, f32=False, page_size=P, bf16_operands=False):
+    orc = Oracle(shape, page_size=page_size, f32=f32, bf16_operands=bf16_operands)
     pools = orc.new_pool(n_pages)
     if ctx:
         prefill(orc, glob, layers, pools, page_table, toks[:ctx], step=5)
@@ -44,6 +44,58 @@ def test_chunk_logits_equal_dense_full_matrix_forward(shape, ctx, n):
             page, row = pt[p // P], p % P
             assert np.abs(pools[l][page, 0, :, row, :] - k[p]).max() <= 1e-11 * max(1.0, np.abs(k).max())
             assert np.abs(pools[l][page, 1, :, row, :] - v[p]).max() <= 1e-11 * max(1.0, np.abs(v).max())
+
+
+# ---------------------------------------------------------------- the bf16-operand mode
+def test_bf16_rounding_is_round_to_nearest_even():
+    orc = Oracle(PIN)
+    g = np.random.default_rng(3)
+    vals = np.concatenate([g.standard_normal(4000) * 10.0 ** g.integers(-6, 6, 4000),
+                           # exact ties between two bf16 neighbours, and values one float ulp off a tie
+                           np.array([1.00390625, 1.01171875, -2.0078125, 3.0e-39, 0.0, -0.0, 65280.0 * 2.0 ** 100]),
+                           np.nextafter(np.float32(1.00390625), np.float32(2.0)).astype(np.float64).reshape(1),
+                           np.nextafter(np.float32(1.00390625), np.float32(0.0)).astype(np.float64).reshape(1)])
+    vals = vals.astype(np.float32).astype(np.float64)
+    ref = torch.from_numpy(vals).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(orc.bf16_round(vals), ref)
+    assert orc.bf16_round([1.00390625])[0] == 1.0 and orc.bf16_round([1.01171875])[0] == 1.015625   # ties to even
+
+
+@pytest.mark.parametrize("shape,ctx,n", [(PIN, 13, 5), (TINY, 21, 4)])
+def test_bf16_operand_mode_equals_dense_forward_with_the_same_roundings(shape, ctx, n):
+    """The bf16 model: activations entering a matrix product or the cache are bf16, sums are wide.
+    The dense full-matrix forward rounds at the same places with torch's conversion."""
+    glob, layers = model(shape)
+    toks = tokens_for(shape, ctx + n)
+    n_pages = -(-(ctx + n) // P) + 2
+    pt = np.random.default_rng(2).permutation(n_pages).astype(np.int32)
+    res, pools = _run(shape, glob, layers, toks, ctx, pt, n_pages, bf16_operands=True)
+    ref, kvs = dense_forward(shape, glob, layers, toks, bf16_operands=True)
+    sigma = ref.std()
+    # a value that sits on a rounding boundary may round differently after a different summation order:
+    # allow a handful of one-ulp flips, nothing systematic
+    assert np.abs(res.logits - ref[ctx:]).max() <= 2e-3 * sigma
+    assert np.sqrt(((res.logits - ref[ctx:]) ** 2).mean()) <= 1e-4 * sigma
+    exact, _ = _run(shape, glob, layers, toks, ctx, pt, n_pages)
+    d = np.sqrt(((res.logits - exact.logits) ** 2).mean()) / sigma
+    assert 1e-4 < d < 2e-2          # the roundings are there, and are small
+    # cached K and V are bf16 values
+    k = pools[0][pt[0], 0, :, 0, :]
+    assert np.array_equal(k, Oracle(shape).bf16_round(k).reshape(k.shape))
+
+
+def test_bf16_operand_mode_keeps_the_chunking_and_paging_invariants():
+    shape = PIN
+    glob, layers = model(shape)
+    toks = tokens_for(shape, 19)
+    pt = np.arange(6, dtype=np.int32)
+    a, _ = _run(shape, glob, layers, toks, 12, pt, 6, bf16_operands=True)
+    orc = Oracle(shape, page_size=P, bf16_operands=True)
+    pools = orc.new_pool(6)
+    pt2 = np.array([4, 0, 5, 2, 1, 3], dtype=np.int32)
+    prefill(orc, glob, layers, pools, pt2, toks[:12], step=3)
+    rows = [orc.forward_chunk(glob, lambda l: layers[l], pools, pt2, 12 + j, [int(toks[12 + j])]).logits[0] for j in range(7)]
+    assert np.array_equal(np.stack(rows), a.logits)
 
 
 def test_runner_up_and_gap_match_sorted_logits():
