@@ -175,12 +175,15 @@ __device__ __forceinline__ void attn_consume_stage(const uint8_t* stage, int fir
         m[r] = mx[r];
         l[r] *= corr[r];
     }
+    // once the running maxima have settled the factors are exactly 1 in every lane: skip the pass
+    if (!__all_sync(0xFFFFFFFFu, corr[0] == 1.f && corr[1] == 1.f)) {
 #pragma unroll
-    for (int nt = 0; nt < HD / 8; ++nt) {
-        o[nt][0] *= corr[0];
-        o[nt][1] *= corr[0];
-        o[nt][2] *= corr[1];
-        o[nt][3] *= corr[1];
+        for (int nt = 0; nt < HD / 8; ++nt) {
+            o[nt][0] *= corr[0];
+            o[nt][1] *= corr[0];
+            o[nt][2] *= corr[1];
+            o[nt][3] *= corr[1];
+        }
     }
     // P = exp2(S * scale - m), O += P V
     const int tokv = ((mi & 1) << 3) + (lane & 7);

@@ -619,8 +619,8 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
     // CTA's fair share: every split costs an fp32 partial and a merge.
     const int n_cta_max = n_sm;
     const int tok_per_group = std::min(16, 64 / G);
-    static const int STAGE_COST[5] = {0, 20, 21, 30, 31};
-    const int ITEM_COST = 60, PART_COST = 40;
+    static const int STAGE_COST[5] = {0, 20, 22, 34, 36};   // measured cycles per stage, in units of ~58
+    const int ITEM_COST = 110, PART_COST = 60;
     auto unit_cost = [&](int L, int nj) { return (int64_t)((L + 63) / 64) * STAGE_COST[(nj * G + 15) / 16] + ITEM_COST; };
     int64_t total_cost = 0;
     for (int i = 0; i < n_req; ++i) {
@@ -630,7 +630,7 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
             total_cost += unit_cost(ctx_lens[i] + j0 + nj, nj) * Hkv;
         }
     }
-    const int64_t share = std::max<int64_t>(8 * 31 + ITEM_COST, (total_cost + n_cta_max - 1) / n_cta_max);
+    const int64_t share = std::max<int64_t>(8 * 36 + ITEM_COST, (total_cost + n_cta_max - 1) / n_cta_max);
     std::vector<AttnItem> items;
     std::vector<int> item_cost;
     std::vector<MergeGroup>& groups = hp.groups;
