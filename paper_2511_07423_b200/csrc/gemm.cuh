@@ -4,17 +4,18 @@
 // PAIR of such tiles that share one token tile), the ragged token batch is the UMMA B operand
 // (N = 16..256 tokens), so a batch of T tokens pads to a multiple of 16 instead of 128.  Weights are
 // stored pre-tiled and pre-swizzled ([feature pair][k-block][2][128 x 64] images of the
-// 128-byte-swizzled shared-memory tile), so a stage's weights are ONE contiguous bulk copy that is
-// also prefetched into L2 several k-blocks ahead; activations come through a TMA tensor map.
-// One persistent CTA per SM walks a static schedule: whole pair tiles in full waves, the remainder as
-// single 128-feature tiles; projections with few output tiles (o, down) split K over CTAs and write
-// fp32 partials that resid_norm_kernel adds to the residual stream in a fixed order.  Accumulation is
-// tcgen05.mma into TMEM, read back with tcgen05.ld and transposed through shared memory into a
-// token-major tile for the epilogues:
-//   EPI_QKV    : RMSNorm row scale, RoPE on q and k, q store, paged-KV append of k and v
+// 128-byte-swizzled shared-memory tile), so a stage's weights are ONE contiguous bulk copy;
+// activations come through a TMA tensor map.  One persistent CTA per SM walks a static schedule:
+// whole pair tiles in full waves, the remainder as single 128-feature tiles; projections with few
+// output tiles (o, down) split K over CTAs and write fp32 partials that resid_norm_kernel adds to the
+// residual stream in a fixed order.  Every CTA starts its k loop at a different k-block, so the CTAs
+// that share a token tile do not ask L2 for the same lines at the same moment.  Accumulation is
+// tcgen05.mma into TMEM, read back with tcgen05.ld by sixteen epilogue warps; a thread then holds one
+// output feature for sixteen tokens, and the epilogues work on those registers:
+//   EPI_QKV    : RoPE on q and k (the partner dimension sits 16 lanes away), q store, paged-KV append
 //   EPI_PART   : fp32 partial of a split-K projection (residual added by resid_norm_kernel)
-//   EPI_SWIGLU : RMSNorm row scale, silu(gate) * up
-//   EPI_LMHEAD : RMSNorm row scale, optional logits, vocabulary argmax (packed 64-bit atomicMax)
+//   EPI_SWIGLU : silu(gate) * up (a gate feature and its up feature sit 16 lanes apart)
+//   EPI_LMHEAD : optional logits, vocabulary argmax (warp reduction, packed 64-bit atomicMax)
 //   EPI_PLAIN  : fp32 store (test hook)
 // The token operand of the QKV, gate/up and lm_head projections is the RMSNorm of the residual stream,
 // bf16(x * rstd * gain), written by resid_norm_kernel (prep_kernel for the first layer).
@@ -272,7 +273,7 @@ constexpr int GEMM_SMEM_MAX = 232448;
 constexpr int GEMM_PREFETCH_KB = 12;               // L2 prefetch distance in k-blocks
 
 __host__ __device__ inline int gemm_stage_bytes(int TN) { return GEMM_A_BYTES + ((TN + 31) / 32) * GEMM_BOX_BYTES; }
-__host__ inline int gemm_fixed_smem() { return 1024 /*align*/ + 2 * 2 * 128 * 8 /*argmax scratch*/ + 512; }
+__host__ inline int gemm_fixed_smem() { return 1024 /*align*/ + 512 /*barriers*/; }
 __host__ inline int gemm_stages(int TN) {
     int s = (GEMM_SMEM_MAX - gemm_fixed_smem()) / gemm_stage_bytes(TN);
     return s > GEMM_MAX_STAGES ? GEMM_MAX_STAGES : s;
@@ -351,8 +352,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int stage_bytes = gemm_stage_bytes(g.TN);
-    unsigned long long* comb = reinterpret_cast<unsigned long long*>(smem + g.n_stages * stage_bytes);   // [2 groups][2][128]
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(comb + 2 * 2 * 128);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + g.n_stages * stage_bytes);
     uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
     uint64_t* accf_bar = empty_bar + GEMM_MAX_STAGES;   // accumulators complete (MMA -> epilogue)
     uint64_t* acce_bar = accf_bar + 1;                  // accumulators drained (epilogue -> MMA)
