@@ -7,7 +7,7 @@
 // host-planned list of items.  One producer warp streams pages (TMA, 128-byte swizzle, one box of
 // 32 rows x 128 bytes per page and 64-element half: K and V of 16 tokens) and the item's Q tile
 // through mbarrier rings; its lanes fetch the page-table entries of the next stage while the
-// current one is in flight.  Eight consumer warps form two groups that take alternate stages, so
+// current one is in flight (its warpgroup gives most of its registers to the consumers).  Eight consumer warps form two groups that take alternate stages, so
 // every scheduler of the SM holds two warps; inside a group the four warps split the item's row
 // tiles and, when there are fewer than four row tiles, the pages of the stage.  QK^T and PV run on
 // warp-level MMAs (m16n8k16, bf16 in, fp32 accumulate) with an online softmax in fp32 (base 2).
@@ -69,7 +69,8 @@ __device__ __forceinline__ bool attn_item_ok(const AttnItem& it, const AttnParam
 
 constexpr int ATT_STAGE_PAGES = 4;
 constexpr int ATT_CONSUMER_WARPS = 8;
-constexpr int ATT_THREADS = (ATT_CONSUMER_WARPS + 1) * 32;
+constexpr int ATT_THREADS = (ATT_CONSUMER_WARPS + 4) * 32;   // two consumer warpgroups + the producer's warpgroup
+constexpr int ATT_PRODUCER_REGS = 40, ATT_CONSUMER_REGS = 232;   // 2 x 232 + 40 per scheduler slot <= 512
 
 template <int HD>
 struct AttnSmem {
@@ -298,8 +299,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     __syncthreads();
     pdl_wait();   // Q and the chunk's K/V come from the preceding projection kernel
 
-    if (warp == ATT_CONSUMER_WARPS) {
-        // ------------------------------------------------------------ producer (whole warp)
+    if (warp >= ATT_CONSUMER_WARPS) {
+        // ------------------------------------------------------------ producer (one warp of its warpgroup)
+        reg_dealloc<ATT_PRODUCER_REGS>();   // the whole warpgroup hands registers to the consumers
+        if (warp > ATT_CONSUMER_WARPS) return;
         uint32_t st = 0;  // running stage counter
         bool ok = true;
         const int my_pg = lane / HALVES, my_half = lane % HALVES;
@@ -350,6 +353,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     }
 
     // ---------------------------------------------------------------- consumers (warps 0..7)
+    reg_alloc<ATT_CONSUMER_REGS>();
     // A wait that runs out sets `ok` = false; the warp then skips all further waits and arithmetic
     // but still walks the items and takes part in every named barrier, so no other warp is left
     // waiting for it.
