@@ -71,6 +71,9 @@ constexpr int ATT_STAGE_PAGES = 4;
 constexpr int ATT_CONSUMER_WARPS = 8;
 constexpr int ATT_THREADS = (ATT_CONSUMER_WARPS + 4) * 32;   // two consumer warpgroups + the producer's warpgroup
 constexpr int ATT_PRODUCER_REGS = 40, ATT_CONSUMER_REGS = 232;   // 2 x 232 + 40 per scheduler slot <= 512
+constexpr int ATT_LAUNCH_REGS = 168;                              // what ptxas grants 384 threads per CTA
+static_assert(ATT_CONSUMER_WARPS * ATT_CONSUMER_REGS + 4 * ATT_PRODUCER_REGS <= (ATT_CONSUMER_WARPS + 4) * ATT_LAUNCH_REGS,
+              "the consumers' increase must fit in what the producer's warpgroup gives back");
 
 template <int HD>
 struct AttnSmem {

@@ -36,6 +36,8 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 // ---------------------------------------------------------------- register re-allocation between warpgroups
 // Executed by all four warps of a warpgroup (warps 4k .. 4k+3).  A kernel compiled for an even split of
 // the register file lets its data-movement warpgroup give registers back and its math warpgroups take them.
+// The increase waits, without any limit, until the registers are free: the totals after re-allocation
+// must not exceed what the launch allocated (threads x registers per thread), or the kernel hangs.
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
