@@ -395,8 +395,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                 const int nbox = (((min(g.TN, p.T - n0) + 15) & ~15) + 31) >> 5;
                 const uint32_t a_bytes = (uint32_t)(w.mt_hi - w.mt_lo) * GEMM_TILE_BYTES;
                 const __nv_bfloat16* wsrc = g.w + ((size_t)w.pair * g.num_kb) * (2 * 128 * 64) + (size_t)w.mt_lo * (128 * 64);
-                if (i == 0) pdl_wait();   // the token operand is the predecessor's output
                 const int nk = w.kb1 - w.kb0, rot = gemm_k_rotation(cta, n_cta, nk);
+                // The weights never depend on an earlier kernel: the first item's weight tiles of the
+                // whole ring are requested before waiting for the predecessor, whose output is only the
+                // token operand.
+                const int n_early = i == 0 ? min(nk, g.n_stages) : 0;
+                for (int j = 0; j < n_early; ++j) {
+                    const int kb = w.kb0 + (j + rot) % nk;
+                    uint8_t* a_s = smem + j * stage_bytes;
+                    mbar_expect_tx(&full_bar[j], a_bytes + nbox * GEMM_BOX_BYTES);
+                    bulk_load(a_s + w.mt_lo * GEMM_TILE_BYTES, wsrc + (size_t)kb * (2 * 128 * 64), a_bytes, &full_bar[j]);
+                }
+                if (i == 0) pdl_wait();
                 for (int j = 0; j < nk; ++j, ++it) {
                     const int kb = w.kb0 + (j + rot) % nk;
                     const int s = it % g.n_stages;
@@ -406,8 +416,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                     }
                     uint8_t* a_s = smem + s * stage_bytes;
                     uint8_t* b_s = a_s + GEMM_A_BYTES;
-                    mbar_expect_tx(&full_bar[s], a_bytes + nbox * GEMM_BOX_BYTES);
-                    bulk_load(a_s + w.mt_lo * GEMM_TILE_BYTES, wsrc + (size_t)kb * (2 * 128 * 64), a_bytes, &full_bar[s]);
+                    if (j >= n_early) {
+                        mbar_expect_tx(&full_bar[s], a_bytes + nbox * GEMM_BOX_BYTES);
+                        bulk_load(a_s + w.mt_lo * GEMM_TILE_BYTES, wsrc + (size_t)kb * (2 * 128 * 64), a_bytes, &full_bar[s]);
+                    }
                     for (int b = 0; b < nbox; ++b)
                         tma_load_2d(b_s + b * GEMM_BOX_BYTES, &tmB, &full_bar[s], kb * GEMM_BK, n0 + b * GEMM_BOX_ROWS);
                 }

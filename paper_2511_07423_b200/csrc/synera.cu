@@ -1052,6 +1052,7 @@ extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, 
         ps.p[0] = (const bf16*)w; ps.rows[0] = N; ps.src_k = K;
         pack_weight_kernel<<<dim3(n_mt, nkb), 256, 0, st>>>(ps, packed, nkb);
         if (!launch_ok()) return SYN_E_CUDA;
+        CU_OK(cudaStreamSynchronize(st));   // the GEMM requests weight tiles before it waits for its predecessor
         packed_src = w; packed_n = N; packed_k = K;
     }
     CUtensorMap tmB;
