@@ -613,14 +613,16 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
         for (int t = 1; t < T; ++t)
             if (s2[t] == s2[t - 1]) return SYN_E_PAGE_ALIAS;
     }
-    // Attention work list: (request, kv head, token group, key range).  Cost of an item = its 64-key
-    // stages weighted by the number of 16-row query tiles (more tiles = more tensor work per key
-    // byte) plus a fixed overhead.  A key range is split only when one unit alone would exceed a
-    // CTA's fair share: every split costs an fp32 partial and a merge.
+    // Attention work list: (request, kv head, token group, key range).  Cost of an item, in SM
+    // cycles: its 64-key stages times a per-stage time that grows with the number of 16-row query
+    // tiles (more tensor work per key byte), plus a fixed overhead per item; the figures are a
+    // least-squares fit to per-CTA durations measured on full batches.  A key range is split only
+    // when one unit alone would exceed a CTA's fair share: every split costs an fp32 partial and a
+    // merge.
     const int n_cta_max = n_sm;
     const int tok_per_group = std::min(16, 64 / G);
-    static const int STAGE_COST[5] = {0, 20, 22, 34, 36};   // measured cycles per stage, in units of ~58
-    const int ITEM_COST = 110, PART_COST = 60;
+    static const int STAGE_COST[5] = {0, 1040, 1200, 1500, 1540};
+    const int ITEM_COST = 5500, PART_COST = 3000;
     auto unit_cost = [&](int L, int nj) { return (int64_t)((L + 63) / 64) * STAGE_COST[(nj * G + 15) / 16] + ITEM_COST; };
     int64_t total_cost = 0;
     for (int i = 0; i < n_req; ++i) {
@@ -630,7 +632,7 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
             total_cost += unit_cost(ctx_lens[i] + j0 + nj, nj) * Hkv;
         }
     }
-    const int64_t share = std::max<int64_t>(8 * 36 + ITEM_COST, (total_cost + n_cta_max - 1) / n_cta_max);
+    const int64_t share = std::max<int64_t>(8 * STAGE_COST[4] + ITEM_COST, (total_cost + n_cta_max - 1) / n_cta_max);
     std::vector<AttnItem> items;
     std::vector<int> item_cost;
     std::vector<MergeGroup>& groups = hp.groups;
@@ -676,6 +678,67 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
         owner[i] = l.second;
         count[l.second + 1]++;
         heap.push(Load(l.first + cost(i), l.second));
+    }
+    // Local search on the greedy result: relieve the most loaded CTA by moving one of its items to
+    // another CTA, or by exchanging it for a cheaper one, as long as that lowers the larger of the
+    // two loads; partners are the least loaded CTAs.  Stops when the maximum is within 0.3 % of
+    // the mean.
+    if (n_cta > 1) {
+        std::vector<int64_t> load(n_cta, 0);
+        std::vector<std::vector<int>> held(n_cta);
+        int64_t sum = 0;
+        for (int i = 0; i < n_items; ++i) {
+            load[owner[i]] += cost(i);
+            held[owner[i]].push_back(i);
+            sum += cost(i);
+        }
+        const int64_t good = sum / n_cta + sum / n_cta / 333;
+        std::vector<int> by_load(n_cta);
+        for (int k = 0; k < n_cta; ++k) by_load[k] = k;
+        for (int round = 0; round < 2 * n_cta; ++round) {
+            const int hi = (int)(std::max_element(load.begin(), load.end()) - load.begin());
+            if (load[hi] <= good) break;
+            // partners: the least loaded CTAs
+            const int n_cand = std::min(n_cta - 1, 24);
+            std::partial_sort(by_load.begin(), by_load.begin() + n_cand + 1, by_load.end(),
+                              [&](int x, int y) { return load[x] != load[y] ? load[x] < load[y] : x < y; });
+            int64_t best = load[hi];
+            int bi = -1, bk = -1, bj = -1;   // positions in held[hi], the other CTA, position in held[bk] (-1: move)
+            for (int a = 0; a < (int)held[hi].size(); ++a) {
+                const int64_t ca = cost(held[hi][a]);
+                for (int q = 0; q <= n_cand; ++q) {
+                    const int k = by_load[q];
+                    if (k == hi) continue;
+                    if (std::max(load[hi] - ca, load[k] + ca) < best) {
+                        best = std::max(load[hi] - ca, load[k] + ca);
+                        bi = a; bk = k; bj = -1;
+                    }
+                    for (int b2 = 0; b2 < (int)held[k].size(); ++b2) {
+                        const int64_t dlt = ca - cost(held[k][b2]);
+                        if (dlt > 0 && std::max(load[hi] - dlt, load[k] + dlt) < best) {
+                            best = std::max(load[hi] - dlt, load[k] + dlt);
+                            bi = a; bk = k; bj = b2;
+                        }
+                    }
+                }
+            }
+            if (bi < 0) break;
+            const int ia = held[hi][bi];
+            if (bj < 0) {
+                load[hi] -= cost(ia); load[bk] += cost(ia);
+                owner[ia] = bk;
+                held[bk].push_back(ia);
+                held[hi].erase(held[hi].begin() + bi);
+            } else {
+                const int ib = held[bk][bj];
+                const int64_t dlt = cost(ia) - cost(ib);
+                load[hi] -= dlt; load[bk] += dlt;
+                owner[ia] = bk; owner[ib] = hi;
+                held[hi][bi] = ib; held[bk][bj] = ia;
+            }
+        }
+        std::fill(count.begin(), count.end(), 0);
+        for (int i = 0; i < n_items; ++i) count[owner[i] + 1]++;
     }
     for (int k = 0; k < n_cta; ++k) count[k + 1] += count[k];
     hp.items.assign(n_items, AttnItem());
