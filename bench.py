@@ -28,24 +28,28 @@ from workloads.configs import CONFIGS  # noqa: E402
 METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant kernel from an
-# ncu capture, keyed by workload, with the hash of the kernel source the capture was taken on: the
-# figure is reported only while the source is unchanged.  Summaries of the captures: profiles/.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from an ncu capture of two timed
+# steps of the workload (mean over all launches of the kernel function), with the hash of the kernel's
+# source file at capture time: the figure is reported only while that source is unchanged.  Summaries of
+# the captures: profiles/.
 NCU_TRAFFIC = {
-    # workload: (kernel, bytes per launch, sha256 of the kernel's source file at capture time)
-    "cfg3-8b": ("attention", 613997568 + 15093760, "f3662d421ffde0ac70fbe1b3bc7ab49d1c1963e78556f304f1f5d10136cd3ec8"),
+    # workload: {kernel: (bytes per launch, sha256 of the kernel's source file)}
+    "cfg3-8b": {
+        "attention": (615960044, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
+        "gemm": (132391874, "42ce693f7884da27f7771dbf960c769188f0682013ec67c8c82d0e8fe36d9254"),
+    },
 }
 
 
 def _traffic(workload: str, kernel: str):
     import hashlib
-    ent = NCU_TRAFFIC.get(workload)
-    if not ent or ent[0] != kernel:
+    ent = NCU_TRAFFIC.get(workload, {}).get(kernel)
+    if not ent:
         return None
     src = os.path.join(ROOT, "paper_2511_07423_b200", "csrc", "attention.cuh" if kernel == "attention" else "gemm.cuh")
-    if hashlib.sha256(open(src, "rb").read()).hexdigest() != ent[2]:
+    if hashlib.sha256(open(src, "rb").read()).hexdigest() != ent[1]:
         return None
-    return ent[1]
+    return ent[0]
 
 
 def _peaks():
@@ -203,7 +207,7 @@ def run_ours(args):
     kv = syn.KVCache(model, batch.n_pages)
     synthetic.fill_cache(kv, shape, wl.seed, batch)
     toks = synthetic.teacher_forced_chunks(kv, wl, batch)
-    plan = syn.Plan(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+    plan = syn.Plan(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, batch.n_uncached)
     st = plan.stats()
     B, T = batch.n_req, batch.n_tokens
     acc = torch.empty(B, dtype=torch.int32, device="cuda")
@@ -231,12 +235,13 @@ def run_ours(args):
     # ---- end to end through the blocking C-ABI call with host buffers
     pin = lambda t: t.pin_memory()
     h_tok, h_off, h_pt, h_ctx = pin(toks), pin(batch.chunk_offsets), pin(batch.page_tables), pin(batch.ctx_lens)
+    h_unc = pin(batch.n_uncached)
     for _ in range(3):
-        kv.verify_batch(h_tok, h_off, h_pt, h_ctx)
+        kv.verify_batch(h_tok, h_off, h_pt, h_ctx, n_uncached=h_unc)
     barrier()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        a_h, c_h = kv.verify_batch(h_tok, h_off, h_pt, h_ctx)
+        a_h, c_h = kv.verify_batch(h_tok, h_off, h_pt, h_ctx, n_uncached=h_unc)
     barrier()
     ms_e2e = (time.perf_counter() - t0) * 1e3 / args.steps
     clocks = sampler.stop() if sampler else None
@@ -284,9 +289,9 @@ def run_ours(args):
         avg_s = gemm_ms_step * 1e-3 / gemm_launches
         if T >= ridge:
             return {"kernel": "gemm_kernel", "bound": "tensor", "achieved": st.dense_flops / gemm_launches / avg_s / 1e12,
-                    "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "traffic": None}
+                    "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "traffic": _traffic(wl.name, "gemm")}
         return {"kernel": "gemm_kernel", "bound": "hbm", "achieved": st.weight_bytes / gemm_launches / avg_s / 1e9,
-                "peak": peaks["hbm_gbs"], "unit": "GB/s", "traffic": None}
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "traffic": _traffic(wl.name, "gemm")}
     def attn_roof():
         return {"kernel": "attn_kernel", "bound": "hbm", "achieved": kernels["attention"]["kv_gbs"], "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "traffic": _traffic(wl.name, "attention")}
@@ -356,7 +361,7 @@ def cpu_baseline(wl, batch, toks, acc_gpu, cor_gpu, min_seconds: float = 12.0, m
         chunk = toks[b:b + n].tolist()
         orc, pools, pt, ctx = oracle_sample(wl, batch, None, glob, req, n)
         t0 = time.perf_counter()
-        res = orc.forward_chunk(glob, layer_w, pools, pt, ctx, chunk, want_logits=False)
+        res = orc.forward_chunk(glob, layer_w, pools, pt, ctx, chunk, u=int(batch.n_uncached[req]), want_logits=False)
         seconds += time.perf_counter() - t0
         tokens += n
         done.append(req)
@@ -375,7 +380,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=3, help="1..5; 3 = the 8B-shape step the metric is quoted on")
+    ap.add_argument("--config", type=int, default=3, help="1..6; 3 = the 8B-shape step the metric is quoted on; 6 = 32-token chunked partial prefill")
     ap.add_argument("--pool-tokens", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -46,7 +46,10 @@ enum {
     SYN_E_DEVICE_TIMEOUT = -11 /* a bounded wait inside a kernel ran out; results are invalid   */
 };
 
-#define SYN_MAX_CHUNK 16
+/* Longest chunk of one request in one call: the fixed chunk length of the paper's chunked partial
+ * prefill (Sec. 4.5).  Verification chunks are tens of tokens at most (Sec. 3.4); a longer
+ * uncached run is fed in several calls. */
+#define SYN_MAX_CHUNK 32
 
 typedef struct syn_model syn_model; /* packed device copy of the weights + workspaces */
 typedef struct syn_kv syn_kv;       /* paged KV pool                                   */
@@ -82,8 +85,10 @@ typedef struct {
 } syn_weights;
 
 /* The LLM that verifies (paper Sec. 3.1).  Makes the library's own packed device copy of the
- * weights, layer by layer (q|k|v rows concatenated, gate/up rows interleaved in blocks of 64,
- * d_ffn padded to a multiple of 64 with zeros), so the caller's copy may be freed afterwards.
+ * weights, layer by layer (tiles of 128 output features x 64 inputs in the tensor cores' shared-
+ * memory order; q|k|v in one matrix with the two halves of a head's rotation side by side, gate
+ * and up features of the same 64 columns in one tile, d_ffn padded to a multiple of 64 with
+ * zeros), so the caller's copy may be freed afterwards.
  * Errors: SYN_E_INVALID_ARG (NULL, unsupported shape, flags != 0), SYN_E_ARCH, SYN_E_OOM,
  * SYN_E_CUDA.  *out is written only on success. */
 int syn_model_load(const syn_model_desc *desc, const syn_weights *weights, syn_model **out);

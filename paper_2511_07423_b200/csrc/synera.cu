@@ -433,7 +433,7 @@ extern "C" int syn_model_load(const syn_model_desc* desc, const syn_weights* w, 
             PACK_OR_FAIL(pack(srcs, rows, 1, 0, q_dim, d, &pk));
             m->wo.push_back(pk);
         }
-        {   // gate/up interleaved in blocks of 64 rows; rows of the padded tail are zero
+        {   // a tile holds the gate and the up rows of the same 64 features; rows of the padded tail are zero
             const void* srcs[2] = {w->wg[l], w->wu[l]};
             const int rows[2] = {f, f};
             PACK_OR_FAIL(pack(srcs, rows, 2, 1, d, m->gu_rows, &pk));
@@ -1213,7 +1213,7 @@ extern "C" const char* syn_strerror(int code) {
     switch (code) {
         case SYN_OK: return "ok";
         case SYN_E_INVALID_ARG: return "invalid argument";
-        case SYN_E_CHUNK_LEN: return "chunk length outside [1, 16]";
+        case SYN_E_CHUNK_LEN: return "chunk length outside [1, 32]";
         case SYN_E_UNCACHED: return "n_uncached outside [1, chunk length]";
         case SYN_E_PAGE_OOB: return "page id out of range";
         case SYN_E_CAPACITY: return "context + chunk exceeds the page table";

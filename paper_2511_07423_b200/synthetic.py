@@ -43,29 +43,35 @@ def fill_cache(kv: KVCache, shape: ModelShape, seed: int, batch: gen.Batch, reqs
 
 
 def teacher_forced_chunks(kv: KVCache, wl: Workload, batch: gen.Batch, fixed: Optional[Dict[int, List[int]]] = None):
-    """Chunk tokens of the whole batch by the sequential draft rule, with the argmax supplied by
-    the library itself (one pass per chunk index).  Requests listed in `fixed` keep the given
-    tokens (e.g. chunks whose drafts a test derived by other means)."""
+    """Chunk tokens of the whole batch by the sequential draft rule (u accepted tokens: the anchor,
+    then uniform ids; then drafts), with the argmax supplied by the library itself (one pass per
+    chunk index that precedes a draft).  Requests listed in `fixed` keep the given tokens (e.g.
+    chunks whose drafts a test derived by other means)."""
     fixed = fixed or {}
     B = batch.n_req
     offs = batch.chunk_offsets.tolist()
+    unc = batch.n_uncached.tolist()
     toks = torch.zeros(batch.n_tokens, dtype=torch.int32)
     for r in range(B):
         if r in fixed:
             toks[offs[r]:offs[r + 1]] = torch.tensor(fixed[r], dtype=torch.int32)
         else:
             toks[offs[r]] = gen.gen_anchor(wl, r)
+            if unc[r] > 1:
+                toks[offs[r] + 1:offs[r] + unc[r]] = gen.gen_context_tokens(wl, r, unc[r] - 1)
     acc = torch.empty(B, dtype=torch.int32, device="cuda")
     cor = torch.empty(B, dtype=torch.int32, device="cuda")
     top1 = torch.empty(batch.n_tokens, dtype=torch.int32, device="cuda")
     n_max = int(batch.chunk_lens.max())
     for j in range(n_max - 1):
-        plan = Plan(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+        todo = [r for r in range(B) if r not in fixed and unc[r] <= j + 1 < offs[r + 1] - offs[r]]
+        if not todo:
+            continue
+        plan = Plan(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, batch.n_uncached)
         plan.run(acc, cor, top1)
         torch.cuda.synchronize()
         t1 = top1.cpu()
         plan.close()
-        for r in range(B):
-            if r not in fixed and j + 1 < offs[r + 1] - offs[r]:
-                toks[offs[r] + j + 1] = gen.gen_draft(wl, r, j, int(t1[offs[r] + j]))
+        for r in todo:
+            toks[offs[r] + j + 1] = gen.gen_draft(wl, r, j + 1 - unc[r], int(t1[offs[r] + j]))
     return toks

@@ -35,21 +35,23 @@ class OracleRequest:
 
 
 def oracle_teacher_forced(orc: Oracle, glob, layer_w: Callable[[int], dict], pools, page_table, ctx: int, wl: Workload,
-                          req: int, n: int, want_logits=True) -> OracleRequest:
-    """Build request `req`'s chunk by the sequential rule (anchor uniform; draft j = the oracle's
-    argmax after the actual earlier chunk tokens with probability p_match, else uniform) while
-    running the oracle token by token, which is bit-identical to its one-shot chunk forward."""
-    chunk = [gen.gen_anchor(wl, req)]
+                          req: int, n: int, want_logits=True, u: int = 1) -> OracleRequest:
+    """Build request `req`'s chunk by the sequential rule (u device-accepted tokens: the anchor, then
+    uniform ids; draft j = the oracle's argmax after the actual earlier chunk tokens with
+    probability p_match, else uniform) while running the oracle token by token, which is
+    bit-identical to its one-shot chunk forward."""
+    assert 1 <= u <= n
+    chunk = [gen.gen_anchor(wl, req)] + [int(x) for x in gen.gen_context_tokens(wl, req, u - 1)]
     t1, t2, gp, lg = [], [], [], []
     for j in range(n):
         r = orc.forward_chunk(glob, layer_w, pools, page_table, ctx + j, [chunk[j]], u=1, want_logits=want_logits)
         t1.append(int(r.top1[0])); t2.append(int(r.top2[0])); gp.append(float(r.gap[0]))
         if want_logits:
             lg.append(r.logits[0])
-        if j + 1 < n:
-            chunk.append(gen.gen_draft(wl, req, j, int(r.top1[0])))
-    a, c = verify_greedy(t1, chunk, 1)
-    return OracleRequest(chunk, 1, np.array(t1), np.array(t2), np.array(gp),
+        if u <= j + 1 < n:
+            chunk.append(gen.gen_draft(wl, req, j + 1 - u, int(r.top1[0])))
+    a, c = verify_greedy(t1, chunk, u)
+    return OracleRequest(chunk, u, np.array(t1), np.array(t2), np.array(gp),
                          np.stack(lg) if want_logits else None, a, c)
 
 

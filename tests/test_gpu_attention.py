@@ -26,6 +26,9 @@ CASES = [
     (64, 8, 8, [130, 31], [16, 2]),                                  # G=1
     (128, 8, 2, [1500, 900, 2300], [16, 1, 9]),                      # long contexts: key ranges split over items
     (64, 16, 2, [40], [8]),                                          # G=8
+    (128, 8, 2, [100, 5, 0], [32, 19, 17]),                          # chunks beyond 16: two token groups per request
+    (128, 10, 2, [50], [30]),                                        # G=5, three token groups
+    (64, 16, 2, [200], [32]),                                        # G=8, four token groups
 ]
 
 

@@ -1,4 +1,4 @@
-"""Parity at the full sizes of configurations 2..5, in the launch configuration bench.py times:
+"""Parity at the full sizes of configurations 2..6, in the launch configuration bench.py times:
 the whole batch goes through syn_verify_batch on the GPU (seeded synthetic cache, drafts by the
 sequential rule from the library's own argmax), and a few sampled requests are recomputed one by one
 by the CPU oracle (all intermediates in double) from the same chunk tokens.  For those requests
@@ -36,7 +36,8 @@ def _samples(batch, max_tokens):
     within = [r for r in ids if n[r] <= max_tokens]
     picks.append(max(within, key=lambda r: (n[r], ctx[r])))
     small = [r for r in ids if n[r] <= 4]
-    picks.append(max(small, key=lambda r: ctx[r]))
+    if small:
+        picks.append(max(small, key=lambda r: ctx[r]))
     out = []
     for r in picks:
         if r not in out:
@@ -44,7 +45,7 @@ def _samples(batch, max_tokens):
     return out
 
 
-@pytest.mark.parametrize("cfg,max_tokens", [(2, 8), (3, 16), (4, 16), (5, 6)])
+@pytest.mark.parametrize("cfg,max_tokens", [(2, 8), (3, 16), (4, 16), (5, 6), (6, 32)])
 def test_sampled_requests_match_the_oracle_at_full_size(cfg, max_tokens):
     import paper_2511_07423_b200 as syn
     from paper_2511_07423_b200 import synthetic
@@ -59,14 +60,16 @@ def test_sampled_requests_match_the_oracle_at_full_size(cfg, max_tokens):
     kv = syn.KVCache(model, batch.n_pages)
     synthetic.fill_cache(kv, shape, wl.seed, batch)
     toks = synthetic.teacher_forced_chunks(kv, wl, batch)
-    acc, cor, logits = kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, want_logits=True)
+    unc = batch.n_uncached.tolist()
+    acc, cor, logits = kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens,
+                                       n_uncached=batch.n_uncached, want_logits=True)
     assert model.status() == 0
     offs = batch.chunk_offsets.tolist()
     # every request: results are in range and consistent with the returned logits' argmax
     top1_gpu = logits.argmax(-1).cpu()
     for r in range(batch.n_req):
         chunk = toks[offs[r]:offs[r + 1]].tolist()
-        assert (int(acc[r]), int(cor[r])) == verify_greedy(top1_gpu[offs[r]:offs[r + 1]].tolist(), chunk, 1)
+        assert (int(acc[r]), int(cor[r])) == verify_greedy(top1_gpu[offs[r]:offs[r + 1]].tolist(), chunk, unc[r])
 
     orc = Oracle(shape)
     exact_bound = 2.5 * 6.0 * np.sqrt(7.0 * shape.n_layers + 1.0) * 2.0 ** -9 / np.sqrt(3.0)
@@ -91,8 +94,8 @@ def test_sampled_requests_match_the_oracle_at_full_size(cfg, max_tokens):
             k, v = gen.gen_kv(shape, wl.seed, l, r, 0, ctx)
             orc.load_kv(pools[l], pt, 0, k.float().numpy(), v.float().numpy())
         chunk = toks[offs[r]:offs[r + 1]].tolist()
-        res = orc.forward_chunk(glob, layer_w, pools, pt, ctx, chunk, u=1, want_logits=True)
-        o = OracleRequest(chunk, 1, res.top1, res.top2, np.asarray(res.gap), res.logits, res.accept_len, res.correction)
+        res = orc.forward_chunk(glob, layer_w, pools, pt, ctx, chunk, u=unc[r], want_logits=True)
+        o = OracleRequest(chunk, unc[r], res.top1, res.top2, np.asarray(res.gap), res.logits, res.accept_len, res.correction)
         ok, strict = admissible_results(o)
         got = (int(acc[r]), int(cor[r]))
         if strict:

@@ -24,13 +24,15 @@ def _setup(shape, seed, batch):
     return glob, layers, model, kv, orc, pools
 
 
-def _run_and_judge(wl, shape, batch, glob, layers, kv, orc, pools, check_kv=True):
+def _run_and_judge(wl, shape, batch, glob, layers, kv, orc, pools, check_kv=True, uncached=None):
     reqs = []
     for r in range(batch.n_req):
         reqs.append(oracle_teacher_forced(orc, glob, lambda l: layers[l], pools, batch.page_tables[r].numpy(),
-                                          int(batch.ctx_lens[r]), wl, r, int(batch.chunk_lens[r])))
+                                          int(batch.ctx_lens[r]), wl, r, int(batch.chunk_lens[r]),
+                                          u=1 if uncached is None else uncached[r]))
     tokens = torch.tensor([t for o in reqs for t in o.chunk], dtype=torch.int32)
-    acc, cor, logits = kv.verify_batch(tokens, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, want_logits=True)
+    acc, cor, logits = kv.verify_batch(tokens, batch.chunk_offsets, batch.page_tables, batch.ctx_lens,
+                                       n_uncached=uncached, want_logits=True)
     assert kv.model.status() == 0
     res = judge(reqs, acc, cor, logits, batch.chunk_offsets)
     if check_kv:   # the chunk's K/V landed in exactly the slots the page table names
@@ -98,6 +100,21 @@ def test_mini_shapes_synthetic_cache(shape, ctx, chunk):
     print(shape.name, res)
 
 
+@pytest.mark.parametrize("shape,ctx,chunk,unc", [
+    # chunked partial prefill (paper Sec. 4.5: fixed chunks of 32) and long uncached runs before the drafts
+    (MINI_8B, [0, 40, 300, 1000, 15], [32, 17, 31, 25, 32], [32, 1, 20, 9, 28]),        # G = 4: two token groups
+    (MINI_1B, [7, 260], [32, 29], [1, 29]),                                             # head_dim 64
+    (ModelShape("g5c", 2, 640, 10, 2, 128, 1376, 3000), [100, 33], [32, 27], [16, 3]),  # G = 5: groups of 12
+])
+def test_chunks_up_to_32_and_long_uncached_runs(shape, ctx, chunk, unc):
+    wl = Workload("chunk32", shape, 13, len(ctx), ("list", tuple(ctx)), ("list", tuple(chunk)), 0.7)
+    batch = gen.gen_batch(wl)
+    glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
+    fill_synthetic_kv(shape, wl.seed, batch, range(batch.n_req), kv=kv, orc=orc, pools=pools)
+    res = _run_and_judge(wl, shape, batch, glob, layers, kv, orc, pools, uncached=unc)
+    print(shape.name, res)
+
+
 def test_uncached_prefix_longer_than_one_and_rerun_is_idempotent():
     shape = MINI_1B
     wl = Workload("u", shape, 5, 3, ("list", (20, 64, 7)), ("list", (6, 16, 1)), 0.7)
@@ -153,7 +170,7 @@ def test_host_validation_errors_leave_outputs_untouched():
             kv.verify_batch(**args)
         return e.value.code
 
-    assert code(chunk_offsets=torch.tensor([0, 4, 8, 12, 29])) == -2                      # chunk of 17
+    assert code(chunk_offsets=torch.tensor([0, 4, 8, 12, 45])) == -2                      # chunk of 33
     assert code(chunk_offsets=torch.tensor([0, 4, 4, 12, 16])) == -2                      # empty chunk
     assert code(n_uncached=[1, 5, 1, 1]) == -3
     assert code(n_uncached=[0, 1, 1, 1]) == -3

@@ -124,14 +124,18 @@ def test_paged_equals_contiguous_and_any_page_permutation_bitwise():
 
 
 # ---------------------------------------------------------------- P-3 chunking invariance
-def test_chunk_equals_token_by_token_and_any_split():
+@pytest.mark.parametrize("total,ctx,splits", [
+    (20, 11, ([1] * 9, [4, 5], [2, 3, 4], [8, 1])),
+    (43, 11, ([16, 16], [5, 27], [31, 1], [1] * 32)),   # a 32-token chunk (chunked partial prefill, Sec. 4.5)
+])
+def test_chunk_equals_token_by_token_and_any_split(total, ctx, splits):
     glob, layers = model(PIN)
-    toks = tokens_for(PIN, 20)
-    ctx, n_pages = 11, 7
+    toks = tokens_for(PIN, total)
+    n_pages = -(-total // P) + 2
     pt = np.random.default_rng(5).permutation(n_pages).astype(np.int32)
     whole, _ = _run(PIN, glob, layers, toks, ctx, pt, n_pages)
     orc = Oracle(PIN, page_size=P)
-    for split in ([1] * 9, [4, 5], [2, 3, 4], [8, 1]):
+    for split in splits:
         pools = orc.new_pool(n_pages)
         prefill(orc, glob, layers, pools, pt, toks[:ctx], step=3)
         p, rows = ctx, []

@@ -28,7 +28,7 @@ def test_positions_and_slots_follow_the_page_table():
     assert r["slot"].tolist() == [4 * 16 + 12, 4 * 16 + 13, 4 * 16 + 14, 4 * 16 + 15, 0, 1, 2, 3, 16, 17, 18]
 
 
-@pytest.mark.parametrize("cfg", [1, 2, 3, 4])
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 6])
 def test_work_list_covers_every_key_of_every_row_group_exactly_once(cfg):
     wl = CONFIGS[cfg]
     shape = wl.shape
@@ -89,7 +89,7 @@ def test_validation_codes_match_the_header():
             _plan(shape, batch, **kw)
         return e.value.code
 
-    assert code(chunk_offsets=torch.tensor([0, 4, 8, 12, 29])) == -2
+    assert code(chunk_offsets=torch.tensor([0, 4, 8, 12, 45])) == -2
     assert code(chunk_offsets=torch.tensor([0, 4, 4, 12, 16])) == -2
     assert code(chunk_offsets=torch.tensor([1, 4, 8, 12, 16])) == -1
     assert code(n_uncached=[1, 5, 1, 1]) == -3

@@ -1,4 +1,5 @@
-"""The five benchmark configurations as data: model shapes and request mixes.
+"""The benchmark configurations as data: model shapes and request mixes (1-5: verification
+batches; 6: chunked partial prefill with 32-token chunks).
 
 Shapes and mixes only; seeds follow the rule "configuration k (1-based) uses seed k-1".
 """
@@ -64,6 +65,7 @@ class Workload:
     page_size: int = 16
     real_prefill: bool = False      # context KV produced by prefilling real tokens
     fit_to_pool: bool = False       # scale contexts by a common factor to fit the pool
+    n_drafts: Optional[int] = None  # drafts at the end of a chunk; the rest is uncached accepted tokens (None: all but one)
 
 
 CONFIGS = {
@@ -75,6 +77,8 @@ CONFIGS = {
                 ("mix", ((0.6, 1, 1), (0.3, 2, 8), (0.1, 9, 16))), 0.65),
     5: Workload("cfg5-32b", SHAPE_32B, 4, 128, ("uniform", 1024, 8192), ("uniform", 1, 16), 0.6,
                 fit_to_pool=True),
+    # chunked partial prefill: every request feeds a full 32-token chunk, 28 uncached tokens + 4 drafts
+    6: Workload("cfg6-8b-chunk32", SHAPE_8B, 5, 64, ("uniform", 512, 4096), ("const", 32), 0.6, n_drafts=4),
 }
 
 # Reduced shapes used by tests that need the structure of a large configuration

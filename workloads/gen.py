@@ -157,7 +157,8 @@ def gen_batch(wl: Workload, pool_tokens: Optional[int] = None, n_req: Optional[i
         offs.append(offs[-1] + n)
     return Batch(B, P, n_pages, torch.tensor(ctx, dtype=torch.int32), torch.tensor(chunk, dtype=torch.int32),
                  torch.tensor(offs, dtype=torch.int32), table, max_pages,
-                 torch.ones(B, dtype=torch.int32), scale)
+                 torch.tensor([1 if wl.n_drafts is None else max(1, n - wl.n_drafts) for n in chunk], dtype=torch.int32),
+                 scale)
 
 
 # ----------------------------------------------------------------------------- cached KV and tokens
