@@ -1,4 +1,4 @@
-"""ctypes binding of include/synera.h: argument marshalling only.
+"""ctypes binding of include/synera.h and include/synera_sched.h: argument marshalling only.
 
 PyTorch supplies device memory and streams; every pointer handed to the library is a raw
 ``data_ptr()``.  There is no CPU fallback: if the library is missing or a call fails, a
@@ -58,6 +58,8 @@ EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "s
            "syn_verify_batch", "syn_plan_create", "syn_plan_free", "syn_verify_run", "syn_model_status",
            "syn_last_step_stats", "syn_plan_host", "syn_strerror", "syn_last_cuda_error", "syn_op_linear", "syn_op_attention", "syn_op_attention_static",
            "syn_set_profile", "syn_get_profile"]
+SCHED_EXPORTS = ["syn_sched_create", "syn_sched_free", "syn_sched_add_request", "syn_sched_add_verify", "syn_sched_finish",
+                 "syn_sched_peek", "syn_sched_commit", "syn_sched_step", "syn_sched_get_stats"]
 
 
 def load_library() -> C.CDLL:
@@ -71,7 +73,7 @@ def load_library() -> C.CDLL:
         lib.syn_strerror.argtypes = [C.c_int]
         lib.syn_last_cuda_error.restype = C.c_char_p
         lib.syn_last_cuda_error.argtypes = []
-        for fn in ("syn_model_free", "syn_kv_free", "syn_plan_free"):
+        for fn in ("syn_model_free", "syn_kv_free", "syn_plan_free", "syn_sched_free"):
             getattr(lib, fn).restype = None
             getattr(lib, fn).argtypes = [C.c_void_p]
         _LIB = lib
@@ -317,6 +319,120 @@ def plan_host(shape, n_pages: int, chunk_tokens, chunk_offsets, page_tables, ctx
         items = torch.zeros(max(cap, 1), len(PLAN_ITEM_FIELDS), dtype=torch.int32)
     return {"pos": pos[:T], "slot": slot[:T], "items": items[:n_items.value], "cta_begin": cta[:n_cta.value + 1],
             "n_cta": n_cta.value, "stats": st}
+
+
+# ------------------------------------------------------------------------------------------ scheduler
+
+SCHED_KINDS = ("idle", "prefill", "verify")
+
+
+class _SchedBatch(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("n_req", C.c_int32), ("n_tokens", C.c_int32), ("max_pages", C.c_int32),
+                ("req_ids", C.POINTER(C.c_int64)), ("chunk_tokens", C.POINTER(C.c_int32)),
+                ("chunk_offsets", C.POINTER(C.c_int32)), ("page_tables", C.POINTER(C.c_int32)),
+                ("ctx_lens", C.POINTER(C.c_int32)), ("n_uncached", C.POINTER(C.c_int32))]
+
+
+class _SchedResult(C.Structure):
+    _fields_ = [("req_id", C.c_int64)] + [(n, C.c_int32) for n in ("kind", "n_tokens", "accept_len", "correction_token",
+                                                                    "ctx_len", "prompt_done")]
+
+
+class SchedStats(C.Structure):
+    _fields_ = [("iterations", C.c_int64 * 3), ("tokens", C.c_int64 * 3), ("requests", C.c_int64 * 3),
+                ("deferred", C.c_int64), ("host_seconds", C.c_double), ("execute_seconds", C.c_double),
+                ("live_requests", C.c_int32), ("free_pages", C.c_int32)]
+
+
+class Scheduler:
+    """syn_sched_*: the verification-aware scheduler over one KV cache, or, with ``kv=None``, its
+    policy alone (peek / commit without a device)."""
+
+    def __init__(self, kv: Optional["KVCache"], n_pages: Optional[int] = None, page_size: int = 16,
+                 max_batch_tokens: int = 2048):
+        self._lib = load_library()
+        self.kv = kv
+        if kv is not None:
+            n_pages, page_size = kv.n_pages, kv.page_size
+        self._h = C.c_void_p()
+        _check(self._lib.syn_sched_create(kv.model._h if kv is not None else None, kv._h if kv is not None else None,
+                                          C.c_uint32(n_pages), C.c_uint32(page_size), C.c_int32(max_batch_tokens),
+                                          C.byref(self._h)), "syn_sched_create")
+        self._cap = 0
+        self._res = None
+
+    def add_request(self, req_id: int, prompt) -> None:
+        p = _i32(prompt)
+        _check(self._lib.syn_sched_add_request(self._h, C.c_int64(req_id), C.c_void_p(p.data_ptr()), C.c_int32(p.numel())),
+               "syn_sched_add_request")
+
+    def add_verify(self, req_id: int, tokens, n_uncached: int = 1) -> None:
+        t = _i32(tokens)
+        _check(self._lib.syn_sched_add_verify(self._h, C.c_int64(req_id), C.c_void_p(t.data_ptr()), C.c_int32(t.numel()),
+                                              C.c_int32(n_uncached)), "syn_sched_add_verify")
+
+    def finish(self, req_id: int) -> None:
+        _check(self._lib.syn_sched_finish(self._h, C.c_int64(req_id)), "syn_sched_finish")
+
+    def peek(self) -> Dict[str, object]:
+        """The next iteration's batch, copied into tensors (page_tables [n_req, max_pages])."""
+        b = _SchedBatch()
+        _check(self._lib.syn_sched_peek(self._h, C.byref(b)), "syn_sched_peek")
+        out = {"kind": SCHED_KINDS[b.kind], "n_req": b.n_req, "n_tokens": b.n_tokens, "max_pages": b.max_pages}
+        if b.kind == 0:
+            return out
+        B = b.n_req
+        out["req_ids"] = [b.req_ids[i] for i in range(B)]
+        out["chunk_offsets"] = torch.tensor([b.chunk_offsets[i] for i in range(B + 1)], dtype=torch.int32)
+        out["chunk_tokens"] = torch.tensor([b.chunk_tokens[i] for i in range(b.n_tokens)], dtype=torch.int32)
+        out["page_tables"] = torch.tensor([b.page_tables[i] for i in range(B * b.max_pages)],
+                                          dtype=torch.int32).view(B, b.max_pages)
+        out["ctx_lens"] = torch.tensor([b.ctx_lens[i] for i in range(B)], dtype=torch.int32)
+        out["n_uncached"] = torch.tensor([b.n_uncached[i] for i in range(B)], dtype=torch.int32)
+        return out
+
+    def _results(self, n: int) -> List[Dict[str, int]]:
+        return [{f: getattr(self._res[i], f) for f, _ in _SchedResult._fields_} for i in range(n)]
+
+    def _room(self, n: int) -> None:
+        if n > self._cap:
+            self._cap = max(n, 64)
+            self._res = (_SchedResult * self._cap)()
+
+    def commit(self, accept_len=None, correction_token=None) -> List[Dict[str, int]]:
+        a = _i32(accept_len) if accept_len is not None else None
+        c = _i32(correction_token) if correction_token is not None else None
+        self._room(a.numel() if a is not None else 1)
+        n = C.c_int32(0)
+        _check(self._lib.syn_sched_commit(self._h, C.c_void_p(a.data_ptr()) if a is not None else None,
+                                          C.c_void_p(c.data_ptr()) if c is not None else None, self._res,
+                                          C.c_int32(self._cap), C.byref(n)), "syn_sched_commit")
+        return self._results(n.value)
+
+    def step(self, stream=None, max_results: int = 4096):
+        """One iteration: (kind, results)."""
+        self._room(max_results)
+        n, kind = C.c_int32(0), C.c_int32(0)
+        sp = _stream_ptr(stream) if self.kv is not None else None   # without a model the library refuses the call
+        _check(self._lib.syn_sched_step(self._h, self._res, C.c_int32(self._cap), C.byref(n), C.byref(kind), sp),
+               "syn_sched_step")
+        return SCHED_KINDS[kind.value], self._results(n.value)
+
+    def stats(self) -> SchedStats:
+        st = SchedStats()
+        _check(self._lib.syn_sched_get_stats(self._h, C.byref(st)), "syn_sched_get_stats")
+        return st
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.syn_sched_free(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def syn_op_linear(x: torch.Tensor, w: torch.Tensor, stream=None) -> torch.Tensor:

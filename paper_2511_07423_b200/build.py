@@ -8,8 +8,9 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsynera.so")
-SOURCES = ["synera.cu"]
-HEADERS = ["ptx.cuh", "gemm.cuh", "attention.cuh", os.path.join("..", "..", "include", "synera.h")]
+SOURCES = ["synera.cu", "scheduler.cpp"]
+HEADERS = ["ptx.cuh", "gemm.cuh", "attention.cuh", os.path.join("..", "..", "include", "synera.h"),
+           os.path.join("..", "..", "include", "synera_sched.h")]
 
 
 def _nvcc() -> str:

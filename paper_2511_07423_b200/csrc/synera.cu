@@ -1214,6 +1214,10 @@ extern "C" const char* syn_strerror(int code) {
         case SYN_OK: return "ok";
         case SYN_E_INVALID_ARG: return "invalid argument";
         case SYN_E_CHUNK_LEN: return "chunk length outside [1, 32]";
+        case -20: return "scheduler: no live request with this id";
+        case -21: return "scheduler: a live request with this id exists already";
+        case -22: return "scheduler: the request cannot take this call in its present state";
+        case -23: return "scheduler: commit without a peeked batch";
         case SYN_E_UNCACHED: return "n_uncached outside [1, chunk length]";
         case SYN_E_PAGE_OOB: return "page id out of range";
         case SYN_E_CAPACITY: return "context + chunk exceeds the page table";

@@ -2,10 +2,14 @@
 
     python -m paper_2511_07423_b200.opbench linear --T 544 --N 28672 --K 4096
     python -m paper_2511_07423_b200.opbench attention --config 3
+    python -m paper_2511_07423_b200.opbench sched --config 2 --rounds 8
 
 `attention` builds a one-layer model with the attention geometry of the chosen configuration
 and that configuration's request mix (seeded synthetic cache), so one launch reads one layer's
-worth of the configuration's KV.
+worth of the configuration's KV.  `sched` drives the verification-aware scheduler with the
+configuration's request mix: every request's context arrives as a prompt (prefilled in 32-token
+chunks, prompts first), then each request offloads `--rounds` chunks drawn from the mix; it
+reports the iterations by kind and the share of the wall time spent in the scheduler's own code.
 """
 from __future__ import annotations
 
@@ -79,6 +83,57 @@ def bench_attention(a):
                       "attn_tflops": st.attn_flops / ms_att / 1e9}))
 
 
+def bench_sched(a):
+    import time
+    wl = CONFIGS[a.config]
+    shape = wl.shape
+    model = synthetic.load_model(shape, wl.seed)
+    batch = gen.gen_batch(wl)
+    B = batch.n_req
+    n_pages = int(batch.n_pages + B * (a.rounds * 2 + 2))
+    kv = syn.KVCache(model, n_pages)
+    sched = syn.Scheduler(kv, max_batch_tokens=a.budget)
+    t_start = time.perf_counter()
+    for r in range(B):
+        sched.add_request(r, gen.gen_context_tokens(wl, r, int(batch.ctx_lens[r])))
+    rounds = [0] * B
+    per_kind = {"prefill": [0, 0.0, 0], "verify": [0, 0.0, 0]}
+    while True:
+        t0 = time.perf_counter()
+        kind, results = sched.step()
+        dt = time.perf_counter() - t0
+        if kind == "idle":
+            break
+        e = per_kind[kind]
+        e[0] += 1
+        e[1] += dt
+        e[2] += sum(x["n_tokens"] for x in results)
+        for x in results:
+            r = x["req_id"]
+            if not x["prompt_done"]:
+                continue
+            if rounds[r] >= a.rounds:
+                sched.finish(r)
+                continue
+            # the device's next chunk: the correction token, then drafts (uniform ids: the timing does
+            # not depend on how many are accepted)
+            n = int(batch.chunk_lens[r])
+            chunk = [x["correction_token"]] + gen.gen_context_tokens(wl, 1000 + r, rounds[r] + n)[rounds[r]:rounds[r] + n - 1].tolist()
+            sched.add_verify(r, chunk, 1)
+            rounds[r] += 1
+    wall = time.perf_counter() - t_start
+    assert model.status() == 0
+    st = sched.stats()
+    out = {"op": "sched", "config": wl.name, "n_req": B, "rounds": a.rounds, "max_batch_tokens": a.budget,
+           "wall_s": wall, "scheduler_host_s": st.host_seconds, "execute_s": st.execute_seconds,
+           "scheduler_share_of_library_time": st.host_seconds / (st.host_seconds + st.execute_seconds),
+           "deferred": st.deferred}
+    for k, (n, t, tok) in per_kind.items():
+        out[k] = {"iterations": n, "tokens": tok, "ms_per_iteration": 1e3 * t / max(1, n), "tokens_per_s": tok / max(t, 1e-9)}
+    out["scheduler_us_per_iteration"] = 1e6 * st.host_seconds / max(1, st.iterations[1] + st.iterations[2])
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="op", required=True)
@@ -91,8 +146,12 @@ def main():
     t.add_argument("--config", type=int, default=3)
     t.add_argument("--pool-tokens", type=int, default=None)
     t.add_argument("--iters", type=int, default=10)
+    c = sub.add_parser("sched")
+    c.add_argument("--config", type=int, default=2)
+    c.add_argument("--rounds", type=int, default=8)
+    c.add_argument("--budget", type=int, default=2048, help="chunk tokens per iteration")
     a = ap.parse_args()
-    {"linear": bench_linear, "attention": bench_attention}[a.op](a)
+    {"linear": bench_linear, "attention": bench_attention, "sched": bench_sched}[a.op](a)
 
 
 if __name__ == "__main__":

@@ -35,13 +35,18 @@ class OracleRequest:
 
 
 def oracle_teacher_forced(orc: Oracle, glob, layer_w: Callable[[int], dict], pools, page_table, ctx: int, wl: Workload,
-                          req: int, n: int, want_logits=True, u: int = 1) -> OracleRequest:
+                          req: int, n: int, want_logits=True, u: int = 1,
+                          head: Optional[Sequence[int]] = None) -> OracleRequest:
     """Build request `req`'s chunk by the sequential rule (u device-accepted tokens: the anchor, then
     uniform ids; draft j = the oracle's argmax after the actual earlier chunk tokens with
     probability p_match, else uniform) while running the oracle token by token, which is
     bit-identical to its one-shot chunk forward."""
     assert 1 <= u <= n
-    chunk = [gen.gen_anchor(wl, req)] + [int(x) for x in gen.gen_context_tokens(wl, req, u - 1)]
+    if head is not None:   # the accepted tokens are given (a running draft-and-verify loop)
+        assert len(head) == u
+        chunk = [int(x) for x in head]
+    else:
+        chunk = [gen.gen_anchor(wl, req)] + [int(x) for x in gen.gen_context_tokens(wl, req, u - 1)]
     t1, t2, gp, lg = [], [], [], []
     for j in range(n):
         r = orc.forward_chunk(glob, layer_w, pools, page_table, ctx + j, [chunk[j]], u=1, want_logits=want_logits)

@@ -1,4 +1,4 @@
-"""The C-ABI library loads without a GPU and exports every function include/synera.h declares;
+"""The C-ABI library loads without a GPU and exports every function include/*.h declares;
 the Python binding lists the same names.  No compute call is made here."""
 import ctypes
 import os
@@ -8,9 +8,13 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared():
-    text = open(os.path.join(ROOT, "include", "synera.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(syn_[a-z0-9_]+)\s*\(", text)))
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in sorted(os.listdir(inc)):
+        if f.endswith(".h"):
+            text = re.sub(r"/\*.*?\*/", "", open(os.path.join(inc, f)).read(), flags=re.S)
+            names |= set(re.findall(r"\b(syn_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_header_declares_the_three_calls_of_the_problem_statement():
@@ -28,7 +32,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_binding_lists_the_header_names():
     from paper_2511_07423_b200 import binding
-    assert sorted(binding.EXPORTS) == _declared()
+    assert sorted(binding.EXPORTS + binding.SCHED_EXPORTS) == _declared()
 
 
 def test_strerror_names_every_code_without_a_device():
@@ -40,6 +44,8 @@ def test_strerror_names_every_code_without_a_device():
         assert s and s != "unknown error"
         seen.add(s)
     assert len(seen) == 12
+    for code in range(-20, -24, -1):   # the scheduler's codes
+        assert lib.syn_strerror(code).decode().startswith("scheduler:")
     assert lib.syn_strerror(-99).decode() == "unknown error"
 
 
