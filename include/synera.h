@@ -197,7 +197,8 @@ int syn_plan_host(const syn_model_desc *desc, uint32_t n_pages, uint32_t page_si
  * every launch with CUDA events on the caller's stream.  syn_get_profile synchronises the device,
  * adds up the elapsed time and launch count of each class since the last call, and clears them.
  * Classes: 0 prep, 1 qkv GEMM, 2 attention, 3 attention merge, 4 o GEMM, 5 gate/up GEMM,
- * 6 down GEMM, 7 lm_head GEMM, 8 verify, 9 residual + norm statistic.  ms, launches: HOST arrays
+ * 6 down GEMM, 7 lm_head GEMM, 8 verify (greedy compare, and the sampling stage of
+ * syn_verify_batch_sampled), 9 residual + norm statistic.  ms, launches: HOST arrays
  * of SYN_N_KERNEL_CLASSES. */
 #define SYN_N_KERNEL_CLASSES 10
 int syn_set_profile(syn_model *m, int on);
@@ -244,6 +245,48 @@ int syn_op_attention(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer
 #define SYN_STATIC_MAX_PARTS 256
 int syn_op_attention_static(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer, const void *q, void *out,
                             void *cuda_stream);
+
+/* Sampling-based verification (paper Sec. 4.2, "Compression before transmission": for
+ * verification the LLM needs the drafts and the SLM's distributions, of which the device sends
+ * the most probable entries as its sampling method, top-1 / top-k / top-p, keeps them; Sec. 3.1:
+ * draft and verify).  The step is syn_verify_batch's; the greedy compare is replaced by:
+ *   q_t  = the LLM's distribution at chunk index t as its own sampling method keeps it:
+ *          softmax(logits / temperature) over the top_k largest logits (ties: lower id), then the
+ *          shortest prefix, in decreasing probability, whose mass reaches top_p of that; renormalised;
+ *   draft at chunk index t >= u_i (token x) with transmitted SLM probability p_t(x) is kept iff
+ *          rand_accept[t] * p_t(x) < q_{t-1}(x)           (probability min(1, q / p));
+ *   accept_len = number of leading drafts kept; at the first draft not kept the correction token
+ *          is drawn from the positive part of q_{t-1} - p_t, otherwise from q at the last chunk
+ *          index: inverse CDF at rand_sample[i] over the candidates in increasing token id.
+ * top_k = 1 with the SLM sending its top-1 is the greedy rule.
+ * HOST inputs beside syn_verify_batch's: slm_ids / slm_probs [T][slm_k], row t = the transmitted
+ * distribution chunk token t was drawn from (rows of the u_i accepted tokens are ignored; id -1 =
+ * unused entry; probabilities in [0, 1], used as sent); rand_accept [T] and rand_sample [n_req],
+ * uniform in [0, 1), drawn by the caller.
+ * logits_out: NULL (the library keeps the step's logits in its own workspace) or DEVICE fp32
+ * [T][vocab].  Errors: those of syn_verify_batch; SYN_E_INVALID_ARG for a configuration outside
+ * 1 <= top_k, slm_k <= SYN_SAMPLE_MAX_K, 0 < top_p <= 1, temperature > 0, or a draw outside [0, 1);
+ * SYN_E_TOKEN_OOB for an SLM id outside [-1, vocab). */
+#define SYN_SAMPLE_MAX_K 64
+typedef struct {
+    int32_t top_k;
+    float top_p;
+    float temperature;
+    int32_t slm_k;
+} syn_sampling;
+int syn_verify_batch_sampled(syn_model *m, syn_kv *kv, int32_t n_req, const int64_t *req_ids,
+                             const int32_t *chunk_tokens, const int32_t *chunk_offsets, const int32_t *page_tables,
+                             int32_t max_pages, const int32_t *ctx_lens, const int32_t *n_uncached,
+                             const syn_sampling *cfg, const int32_t *slm_ids, const float *slm_probs,
+                             const float *rand_accept, const float *rand_sample, int32_t *accept_len,
+                             int32_t *correction_token, float *logits_out, void *cuda_stream);
+
+/* The sampling stage alone, on logits the caller supplies (DEVICE fp32 [T][vocab]; everything
+ * else HOST, as above): per-kernel parity and timing.  Needs no model.  Synchronises cuda_stream. */
+int syn_op_sample_verify(const float *logits, int32_t T, int32_t vocab, int32_t n_req, const int32_t *chunk_tokens,
+                         const int32_t *chunk_offsets, const int32_t *n_uncached, const syn_sampling *cfg,
+                         const int32_t *slm_ids, const float *slm_probs, const float *rand_accept,
+                         const float *rand_sample, int32_t *accept_len, int32_t *correction_token, void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -1,4 +1,5 @@
 """B200-native cloud verification step of Synera (arxiv 2511.07423): thin Python binding
 over the C ABI of libsynera.so.  All computation runs in the library's CUDA kernels."""
 from .binding import (SynError, Model, KVCache, Plan, StepStats, lib_path, load_library,  # noqa: F401
-                      syn_op_linear, plan_host, Scheduler, SchedStats)
+                      syn_op_linear, plan_host, Scheduler, SchedStats, Sampling, verify_batch_sampled,
+                      syn_op_sample_verify)

@@ -57,7 +57,7 @@ _LIB: Optional[C.CDLL] = None
 EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "syn_kv_import", "syn_kv_export",
            "syn_verify_batch", "syn_plan_create", "syn_plan_free", "syn_verify_run", "syn_model_status",
            "syn_last_step_stats", "syn_plan_host", "syn_strerror", "syn_last_cuda_error", "syn_op_linear", "syn_op_attention", "syn_op_attention_static",
-           "syn_set_profile", "syn_get_profile"]
+           "syn_set_profile", "syn_get_profile", "syn_verify_batch_sampled", "syn_op_sample_verify"]
 SCHED_EXPORTS = ["syn_sched_create", "syn_sched_free", "syn_sched_add_request", "syn_sched_add_verify", "syn_sched_finish",
                  "syn_sched_peek", "syn_sched_commit", "syn_sched_step", "syn_sched_get_stats"]
 
@@ -219,6 +219,52 @@ class KVCache:
             C.c_void_p(acc.data_ptr()), C.c_void_p(cor.data_ptr()),
             C.c_void_p(logits.data_ptr()) if logits is not None else None, _stream_ptr(stream)), "syn_verify_batch")
         return (acc, cor, logits) if want_logits else (acc, cor)
+
+
+class Sampling(C.Structure):
+    """syn_sampling: the LLM's sampling method and the width of the transmitted SLM rows."""
+    _fields_ = [("top_k", C.c_int32), ("top_p", C.c_float), ("temperature", C.c_float), ("slm_k", C.c_int32)]
+
+
+def _f32(t) -> torch.Tensor:
+    return torch.as_tensor(t, dtype=torch.float32, device="cpu").contiguous()
+
+
+def verify_batch_sampled(kv: "KVCache", chunk_tokens, chunk_offsets, page_tables, ctx_lens, n_uncached, cfg: Sampling,
+                         slm_ids, slm_probs, rand_accept, rand_sample, want_logits: bool = False, stream=None):
+    """syn_verify_batch_sampled with HOST metadata.  Returns (accept_len, correction_token[, logits])."""
+    tok, off, ctx, pt = _i32(chunk_tokens), _i32(chunk_offsets), _i32(ctx_lens), _i32(page_tables)
+    n_req = ctx.numel()
+    unc = _i32(n_uncached) if n_uncached is not None else None
+    sid, sp, ra, rs = _i32(slm_ids), _f32(slm_probs), _f32(rand_accept), _f32(rand_sample)
+    acc = torch.empty(n_req, dtype=torch.int32)
+    cor = torch.empty(n_req, dtype=torch.int32)
+    logits = torch.empty(int(off[-1]), kv.model.shape.vocab, dtype=torch.float32, device="cuda") if want_logits else None
+    _check(load_library().syn_verify_batch_sampled(
+        kv.model._h, kv._h, C.c_int32(n_req), None, C.c_void_p(tok.data_ptr()), C.c_void_p(off.data_ptr()),
+        C.c_void_p(pt.data_ptr()), C.c_int32(pt.shape[1]), C.c_void_p(ctx.data_ptr()),
+        C.c_void_p(unc.data_ptr()) if unc is not None else None, C.byref(cfg), C.c_void_p(sid.data_ptr()),
+        C.c_void_p(sp.data_ptr()), C.c_void_p(ra.data_ptr()), C.c_void_p(rs.data_ptr()), C.c_void_p(acc.data_ptr()),
+        C.c_void_p(cor.data_ptr()), C.c_void_p(logits.data_ptr()) if logits is not None else None, _stream_ptr(stream)),
+        "syn_verify_batch_sampled")
+    return (acc, cor, logits) if want_logits else (acc, cor)
+
+
+def syn_op_sample_verify(logits: torch.Tensor, chunk_tokens, chunk_offsets, n_uncached, cfg: Sampling, slm_ids, slm_probs,
+                         rand_accept, rand_sample, stream=None):
+    """The sampling stage alone on device logits fp32 [T, vocab].  Returns (accept_len, correction_token)."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    tok, off, unc = _i32(chunk_tokens), _i32(chunk_offsets), _i32(n_uncached)
+    sid, sp, ra, rs = _i32(slm_ids), _f32(slm_probs), _f32(rand_accept), _f32(rand_sample)
+    n_req = unc.numel()
+    acc = torch.empty(n_req, dtype=torch.int32)
+    cor = torch.empty(n_req, dtype=torch.int32)
+    _check(load_library().syn_op_sample_verify(
+        C.c_void_p(logits.data_ptr()), C.c_int32(logits.shape[0]), C.c_int32(logits.shape[1]), C.c_int32(n_req),
+        C.c_void_p(tok.data_ptr()), C.c_void_p(off.data_ptr()), C.c_void_p(unc.data_ptr()), C.byref(cfg),
+        C.c_void_p(sid.data_ptr()), C.c_void_p(sp.data_ptr()), C.c_void_p(ra.data_ptr()), C.c_void_p(rs.data_ptr()),
+        C.c_void_p(acc.data_ptr()), C.c_void_p(cor.data_ptr()), _stream_ptr(stream)), "syn_op_sample_verify")
+    return acc, cor
 
 
 class Plan:

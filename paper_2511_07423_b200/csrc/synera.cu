@@ -14,6 +14,7 @@
 
 #include "attention.cuh"
 #include "gemm.cuh"
+#include "sampling.cuh"
 
 using namespace syn;
 typedef __nv_bfloat16 bf16;
@@ -182,6 +183,14 @@ struct syn_model {
     int* group_count = nullptr;     // per merge group: partial items completed (zero between launches)
     int part_cap = 0;
     syn_plan* scratch_plan = nullptr;
+    // sampling-based verification (grow-only): logits of a step, the rows' top-k lists, the
+    // transmitted SLM distributions and the uniform draws
+    struct SampleWs {
+        float *logits = nullptr, *topk_logit = nullptr, *slm_prob = nullptr, *rand_accept = nullptr, *rand_sample = nullptr;
+        int *topk_id = nullptr, *slm_id = nullptr;
+        size_t logits_cap = 0;
+        int t_cap = 0, b_cap = 0, slm_cap = 0;
+    } sw;
     int* pinned_out = nullptr;
     int pinned_out_cap = 0;
     // per-class event timing
@@ -301,6 +310,8 @@ extern "C" void syn_model_free(syn_model* m) {
     free_workspace(m);
     cudaFree(m->acc_dev); cudaFree(m->corr_dev); cudaFree(m->part_o); cudaFree(m->part_ml); cudaFree(m->group_count);
     if (m->pinned_out) cudaFreeHost(m->pinned_out);
+    cudaFree(m->sw.logits); cudaFree(m->sw.topk_logit); cudaFree(m->sw.topk_id); cudaFree(m->sw.slm_id);
+    cudaFree(m->sw.slm_prob); cudaFree(m->sw.rand_accept); cudaFree(m->sw.rand_sample);
     if (m->scratch_plan) syn_plan_free(m->scratch_plan);
     for (auto* v : {&m->ev_used, &m->ev_free})
         for (auto& e : *v) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
@@ -1079,7 +1090,187 @@ extern "C" int syn_verify_batch(syn_model* m, syn_kv* kv, int32_t n_req, const i
     return SYN_OK;
 }
 
+// ------------------------------------------------------------------------------------------ sampling-based verification
+
+static int check_sampling(const syn_sampling* cfg, int vocab, int T, int n_req, const int32_t* slm_ids, const float* slm_probs,
+                          const float* rand_accept, const float* rand_sample) {
+    if (!cfg || !slm_ids || !slm_probs || !rand_accept || !rand_sample) return SYN_E_INVALID_ARG;
+    if (cfg->top_k < 1 || cfg->top_k > SYN_SAMPLE_MAX_K || cfg->slm_k < 1 || cfg->slm_k > SYN_SAMPLE_MAX_K) return SYN_E_INVALID_ARG;
+    if (!(cfg->top_p > 0.f && cfg->top_p <= 1.f) || !(cfg->temperature > 0.f)) return SYN_E_INVALID_ARG;
+    for (size_t i = 0; i < (size_t)T * cfg->slm_k; ++i) {
+        if (slm_ids[i] < -1 || slm_ids[i] >= vocab) return SYN_E_TOKEN_OOB;
+        if (!(slm_probs[i] >= 0.f && slm_probs[i] <= 1.f)) return SYN_E_INVALID_ARG;
+    }
+    for (int t = 0; t < T; ++t)
+        if (!(rand_accept[t] >= 0.f && rand_accept[t] < 1.f)) return SYN_E_INVALID_ARG;
+    for (int i = 0; i < n_req; ++i)
+        if (!(rand_sample[i] >= 0.f && rand_sample[i] < 1.f)) return SYN_E_INVALID_ARG;
+    return SYN_OK;
+}
+
+// The two kernels behind the lm_head; every pointer is device memory.
+static int sample_stage(syn_model* prof_m, cudaStream_t st, const float* logits, int T, int V, int n_req, const int* tokens,
+                        const int* offsets, const int* uncached, const syn_sampling& cfg, int* topk_id, float* topk_logit,
+                        const int* slm_id, const float* slm_prob, const float* rand_accept, const float* rand_sample,
+                        int* acc_dev, int* corr_dev) {
+    ProfScope prof(prof_m, 8, st);
+    if (launch_pdl(topk_rows_kernel, dim3(T), dim3(TOPK_THREADS), 0, st, logits, V, offsets, uncached, n_req, (int)cfg.top_k,
+                   topk_id, topk_logit) != cudaSuccess)
+        return SYN_E_CUDA;
+    SampleParams sp;
+    sp.tokens = tokens; sp.offsets = offsets; sp.uncached = uncached;
+    sp.topk_id = topk_id; sp.topk_logit = topk_logit;
+    sp.slm_id = slm_id; sp.slm_prob = slm_prob; sp.rand_accept = rand_accept; sp.rand_sample = rand_sample;
+    sp.accept_len = acc_dev; sp.correction = corr_dev;
+    sp.n_req = n_req; sp.top_k = cfg.top_k; sp.slm_k = cfg.slm_k;
+    sp.top_p = cfg.top_p; sp.inv_temperature = 1.0f / cfg.temperature;
+    if (launch_pdl(sample_verify_kernel, dim3(n_req), dim3(SAMPLE_MAX_K), 0, st, sp) != cudaSuccess) return SYN_E_CUDA;
+    return SYN_OK;
+}
+
+static int ensure_sample_ws(syn_model* m, int T, int B, int slm_k, bool own_logits) {
+    syn_model::SampleWs& w = m->sw;
+    const size_t need_logits = own_logits ? (size_t)T * m->desc.vocab : 0;
+    if (need_logits > w.logits_cap) {
+        cudaFree(w.logits); w.logits = nullptr; w.logits_cap = 0;
+        CU_OK(cudaMalloc(&w.logits, need_logits * 4));
+        w.logits_cap = need_logits;
+    }
+    if (T > w.t_cap) {
+        cudaFree(w.topk_id); cudaFree(w.topk_logit); cudaFree(w.rand_accept);
+        w.topk_id = nullptr; w.topk_logit = nullptr; w.rand_accept = nullptr; w.t_cap = 0;
+        const int cap = (T + 255) / 256 * 256;
+        CU_OK(cudaMalloc(&w.topk_id, (size_t)cap * SAMPLE_MAX_K * 4));
+        CU_OK(cudaMalloc(&w.topk_logit, (size_t)cap * SAMPLE_MAX_K * 4));
+        CU_OK(cudaMalloc(&w.rand_accept, (size_t)cap * 4));
+        w.t_cap = cap;
+        w.slm_cap = 0;
+    }
+    if (T * slm_k > w.slm_cap) {
+        cudaFree(w.slm_id); cudaFree(w.slm_prob);
+        w.slm_id = nullptr; w.slm_prob = nullptr; w.slm_cap = 0;
+        const int cap = w.t_cap * slm_k;
+        CU_OK(cudaMalloc(&w.slm_id, (size_t)cap * 4));
+        CU_OK(cudaMalloc(&w.slm_prob, (size_t)cap * 4));
+        w.slm_cap = cap;
+    }
+    if (B > w.b_cap) {
+        cudaFree(w.rand_sample); w.rand_sample = nullptr; w.b_cap = 0;
+        const int cap = (B + 255) / 256 * 256;
+        CU_OK(cudaMalloc(&w.rand_sample, (size_t)cap * 4));
+        w.b_cap = cap;
+    }
+    return SYN_OK;
+}
+
+extern "C" int syn_verify_batch_sampled(syn_model* m, syn_kv* kv, int32_t n_req, const int64_t* req_ids,
+                                        const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables,
+                                        int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached,
+                                        const syn_sampling* cfg, const int32_t* slm_ids, const float* slm_probs,
+                                        const float* rand_accept, const float* rand_sample, int32_t* accept_len,
+                                        int32_t* correction_token, float* logits_out, void* cuda_stream) {
+    (void)req_ids;
+    if (!m || !accept_len || !correction_token) return SYN_E_INVALID_ARG;
+    if (!m->scratch_plan) {
+        m->scratch_plan = new (std::nothrow) syn_plan();
+        if (!m->scratch_plan) return SYN_E_OOM;
+    }
+    syn_plan* p = m->scratch_plan;
+    int r = plan_build(p, m, kv, n_req, chunk_tokens, chunk_offsets, page_tables, max_pages, ctx_lens, n_uncached);
+    if (r) return r;
+    if ((r = check_sampling(cfg, (int)m->desc.vocab, p->T, n_req, slm_ids, slm_probs, rand_accept, rand_sample))) return r;
+    if ((r = ensure_workspace(m, p->T, p->n_req, p->n_parts))) return r;
+    if ((r = ensure_sample_ws(m, p->T, n_req, cfg->slm_k, logits_out == nullptr))) return r;
+    if (n_req > m->pinned_out_cap) {
+        if (m->pinned_out) cudaFreeHost(m->pinned_out);
+        m->pinned_out = nullptr; m->pinned_out_cap = 0;
+        const int cap = (n_req + 255) / 256 * 256;
+        CU_OK(cudaMallocHost(&m->pinned_out, (size_t)cap * 12));
+        m->pinned_out_cap = cap;
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    syn_model::SampleWs& w = m->sw;
+    float* logits = logits_out ? logits_out : w.logits;
+    CU_OK(cudaMemcpyAsync(p->dev, p->host, p->used, cudaMemcpyHostToDevice, st));
+    CU_OK(cudaMemcpyAsync(w.slm_id, slm_ids, (size_t)p->T * cfg->slm_k * 4, cudaMemcpyHostToDevice, st));
+    CU_OK(cudaMemcpyAsync(w.slm_prob, slm_probs, (size_t)p->T * cfg->slm_k * 4, cudaMemcpyHostToDevice, st));
+    CU_OK(cudaMemcpyAsync(w.rand_accept, rand_accept, (size_t)p->T * 4, cudaMemcpyHostToDevice, st));
+    CU_OK(cudaMemcpyAsync(w.rand_sample, rand_sample, (size_t)n_req * 4, cudaMemcpyHostToDevice, st));
+    if ((r = run_step(m, kv, p, m->acc_dev, m->corr_dev, nullptr, logits, st))) return r;
+    // the greedy results of the step are replaced by the sampled ones
+    if ((r = sample_stage(m, st, logits, p->T, (int)m->desc.vocab, n_req, p->d<int>(p->o_tokens), p->d<int>(p->o_offsets),
+                          p->d<int>(p->o_uncached), *cfg, w.topk_id, w.topk_logit, w.slm_id, w.slm_prob, w.rand_accept,
+                          w.rand_sample, m->acc_dev, m->corr_dev)))
+        return r;
+    int* po = m->pinned_out;
+    CU_OK(cudaMemcpyAsync(po, m->acc_dev, (size_t)n_req * 4, cudaMemcpyDeviceToHost, st));
+    CU_OK(cudaMemcpyAsync(po + m->pinned_out_cap, m->corr_dev, (size_t)n_req * 4, cudaMemcpyDeviceToHost, st));
+    CU_OK(cudaMemcpyAsync(po + 2 * m->pinned_out_cap, m->status_dev, 4, cudaMemcpyDeviceToHost, st));
+    CU_OK(cudaStreamSynchronize(st));
+    if (po[2 * m->pinned_out_cap]) {
+        cudaMemset(m->status_dev, 0, 4);
+        if (m->group_count) cudaMemset(m->group_count, 0, (size_t)m->part_cap * 4);
+        return SYN_E_DEVICE_TIMEOUT;
+    }
+    memcpy(accept_len, po, (size_t)n_req * 4);
+    memcpy(correction_token, po + m->pinned_out_cap, (size_t)n_req * 4);
+    return SYN_OK;
+}
+
 // ------------------------------------------------------------------------------------------ single ops
+
+// The sampling stage alone on logits the caller supplies (device, fp32 [T][vocab]).
+extern "C" int syn_op_sample_verify(const float* logits, int32_t T, int32_t vocab, int32_t n_req, const int32_t* chunk_tokens,
+                                    const int32_t* chunk_offsets, const int32_t* n_uncached, const syn_sampling* cfg,
+                                    const int32_t* slm_ids, const float* slm_probs, const float* rand_accept,
+                                    const float* rand_sample, int32_t* accept_len, int32_t* correction_token,
+                                    void* cuda_stream) {
+    if (!logits || T <= 0 || vocab <= 0 || n_req <= 0 || !chunk_tokens || !chunk_offsets || !n_uncached || !accept_len ||
+        !correction_token)
+        return SYN_E_INVALID_ARG;
+    if (chunk_offsets[0] != 0 || chunk_offsets[n_req] != T) return SYN_E_INVALID_ARG;
+    for (int i = 0; i < n_req; ++i) {
+        const int n = chunk_offsets[i + 1] - chunk_offsets[i];
+        if (n < 1 || n > SYN_MAX_CHUNK) return SYN_E_CHUNK_LEN;
+        if (n_uncached[i] < 1 || n_uncached[i] > n) return SYN_E_UNCACHED;
+    }
+    for (int t = 0; t < T; ++t)
+        if (chunk_tokens[t] < 0 || chunk_tokens[t] >= vocab) return SYN_E_TOKEN_OOB;
+    int r = check_sampling(cfg, vocab, T, n_req, slm_ids, slm_probs, rand_accept, rand_sample);
+    if (r) return r;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const size_t n_slm = (size_t)T * cfg->slm_k;
+    // one device block: tokens, offsets, uncached, slm ids | slm probs, draws | top-k lists | results
+    const size_t n_i = (size_t)T + (n_req + 1) + n_req + n_slm + (size_t)T * SAMPLE_MAX_K + 2 * (size_t)n_req;
+    const size_t n_f = n_slm + T + n_req + (size_t)T * SAMPLE_MAX_K;
+    int* di = nullptr;
+    float* df = nullptr;
+    CU_OK(cudaMalloc(&di, n_i * 4));
+    if (note_cuda(cudaMalloc(&df, n_f * 4)) != cudaSuccess) { cudaFree(di); return SYN_E_OOM; }
+    int *d_tok = di, *d_off = d_tok + T, *d_unc = d_off + n_req + 1, *d_sid = d_unc + n_req, *d_tid = d_sid + n_slm,
+        *d_acc = d_tid + (size_t)T * SAMPLE_MAX_K, *d_cor = d_acc + n_req;
+    float *d_sp = df, *d_ra = d_sp + n_slm, *d_rs = d_ra + T, *d_tl = d_rs + n_req;
+    std::vector<int> out(2 * (size_t)n_req);
+    bool ok = cudaMemcpyAsync(d_tok, chunk_tokens, (size_t)T * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(d_off, chunk_offsets, (size_t)(n_req + 1) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(d_unc, n_uncached, (size_t)n_req * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(d_sid, slm_ids, n_slm * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(d_sp, slm_probs, n_slm * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(d_ra, rand_accept, (size_t)T * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(d_rs, rand_sample, (size_t)n_req * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    r = ok ? sample_stage(nullptr, st, logits, T, vocab, n_req, d_tok, d_off, d_unc, *cfg, d_tid, d_tl, d_sid, d_sp, d_ra, d_rs,
+                          d_acc, d_cor)
+           : SYN_E_CUDA;
+    if (r == SYN_OK && (note_cuda(cudaMemcpyAsync(out.data(), d_acc, 2 * (size_t)n_req * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+                        note_cuda(cudaStreamSynchronize(st)) != cudaSuccess))
+        r = SYN_E_CUDA;
+    cudaFree(di);
+    cudaFree(df);
+    if (r) return r;
+    memcpy(accept_len, out.data(), (size_t)n_req * 4);
+    memcpy(correction_token, out.data() + n_req, (size_t)n_req * 4);
+    return SYN_OK;
+}
 
 extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, int32_t N, int32_t K, void* cuda_stream) {
     if (!x || !w || !y || T <= 0 || N <= 0 || K <= 0 || K % 8 != 0) return SYN_E_INVALID_ARG;

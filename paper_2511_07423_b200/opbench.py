@@ -3,6 +3,7 @@
     python -m paper_2511_07423_b200.opbench linear --T 544 --N 28672 --K 4096
     python -m paper_2511_07423_b200.opbench attention --config 3
     python -m paper_2511_07423_b200.opbench sched --config 2 --rounds 8
+    python -m paper_2511_07423_b200.opbench sample --config 3
 
 `attention` builds a one-layer model with the attention geometry of the chosen configuration
 and that configuration's request mix (seeded synthetic cache), so one launch reads one layer's
@@ -10,6 +11,8 @@ worth of the configuration's KV.  `sched` drives the verification-aware schedule
 configuration's request mix: every request's context arrives as a prompt (prefilled in 32-token
 chunks, prompts first), then each request offloads `--rounds` chunks drawn from the mix; it
 reports the iterations by kind and the share of the wall time spent in the scheduler's own code.
+`sample` times the sampling-verification stage (top-k of the logits rows + the per-request kernel)
+behind a one-layer model with the configuration's vocabulary and request mix.
 """
 from __future__ import annotations
 
@@ -134,6 +137,41 @@ def bench_sched(a):
     print(json.dumps(out))
 
 
+def bench_sample(a):
+    wl = CONFIGS[a.config]
+    s = wl.shape
+    shape = ModelShape(f"sample-{s.name}", 1, s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, 1024, s.vocab)
+    model = synthetic.load_model(shape, wl.seed)
+    batch = gen.gen_batch(wl)
+    kv = syn.KVCache(model, batch.n_pages)
+    T, B = batch.n_tokens, batch.n_req
+    toks = gen.gen_context_tokens(wl, 0, T)
+    key = rng.stream_key(wl.seed, 4242)
+    slm_k = a.slm_k
+    # transmitted rows: the draft itself with probability 0.5, the rest spread over random ids
+    slm_ids = rng.randint(key, 0, T * slm_k, 0, s.vocab - 1).to(torch.int32).view(T, slm_k)
+    slm_ids[:, 0] = toks
+    slm_probs = torch.full((T, slm_k), 0.5 / max(1, slm_k - 1))
+    slm_probs[:, 0] = 0.5 if slm_k > 1 else 1.0
+    ra = rng.uniform01(key, 1 << 20, T).float().clamp_(0, 0.999999)
+    rs = rng.uniform01(key, 2 << 20, B).float().clamp_(0, 0.999999)
+    cfg = syn.Sampling(a.top_k, a.top_p, 1.0, slm_k)
+    args = (kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, batch.n_uncached, cfg, slm_ids, slm_probs, ra, rs)
+    for _ in range(3):
+        syn.verify_batch_sampled(*args)
+    model.set_profile(True)
+    model.get_profile()
+    for _ in range(a.iters):
+        syn.verify_batch_sampled(*args)
+    prof = model.get_profile()
+    ms = prof["verify"][0] / a.iters          # greedy compare + top-k rows + sampling kernel, per step
+    rows = int((batch.chunk_lens - batch.n_uncached + 1).sum())
+    by = rows * s.vocab * 4
+    print(json.dumps({"op": "sample", "config": wl.name, "T": T, "rows_with_a_distribution": rows, "vocab": s.vocab,
+                      "top_k": a.top_k, "top_p": a.top_p, "slm_k": slm_k, "ms_sampling_stage": ms, "logit_bytes_read_once": by,
+                      "gbs": by / ms / 1e6}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="op", required=True)
@@ -146,12 +184,18 @@ def main():
     t.add_argument("--config", type=int, default=3)
     t.add_argument("--pool-tokens", type=int, default=None)
     t.add_argument("--iters", type=int, default=10)
+    m = sub.add_parser("sample")
+    m.add_argument("--config", type=int, default=3)
+    m.add_argument("--top-k", type=int, default=50)
+    m.add_argument("--top-p", type=float, default=0.9)
+    m.add_argument("--slm-k", type=int, default=20)
+    m.add_argument("--iters", type=int, default=10)
     c = sub.add_parser("sched")
     c.add_argument("--config", type=int, default=2)
     c.add_argument("--rounds", type=int, default=8)
     c.add_argument("--budget", type=int, default=2048, help="chunk tokens per iteration")
     a = ap.parse_args()
-    {"linear": bench_linear, "attention": bench_attention, "sched": bench_sched}[a.op](a)
+    {"linear": bench_linear, "attention": bench_attention, "sched": bench_sched, "sample": bench_sample}[a.op](a)
 
 
 if __name__ == "__main__":

@@ -1,0 +1,177 @@
+"""Sampling-based verification on the GPU against the float64 oracle (oracle/sampling.py).
+
+Kernel level (syn_op_sample_verify): both sides get the same fp32 logits, so the decisions differ only
+by float32 rounding of the probabilities; results must be equal wherever the oracle's margin (relative
+distance of the nearest consulted decision from flipping) exceeds 1e-4.  End to end
+(syn_verify_batch_sampled): the logits differ by the bf16 operand rounding of the forward, at most
+eps = 0.03 x the standard deviation of the oracle's logits (asserted).  A logit error eps moves a kept
+probability by at most a factor exp(2 eps / temperature) and can swap two tokens at the top-k boundary
+only if they are closer than 2 eps; so equality is required where every consulted top-k boundary is
+wider than 2 eps and the margin exceeds 4 eps / temperature (twice the first-order bound).  Every
+result must be in range.  With random weights the logits are near-Gaussian and the boundary of a wide
+top-k is almost never 2 eps wide (the k-th and (k+1)-th of thousands of logits are close), so the
+wide case asserts the overall agreement rate instead (a swap of two near-equal boundary tokens changes
+the outcome only when one of them is the draft or is drawn)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import Oracle
+from oracle.sampling import llm_distribution, verify_sampled
+from workloads import gen
+from workloads.configs import MINI_8B, TINY, Workload
+
+from harness import cpu_model, fill_synthetic_kv, to_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+def _slm_rows(rng, logits_prev, chunk, u, slm_k, V, temp, mode):
+    """Transmitted SLM distributions and drafts: the SLM is a noisy copy of the LLM's logits; draft t
+    is drawn from the SLM's kept distribution (or, mode 'greedy', is its top-1)."""
+    n = len(chunk)
+    ids = np.full((n, slm_k), -1, dtype=np.int32)
+    probs = np.zeros((n, slm_k), dtype=np.float32)
+    for t in range(u, n):
+        noisy = logits_prev[t - 1] + rng.normal(size=V) * 1.0
+        kid, q, _, _ = llm_distribution(noisy, slm_k, 1.0, temp)
+        ids[t, :len(kid)] = kid
+        probs[t, :len(kid)] = q.astype(np.float32)
+        chunk[t] = int(kid[0]) if mode == "greedy" else int(rng.choice(kid, p=q))
+    return ids, probs
+
+
+@pytest.mark.parametrize("V,top_k,top_p,temp,slm_k", [
+    (1000, 8, 1.0, 1.0, 8), (32000, 50, 0.9, 0.7, 20), (151, 64, 0.5, 1.3, 64), (4099, 1, 1.0, 1.0, 1),
+    (128256, 40, 0.95, 1.0, 40),
+])
+def test_sampling_stage_matches_the_oracle_on_the_same_logits(V, top_k, top_p, temp, slm_k):
+    import paper_2511_07423_b200 as syn
+    rng = np.random.default_rng(V + top_k)
+    chunks = [(5, 1), (9, 3), (1, 1), (16, 16), (32, 2), (7, 6)]      # (n, u)
+    T = sum(n for n, _ in chunks)
+    logits = (rng.normal(size=(T, V)) * 2.0).astype(np.float32)
+    logits[3, 10:14] = logits[3].max() + 1.0                      # exact ties at the top: lower ids first
+    logits[1, :] = 1.0                                            # a constant row: the first k ids
+    logits[2, ::3] = logits[2].max() + 2.0                        # a third of the row ties at the top
+    offs, toks, unc = [0], [], []
+    slm_ids = np.full((T, slm_k), -1, dtype=np.int32)
+    slm_probs = np.zeros((T, slm_k), dtype=np.float32)
+    for n, u in chunks:
+        b = offs[-1]
+        chunk = [int(x) for x in rng.integers(0, V, size=n)]
+        ids, probs = _slm_rows(rng, logits[b:b + n].astype(np.float64), chunk, u, slm_k, V, temp,
+                               "greedy" if top_k == 1 else "sample")
+        slm_ids[b:b + n], slm_probs[b:b + n] = ids, probs
+        toks += chunk
+        unc.append(u)
+        offs.append(b + n)
+    n_strict = 0
+    for trial in range(6):
+        ra = rng.random(T).astype(np.float32)
+        rs = rng.random(len(chunks)).astype(np.float32)
+        cfg = syn.Sampling(top_k, top_p, temp, slm_k)
+        acc, cor = syn.syn_op_sample_verify(torch.from_numpy(logits).cuda(), toks, offs, unc, cfg, slm_ids, slm_probs, ra, rs)
+        for i, (n, u) in enumerate(chunks):
+            b = offs[i]
+            o = verify_sampled(logits[b:b + n].astype(np.float64), toks[b:b + n], u, slm_ids[b:b + n],
+                               slm_probs[b:b + n].astype(np.float64), ra[b:b + n], float(rs[i]), top_k, top_p, temp)
+            assert 0 <= int(acc[i]) <= n - u and 0 <= int(cor[i]) < V
+            if o.margin > 1e-4:
+                n_strict += 1
+                assert (int(acc[i]), int(cor[i])) == (o.accept_len, o.correction), (trial, i, o)
+    assert n_strict >= 15, n_strict
+
+
+def test_rejects_bad_configurations_and_draws():
+    import paper_2511_07423_b200 as syn
+    lg = torch.zeros(2, 10, device="cuda")
+    ok = dict(chunk_tokens=[1, 2], chunk_offsets=[0, 2], n_uncached=[1], slm_ids=[[1], [2]], slm_probs=[[1.0], [1.0]],
+              rand_accept=[0.1, 0.2], rand_sample=[0.3])
+
+    def code(cfg, **kw):
+        a = dict(ok); a.update(kw)
+        with pytest.raises(syn.SynError) as e:
+            syn.syn_op_sample_verify(lg, a["chunk_tokens"], a["chunk_offsets"], a["n_uncached"], cfg, a["slm_ids"],
+                                     a["slm_probs"], a["rand_accept"], a["rand_sample"])
+        return e.value.code
+
+    good = syn.Sampling(1, 1.0, 1.0, 1)
+    acc, cor = syn.syn_op_sample_verify(lg, ok["chunk_tokens"], ok["chunk_offsets"], ok["n_uncached"], good, ok["slm_ids"],
+                                        ok["slm_probs"], ok["rand_accept"], ok["rand_sample"])
+    assert (int(acc[0]), int(cor[0])) == (0, 0)      # all logits equal: the LLM's top-1 is token 0, the draft 2 is not kept
+    assert code(syn.Sampling(0, 1.0, 1.0, 1)) == -1 and code(syn.Sampling(65, 1.0, 1.0, 1)) == -1
+    assert code(syn.Sampling(1, 0.0, 1.0, 1)) == -1 and code(syn.Sampling(1, 1.0, 0.0, 1)) == -1
+    assert code(good, rand_accept=[0.1, 1.0]) == -1 and code(good, rand_sample=[-0.1]) == -1
+    assert code(good, slm_ids=[[1], [10]]) == -6 and code(good, slm_probs=[[1.0], [1.5]]) == -1
+    assert code(good, n_uncached=[3]) == -3
+
+
+@pytest.mark.parametrize("shape,top_k,top_p,temp,min_strict", [
+    (TINY, 8, 1.0, 1.0, 6), (MINI_8B, 3, 1.0, 0.8, 6), (MINI_8B, 20, 0.9, 0.8, 0)])
+def test_step_with_sampled_verification_matches_the_oracle(shape, top_k, top_p, temp, min_strict):
+    import paper_2511_07423_b200 as syn
+    ctx, chunk_lens, unc = [0, 40, 130, 61, 300], [6, 9, 16, 1, 24], [1, 2, 1, 1, 20]
+    wl = Workload("s", shape, 31, len(ctx), ("list", tuple(ctx)), ("list", tuple(chunk_lens)), 0.7)
+    batch = gen.gen_batch(wl)
+    glob, layers = cpu_model(shape, wl.seed)
+    gg, gl = to_cuda(glob, layers)
+    model = syn.Model(shape, gg, gl)
+    kv = syn.KVCache(model, batch.n_pages)
+    orc = Oracle(shape)
+    pools = orc.new_pool(batch.n_pages)
+    fill_synthetic_kv(shape, wl.seed, batch, range(batch.n_req), kv=kv, orc=orc, pools=pools)
+    rng = np.random.default_rng(3)
+    V, slm_k = shape.vocab, 12
+    offs = batch.chunk_offsets.tolist()
+    T = batch.n_tokens
+    toks = np.zeros(T, dtype=np.int32)
+    slm_ids = np.full((T, slm_k), -1, dtype=np.int32)
+    slm_probs = np.zeros((T, slm_k), dtype=np.float32)
+    ora_logits = []
+    # the oracle runs token by token; the SLM's row for chunk index t is a noisy copy of the oracle's logits at t - 1
+    for r in range(batch.n_req):
+        n, u, c0 = chunk_lens[r], unc[r], ctx[r]
+        chunk = [int(x) for x in rng.integers(0, V, size=n)]
+        rows = []
+        for t in range(n):
+            if t >= u:
+                noisy = rows[t - 1] + rng.normal(size=V) * 0.5 * rows[t - 1].std()
+                kid, q, _, _ = llm_distribution(noisy, slm_k, 1.0, temp)
+                slm_ids[offs[r] + t, :len(kid)] = kid
+                slm_probs[offs[r] + t, :len(kid)] = q.astype(np.float32)
+                chunk[t] = int(rng.choice(kid, p=q))
+            res = orc.forward_chunk(glob, lambda l: layers[l], pools, batch.page_tables[r].numpy(), c0 + t, [chunk[t]], u=1,
+                                    want_logits=True)
+            rows.append(res.logits[0])
+        toks[offs[r]:offs[r + 1]] = chunk
+        ora_logits.append(np.stack(rows))
+    n_strict = n_equal = n_all = 0
+    cfg = syn.Sampling(top_k, top_p, temp, slm_k)
+    eps = 0.03 * float(np.concatenate(ora_logits).std())
+    for trial in range(12):
+        ra = rng.random(T).astype(np.float32)
+        rs = rng.random(batch.n_req).astype(np.float32)
+        acc, cor, lg = syn.verify_batch_sampled(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, unc, cfg,
+                                                slm_ids, slm_probs, ra, rs, want_logits=True)
+        assert model.status() == 0
+        if trial == 0:
+            ref = np.concatenate(ora_logits)
+            assert np.abs(lg.cpu().numpy() - ref).max() <= 0.03 * ref.std()
+        for r in range(batch.n_req):
+            b, n = offs[r], chunk_lens[r]
+            o = verify_sampled(ora_logits[r], toks[b:b + n], unc[r], slm_ids[b:b + n], slm_probs[b:b + n].astype(np.float64),
+                               ra[b:b + n], float(rs[r]), top_k, top_p, temp)
+            assert 0 <= int(acc[r]) <= n - unc[r] and 0 <= int(cor[r]) < V
+            n_all += 1
+            n_equal += (int(acc[r]), int(cor[r])) == (o.accept_len, o.correction)
+            if o.margin > 4 * eps / temp and o.topk_gap > 2 * eps:
+                n_strict += 1
+                assert (int(acc[r]), int(cor[r])) == (o.accept_len, o.correction), (trial, r, o)
+        # without its own logits buffer the library keeps them itself: same results
+        acc2, cor2 = syn.verify_batch_sampled(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, unc, cfg,
+                                              slm_ids, slm_probs, ra, rs)
+        assert torch.equal(acc, acc2) and torch.equal(cor, cor2)
+    print(shape.name, "top_k", top_k, "strict", n_strict, "equal", n_equal, "of", n_all, "eps", eps)
+    assert n_strict >= min_strict, n_strict
+    assert n_equal >= 0.6 * n_all, (n_equal, n_all)
