@@ -4,6 +4,7 @@
     python -m paper_2511_07423_b200.opbench attention --config 3
     python -m paper_2511_07423_b200.opbench sched --config 2 --rounds 8
     python -m paper_2511_07423_b200.opbench sample --config 3
+    python -m paper_2511_07423_b200.opbench scale --config 2 --budgets 0.3,0.6,0.9 --rates 2,4,8,16,32
 
 `attention` builds a one-layer model with the attention geometry of the chosen configuration
 and that configuration's request mix (seeded synthetic cache), so one launch reads one layer's
@@ -13,6 +14,12 @@ chunks, prompts first), then each request offloads `--rounds` chunks drawn from 
 reports the iterations by kind and the share of the wall time spent in the scheduler's own code.
 `sample` times the sampling-verification stage (top-k of the logits rows + the per-request kernel)
 behind a one-layer model with the configuration's vocabulary and request mix.
+`scale` is the scalability experiment of the paper's Sec. 6.4 in shape: sessions arrive at a given
+rate, every session's device drafts chunks of gamma tokens at a fixed pace and offloads a chunk with
+probability = the offloading budget (tokens of chunks it keeps to itself ride along as uncached
+tokens of the next offload); the cloud is the scheduler over the real model on this GPU.  Device
+time is simulated, cloud time is the measured wall time of every iteration; the output is the
+verification latency per request (submission to result) against the arrival rate.
 """
 from __future__ import annotations
 
@@ -172,6 +179,109 @@ def bench_sample(a):
                       "gbs": by / ms / 1e6}))
 
 
+def bench_scale(a):
+    import heapq
+    import math
+    import random
+    import time
+    wl = CONFIGS[a.config]
+    shape = wl.shape
+    model = synthetic.load_model(shape, wl.seed)
+    lo, hi = wl.ctx[1], wl.ctx[2]                      # prompt lengths: the configuration's context range
+    n_pages = int(a.max_sessions * ((hi + a.out_tokens + 64) // 16 + 1))
+    kv = syn.KVCache(model, n_pages)
+    for budget in [float(x) for x in a.budgets.split(",")]:
+        for rate in [float(x) for x in a.rates.split(",")]:
+            rnd = random.Random(int(1000 * budget) * 7919 + int(100 * rate))
+            sched = syn.Scheduler(kv, max_batch_tokens=a.budget_tokens)
+            ev = []                                    # (time, seq, kind, session)
+            seq = 0
+            t = 0.0
+            while t < a.horizon:                       # Poisson arrivals
+                t += rnd.expovariate(rate)
+                heapq.heappush(ev, (t, seq, "arrive", seq)); seq += 1
+            sess = {}
+            now, busy = 0.0, 0.0
+            lat, n_done, n_drop, iters = [], 0, 0, {"prefill": 0, "verify": 0}
+            submitted = {}
+            while True:
+                while ev and ev[0][0] <= now:
+                    _, _, kind, sid = heapq.heappop(ev)
+                    if kind == "arrive":
+                        if len(sess) >= a.max_sessions:
+                            n_drop += 1
+                            continue
+                        sess[sid] = {"gen": 0, "pend": []}
+                        sched.add_request(sid, [rnd.randrange(shape.vocab) for _ in range(rnd.randint(lo, hi))])
+                    elif sid in sess:                  # the device has drafted its next chunk
+                        s = sess[sid]
+                        drafts = [rnd.randrange(shape.vocab) for _ in range(a.gamma)]
+                        if rnd.random() < budget or len(s["pend"]) + 2 * a.gamma > 32:
+                            sched.add_verify(sid, s["pend"] + drafts, len(s["pend"]))
+                            submitted[sid] = now
+                        else:                          # kept on the device: accepted locally, cached at the next offload
+                            s["pend"] += drafts
+                            s["gen"] += a.gamma
+                            if s["gen"] >= a.out_tokens:
+                                sched.finish(sid); del sess[sid]; n_done += 1
+                            else:
+                                heapq.heappush(ev, (now + a.gamma * a.device_ms * 1e-3, seq, "chunk", sid)); seq += 1
+                b = sched.peek()
+                if b["kind"] == "idle":
+                    sched.commit()
+                    if not ev:
+                        break
+                    now = max(now, ev[0][0])
+                    if now > a.horizon * 3:
+                        break
+                    continue
+                t0 = time.perf_counter()
+                acc, cor = kv.verify_batch(b["chunk_tokens"], b["chunk_offsets"], b["page_tables"], b["ctx_lens"],
+                                           n_uncached=b["n_uncached"])
+                dt = time.perf_counter() - t0
+                now += dt
+                busy += dt
+                iters[b["kind"]] += 1
+                offs = b["chunk_offsets"].tolist()
+                if b["kind"] == "verify":   # accepted drafts: capped geometric with the workload's match probability
+                    acc_syn = []
+                    for i in range(b["n_req"]):
+                        g = offs[i + 1] - offs[i] - int(b["n_uncached"][i])
+                        k = 0
+                        while k < g and rnd.random() < wl.p_match:
+                            k += 1
+                        acc_syn.append(k)
+                    res = sched.commit(acc_syn, cor)
+                else:
+                    res = sched.commit([0] * b["n_req"], cor)
+                for x in res:
+                    sid = x["req_id"]
+                    if sid not in sess or not x["prompt_done"]:
+                        continue
+                    s = sess[sid]
+                    if x["kind"] == 2:
+                        lat.append(now - submitted.pop(sid) + 2e-3 * a.rtt_ms)
+                        s["gen"] += x["accept_len"] + 1
+                    s["pend"] = [x["correction_token"]]
+                    if s["gen"] >= a.out_tokens:
+                        sched.finish(sid); del sess[sid]; n_done += 1
+                    else:
+                        heapq.heappush(ev, (now + 2e-3 * a.rtt_ms + a.gamma * a.device_ms * 1e-3, seq, "chunk", sid)); seq += 1
+                if now > a.horizon * 3:
+                    break
+            for sid in list(sess):
+                sched.finish(sid)
+            sched.peek(); sched.commit()
+            sched.close()
+            lat.sort()
+            print(json.dumps({"op": "scale", "config": wl.name, "offload_budget": budget, "arrival_rate_per_s": rate,
+                              "sessions_done": n_done, "sessions_dropped": n_drop, "verify_requests": len(lat),
+                              "verify_latency_ms_mean": 1e3 * sum(lat) / max(1, len(lat)),
+                              "verify_latency_ms_p95": 1e3 * lat[int(0.95 * (len(lat) - 1))] if lat else None,
+                              "gpu_busy_fraction": busy / max(now, 1e-9), "virtual_seconds": now,
+                              "iterations": iters}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="op", required=True)
@@ -190,12 +300,23 @@ def main():
     m.add_argument("--top-p", type=float, default=0.9)
     m.add_argument("--slm-k", type=int, default=20)
     m.add_argument("--iters", type=int, default=10)
+    z = sub.add_parser("scale")
+    z.add_argument("--config", type=int, default=2)
+    z.add_argument("--budgets", default="0.3,0.6,0.9")
+    z.add_argument("--rates", default="2,4,8,16,32", help="session arrivals per second")
+    z.add_argument("--horizon", type=float, default=10.0, help="seconds of arrivals (virtual time)")
+    z.add_argument("--out-tokens", type=int, default=128)
+    z.add_argument("--gamma", type=int, default=4)
+    z.add_argument("--device-ms", type=float, default=25.0, help="device time per drafted token")
+    z.add_argument("--rtt-ms", type=float, default=10.0, help="one-way network delay")
+    z.add_argument("--max-sessions", type=int, default=512)
+    z.add_argument("--budget-tokens", type=int, default=2048, help="chunk tokens per iteration")
     c = sub.add_parser("sched")
     c.add_argument("--config", type=int, default=2)
     c.add_argument("--rounds", type=int, default=8)
     c.add_argument("--budget", type=int, default=2048, help="chunk tokens per iteration")
     a = ap.parse_args()
-    {"linear": bench_linear, "attention": bench_attention, "sched": bench_sched, "sample": bench_sample}[a.op](a)
+    {"linear": bench_linear, "attention": bench_attention, "sched": bench_sched, "sample": bench_sample, "scale": bench_scale}[a.op](a)
 
 
 if __name__ == "__main__":
