@@ -18,7 +18,7 @@
 
 using namespace syn;
 typedef __nv_bfloat16 bf16;
-constexpr int GEMM_MAX_SPLITS = 4;   // split-K partial buffers of the o / down projections
+constexpr int GEMM_MAX_SPLITS = 8;   // split-K partial buffers of the o / down projections
 
 // Name of the last CUDA error a call of this library met on this thread (for syn_last_cuda_error).
 static thread_local const char* g_last_cuda_error = "";
@@ -904,7 +904,7 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     g.pair_mode = tiles >= n_sm;
     int n_cta;
     if (ep.mode == EPI_PART && tiles < n_sm) {
-        int sp = std::min(GEMM_MAX_SPLITS, std::min(n_sm / tiles, std::max(1, g.num_kb / 8)));
+        int sp = std::min(GEMM_MAX_SPLITS, std::min(n_sm / tiles, std::max(1, g.num_kb / 4)));
         g.kb_per_split = (g.num_kb + sp - 1) / sp;
         g.splits = (g.num_kb + g.kb_per_split - 1) / g.kb_per_split;
         g.pair_mode = 1;
