@@ -894,12 +894,20 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     g.num_kb = (K + 63) / 64;
     g.n_pairs = (packed_rows + 255) / 256;
     g.n_tt = (T + 255) / 256;
+    if (ep.mode != EPI_PART) {
+        // Few feature tiles and few tokens: narrower token tiles (32 tokens at least) put more SMs to
+        // work; the weights are then read by several CTAs, which costs only L2 bandwidth.
+        const int want = n_sm / std::max(1, 2 * g.n_pairs), most = (T + 31) / 32;
+        g.n_tt = std::max(g.n_tt, std::min(want, most));
+    }
     g.TN = (((T + g.n_tt - 1) / g.n_tt) + 15) / 16 * 16;
+    g.n_tt = (T + g.TN - 1) / g.TN;   // rounding the width up may leave the last tiles without tokens
     g.n_stages = gemm_stages(g.TN);
     g.status = status;
     g.splits = 1;
     g.kb_per_split = g.num_kb;
-    if (g.n_stages < 2) return SYN_E_INVALID_ARG;
+    // every token tile must hold a token: an empty one would issue an MMA of width 0
+    if (g.n_stages < 2 || g.TN < 16 || g.TN > 256 || (g.n_tt - 1) * g.TN >= T) return SYN_E_INVALID_ARG;
     const int tiles = g.n_pairs * g.n_tt;
     g.pair_mode = tiles >= n_sm;
     int n_cta;
