@@ -1,7 +1,7 @@
 """Compile the CPU oracle (plain C + OpenMP) into shared objects next to this file.
 
 Two builds of the same source: double precision (the one parity is judged against) and
-single precision (the precision the project brief names; tests show the two agree far
+single precision (a plain fp32 build; tests show the two agree far
 inside the parity tolerance).  TEST INFRASTRUCTURE: the product never loads these.
 """
 from __future__ import annotations

@@ -1,7 +1,7 @@
 """Shared machinery of the GPU parity tests: build the same seeded batch on both sides,
 run the CPU oracle request by request, and judge the CUDA result by the stated rule.
 
-Rule (project brief): accept_len and correction_token bit-exact, except that a chunk
+Parity rule: accept_len and correction_token bit-exact, except that a chunk
 position whose oracle top-2 logit gap is below 0.05 ("soft") may resolve to either of the
 oracle's two best ids; logits within 3e-2 x the standard deviation of the oracle's logits.
 """

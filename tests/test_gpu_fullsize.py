@@ -12,7 +12,7 @@ operands (two normalised hidden states, q/k/v, softmax weights, attention output
 relative rms 2^-9/sqrt(3) each, the errors of the layers add in quadrature, and the maximum over
 millions of logits sits near six standard deviations.  The bound asserted here is that arithmetic
 with a factor 2.5 of slack (wider contractions, K up to 27648, sit above the simple count); the
-measured values are printed and recorded in the design doc."""
+measured values are printed."""
 import numpy as np
 import pytest
 import torch
