@@ -22,8 +22,11 @@ def _case(T, N, K, seed):
     (16, 128, 256),       # several k-blocks, fewer than the ring
     (32, 256, 1024),      # ring wraps (16 k-blocks)
     (50, 300, 192),       # ragged tokens and features
-    (129, 384, 2048),     # token tile of 144 columns
-    (544, 640, 4096),     # three token tiles (192/176/176), 64 k-blocks
+    (129, 384, 2048),     # few feature tiles: five token tiles of 32 columns, the last with one token
+    (544, 640, 4096),     # seventeen token tiles of 32 columns, 64 k-blocks
+    (544, 28672, 512),    # many feature tiles: three token tiles of 192 columns, pair items in full waves + single tiles
+    (137, 4096, 512),     # token tiles of 48 columns: 3 x 48 covers 137, no fourth tile
+    (300, 1024, 320),     # ten token tiles of 32 columns, the last with 12 tokens
     (16, 128, 688),       # K tail: 688 = 10.75 k-blocks (zero-filled by TMA)
     (257, 128, 128),      # two token tiles, the second nearly empty
     (1, 128, 64),         # a single token
