@@ -6,9 +6,11 @@
 // stored pre-tiled and pre-swizzled ([feature pair][k-block][2][128 x 64] images of the
 // 128-byte-swizzled shared-memory tile), so a stage's weights are ONE contiguous bulk copy;
 // activations come through a TMA tensor map.  One persistent CTA per SM walks a static schedule:
-// whole pair tiles in full waves, the remainder as single 128-feature tiles; projections with few
-// output tiles (o, down) split K over CTAs and write fp32 partials that resid_norm_kernel adds to the
-// residual stream in a fixed order.  Every CTA starts its k loop at a different k-block, so the CTAs
+// whole pair tiles in full waves; the pair tiles left over are cut along K into parts on different
+// CTAs (the "helper" parts run first and store their fp32 accumulators, the "owner" part runs last
+// on another CTA, adds them in part order and finishes the tile), or, where K is too short for
+// that, run as single 128-feature tiles; projections with few output tiles (o, down) split K over
+// CTAs and write fp32 partials that resid_norm_kernel adds to the residual stream in a fixed order.  Every CTA starts its k loop at a different k-block, so the CTAs
 // that share a token tile do not ask L2 for the same lines at the same moment.  Accumulation is
 // tcgen05.mma into TMEM, read back with tcgen05.ld by sixteen epilogue warps; a thread then holds one
 // output feature for sixteen tokens, and the epilogues work on those registers:
@@ -287,17 +289,30 @@ struct GemmParams {
     int n_stages;
     int splits, kb_per_split;   // splits > 1: every CTA owns one (pair tile, k range)
     int pair_mode;              // 1: pair tiles in full waves + remainder as singles; 0: all singles
+    int ksplit;                 // pair mode, > 1: the remainder's pair tiles are cut along K into this many parts
+    int kper;                   // ksplit: k-blocks of a helper part, (ksplit - 1) * kper < num_kb
+    float* fix_part;            // ksplit: fp32 partial accumulators of the helper parts, [slot][2][TN/16][4][32][16]
+    int* fix_flag;              // ksplit: per remainder tile, epilogue warps of helpers that have stored; then
+                                // [n_sm + tile]: owner warps that are done reading (the last one clears both)
+    int n_sm;
     int* status;
 };
 
 struct GemmWork {
     int pair, tt, mt_lo, mt_hi, kb0, kb1, split;
+    int role;    // 0: the item's whole K; 1: helper part (accumulators go to fix_part); 2: owner part (adds the helpers')
+    int rtile;   // role 1, 2: index of the remainder tile
+    int hpart;   // role 1: which helper part
 };
 
 // Static schedule: work item i of CTA `cta`.  Returns false when the CTA is done.
+// KSPLIT: the kernel variant that cuts the remainder's pair tiles along K (launched only when
+// GemmParams::ksplit > 1; the plain variant carries none of that code).
+template <bool KSPLIT>
 __device__ __forceinline__ bool gemm_work(const GemmParams& g, int cta, int n_cta, int i, GemmWork& w) {
     const int n_tiles = g.n_pairs * g.n_tt;
     w.split = 0; w.kb0 = 0; w.kb1 = g.num_kb; w.mt_lo = 0; w.mt_hi = 2;
+    w.role = 0; w.rtile = 0; w.hpart = 0;
     if (g.splits > 1) {
         if (i > 0 || cta >= n_tiles * g.splits) return false;
         const int tile = cta / g.splits;
@@ -306,6 +321,39 @@ __device__ __forceinline__ bool gemm_work(const GemmParams& g, int cta, int n_ct
         w.kb0 = w.split * g.kb_per_split;
         w.kb1 = min(g.num_kb, w.kb0 + g.kb_per_split);
         return true;
+    }
+    if (KSPLIT) {
+        // Full waves of pair tiles; the R tiles of the remainder are cut along K into ksplit parts on
+        // different CTAs.  The helper parts run FIRST on CTAs 0 .. R (ksplit - 1) - 1, the owner part
+        // (the last k range) runs LAST on the last R CTAs and adds the helpers' stored accumulators,
+        // which by then have long been written.
+        const int fw = n_tiles / n_cta, R = n_tiles - fw * n_cta, H = g.ksplit - 1;
+        const int kper = g.kper;   // k-blocks of a helper part; the owner takes the (shorter) rest
+        const bool helper = cta < R * H, owner = cta >= n_cta - R;
+        int wave = i;
+        if (helper) {
+            if (i == 0) {
+                w.role = 1; w.rtile = cta / H; w.hpart = cta - w.rtile * H;
+                const int tile = fw * n_cta + w.rtile;
+                w.pair = tile / g.n_tt; w.tt = tile - w.pair * g.n_tt;
+                w.kb0 = w.hpart * kper; w.kb1 = w.kb0 + kper;
+                return true;
+            }
+            wave = i - 1;
+        }
+        if (wave < fw) {
+            const int tile = wave * n_cta + cta;
+            w.pair = tile / g.n_tt; w.tt = tile - w.pair * g.n_tt;
+            return true;
+        }
+        if (owner && wave == fw) {
+            w.role = 2; w.rtile = cta - (n_cta - R);
+            const int tile = fw * n_cta + w.rtile;
+            w.pair = tile / g.n_tt; w.tt = tile - w.pair * g.n_tt;
+            w.kb0 = H * kper; w.kb1 = g.num_kb;
+            return true;
+        }
+        return false;
     }
     if (g.pair_mode) {
         const int fw = n_tiles / n_cta;
@@ -347,6 +395,7 @@ __device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes
                  : "memory");
 }
 
+template <bool KSPLIT>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -390,7 +439,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
             uint32_t it = 0;
             bool ok = true;
             GemmWork w;
-            for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
+            for (int i = 0; ok && gemm_work<KSPLIT>(g, cta, n_cta, i, w); ++i) {
                 const int n0 = w.tt * g.TN;
                 const int nbox = (((min(g.TN, p.T - n0) + 15) & ~15) + 31) >> 5;
                 const uint32_t a_bytes = (uint32_t)(w.mt_hi - w.mt_lo) * GEMM_TILE_BYTES;
@@ -432,7 +481,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
             uint32_t it = 0;
             bool ok = true;
             GemmWork w;
-            for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
+            for (int i = 0; ok && gemm_work<KSPLIT>(g, cta, n_cta, i, w); ++i) {
                 const uint32_t nn = (uint32_t)((min(g.TN, p.T - w.tt * g.TN) + 15) & ~15);
                 const uint32_t idesc = umma_idesc_bf16(128, nn);
                 if (i > 0) {   // the epilogue must have drained the previous item's accumulators
@@ -471,7 +520,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
         bool ok = true;
         GemmWork w;
         pdl_wait();   // the epilogues write buffers that earlier kernels may still read
-        for (int i = 0; ok && gemm_work(g, cta, n_cta, i, w); ++i) {
+        for (int i = 0; ok && gemm_work<KSPLIT>(g, cta, n_cta, i, w); ++i) {
             const int n0 = w.tt * g.TN;
             const int n_valid = min(g.TN, p.T - n0);
             const int nchunks = (n_valid + EPI_COLS - 1) / EPI_COLS;
@@ -479,30 +528,116 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
             if (!ok) break;
             tc_fence_after();
             const int total_chunks = (w.mt_hi - w.mt_lo) * nchunks;
+            if (!KSPLIT || w.role == 0) {
+                for (int ci = grp; ci < total_chunks; ci += NGRP) {
+                    const int mt = w.mt_lo + ci / nchunks, c = ci % nchunks;
+                    const int m0 = w.pair * 256 + mt * 128;
+                    uint32_t r[EPI_COLS];
+                    tmem_ld16(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * EPI_COLS), r);
+                    tmem_ld_wait();
+                    if (ci + NGRP >= total_chunks) {   // last TMEM read of this warp for this item
+                        tc_fence_before();
+                        if (lane == 0) mbar_arrive(acce_bar);
+                    }
+                    const int tc0 = n0 + c * EPI_COLS, ncols = min(EPI_COLS, n_valid - c * EPI_COLS);
+                    if (m0 < p.N) {
+                        switch (p.mode) {
+                            case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                            case EPI_QKV: epi_direct<EPI_QKV>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                            case EPI_PART: epi_direct<EPI_PART>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                            case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                            default: epi_direct<EPI_LMHEAD>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                        }
+                    }
+                }
+                if (grp >= total_chunks) {   // a group without any chunk still releases the accumulators
+                    tc_fence_before();
+                    if (lane == 0) mbar_arrive(acce_bar);
+                }
+                continue;
+            }
+            // ---- a part of a K-split remainder tile.  Stored accumulators:
+            // [part][tile of the pair][chunk][lane quarter][4][lane][4 floats], so that one 16-byte access
+            // per lane covers 512 contiguous bytes per warp.
+            const int H = g.ksplit - 1, cpt = g.TN / EPI_COLS;   // helper parts per tile, chunk slots per tile
+            const size_t part_elems = (size_t)2 * cpt * 128 * EPI_COLS;
+            if (w.role == 1) {
+                float* mine = g.fix_part + (size_t)(w.rtile * H + w.hpart) * part_elems;
+                for (int ci = grp; ci < total_chunks; ci += NGRP) {
+                    const int mt = w.mt_lo + ci / nchunks, c = ci % nchunks;
+                    uint32_t r[EPI_COLS];
+                    tmem_ld16(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * EPI_COLS), r);
+                    tmem_ld_wait();
+                    if (ci + NGRP >= total_chunks) {
+                        tc_fence_before();
+                        if (lane == 0) mbar_arrive(acce_bar);
+                    }
+                    uint4* dst = reinterpret_cast<uint4*>(mine + (((size_t)mt * cpt + c) * 4 + quarter) * 32 * EPI_COLS) + lane;
+#pragma unroll
+                    for (int v = 0; v < EPI_COLS / 4; ++v) dst[v * 32] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                }
+                if (grp >= total_chunks) {
+                    tc_fence_before();
+                    if (lane == 0) mbar_arrive(acce_bar);
+                }
+                __threadfence();        // this warp's part of the accumulators is in memory
+                __syncwarp();
+                if (lane == 0) atomicAdd(g.fix_flag + w.rtile, 1);
+                continue;
+            }
+            // owner: the helpers ran first; the wait is bounded all the same
+            if (lane == 0) {
+                const int want = H * GEMM_EPI_WARPS;
+                const long long t_end = clock64() + SYN_SPIN_LIMIT_CYCLES;
+                while (ld_acquire_gpu(g.fix_flag + w.rtile) < want) {
+                    if (clock64() > t_end) {
+                        atomicExch(g.status, 1);
+                        break;
+                    }
+                }
+            }
+            __syncwarp();
             for (int ci = grp; ci < total_chunks; ci += NGRP) {
                 const int mt = w.mt_lo + ci / nchunks, c = ci % nchunks;
                 const int m0 = w.pair * 256 + mt * 128;
                 uint32_t r[EPI_COLS];
                 tmem_ld16(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * EPI_COLS), r);
                 tmem_ld_wait();
-                if (ci + NGRP >= total_chunks) {   // last TMEM read of this warp for this item
+                if (ci + NGRP >= total_chunks) {
                     tc_fence_before();
                     if (lane == 0) mbar_arrive(acce_bar);
+                }
+                const size_t at = (((size_t)mt * cpt + c) * 4 + quarter) * 32 * EPI_COLS;
+                for (int h = 0; h < H; ++h) {   // fixed order: own k range, then the helpers' in part order
+                    const float4* src = reinterpret_cast<const float4*>(g.fix_part + (size_t)(w.rtile * H + h) * part_elems + at) + lane;
+#pragma unroll
+                    for (int v = 0; v < EPI_COLS / 4; ++v) {
+                        const float4 q4 = __ldcg(src + v * 32);
+                        r[4 * v] = __float_as_uint(__uint_as_float(r[4 * v]) + q4.x);
+                        r[4 * v + 1] = __float_as_uint(__uint_as_float(r[4 * v + 1]) + q4.y);
+                        r[4 * v + 2] = __float_as_uint(__uint_as_float(r[4 * v + 2]) + q4.z);
+                        r[4 * v + 3] = __float_as_uint(__uint_as_float(r[4 * v + 3]) + q4.w);
+                    }
                 }
                 const int tc0 = n0 + c * EPI_COLS, ncols = min(EPI_COLS, n_valid - c * EPI_COLS);
                 if (m0 < p.N) {
                     switch (p.mode) {
-                        case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
-                        case EPI_QKV: epi_direct<EPI_QKV>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
-                        case EPI_PART: epi_direct<EPI_PART>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
-                        case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
-                        default: epi_direct<EPI_LMHEAD>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
+                        case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, m0, tc0, ncols, 0, quarter, lane); break;
+                        case EPI_QKV: epi_direct<EPI_QKV>(p, r, m0, tc0, ncols, 0, quarter, lane); break;
+                        case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, m0, tc0, ncols, 0, quarter, lane); break;
+                        default: epi_direct<EPI_LMHEAD>(p, r, m0, tc0, ncols, 0, quarter, lane); break;
                     }
                 }
             }
-            if (grp >= total_chunks) {   // a group without any chunk still releases the accumulators
+            if (grp >= total_chunks) {
                 tc_fence_before();
                 if (lane == 0) mbar_arrive(acce_bar);
+            }
+            // the last warp to finish reading clears the tile's counters for the next launch
+            __syncwarp();
+            if (lane == 0 && atomicAdd(g.fix_flag + g.n_sm + w.rtile, 1) == GEMM_EPI_WARPS - 1) {
+                g.fix_flag[w.rtile] = 0;
+                g.fix_flag[g.n_sm + w.rtile] = 0;
             }
         }
     }

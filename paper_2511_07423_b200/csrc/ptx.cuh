@@ -11,6 +11,12 @@ namespace syn {
 
 constexpr long long SYN_SPIN_LIMIT_CYCLES = 4000000000LL;  // ~2 s at 2 GHz
 
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }

@@ -18,6 +18,8 @@
 
 using namespace syn;
 typedef __nv_bfloat16 bf16;
+// Slot of one helper part's stored accumulators: two tiles of 128 features x up to 256 tokens, fp32.
+constexpr size_t GEMM_FIX_SLOT_BYTES = (size_t)2 * 128 * 256 * 4;
 constexpr int GEMM_MAX_SPLITS = 8;   // split-K partial buffers of the o / down projections
 
 // Name of the last CUDA error a call of this library met on this thread (for syn_last_cuda_error).
@@ -178,6 +180,8 @@ struct syn_model {
     int *acc_dev = nullptr, *corr_dev = nullptr;
     int b_cap = 0;
     CUtensorMap tm_xn, tm_attn, tm_act, tm_q;
+    float* fix_part = nullptr;      // stored accumulators of K-split remainder tiles (one slot per SM)
+    int* fix_flag = nullptr;        // their arrival / release counters, [2 * n_sm], zero between launches
     float* part_o = nullptr;
     float2* part_ml = nullptr;
     int* group_count = nullptr;     // per merge group: partial items completed (zero between launches)
@@ -279,6 +283,11 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return SYN_E_CUDA;
     }
+    if (!m->fix_part) {
+        CU_OK(cudaMalloc(&m->fix_part, (size_t)m->n_sm * GEMM_FIX_SLOT_BYTES));
+        CU_OK(cudaMalloc(&m->fix_flag, (size_t)2 * m->n_sm * 4));
+        CU_OK(cudaMemset(m->fix_flag, 0, (size_t)2 * m->n_sm * 4));
+    }
     if (B > m->b_cap) {
         cudaFree(m->acc_dev); cudaFree(m->corr_dev);
         m->acc_dev = m->corr_dev = nullptr; m->b_cap = 0;
@@ -309,6 +318,7 @@ extern "C" void syn_model_free(syn_model* m) {
     cudaFree(m->embed); cudaFree(m->lm_head); cudaFree(m->final_norm); cudaFree(m->inv_freq); cudaFree(m->status_dev);
     free_workspace(m);
     cudaFree(m->acc_dev); cudaFree(m->corr_dev); cudaFree(m->part_o); cudaFree(m->part_ml); cudaFree(m->group_count);
+    cudaFree(m->fix_part); cudaFree(m->fix_flag);
     if (m->pinned_out) cudaFreeHost(m->pinned_out);
     cudaFree(m->sw.logits); cudaFree(m->sw.topk_logit); cudaFree(m->sw.topk_id); cudaFree(m->sw.slm_id);
     cudaFree(m->sw.slm_prob); cudaFree(m->sw.rand_accept); cudaFree(m->sw.rand_sample);
@@ -469,7 +479,8 @@ extern "C" int syn_model_load(const syn_model_desc* desc, const syn_weights* w, 
     CU_M(cudaMemcpy(m->inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice));
     CU_M(cudaMalloc(&m->status_dev, 4));
     CU_M(cudaMemset(m->status_dev, 0, 4));
-    CU_M(cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_M(cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_M(cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_M(cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::TOTAL));
     CU_M(cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::TOTAL));
     CU_M(cudaDeviceSynchronize());
@@ -886,7 +897,8 @@ extern "C" int syn_last_step_stats(const syn_plan* p, syn_step_stats* out) {
 // for partial-sum epilogues with few output tiles, pair tiles when they fill the SMs, else singles.
 // Returns the number of splits through *splits_out (EPI_PART only).
 static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const bf16* w_packed, int packed_rows, int K,
-                       const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, int* splits_out = nullptr) {
+                       const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, int* splits_out = nullptr,
+                       float* fix_part = nullptr, int* fix_flag = nullptr) {
     ProfScope prof(cls >= 0 ? prof_m : nullptr, cls, st);
     const int T = ep.T;
     GemmParams g;
@@ -904,6 +916,7 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     g.n_tt = (T + g.TN - 1) / g.TN;   // rounding the width up may leave the last tiles without tokens
     g.n_stages = gemm_stages(g.TN);
     g.status = status;
+    g.ksplit = 1; g.kper = 0; g.fix_part = fix_part; g.fix_flag = fix_flag; g.n_sm = n_sm;
     g.splits = 1;
     g.kb_per_split = g.num_kb;
     // every token tile must hold a token: an empty one would issue an MMA of width 0
@@ -919,9 +932,27 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     }
     if (g.splits > 1) n_cta = tiles * g.splits;
     else n_cta = std::min(n_sm, g.pair_mode ? tiles : 2 * tiles);
+    if (g.splits == 1 && g.pair_mode && fix_part && fix_flag) {
+        // The tiles left after the full waves: cut along K over otherwise idle CTAs (parts of at
+        // least 8 k-blocks; helpers and owners are different CTAs, so R * parts <= n_cta).
+        const int rem = tiles % n_cta;
+        if (rem > 0) {
+            const int parts = std::min(std::min(8, n_cta / rem), g.num_kb / 8);
+            if (parts >= 2) {
+                // the owner part also adds the others and finishes the tile: about half a helper's k range
+                const int H = parts - 1;
+                int kper = (2 * g.num_kb + 2 * H) / (2 * H + 1);
+                while (H * kper >= g.num_kb) --kper;
+                g.ksplit = parts;
+                g.kper = kper;
+            }
+        }
+    }
     if (splits_out) *splits_out = g.splits;
     const int smem = gemm_fixed_smem() + g.n_stages * gemm_stage_bytes(g.TN);
-    return launch_pdl(gemm_kernel, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep) == cudaSuccess ? SYN_OK : SYN_E_CUDA;
+    const cudaError_t le = g.ksplit > 1 ? launch_pdl(gemm_kernel<true>, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep)
+                                        : launch_pdl(gemm_kernel<false>, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep);
+    return le == cudaSuccess ? SYN_OK : SYN_E_CUDA;
 }
 
 static void attn_params(AttnParams& ap, const syn_model* m, const syn_kv* kv, const syn_plan* p, uint32_t layer, bf16* out,
@@ -993,7 +1024,9 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
         e.q = m->q; e.q_dim = q_dim; e.kv_dim = kv_dim; e.hd = c.head_dim; e.n_kv_heads = c.n_kv_heads;
         e.page_size = kv->page_size; e.rope = m->rope; e.pool = kv->pool + kv->layer_elems * l;
         e.slot = p->d<int>(p->o_slot);
-        if ((r = launch_gemm(m, 1, m->n_sm, m->status_dev, m->wqkv[l], m->qkv_rows, d, m->tm_xn, e, st))) return r;
+        if ((r = launch_gemm(m, 1, m->n_sm, m->status_dev, m->wqkv[l], m->qkv_rows, d, m->tm_xn, e, st, nullptr, m->fix_part,
+                             m->fix_flag)))
+            return r;
         if ((r = launch_attention(m, kv, p, l, m->tm_q, m->attn, st))) return r;
         e = base;
         e.mode = EPI_PART; e.N = d; e.d = d; e.part = m->part; e.part_stride = part_stride;
@@ -1001,7 +1034,9 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
         if ((r = resid(9, m->norm2[l]))) return r;
         e = base;
         e.mode = EPI_SWIGLU; e.N = m->gu_rows; e.act = m->act; e.f_pad = m->f_pad;
-        if ((r = launch_gemm(m, 5, m->n_sm, m->status_dev, m->wgu[l], m->gu_rows, d, m->tm_xn, e, st))) return r;
+        if ((r = launch_gemm(m, 5, m->n_sm, m->status_dev, m->wgu[l], m->gu_rows, d, m->tm_xn, e, st, nullptr, m->fix_part,
+                             m->fix_flag)))
+            return r;
         e = base;
         e.mode = EPI_PART; e.N = d; e.d = d; e.part = m->part; e.part_stride = part_stride;
         if ((r = launch_gemm(m, 6, m->n_sm, m->status_dev, m->wd[l], d, m->f_pad, m->tm_act, e, st, &splits))) return r;
@@ -1009,7 +1044,8 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
     }
     EpiParams e = base;
     e.mode = EPI_LMHEAD; e.N = m->v_rows; e.vocab = c.vocab; e.logits = logits_out; e.best = m->best;
-    if ((r = launch_gemm(m, 7, m->n_sm, m->status_dev, m->lm_head, m->v_rows, d, m->tm_xn, e, st))) return r;
+    if ((r = launch_gemm(m, 7, m->n_sm, m->status_dev, m->lm_head, m->v_rows, d, m->tm_xn, e, st, nullptr, m->fix_part, m->fix_flag)))
+        return r;
     {
         ProfScope prof(m, 8, st);
         if (launch_pdl(verify_kernel, dim3((p->n_req + 127) / 128), dim3(128), 0, st, m->best, tokens, p->d<int>(p->o_offsets),
@@ -1054,6 +1090,7 @@ extern "C" int syn_model_status(syn_model* m) {
     if (s) {
         cudaMemset(m->status_dev, 0, 4);
         if (m->group_count) cudaMemset(m->group_count, 0, (size_t)m->part_cap * 4);   // an aborted step may leave counts
+        if (m->fix_flag) cudaMemset(m->fix_flag, 0, (size_t)2 * m->n_sm * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     return SYN_OK;
@@ -1091,6 +1128,7 @@ extern "C" int syn_verify_batch(syn_model* m, syn_kv* kv, int32_t n_req, const i
     if (po[2 * m->pinned_out_cap]) {
         cudaMemset(m->status_dev, 0, 4);
         if (m->group_count) cudaMemset(m->group_count, 0, (size_t)m->part_cap * 4);
+        if (m->fix_flag) cudaMemset(m->fix_flag, 0, (size_t)2 * m->n_sm * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     memcpy(accept_len, po, (size_t)n_req * 4);
@@ -1218,6 +1256,7 @@ extern "C" int syn_verify_batch_sampled(syn_model* m, syn_kv* kv, int32_t n_req,
     if (po[2 * m->pinned_out_cap]) {
         cudaMemset(m->status_dev, 0, 4);
         if (m->group_count) cudaMemset(m->group_count, 0, (size_t)m->part_cap * 4);
+        if (m->fix_flag) cudaMemset(m->fix_flag, 0, (size_t)2 * m->n_sm * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     memcpy(accept_len, po, (size_t)n_req * 4);
@@ -1288,6 +1327,8 @@ extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, 
     // the last weight matrix seen (re-packed when the pointer or the shape changes)
     static int n_sm = 0;
     static int* status = nullptr;
+    static float* fix_part = nullptr;
+    static int* fix_flag = nullptr;
     static bf16* packed = nullptr;
     static const void* packed_src = nullptr;
     static int packed_n = 0, packed_k = 0;
@@ -1299,7 +1340,11 @@ extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, 
         CU_OK(cudaGetDeviceProperties(&prop, dev));
         if (prop.major != 10) return SYN_E_ARCH;
         n_sm = prop.multiProcessorCount;
-        CU_OK(cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+        CU_OK(cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+        CU_OK(cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+        CU_OK(cudaMalloc(&fix_part, (size_t)n_sm * GEMM_FIX_SLOT_BYTES));
+        CU_OK(cudaMalloc(&fix_flag, (size_t)2 * n_sm * 4));
+        CU_OK(cudaMemset(fix_flag, 0, (size_t)2 * n_sm * 4));
         CU_OK(cudaMalloc(&status, 4));
         CU_OK(cudaMemset(status, 0, 4));
     }
@@ -1322,13 +1367,14 @@ extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, 
     EpiParams e;
     memset(&e, 0, sizeof(e));
     e.mode = EPI_PLAIN; e.T = T; e.N = N; e.y = y; e.ldy = N;
-    r = launch_gemm(nullptr, -1, n_sm, status, packed, n_mt * 128, K, tmB, e, st);
+    r = launch_gemm(nullptr, -1, n_sm, status, packed, n_mt * 128, K, tmB, e, st, nullptr, fix_part, fix_flag);
     if (r) return r;
     CU_OK(cudaStreamSynchronize(st));
     int s = 0;
     CU_OK(cudaMemcpy(&s, status, 4, cudaMemcpyDeviceToHost));
     if (s) {
         cudaMemset(status, 0, 4);
+        cudaMemset(fix_flag, 0, (size_t)2 * n_sm * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     return SYN_OK;

@@ -25,6 +25,8 @@ def _case(T, N, K, seed):
     (129, 384, 2048),     # few feature tiles: five token tiles of 32 columns, the last with one token
     (544, 640, 4096),     # seventeen token tiles of 32 columns, 64 k-blocks
     (544, 28672, 512),    # many feature tiles: three token tiles of 192 columns, pair items in full waves + single tiles
+    (544, 28672, 4096),   # 336 pair tiles on 148 SMs: two full waves, the other 40 cut along K into 3 parts each
+    (300, 38144, 1024),   # 298 pair tiles: two left over, each cut in two
     (137, 4096, 512),     # token tiles of 48 columns: 3 x 48 covers 137, no fourth tile
     (300, 1024, 320),     # ten token tiles of 32 columns, the last with 12 tokens
     (16, 128, 688),       # K tail: 688 = 10.75 k-blocks (zero-filled by TMA)
