@@ -35,8 +35,8 @@ UNIT = "tokens/s"
 NCU_TRAFFIC = {
     # workload: {kernel: (bytes per launch, sha256 of the kernel's source file)}
     "cfg3-8b": {
-        "attention": (615960044, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
-        "gemm": (132391874, "42ce693f7884da27f7771dbf960c769188f0682013ec67c8c82d0e8fe36d9254"),
+        "attention": (616096960, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
+        "gemm": (140730384, "4786f9dcd7d970e8807400e55431d7e567a4aca3e5d5da168b92384152844ce7"),
     },
 }
 
