@@ -608,10 +608,10 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
         if (ctx_lens[i] < 0) return SYN_E_INVALID_ARG;
         if ((int64_t)ctx_lens[i] + n > (int64_t)max_pages * P) return SYN_E_CAPACITY;
         const int used = (int)((ctx_lens[i] + n + P - 1) / P);
-        for (int k = 0; k < used; ++k) {
-            const int pg = page_tables[(size_t)i * max_pages + k];
-            if (pg < 0 || (uint32_t)pg >= n_pages) return SYN_E_PAGE_OOB;
-        }
+        const int32_t* row = page_tables + (size_t)i * max_pages;
+        uint32_t worst = 0;   // a negative id is a large unsigned one
+        for (int k = 0; k < used; ++k) worst = std::max(worst, (uint32_t)row[k]);
+        if (worst >= n_pages) return SYN_E_PAGE_OOB;
         ctx_sum += ctx_lens[i];
         kv_units += ctx_lens[i] + n;
         keys_seen += n * (int64_t)ctx_lens[i] + n * (n + 1) / 2;
@@ -630,10 +630,22 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
             slot[b + j] = page_tables[(size_t)i * max_pages + pp / P] * P + pp % P;
         }
     {
-        std::vector<int> s2(slot);
-        std::sort(s2.begin(), s2.end());
-        for (int t = 1; t < T; ++t)
-            if (s2[t] == s2[t - 1]) return SYN_E_PAGE_ALIAS;
+        // Two chunk tokens may not share a KV slot.  Inside a request the chunk's slots differ unless
+        // two of its (at most three) pages are the same page; between requests they can only meet in
+        // a page both chunks write.  So look at the pages first, and at the slots only if a page
+        // is written twice.
+        std::vector<int> pg;
+        pg.reserve((size_t)n_req * 3);
+        for (int i = 0; i < n_req; ++i) {
+            const int first = ctx_lens[i] / P, last = (ctx_lens[i] + (chunk_offsets[i + 1] - chunk_offsets[i]) - 1) / P;
+            for (int k = first; k <= last; ++k) pg.push_back(page_tables[(size_t)i * max_pages + k]);
+        }
+        std::sort(pg.begin(), pg.end());
+        if (std::adjacent_find(pg.begin(), pg.end()) != pg.end()) {
+            std::vector<int> s2(slot);
+            std::sort(s2.begin(), s2.end());
+            if (std::adjacent_find(s2.begin(), s2.end()) != s2.end()) return SYN_E_PAGE_ALIAS;
+        }
     }
     // Attention work list: (request, kv head, token group, key range).  Cost of an item, in SM
     // cycles: its 64-key stages times a per-stage time that grows with the number of 16-row query
@@ -685,82 +697,118 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
     }
     const int n_items = (int)items.size();
     const int n_cta = std::min(n_cta_max, n_items);
+    // longest first (equal costs: lower index first), each to the least loaded CTA (ties: lower CTA);
+    // both orders are carried in one 64-bit key
     std::vector<int> order(n_items), owner(n_items);
-    for (int i = 0; i < n_items; ++i) order[i] = i;
     auto cost = [&](int i) { return item_cost[i]; };
-    std::stable_sort(order.begin(), order.end(), [&](int a, int bb) { return cost(a) > cost(bb); });
-    typedef std::pair<int64_t, int> Load;
-    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-    for (int k = 0; k < n_cta; ++k) heap.push(Load(0, k));
+    {
+        // stable radix sort of the indices by decreasing cost, 11 bits a pass
+        int top = 0;
+        for (int i = 0; i < n_items; ++i) top = std::max(top, item_cost[i]);
+        std::vector<int> tmp(n_items);
+        for (int i = 0; i < n_items; ++i) order[i] = i;
+        int hist[2048];
+        for (int shift = 0; shift < 32 && (top >> shift) != 0; shift += 11) {
+            memset(hist, 0, sizeof(hist));
+            for (int i = 0; i < n_items; ++i) hist[2047 - ((item_cost[order[i]] >> shift) & 2047)]++;
+            int run = 0;
+            for (int b = 0; b < 2048; ++b) { const int h = hist[b]; hist[b] = run; run += h; }
+            for (int i = 0; i < n_items; ++i) tmp[hist[2047 - ((item_cost[order[i]] >> shift) & 2047)]++] = order[i];
+            order.swap(tmp);
+        }
+    }
     std::vector<int>& count = hp.cta_begin;
     count.assign(n_cta + 1, 0);
-    for (int i : order) {
-        Load l = heap.top();
-        heap.pop();
-        owner[i] = l.second;
-        count[l.second + 1]++;
-        heap.push(Load(l.first + cost(i), l.second));
+    {
+        std::vector<uint64_t> heap(n_cta);   // (load << 16) | cta, smallest at the root
+        for (int k = 0; k < n_cta; ++k) heap[k] = (uint64_t)k;   // all loads 0: already a heap
+        for (int i : order) {
+            const uint64_t top = heap[0];
+            const int k = (int)(top & 0xFFFFu);
+            owner[i] = k;
+            count[k + 1]++;
+            const uint64_t v = (((top >> 16) + (uint64_t)cost(i)) << 16) | (uint64_t)k;
+            int at = 0;   // the root grows: sift it down
+            for (;;) {
+                int ch = 2 * at + 1;
+                if (ch >= n_cta) break;
+                if (ch + 1 < n_cta && heap[ch + 1] < heap[ch]) ++ch;
+                if (heap[ch] >= v) break;
+                heap[at] = heap[ch];
+                at = ch;
+            }
+            heap[at] = v;
+        }
     }
     // Local search on the greedy result: relieve the most loaded CTA by moving one of its items to
     // another CTA, or by exchanging it for a cheaper one, as long as that lowers the larger of the
-    // two loads; partners are the least loaded CTAs.  Stops when the maximum is within 0.3 % of
-    // the mean.
+    // two loads; partners are the least loaded CTAs.  Only when the greedy result is more than 1 %
+    // above the mean; stops within 0.3 % of it.
     if (n_cta > 1) {
         std::vector<int64_t> load(n_cta, 0);
-        std::vector<std::vector<int>> held(n_cta);
         int64_t sum = 0;
         for (int i = 0; i < n_items; ++i) {
             load[owner[i]] += cost(i);
-            held[owner[i]].push_back(i);
             sum += cost(i);
         }
-        const int64_t good = sum / n_cta + sum / n_cta / 333;
-        std::vector<int> by_load(n_cta);
-        for (int k = 0; k < n_cta; ++k) by_load[k] = k;
-        for (int round = 0; round < 2 * n_cta; ++round) {
-            const int hi = (int)(std::max_element(load.begin(), load.end()) - load.begin());
-            if (load[hi] <= good) break;
-            // partners: the least loaded CTAs
-            const int n_cand = std::min(n_cta - 1, 24);
-            std::partial_sort(by_load.begin(), by_load.begin() + n_cand + 1, by_load.end(),
-                              [&](int x, int y) { return load[x] != load[y] ? load[x] < load[y] : x < y; });
-            int64_t best = load[hi];
-            int bi = -1, bk = -1, bj = -1;   // positions in held[hi], the other CTA, position in held[bk] (-1: move)
-            for (int a = 0; a < (int)held[hi].size(); ++a) {
-                const int64_t ca = cost(held[hi][a]);
-                for (int q = 0; q <= n_cand; ++q) {
-                    const int k = by_load[q];
-                    if (k == hi) continue;
-                    if (std::max(load[hi] - ca, load[k] + ca) < best) {
-                        best = std::max(load[hi] - ca, load[k] + ca);
-                        bi = a; bk = k; bj = -1;
-                    }
-                    for (int b2 = 0; b2 < (int)held[k].size(); ++b2) {
-                        const int64_t dlt = ca - cost(held[k][b2]);
-                        if (dlt > 0 && std::max(load[hi] - dlt, load[k] + dlt) < best) {
-                            best = std::max(load[hi] - dlt, load[k] + dlt);
-                            bi = a; bk = k; bj = b2;
+        const int64_t mean = sum / n_cta;
+        if (*std::max_element(load.begin(), load.end()) > mean + mean / 100) {
+            std::vector<std::vector<int>> held(n_cta);
+            for (int i = 0; i < n_items; ++i) held[owner[i]].push_back(i);
+            std::vector<int> by_load(n_cta);   // CTAs by increasing load, kept sorted
+            for (int k = 0; k < n_cta; ++k) by_load[k] = k;
+            auto lighter = [&](int x, int y) { return load[x] != load[y] ? load[x] < load[y] : x < y; };
+            std::sort(by_load.begin(), by_load.end(), lighter);
+            auto resort = [&](int k) {   // k's load changed: move it to its place
+                int at = (int)(std::find(by_load.begin(), by_load.end(), k) - by_load.begin());
+                while (at + 1 < n_cta && lighter(by_load[at + 1], k)) { by_load[at] = by_load[at + 1]; ++at; }
+                while (at > 0 && lighter(k, by_load[at - 1])) { by_load[at] = by_load[at - 1]; --at; }
+                by_load[at] = k;
+            };
+            const int64_t good = mean + mean / 333;
+            const int n_cand = std::min(n_cta - 1, 16);
+            for (int round = 0; round < 128; ++round) {
+                const int hi = by_load[n_cta - 1];
+                if (load[hi] <= good) break;
+                int64_t best = load[hi];
+                int bi = -1, bk = -1, bj = -1;   // position in held[hi], the other CTA, position in held[bk] (-1: move)
+                for (int a = 0; a < (int)held[hi].size(); ++a) {
+                    const int64_t ca = cost(held[hi][a]);
+                    for (int q = 0; q < n_cand; ++q) {
+                        const int k = by_load[q];
+                        if (std::max(load[hi] - ca, load[k] + ca) < best) {
+                            best = std::max(load[hi] - ca, load[k] + ca);
+                            bi = a; bk = k; bj = -1;
+                        }
+                        for (int b2 = 0; b2 < (int)held[k].size(); ++b2) {
+                            const int64_t dlt = ca - cost(held[k][b2]);
+                            if (dlt > 0 && std::max(load[hi] - dlt, load[k] + dlt) < best) {
+                                best = std::max(load[hi] - dlt, load[k] + dlt);
+                                bi = a; bk = k; bj = b2;
+                            }
                         }
                     }
                 }
+                if (bi < 0 || load[hi] - best < mean / 1000) break;   // nothing, or next to nothing, to gain
+                const int ia = held[hi][bi];
+                if (bj < 0) {
+                    load[hi] -= cost(ia); load[bk] += cost(ia);
+                    owner[ia] = bk;
+                    held[bk].push_back(ia);
+                    held[hi].erase(held[hi].begin() + bi);
+                } else {
+                    const int ib = held[bk][bj];
+                    const int64_t dlt = cost(ia) - cost(ib);
+                    load[hi] -= dlt; load[bk] += dlt;
+                    owner[ia] = bk; owner[ib] = hi;
+                    held[hi][bi] = ib; held[bk][bj] = ia;
+                }
+                resort(hi);
+                resort(bk);
             }
-            if (bi < 0) break;
-            const int ia = held[hi][bi];
-            if (bj < 0) {
-                load[hi] -= cost(ia); load[bk] += cost(ia);
-                owner[ia] = bk;
-                held[bk].push_back(ia);
-                held[hi].erase(held[hi].begin() + bi);
-            } else {
-                const int ib = held[bk][bj];
-                const int64_t dlt = cost(ia) - cost(ib);
-                load[hi] -= dlt; load[bk] += dlt;
-                owner[ia] = bk; owner[ib] = hi;
-                held[hi][bi] = ib; held[bk][bj] = ia;
-            }
+            std::fill(count.begin(), count.end(), 0);
+            for (int i = 0; i < n_items; ++i) count[owner[i] + 1]++;
         }
-        std::fill(count.begin(), count.end(), 0);
-        for (int i = 0; i < n_items; ++i) count[owner[i] + 1]++;
     }
     for (int k = 0; k < n_cta; ++k) count[k + 1] += count[k];
     hp.items.assign(n_items, AttnItem());
