@@ -52,6 +52,8 @@ struct EpiParams {
     float* logits;
     int vocab;
     unsigned long long* best;
+    uint32_t* warp_max;   // NULL, or [T][n_warp_max]: the ordered bit pattern of the largest logit of every
+    int n_warp_max;       // 32-feature group of a token (0 for a group without a valid feature)
 };
 
 __device__ __forceinline__ uint32_t orderable_f32(float v) {   // monotone map of a float to unsigned
@@ -160,6 +162,13 @@ __device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&
             if (lane == j && hit) mine = pack_argmax_key(mx[j], m0 + quarter * 32 + (__ffs(hit) - 1));
         }
         if (lane < ncols && mine) atomicMax(p.best + t0 + lane, mine);
+        if (p.warp_max) {   // lane j keeps the group's maximum of token j: a threshold source for a later top-k
+            uint32_t gm = 0u;
+#pragma unroll
+            for (int j = 0; j < EPI_COLS; ++j)
+                if (lane == j) gm = mx[j];
+            if (lane < ncols) p.warp_max[(size_t)(t0 + lane) * p.n_warp_max + (m0 >> 5) + quarter] = gm;
+        }
     }
 }
 

@@ -38,22 +38,25 @@ constexpr int TOPK_CAND_CAP = 1024;
 // out_id / out_logit [T][SAMPLE_MAX_K]: the k largest logits in decreasing order (equal logits:
 // increasing id); entries k.. hold id -1.
 //
-// Fast path, two passes over the row: the k-th largest of the threads' own maxima is a threshold
-// that at least k elements reach; the elements that reach it (about k in a row of distinct
-// values) are collected and ranked exactly.  A row with so many elements at the threshold that
+// Fast path: the k-th largest of the threads' own maxima is a threshold that at least k elements
+// reach; the elements that reach it (about k in a row of distinct values) are collected and
+// ranked exactly.  The maxima come from a pass over the row, or, when the projection that wrote
+// the logits also stored the maximum of every 32-feature group (warp_max), from those few
+// thousand values, so that the row itself is read once.  A row with so many elements at the threshold that
 // they overflow the candidate buffer (long runs of equal logits) takes the radix path instead:
 // select the k-th largest bit pattern byte by byte, then gather in index order.
 __global__ void __launch_bounds__(TOPK_THREADS)
 topk_rows_kernel(const float* __restrict__ logits, int V, const int* __restrict__ offsets, const int* __restrict__ uncached,
-                 int n_req, int k, int* __restrict__ out_id, float* __restrict__ out_logit) {
-    __shared__ float tmax[TOPK_THREADS];
+                 int n_req, int k, const uint32_t* __restrict__ warp_max, int n_warp_max, int* __restrict__ out_id,
+                 float* __restrict__ out_logit) {
+    __shared__ uint32_t tmax[TOPK_THREADS];
     __shared__ int cand_id[TOPK_CAND_CAP];
     __shared__ float cand_logit[TOPK_CAND_CAP];
     __shared__ uint32_t hist[256];
     __shared__ uint32_t sel[2];                 // radix path: prefix, remaining count
     __shared__ int warp_gt[TOPK_THREADS / 32], warp_eq[TOPK_THREADS / 32];
     __shared__ int needed, n_cand;
-    __shared__ float tau;
+    __shared__ uint32_t tau;
     const int row = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     pdl_wait();
     if (tid == 0) {
@@ -69,9 +72,14 @@ topk_rows_kernel(const float* __restrict__ logits, int V, const int* __restrict_
     float* ol = out_logit + (size_t)row * SAMPLE_MAX_K;
     if (tid < SAMPLE_MAX_K && tid >= kk) { oid[tid] = -1; ol[tid] = 0.f; }
 
-    // ---- fast path
-    float mx = -INFINITY;
-    for (int i = tid; i < V; i += TOPK_THREADS) mx = fmaxf(mx, x[i]);
+    // ---- fast path (all comparisons on the ordered bit patterns; 0 stands for "no element")
+    uint32_t mx = 0u;
+    if (warp_max && n_warp_max * 32 >= V) {
+        const uint32_t* gm = warp_max + (size_t)row * n_warp_max;
+        for (int i = tid; i < n_warp_max; i += TOPK_THREADS) mx = max(mx, gm[i]);
+    } else {
+        for (int i = tid; i < V; i += TOPK_THREADS) mx = max(mx, f32_order_key(x[i]));
+    }
     tmax[tid] = mx;
     __syncthreads();
     {
@@ -80,10 +88,10 @@ topk_rows_kernel(const float* __restrict__ logits, int V, const int* __restrict_
         if (rank == kk - 1) tau = mx;
     }
     __syncthreads();
-    const float thr = tau;
+    const uint32_t thr = tau;   // 0 when fewer than kk threads saw an element: then every element is a candidate
     for (int i = tid; i < V; i += TOPK_THREADS) {
         const float v = x[i];
-        if (v >= thr) {
+        if (f32_order_key(v) >= thr) {
             const int pos = atomicAdd(&n_cand, 1);
             if (pos < TOPK_CAND_CAP) { cand_id[pos] = i; cand_logit[pos] = v; }
         }

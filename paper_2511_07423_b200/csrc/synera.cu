@@ -192,6 +192,7 @@ struct syn_model {
     struct SampleWs {
         float *logits = nullptr, *topk_logit = nullptr, *slm_prob = nullptr, *rand_accept = nullptr, *rand_sample = nullptr;
         int *topk_id = nullptr, *slm_id = nullptr;
+        uint32_t* warp_max = nullptr;   // [t_cap][v_rows / 32]: per-group maxima stored by the lm_head epilogue
         size_t logits_cap = 0;
         int t_cap = 0, b_cap = 0, slm_cap = 0;
     } sw;
@@ -321,7 +322,7 @@ extern "C" void syn_model_free(syn_model* m) {
     cudaFree(m->fix_part); cudaFree(m->fix_flag);
     if (m->pinned_out) cudaFreeHost(m->pinned_out);
     cudaFree(m->sw.logits); cudaFree(m->sw.topk_logit); cudaFree(m->sw.topk_id); cudaFree(m->sw.slm_id);
-    cudaFree(m->sw.slm_prob); cudaFree(m->sw.rand_accept); cudaFree(m->sw.rand_sample);
+    cudaFree(m->sw.slm_prob); cudaFree(m->sw.rand_accept); cudaFree(m->sw.rand_sample); cudaFree(m->sw.warp_max);
     if (m->scratch_plan) syn_plan_free(m->scratch_plan);
     for (auto* v : {&m->ev_used, &m->ev_free})
         for (auto& e : *v) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
@@ -1044,7 +1045,7 @@ static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_
 }
 
 static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, int* corr_dev, int* top1_dev,
-                    float* logits_out, cudaStream_t st) {
+                    float* logits_out, cudaStream_t st, uint32_t* warp_max = nullptr) {
     const syn_model_desc& c = m->desc;
     const int T = p->T, d = c.d_model, q_dim = c.n_q_heads * c.head_dim, kv_dim = c.n_kv_heads * c.head_dim;
     if (T > m->t_cap || p->n_req > m->b_cap || p->n_parts > m->part_cap) return SYN_E_INVALID_ARG;
@@ -1092,6 +1093,7 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
     }
     EpiParams e = base;
     e.mode = EPI_LMHEAD; e.N = m->v_rows; e.vocab = c.vocab; e.logits = logits_out; e.best = m->best;
+    e.warp_max = warp_max; e.n_warp_max = m->v_rows / 32;
     if ((r = launch_gemm(m, 7, m->n_sm, m->status_dev, m->lm_head, m->v_rows, d, m->tm_xn, e, st, nullptr, m->fix_part, m->fix_flag)))
         return r;
     {
@@ -1206,10 +1208,10 @@ static int check_sampling(const syn_sampling* cfg, int vocab, int T, int n_req, 
 static int sample_stage(syn_model* prof_m, cudaStream_t st, const float* logits, int T, int V, int n_req, const int* tokens,
                         const int* offsets, const int* uncached, const syn_sampling& cfg, int* topk_id, float* topk_logit,
                         const int* slm_id, const float* slm_prob, const float* rand_accept, const float* rand_sample,
-                        int* acc_dev, int* corr_dev) {
+                        int* acc_dev, int* corr_dev, const uint32_t* warp_max = nullptr, int n_warp_max = 0) {
     ProfScope prof(prof_m, 8, st);
     if (launch_pdl(topk_rows_kernel, dim3(T), dim3(TOPK_THREADS), 0, st, logits, V, offsets, uncached, n_req, (int)cfg.top_k,
-                   topk_id, topk_logit) != cudaSuccess)
+                   warp_max, n_warp_max, topk_id, topk_logit) != cudaSuccess)
         return SYN_E_CUDA;
     SampleParams sp;
     sp.tokens = tokens; sp.offsets = offsets; sp.uncached = uncached;
@@ -1231,9 +1233,10 @@ static int ensure_sample_ws(syn_model* m, int T, int B, int slm_k, bool own_logi
         w.logits_cap = need_logits;
     }
     if (T > w.t_cap) {
-        cudaFree(w.topk_id); cudaFree(w.topk_logit); cudaFree(w.rand_accept);
-        w.topk_id = nullptr; w.topk_logit = nullptr; w.rand_accept = nullptr; w.t_cap = 0;
+        cudaFree(w.topk_id); cudaFree(w.topk_logit); cudaFree(w.rand_accept); cudaFree(w.warp_max);
+        w.topk_id = nullptr; w.topk_logit = nullptr; w.rand_accept = nullptr; w.warp_max = nullptr; w.t_cap = 0;
         const int cap = (T + 255) / 256 * 256;
+        CU_OK(cudaMalloc(&w.warp_max, (size_t)cap * (m->v_rows / 32) * 4));
         CU_OK(cudaMalloc(&w.topk_id, (size_t)cap * SAMPLE_MAX_K * 4));
         CU_OK(cudaMalloc(&w.topk_logit, (size_t)cap * SAMPLE_MAX_K * 4));
         CU_OK(cudaMalloc(&w.rand_accept, (size_t)cap * 4));
@@ -1290,11 +1293,11 @@ extern "C" int syn_verify_batch_sampled(syn_model* m, syn_kv* kv, int32_t n_req,
     CU_OK(cudaMemcpyAsync(w.slm_prob, slm_probs, (size_t)p->T * cfg->slm_k * 4, cudaMemcpyHostToDevice, st));
     CU_OK(cudaMemcpyAsync(w.rand_accept, rand_accept, (size_t)p->T * 4, cudaMemcpyHostToDevice, st));
     CU_OK(cudaMemcpyAsync(w.rand_sample, rand_sample, (size_t)n_req * 4, cudaMemcpyHostToDevice, st));
-    if ((r = run_step(m, kv, p, m->acc_dev, m->corr_dev, nullptr, logits, st))) return r;
+    if ((r = run_step(m, kv, p, m->acc_dev, m->corr_dev, nullptr, logits, st, w.warp_max))) return r;
     // the greedy results of the step are replaced by the sampled ones
     if ((r = sample_stage(m, st, logits, p->T, (int)m->desc.vocab, n_req, p->d<int>(p->o_tokens), p->d<int>(p->o_offsets),
                           p->d<int>(p->o_uncached), *cfg, w.topk_id, w.topk_logit, w.slm_id, w.slm_prob, w.rand_accept,
-                          w.rand_sample, m->acc_dev, m->corr_dev)))
+                          w.rand_sample, m->acc_dev, m->corr_dev, w.warp_max, m->v_rows / 32)))
         return r;
     int* po = m->pinned_out;
     CU_OK(cudaMemcpyAsync(po, m->acc_dev, (size_t)n_req * 4, cudaMemcpyDeviceToHost, st));
