@@ -89,12 +89,20 @@ topk_rows_kernel(const float* __restrict__ logits, int V, const int* __restrict_
     }
     __syncthreads();
     const uint32_t thr = tau;   // 0 when fewer than kk threads saw an element: then every element is a candidate
-    for (int i = tid; i < V; i += TOPK_THREADS) {
-        const float v = x[i];
+    auto offer = [&](int i, float v) {
         if (f32_order_key(v) >= thr) {
             const int pos = atomicAdd(&n_cand, 1);
             if (pos < TOPK_CAND_CAP) { cand_id[pos] = i; cand_logit[pos] = v; }
         }
+    };
+    if ((V & 3) == 0) {   // rows start 16-byte aligned: four logits a load
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        for (int i = tid; i < (V >> 2); i += TOPK_THREADS) {
+            const float4 v = x4[i];
+            offer(4 * i, v.x); offer(4 * i + 1, v.y); offer(4 * i + 2, v.z); offer(4 * i + 3, v.w);
+        }
+    } else {
+        for (int i = tid; i < V; i += TOPK_THREADS) offer(i, x[i]);
     }
     __syncthreads();
     int nc = n_cand;
