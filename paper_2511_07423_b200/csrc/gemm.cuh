@@ -297,7 +297,8 @@ struct GemmParams {
     int n_tt, TN;               // token tiles of TN columns (multiple of 16, <= 256)
     int n_stages;
     int splits, kb_per_split;   // splits > 1: every CTA owns one (pair tile, k range)
-    int pair_mode;              // 1: pair tiles in full waves + remainder as singles; 0: all singles
+    int pair_mode;              // 1: pair tiles in full waves + remainder as singles; 0: all singles;
+                                // 2: one wave of n_cta items, pair tiles first, the rest as singles
     int ksplit;                 // pair mode, > 1: the remainder's pair tiles are cut along K into this many parts
     int kper;                   // ksplit: k-blocks of a helper part, (ksplit - 1) * kper < num_kb
     float* fix_part;            // ksplit: fp32 partial accumulators of the helper parts, [slot][2][TN/16][4][32][16]
@@ -364,7 +365,7 @@ __device__ __forceinline__ bool gemm_work(const GemmParams& g, int cta, int n_ct
         }
         return false;
     }
-    if (g.pair_mode) {
+    if (g.pair_mode == 1) {
         const int fw = n_tiles / n_cta;
         if (i < fw) {
             const int tile = i * n_cta + cta;
@@ -374,6 +375,20 @@ __device__ __forceinline__ bool gemm_work(const GemmParams& g, int cta, int n_ct
         const int r = (i - fw) * n_cta + cta;
         if (r >= (n_tiles - fw * n_cta) * 2) return false;
         const int tile = fw * n_cta + (r >> 1);
+        w.pair = tile / g.n_tt; w.tt = tile - w.pair * g.n_tt;
+        w.mt_lo = r & 1; w.mt_hi = w.mt_lo + 1;
+        return true;
+    }
+    if (g.pair_mode == 2) {
+        // One item per CTA and more single tiles than CTAs: the first 2 n_tiles - n_cta pair tiles stay
+        // whole, the others run as two single tiles, so that n_cta CTAs cover everything in one wave.
+        if (i > 0) return false;
+        const int whole = 2 * n_tiles - n_cta;
+        if (cta < whole) {
+            w.pair = cta / g.n_tt; w.tt = cta - w.pair * g.n_tt;
+            return true;
+        }
+        const int r = cta - whole, tile = whole + (r >> 1);
         w.pair = tile / g.n_tt; w.tt = tile - w.pair * g.n_tt;
         w.mt_lo = r & 1; w.mt_hi = w.mt_lo + 1;
         return true;

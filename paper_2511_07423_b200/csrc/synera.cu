@@ -981,7 +981,10 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     }
     if (g.splits > 1) n_cta = tiles * g.splits;
     else n_cta = std::min(n_sm, g.pair_mode ? tiles : 2 * tiles);
-    if (g.splits == 1 && g.pair_mode && fix_part && fix_flag) {
+    // fewer pair tiles than SMs but more single tiles: one wave that mixes whole pair tiles and single tiles
+    // (two waves of single tiles would take longer than one pair tile)
+    if (g.splits == 1 && !g.pair_mode && 2 * tiles > n_sm) g.pair_mode = 2;
+    if (g.splits == 1 && g.pair_mode == 1 && fix_part && fix_flag) {
         // The tiles left after the full waves: cut along K over otherwise idle CTAs (parts of at
         // least 8 k-blocks; helpers and owners are different CTAs, so R * parts <= n_cta).
         const int rem = tiles % n_cta;

@@ -64,6 +64,11 @@ def test_sampled_requests_match_the_oracle_at_full_size(cfg, max_tokens):
     acc, cor, logits = kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens,
                                        n_uncached=batch.n_uncached, want_logits=True)
     assert model.status() == 0
+    # the same step again: bit-identical (static schedules, fixed summation orders, counters back at zero)
+    acc2, cor2, logits2 = kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens,
+                                          n_uncached=batch.n_uncached, want_logits=True)
+    assert torch.equal(acc, acc2) and torch.equal(cor, cor2) and torch.equal(logits, logits2)
+    del logits2
     offs = batch.chunk_offsets.tolist()
     # every request: results are in range and consistent with the returned logits' argmax
     top1_gpu = logits.argmax(-1).cpu()

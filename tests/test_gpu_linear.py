@@ -27,6 +27,8 @@ def _case(T, N, K, seed):
     (544, 28672, 512),    # many feature tiles: three token tiles of 192 columns, pair items in full waves + single tiles
     (544, 28672, 4096),   # 336 pair tiles on 148 SMs: two full waves, the other 40 cut along K into 3 parts each
     (300, 38144, 1024),   # 298 pair tiles: two left over, each cut in two
+    (921, 6144, 512),     # 96 pair tiles, 192 single tiles on 148 SMs: 44 whole pair tiles + 104 single tiles in one wave
+    (200, 25600, 256),    # 100 pair tiles: 52 whole + 96 single tiles
     (137, 4096, 512),     # token tiles of 48 columns: 3 x 48 covers 137, no fourth tile
     (300, 1024, 320),     # ten token tiles of 32 columns, the last with 12 tokens
     (16, 128, 688),       # K tail: 688 = 10.75 k-blocks (zero-filled by TMA)
