@@ -960,6 +960,12 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
         // work; the weights are then read by several CTAs, which costs only L2 bandwidth.
         const int want = n_sm / std::max(1, 2 * g.n_pairs), most = (T + 31) / 32;
         g.n_tt = std::max(g.n_tt, std::min(want, most));
+    } else if (g.n_pairs * g.n_tt < n_sm && n_sm / (g.n_pairs * g.n_tt) < 2) {
+        // Split-K projection whose pair tiles cover more than half of the SMs but not all: K cannot be
+        // split, so narrower token tiles (64 tokens at least) fill the machine instead; every CTA still
+        // walks the whole K, on a smaller item.
+        const int fit = n_sm / g.n_pairs, most = (T + 63) / 64;
+        g.n_tt = std::max(g.n_tt, std::min(fit, most));
     }
     g.TN = (((T + g.n_tt - 1) / g.n_tt) + 15) / 16 * 16;
     g.n_tt = (T + g.TN - 1) / g.TN;   // rounding the width up may leave the last tiles without tokens
