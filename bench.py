@@ -35,8 +35,8 @@ UNIT = "tokens/s"
 NCU_TRAFFIC = {
     # workload: {kernel: (bytes per launch, sha256 of the kernel's source file)}
     "cfg3-8b": {
-        "attention": (616096960, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
-        "gemm": (140730384, "4786f9dcd7d970e8807400e55431d7e567a4aca3e5d5da168b92384152844ce7"),
+        "attention": (615988028, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
+        "gemm": (140228771, "4c3a6eab1bf16db2df70ee8d4618f27bf6789efe918a66da65d458cbb53f9fff"),
     },
 }
 
