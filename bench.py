@@ -329,6 +329,7 @@ def run_ours(args):
                           "peaks": peaks},
         "kernels": kernels,
         "committed_tokens_per_s": float((a_h.sum() + B)) / (ms * 1e-3),
+        "drafts_per_s": float(T - int(batch.n_uncached.sum())) / (ms * 1e-3),
         "cpu_baseline": cpu,
     }
     print(json.dumps(out))
