@@ -304,6 +304,7 @@ def run_ours(args):
     step_bytes = st.weight_bytes + st.kv_read_bytes + st.kv_write_bytes
     step_flops = st.dense_flops + st.attn_flops
     t_roof = max(step_flops / (peaks["tf_sustained"] * 1e12), step_bytes / (peaks["hbm_gbs"] * 1e9))
+    t_roof_spec = max(step_flops / 2.25e15, step_bytes / 8.0e12)   # nominal dense bf16 rate and HBM3e bandwidth
 
     # ---- CPU oracle on a bounded sample (rank 0, N = 1 only)
     cpu = None
@@ -326,7 +327,7 @@ def run_ours(args):
         "roofline": roof,
         "roofline_second_kernel": other,
         "step_roofline": {"bytes": step_bytes, "flops": step_flops, "t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms,
-                          "peaks": peaks},
+                          "peaks": peaks, "t_roof_ms_nominal": t_roof_spec * 1e3, "frac_of_nominal": t_roof_spec * 1e3 / ms},
         "kernels": kernels,
         "committed_tokens_per_s": float((a_h.sum() + B)) / (ms * 1e-3),
         "drafts_per_s": float(T - int(batch.n_uncached.sum())) / (ms * 1e-3),
