@@ -30,6 +30,39 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, name), name
 
 
+def test_headers_are_plain_c(tmp_path):
+    """The boundary is a C ABI: both headers compile as C99 (no C++ in the signatures), and a C program that
+    uses their types and constants links against the library."""
+    import shutil
+    import subprocess
+    from paper_2511_07423_b200 import build
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        import pytest
+        pytest.skip("no C compiler")
+    src = tmp_path / "use_abi.c"
+    src.write_text(
+        '#include "synera.h"\n#include "synera_sched.h"\n#include <string.h>\n'
+        "int main(void) {\n"
+        "    syn_sampling s = {1, 1.0f, 1.0f, 1};\n"
+        "    syn_sched *sc = 0;\n"
+        "    int32_t prompt[3] = {1, 2, 3};\n"
+        "    syn_sched_batch b;\n"
+        "    (void)s;\n"
+        "    if (strcmp(syn_strerror(SYN_E_CHUNK_LEN), \"unknown error\") == 0) return 1;\n"
+        "    if (syn_sched_create(0, 0, 8, 16, SYN_MAX_CHUNK, &sc) != SYN_OK) return 2;\n"
+        "    if (syn_sched_add_request(sc, 7, prompt, 3) != SYN_OK) return 3;\n"
+        "    if (syn_sched_peek(sc, &b) != SYN_OK || b.kind != SYN_SCHED_PREFILL || b.n_tokens != 3) return 4;\n"
+        "    syn_sched_free(sc);\n"
+        "    return 0;\n}\n")
+    lib = build.build()
+    exe = tmp_path / "use_abi"
+    inc = os.path.join(ROOT, "include")
+    subprocess.check_call([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", inc, str(src), "-o", str(exe),
+                           lib, "-Wl,-rpath," + os.path.dirname(lib)])
+    assert subprocess.call([str(exe)]) == 0
+
+
 def test_binding_lists_the_header_names():
     from paper_2511_07423_b200 import binding
     assert sorted(binding.EXPORTS + binding.SCHED_EXPORTS) == _declared()

@@ -132,6 +132,25 @@ def test_uncached_prefix_longer_than_one_and_rerun_is_idempotent():
                 assert (int(acc[r]), int(cor[r])) == verify_greedy(o.top1, o.chunk, u[r])
 
 
+def test_host_resident_weights_give_the_same_results():
+    """syn_model_load copies from host memory (location 0) as well as from device memory."""
+    import paper_2511_07423_b200 as syn
+    shape = MINI_1B
+    wl = Workload("h", shape, 9, 3, ("list", (30, 0, 77)), ("list", (5, 16, 2)), 0.7)
+    batch = gen.gen_batch(wl)
+    glob, layers = cpu_model(shape, wl.seed)
+    toks = gen.gen_context_tokens(wl, 0, batch.n_tokens)
+    outs = []
+    for on_device in (True, False):
+        g2, l2 = to_cuda(glob, layers) if on_device else (glob, layers)
+        model = syn.Model(shape, g2, l2)
+        kv = syn.KVCache(model, batch.n_pages)
+        fill_synthetic_kv(shape, wl.seed, batch, range(3), kv=kv)
+        outs.append(kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens, want_logits=True))
+        assert model.status() == 0
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
+
+
 def test_plan_run_device_outputs_match_blocking_call():
     import paper_2511_07423_b200 as syn
     shape = MINI_8B
