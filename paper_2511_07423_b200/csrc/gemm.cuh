@@ -552,6 +552,76 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
             if (!ok) break;
             tc_fence_after();
             const int total_chunks = (w.mt_hi - w.mt_lo) * nchunks;
+            if ((!KSPLIT || w.role == 0) && (p.mode == EPI_PART || p.mode == EPI_PLAIN)) {
+                // fp32 stores only: 32 columns a TMEM load (the accumulator's columns beyond the
+                // tile's tokens are allocated, their contents are not stored)
+                const int nch2 = (nchunks + 1) >> 1;
+                const int total2 = (w.mt_hi - w.mt_lo) * nch2;
+                for (int ci = grp; ci < total2; ci += NGRP) {
+                    const int mt = w.mt_lo + ci / nch2, c2 = ci % nch2;
+                    const int m0 = w.pair * 256 + mt * 128;
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c2 * 32), r);
+                    tmem_ld_wait();
+                    if (ci + NGRP >= total2) {
+                        tc_fence_before();
+                        if (lane == 0) mbar_arrive(acce_bar);
+                    }
+                    const int f = m0 + quarter * 32 + lane;
+                    const int tc0 = n0 + c2 * 32, ncols = min(32, n_valid - c2 * 32);
+                    if (f < p.N) {
+                        const size_t ld = p.mode == EPI_PLAIN ? (size_t)p.ldy : (size_t)p.d;
+                        float* base = (p.mode == EPI_PLAIN ? p.y + f : p.part + (size_t)w.split * p.part_stride + f) + (size_t)tc0 * ld;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < ncols) base[(size_t)j * ld] = __uint_as_float(r[j]);
+                    }
+                }
+                if (grp >= total2) {
+                    tc_fence_before();
+                    if (lane == 0) mbar_arrive(acce_bar);
+                }
+                continue;
+            }
+            if ((!KSPLIT || w.role == 0) && p.mode == EPI_SWIGLU) {
+                // silu(gate) * up on 32 columns a TMEM load.  Lanes 0..15 hold gate, lanes 16..31 the
+                // matching up features; the lower half-warp finishes the even tokens, the upper one the
+                // odd tokens, so all lanes evaluate silu and one store covers two rows of 16 features.
+                const int nch2 = (nchunks + 1) >> 1;
+                const int total2 = (w.mt_hi - w.mt_lo) * nch2;
+                const bool up_half = lane >= 16;
+                for (int ci = grp; ci < total2; ci += NGRP) {
+                    const int mt = w.mt_lo + ci / nch2, c2 = ci % nch2;
+                    const int m0 = w.pair * 256 + mt * 128;
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c2 * 32), r);
+                    tmem_ld_wait();
+                    if (ci + NGRP >= total2) {
+                        tc_fence_before();
+                        if (lane == 0) mbar_arrive(acce_bar);
+                    }
+                    const int tc0 = n0 + c2 * 32, ncols = min(32, n_valid - c2 * 32);
+                    float got[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k)   // each half-warp sends what the other one needs
+                        got[k] = __shfl_xor_sync(0xFFFFFFFFu, __uint_as_float(up_half ? r[2 * k] : r[2 * k + 1]), 16);
+                    if (m0 < p.N) {
+                        __nv_bfloat16* const dst = p.act + (size_t)(tc0 + (up_half ? 1 : 0)) * p.f_pad + (m0 >> 1) + 16 * quarter + (lane & 15);
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            const float gate = up_half ? got[k] : __uint_as_float(r[2 * k]);       // upper half: gate of token 2k + 1
+                            const float upv = up_half ? __uint_as_float(r[2 * k + 1]) : got[k];    // lower half: up of token 2k
+                            const float h = __fdividef(gate, 1.0f + __expf(-gate)) * upv;
+                            if (2 * k + (up_half ? 1 : 0) < ncols) dst[(size_t)(2 * k) * p.f_pad] = __float2bfloat16(h);
+                        }
+                    }
+                }
+                if (grp >= total2) {
+                    tc_fence_before();
+                    if (lane == 0) mbar_arrive(acce_bar);
+                }
+                continue;
+            }
             if (!KSPLIT || w.role == 0) {
                 for (int ci = grp; ci < total_chunks; ci += NGRP) {
                     const int mt = w.mt_lo + ci / nchunks, c = ci % nchunks;
