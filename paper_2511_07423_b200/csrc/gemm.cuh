@@ -13,7 +13,9 @@
 // CTAs and write fp32 partials that resid_norm_kernel adds to the residual stream in a fixed order.  Every CTA starts its k loop at a different k-block, so the CTAs
 // that share a token tile do not ask L2 for the same lines at the same moment.  Accumulation is
 // tcgen05.mma into TMEM, read back with tcgen05.ld by sixteen epilogue warps; a thread then holds one
-// output feature for sixteen tokens, and the epilogues work on those registers:
+// output feature for sixteen tokens (thirty-two in the epilogues that need few other registers: the
+// fp32 stores and SwiGLU; an epilogue is bound by the round trips of its loads, not by their width),
+// and the epilogues work on those registers:
 //   EPI_QKV    : RoPE on q and k (the partner dimension sits 16 lanes away), q store, paged-KV append
 //   EPI_PART   : fp32 partial of a split-K projection (residual added by resid_norm_kernel)
 //   EPI_SWIGLU : silu(gate) * up (a gate feature and its up feature sit 16 lanes apart)
