@@ -35,8 +35,8 @@ UNIT = "tokens/s"
 NCU_TRAFFIC = {
     # workload: {kernel: (bytes per launch, sha256 of the kernel's source file)}
     "cfg3-8b": {
-        "attention": (615988028, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
-        "gemm": (140228771, "4c3a6eab1bf16db2df70ee8d4618f27bf6789efe918a66da65d458cbb53f9fff"),
+        "attention": (615890944, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
+        "gemm": (139793337, "9ab6d49fa679f5c805fab39a61aa8098f4ab576763df1b008a48e1fc45c3c420"),
     },
 }
 
