@@ -246,6 +246,21 @@ int syn_op_attention(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer
 int syn_op_attention_static(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer, const void *q, void *out,
                             void *cuda_stream);
 
+/* The projection kernel's schedule without a device (tests): how a y[T][N] = x[T][K] w[N][K]^T
+ * projection with the given epilogue (0 plain store, 1 QKV, 2 split-K partial, 3 SwiGLU, 4 lm_head)
+ * is cut up on n_sm SMs.  syn_gemm_plan_host fills out[SYN_GEMM_PLAN_FIELDS] = {feature pairs of 256,
+ * token tiles, tokens per tile, k-blocks of 64, CTAs, pair mode, split-K parts, k-blocks per part,
+ * K parts of a leftover pair tile, k-blocks of a helper part}.  syn_gemm_work_host returns 1 and
+ * fills out[SYN_GEMM_WORK_FIELDS] = {pair, token tile, first 128-feature tile, one past the last,
+ * first k-block, one past the last, split-K part, role (0 whole K, 1 helper, 2 owner), leftover
+ * tile, helper part} for work item i of CTA cta, 0 when that CTA has no item i.
+ * Errors: SYN_E_INVALID_ARG. */
+#define SYN_GEMM_PLAN_FIELDS 10
+#define SYN_GEMM_WORK_FIELDS 10
+int syn_gemm_plan_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t *out);
+int syn_gemm_work_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t cta, int32_t i,
+                       int32_t *out);
+
 /* Sampling-based verification (paper Sec. 4.2, "Compression before transmission": for
  * verification the LLM needs the drafts and the SLM's distributions, of which the device sends
  * the most probable entries as its sampling method, top-1 / top-k / top-p, keeps them; Sec. 3.1:

@@ -57,7 +57,8 @@ _LIB: Optional[C.CDLL] = None
 EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "syn_kv_import", "syn_kv_export",
            "syn_verify_batch", "syn_plan_create", "syn_plan_free", "syn_verify_run", "syn_model_status",
            "syn_last_step_stats", "syn_plan_host", "syn_strerror", "syn_last_cuda_error", "syn_op_linear", "syn_op_attention", "syn_op_attention_static",
-           "syn_set_profile", "syn_get_profile", "syn_verify_batch_sampled", "syn_op_sample_verify"]
+           "syn_set_profile", "syn_get_profile", "syn_verify_batch_sampled", "syn_op_sample_verify",
+           "syn_gemm_plan_host", "syn_gemm_work_host"]
 SCHED_EXPORTS = ["syn_sched_create", "syn_sched_free", "syn_sched_add_request", "syn_sched_add_verify", "syn_sched_finish",
                  "syn_sched_peek", "syn_sched_commit", "syn_sched_step", "syn_sched_get_stats"]
 
@@ -479,6 +480,29 @@ class Scheduler:
             self.close()
         except Exception:
             pass
+
+
+GEMM_PLAN_FIELDS = ("n_pairs", "n_tt", "TN", "num_kb", "n_cta", "pair_mode", "splits", "kb_per_split", "ksplit", "kper")
+GEMM_WORK_FIELDS = ("pair", "tt", "mt_lo", "mt_hi", "kb0", "kb1", "split", "role", "rtile", "hpart")
+GEMM_EPILOGUES = {"plain": 0, "qkv": 1, "part": 2, "swiglu": 3, "lmhead": 4}
+
+
+def gemm_plan_host(T: int, N: int, K: int, epilogue: str, n_sm: int = 148) -> Dict[str, int]:
+    """syn_gemm_plan_host: the launch shape of one projection, without a device."""
+    out = (C.c_int32 * len(GEMM_PLAN_FIELDS))()
+    _check(load_library().syn_gemm_plan_host(C.c_int32(T), C.c_int32(N), C.c_int32(K), C.c_int32(n_sm),
+                                             C.c_int32(GEMM_EPILOGUES[epilogue]), out), "syn_gemm_plan_host")
+    return dict(zip(GEMM_PLAN_FIELDS, out))
+
+
+def gemm_work_host(T: int, N: int, K: int, epilogue: str, cta: int, i: int, n_sm: int = 148) -> Optional[Dict[str, int]]:
+    """syn_gemm_work_host: work item i of CTA cta, or None."""
+    out = (C.c_int32 * len(GEMM_WORK_FIELDS))()
+    r = load_library().syn_gemm_work_host(C.c_int32(T), C.c_int32(N), C.c_int32(K), C.c_int32(n_sm),
+                                          C.c_int32(GEMM_EPILOGUES[epilogue]), C.c_int32(cta), C.c_int32(i), out)
+    if r < 0:
+        _check(r, "syn_gemm_work_host")
+    return dict(zip(GEMM_WORK_FIELDS, out)) if r == 1 else None
 
 
 def syn_op_linear(x: torch.Tensor, w: torch.Tensor, stream=None) -> torch.Tensor:

@@ -321,7 +321,7 @@ struct GemmWork {
 // KSPLIT: the kernel variant that cuts the remainder's pair tiles along K (launched only when
 // GemmParams::ksplit > 1; the plain variant carries none of that code).
 template <bool KSPLIT>
-__device__ __forceinline__ bool gemm_work(const GemmParams& g, int cta, int n_cta, int i, GemmWork& w) {
+__host__ __device__ __forceinline__ bool gemm_work(const GemmParams& g, int cta, int n_cta, int i, GemmWork& w) {
     const int n_tiles = g.n_pairs * g.n_tt;
     w.split = 0; w.kb0 = 0; w.kb1 = g.num_kb; w.mt_lo = 0; w.mt_hi = 2;
     w.role = 0; w.rtile = 0; w.hpart = 0;
@@ -331,7 +331,7 @@ __device__ __forceinline__ bool gemm_work(const GemmParams& g, int cta, int n_ct
         w.split = cta - tile * g.splits;
         w.pair = tile / g.n_tt; w.tt = tile - w.pair * g.n_tt;
         w.kb0 = w.split * g.kb_per_split;
-        w.kb1 = min(g.num_kb, w.kb0 + g.kb_per_split);
+        w.kb1 = w.kb0 + g.kb_per_split < g.num_kb ? w.kb0 + g.kb_per_split : g.num_kb;
         return true;
     }
     if (KSPLIT) {

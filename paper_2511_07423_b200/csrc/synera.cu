@@ -945,17 +945,13 @@ extern "C" int syn_last_step_stats(const syn_plan* p, syn_step_stats* out) {
 // D[rows][T] = Wpacked[rows][K] * X[T][K]^T with the epilogue `ep`.  Chooses the schedule: split-K
 // for partial-sum epilogues with few output tiles, pair tiles when they fill the SMs, else singles.
 // Returns the number of splits through *splits_out (EPI_PART only).
-static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const bf16* w_packed, int packed_rows, int K,
-                       const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, int* splits_out = nullptr,
-                       float* fix_part = nullptr, int* fix_flag = nullptr) {
-    ProfScope prof(cls >= 0 ? prof_m : nullptr, cls, st);
-    const int T = ep.T;
-    GemmParams g;
-    g.w = w_packed;
+// The launch shape of one projection: token tiling, work decomposition, CTA count.  Host arithmetic only
+// (also exported as syn_gemm_plan_host so that the schedule can be checked without a device).
+static int gemm_plan(int T, int packed_rows, int K, int n_sm, int mode, bool may_ksplit, GemmParams& g, int& n_cta) {
     g.num_kb = (K + 63) / 64;
     g.n_pairs = (packed_rows + 255) / 256;
     g.n_tt = (T + 255) / 256;
-    if (ep.mode != EPI_PART) {
+    if (mode != EPI_PART) {
         // Few feature tiles and few tokens: narrower token tiles (32 tokens at least) put more SMs to
         // work; the weights are then read by several CTAs, which costs only L2 bandwidth.
         const int want = n_sm / std::max(1, 2 * g.n_pairs), most = (T + 31) / 32;
@@ -970,16 +966,14 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     g.TN = (((T + g.n_tt - 1) / g.n_tt) + 15) / 16 * 16;
     g.n_tt = (T + g.TN - 1) / g.TN;   // rounding the width up may leave the last tiles without tokens
     g.n_stages = gemm_stages(g.TN);
-    g.status = status;
-    g.ksplit = 1; g.kper = 0; g.fix_part = fix_part; g.fix_flag = fix_flag; g.n_sm = n_sm;
+    g.ksplit = 1; g.kper = 0; g.n_sm = n_sm;
     g.splits = 1;
     g.kb_per_split = g.num_kb;
     // every token tile must hold a token: an empty one would issue an MMA of width 0
     if (g.n_stages < 2 || g.TN < 16 || g.TN > 256 || (g.n_tt - 1) * g.TN >= T) return SYN_E_INVALID_ARG;
     const int tiles = g.n_pairs * g.n_tt;
     g.pair_mode = tiles >= n_sm;
-    int n_cta;
-    if (ep.mode == EPI_PART && tiles < n_sm) {
+    if (mode == EPI_PART && tiles < n_sm) {
         int sp = std::min(GEMM_MAX_SPLITS, std::min(n_sm / tiles, std::max(1, g.num_kb / 4)));
         g.kb_per_split = (g.num_kb + sp - 1) / sp;
         g.splits = (g.num_kb + g.kb_per_split - 1) / g.kb_per_split;
@@ -990,7 +984,7 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     // fewer pair tiles than SMs but more single tiles: one wave that mixes whole pair tiles and single tiles
     // (two waves of single tiles would take longer than one pair tile)
     if (g.splits == 1 && !g.pair_mode && 2 * tiles > n_sm) g.pair_mode = 2;
-    if (g.splits == 1 && g.pair_mode == 1 && fix_part && fix_flag) {
+    if (g.splits == 1 && g.pair_mode == 1 && may_ksplit) {
         // The tiles left after the full waves: cut along K over otherwise idle CTAs (parts of at
         // least 8 k-blocks; helpers and owners are different CTAs, so R * parts <= n_cta).
         const int rem = tiles % n_cta;
@@ -1006,6 +1000,20 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
             }
         }
     }
+    return SYN_OK;
+}
+
+static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const bf16* w_packed, int packed_rows, int K,
+                       const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, int* splits_out = nullptr,
+                       float* fix_part = nullptr, int* fix_flag = nullptr) {
+    ProfScope prof(cls >= 0 ? prof_m : nullptr, cls, st);
+    GemmParams g;
+    int n_cta = 0;
+    const int pr = gemm_plan(ep.T, packed_rows, K, n_sm, ep.mode, fix_part && fix_flag, g, n_cta);
+    if (pr) return pr;
+    g.w = w_packed;
+    g.status = status;
+    g.fix_part = fix_part; g.fix_flag = fix_flag;
     if (splits_out) *splits_out = g.splits;
     const int smem = gemm_fixed_smem() + g.n_stages * gemm_stage_bytes(g.TN);
     const cudaError_t le = g.ksplit > 1 ? launch_pdl(gemm_kernel<true>, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep)
@@ -1510,6 +1518,38 @@ extern "C" int syn_op_attention_static(syn_model* m, syn_kv* kv, const syn_plan*
     else
         attn_kernel<64><<<p->n_cta, ATT_THREADS, AttnSmem<64>::TOTAL, st>>>(m->tm_q, kv->tm_kv, ap);
     return launch_ok() ? SYN_OK : SYN_E_CUDA;
+}
+
+// The projection schedule without a device (tests): the launch shape, and work item i of CTA `cta`.
+extern "C" int syn_gemm_plan_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t* out) {
+    if (T <= 0 || N <= 0 || K <= 0 || n_sm <= 0 || n_sm > 65535 || epilogue < EPI_PLAIN || epilogue > EPI_LMHEAD || !out)
+        return SYN_E_INVALID_ARG;
+    GemmParams g;
+    memset(&g, 0, sizeof(g));
+    int n_cta = 0;
+    const int r = gemm_plan(T, (N + 255) / 256 * 256, K, n_sm, epilogue, epilogue != EPI_PART, g, n_cta);
+    if (r) return r;
+    const int v[SYN_GEMM_PLAN_FIELDS] = {g.n_pairs, g.n_tt, g.TN, g.num_kb, n_cta, g.pair_mode, g.splits, g.kb_per_split, g.ksplit, g.kper};
+    memcpy(out, v, sizeof(v));
+    return SYN_OK;
+}
+
+extern "C" int syn_gemm_work_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t cta, int32_t i,
+                                  int32_t* out) {
+    if (T <= 0 || N <= 0 || K <= 0 || n_sm <= 0 || n_sm > 65535 || epilogue < EPI_PLAIN || epilogue > EPI_LMHEAD || !out || i < 0)
+        return SYN_E_INVALID_ARG;
+    GemmParams g;
+    memset(&g, 0, sizeof(g));
+    int n_cta = 0;
+    const int r = gemm_plan(T, (N + 255) / 256 * 256, K, n_sm, epilogue, epilogue != EPI_PART, g, n_cta);
+    if (r) return r;
+    if (cta < 0 || cta >= n_cta) return SYN_E_INVALID_ARG;
+    GemmWork w;
+    const bool have = g.ksplit > 1 ? gemm_work<true>(g, cta, n_cta, i, w) : gemm_work<false>(g, cta, n_cta, i, w);
+    if (!have) return 0;
+    const int v[SYN_GEMM_WORK_FIELDS] = {w.pair, w.tt, w.mt_lo, w.mt_hi, w.kb0, w.kb1, w.split, w.role, w.rtile, w.hpart};
+    memcpy(out, v, sizeof(v));
+    return 1;
 }
 
 extern "C" const char* syn_last_cuda_error(void) { return g_last_cuda_error; }
