@@ -35,8 +35,8 @@ UNIT = "tokens/s"
 NCU_TRAFFIC = {
     # workload: {kernel: (bytes per launch, sha256 of the kernel's source file)}
     "cfg3-8b": {
-        "attention": (615890944, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
-        "gemm": (139793337, "9ab6d49fa679f5c805fab39a61aa8098f4ab576763df1b008a48e1fc45c3c420"),
+        "attention": (615966076, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
+        "gemm": (140141518, "4caa57856b234a4a49c91d04f4f6f1c774d7a1598602fd63507e1b776e9f5f84"),
     },
 }
 
