@@ -44,6 +44,8 @@ def _slm_rows(rng, logits_prev, chunk, u, slm_k, V, temp, mode):
 @pytest.mark.parametrize("V,top_k,top_p,temp,slm_k", [
     (1000, 8, 1.0, 1.0, 8), (32000, 50, 0.9, 0.7, 20), (151, 64, 0.5, 1.3, 64), (4099, 1, 1.0, 1.0, 1),
     (128256, 40, 0.95, 1.0, 40),
+    (40, 64, 1.0, 1.0, 8),            # fewer logits than top_k: everything is kept
+    (513, 3, 0.7, 0.5, 5),            # vocabulary not a multiple of four: scalar candidate pass
 ])
 def test_sampling_stage_matches_the_oracle_on_the_same_logits(V, top_k, top_p, temp, slm_k):
     import paper_2511_07423_b200 as syn
