@@ -1,6 +1,7 @@
 """Pins of the CPU oracle against things other than itself: a dense full-matrix numpy
 forward, invariants of paging and chunking, hand-worked integer cases, closed forms,
 and the capped-geometric acceptance expectation (paper Sec. 5)."""
+import itertools
 import math
 
 import numpy as np
@@ -363,16 +364,56 @@ def test_mean_accept_len_follows_capped_geometric():
 @pytest.mark.parametrize("row", _golden("expected_generated_tokens.txt"))
 def test_generated_tokens_per_verification_match_the_papers_expectation(row):
     """Drafts that match the argmax independently with probability alpha: accepted drafts + the
-    correction/bonus token per verification average to the stored closed-form value (Sec. 5)."""
+    correction/bonus token per verification have the stored closed-form expectation (Sec. 5).
+    Exact: every one of the 2^gamma hit patterns goes through the verification routine and is
+    weighted with its probability, so a wrong fourth decimal in the stored value fails."""
     alpha, gamma, expect = float(row[0]), int(row[1]), float(row[2])
-    g = np.random.default_rng(int(alpha * 1000) + gamma)
-    n_req, total = 20000, 0
-    for _ in range(n_req):
-        top1 = g.integers(0, 1000, size=gamma + 1)
-        hit = g.random(gamma) < alpha
-        chunk = [0] + [int(top1[j]) if hit[j] else int(top1[j]) + 1000 for j in range(gamma)]
-        total += verify_greedy(top1, chunk, 1)[0] + 1
-    assert abs(total / n_req - expect) < 4 * 1.3 / math.sqrt(n_req) + 5e-4
+    top1 = [11 + 3 * j for j in range(gamma + 1)]
+    total = 0.0
+    for pattern in itertools.product((False, True), repeat=gamma):
+        prob = 1.0
+        for hit in pattern:
+            prob *= alpha if hit else 1.0 - alpha
+        chunk = [0] + [top1[j] if pattern[j] else top1[j] + 1000 for j in range(gamma)]
+        total += prob * (verify_greedy(top1, chunk, 1)[0] + 1)
+    assert abs(total - expect) < 1e-12
+
+
+# ---------------------------------------------------------------- SwiGLU: hand values, not the formula again
+def test_swiglu_product_against_hand_values_of_silu():
+    """One layer whose attention contributes nothing (zero q/k/v/o projections), unit gains and
+    eps = 0, fed rows of mean square 1, so the normalised hidden state h equals the row itself.
+    With W_g = I, W_d = I and every row of W_u picking h[1], the layer adds silu(h_i) * h[1] to
+    x_i.  The expected numbers are tabulated values of the logistic function, typed in, not the
+    expression under test evaluated again: silu(0) = 0, silu(1) = 0.7310585786,
+    silu(-1) = -0.2689414214, silu(2) = 1.7615941560."""
+    shape = ModelShape("swiglu-pin", 1, 4, 1, 1, 4, 4, 8, rms_eps=0.0)
+    orc = Oracle(shape, page_size=16)
+
+    def bf(a):
+        return torch.tensor(a, dtype=torch.float32).to(torch.bfloat16)
+
+    eye = [[1.0 if i == j else 0.0 for j in range(4)] for i in range(4)]
+    zero = [[0.0] * 4 for _ in range(4)]
+    w = {"wq": bf(zero), "wk": bf(zero), "wv": bf(zero), "wo": bf(zero), "wg": bf(eye),
+         "wu": bf([[0.0, 1.0, 0.0, 0.0]] * 4), "wd": bf(eye), "norm1": bf([1.0] * 4), "norm2": bf([1.0] * 4)}
+    pt = np.array([0], dtype=np.int32)
+    pool = orc.new_pool(1)
+    # h = (0, 1, -1, sqrt 2): up = h[1] = 1;  h = (1, -1, 1, 1): up = -1 (the product's second factor and its sign)
+    x = np.array([[0.0, 1.0, -1.0, math.sqrt(2.0)], [1.0, -1.0, 1.0, 1.0]], dtype=np.float64)
+    before = x.copy()
+    orc.layer(w, x, pool[0], pt, 0)
+    upd = x - before
+    assert np.allclose(upd[0][:3], [0.0, 0.7310585786, -0.2689414214], atol=1e-9)
+    assert np.allclose(upd[1], [-0.7310585786, 0.2689414214, -0.7310585786, -0.7310585786], atol=1e-9)
+    # gate and up from different inputs and with weights other than 0 / 1: g = 2 h[0], u = -2 h[1]
+    w2 = dict(w)
+    w2["wg"] = bf([[2.0, 0, 0, 0]] + [[0.0] * 4] * 3)
+    w2["wu"] = bf([[0, -2.0, 0, 0]] + [[0.0] * 4] * 3)
+    x2 = np.ones((1, 4), dtype=np.float64)
+    orc.layer(w2, x2, pool[0], pt, 0)
+    assert abs((x2[0][0] - 1.0) - 1.7615941560 * -2.0) < 1e-8
+    assert np.allclose(x2[0][1:], 1.0, atol=1e-12)
 
 
 # ---------------------------------------------------------------- the single-precision build agrees
