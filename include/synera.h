@@ -104,7 +104,8 @@ void syn_kv_free(syn_kv *kv);
 /* Place externally produced (already rotated) K and V of one request and one layer at logical
  * positions pos0 .. pos0+n_pos-1, e.g. a prefix computed on another server.  k, v: DEVICE bf16
  * [n_pos][n_kv_heads][head_dim]; page_table: HOST int32, at least ceil((pos0+n_pos)/page_size)
- * entries.  Asynchronous on `cuda_stream` except for a small blocking metadata copy.
+ * entries.  Blocking: the call allocates a small device buffer for the slot list, synchronises
+ * `cuda_stream` and returns when the copy is done.
  * syn_kv_export is the inverse (reads the same positions into k, v).
  * Errors: SYN_E_INVALID_ARG, SYN_E_PAGE_OOB, SYN_E_CUDA. */
 int syn_kv_import(syn_kv *kv, uint32_t layer, const int32_t *page_table, int32_t pos0, int32_t n_pos,
@@ -152,7 +153,11 @@ int syn_verify_batch(syn_model *m, syn_kv *kv, int32_t n_req, const int64_t *req
  * asynchronously on cuda_stream; accept_len_dev / correction_dev are DEVICE int32 [n_req];
  * top1_dev is NULL or DEVICE int32 [T] (argmax per chunk position).  It does not synchronise:
  * call syn_model_status after synchronising the stream to learn of a device-side timeout.
- * A plan may be run any number of times (each run rewrites the same KV slots). */
+ * A plan may be run any number of times (each run rewrites the same KV slots).
+ * A plan belongs to the cache it was created with: its page ids and KV slots were checked against
+ * that cache's size, so syn_verify_run, syn_op_attention and syn_op_attention_static return
+ * SYN_E_INVALID_ARG, before any launch, when they are given another cache (or that cache freed and
+ * another allocated in its place). */
 int syn_plan_create(syn_model *m, syn_kv *kv, int32_t n_req, const int32_t *chunk_tokens,
                     const int32_t *chunk_offsets, const int32_t *page_tables, int32_t max_pages,
                     const int32_t *ctx_lens, const int32_t *n_uncached, syn_plan **out);
@@ -161,7 +166,7 @@ int syn_verify_run(syn_model *m, syn_kv *kv, const syn_plan *p, int32_t *accept_
                    int32_t *correction_dev, int32_t *top1_dev, float *logits_out, void *cuda_stream);
 int syn_model_status(syn_model *m); /* SYN_OK or SYN_E_DEVICE_TIMEOUT / SYN_E_CUDA; blocking */
 
-/* Counters of the last planned step (algorithmic work, for roofline arithmetic). */
+/* Counters of a step (algorithmic work, for roofline arithmetic) and, measured, its times. */
 typedef struct {
     int32_t n_req, n_tokens;       /* B and T                                               */
     int64_t ctx_tokens;            /* sum of ctx_lens                                       */
@@ -173,8 +178,15 @@ typedef struct {
     int32_t attn_items, attn_split_items; /* attention work items per layer / those that are partial */
     int32_t kernel_launches;       /* kernels launched by one syn_verify_run                */
     int64_t h2d_bytes;             /* batch description uploaded per step by syn_verify_batch */
+    double t_gpu_ms;               /* device time of the step, first kernel to last (CUDA events); 0 unless profiling is on */
+    double t_wall_ms;              /* host wall time of the blocking call that ran it; 0 unless profiling is on  */
 } syn_step_stats;
-int syn_last_step_stats(const syn_plan *p, syn_step_stats *out);
+/* The last step launched on this model by syn_verify_batch, syn_verify_batch_sampled or syn_verify_run
+ * (the paper's cloud runtime reports per-iteration execution time, Sec. 6.7).  With syn_set_profile on,
+ * t_gpu_ms is filled (the call then waits for that step to finish) and, for the blocking calls,
+ * t_wall_ms.  SYN_E_INVALID_ARG before the first step.  syn_plan_stats: the counters of a plan. */
+int syn_last_step_stats(syn_model *m, syn_step_stats *out);
+int syn_plan_stats(const syn_plan *p, syn_step_stats *out);
 
 /* The host planner of syn_plan_create / syn_verify_batch on its own, without a device: the same
  * validation (same error codes, same order) and the same outputs, written to caller-provided HOST
@@ -198,8 +210,8 @@ int syn_plan_host(const syn_model_desc *desc, uint32_t n_pages, uint32_t page_si
  * adds up the elapsed time and launch count of each class since the last call, and clears them.
  * Classes: 0 prep, 1 qkv GEMM, 2 attention, 3 attention merge, 4 o GEMM, 5 gate/up GEMM,
  * 6 down GEMM, 7 lm_head GEMM, 8 verify (greedy compare, and the sampling stage of
- * syn_verify_batch_sampled), 9 residual + norm statistic.  ms, launches: HOST arrays
- * of SYN_N_KERNEL_CLASSES. */
+ * syn_verify_batch_sampled), 9 unused (the residual update and the norm statistic are part of the
+ * o and down GEMMs).  ms, launches: HOST arrays of SYN_N_KERNEL_CLASSES. */
 #define SYN_N_KERNEL_CLASSES 10
 int syn_set_profile(syn_model *m, int on);
 int syn_get_profile(syn_model *m, double *ms, int32_t *launches);
@@ -213,10 +225,28 @@ const char *syn_last_cuda_error(void);
 
 /* y[T][N] (fp32, DEVICE) = x[T][K] (bf16, DEVICE) * W[N][K]^T (bf16, DEVICE): the tcgen05
  * GEMM used by every projection, with a plain store epilogue.  The first call with a given w
- * (pointer and shape) packs it into the library's tiled layout; later calls reuse the packed copy.  K a multiple of 64 is not
- * required (TMA zero-fills the tail) but K*2 bytes must be a multiple of 16; N arbitrary.
- * Errors: SYN_E_INVALID_ARG, SYN_E_CUDA. */
+ * (pointer and shape) packs it into the library's tiled layout; later calls reuse the packed copy:
+ * call syn_op_linear_reset after the contents of w changed or w was freed (a new matrix may land at
+ * the old address).  K a multiple of 64 is not required (TMA zero-fills the tail) but K*2 bytes must
+ * be a multiple of 16; N arbitrary.  Blocks until the result is there.
+ * syn_op_linear_as runs the same product under the schedule the step uses for the projection with
+ * epilogue `schedule_as` (0 plain, 1 qkv, 2 residual, 3 SwiGLU, 4 lm_head; see syn_gemm_plan_host), so
+ * that every schedule can be checked against a plain matrix product.
+ * Errors: SYN_E_INVALID_ARG, SYN_E_CUDA, SYN_E_DEVICE_TIMEOUT. */
 int syn_op_linear(const void *x, const void *w, float *y, int32_t T, int32_t N, int32_t K, void *cuda_stream);
+int syn_op_linear_as(const void *x, const void *w, float *y, int32_t T, int32_t N, int32_t K, int32_t schedule_as,
+                     void *cuda_stream);
+int syn_op_linear_reset(void);
+
+/* Test hooks for the bounded device-side waits (SYN_E_DEVICE_TIMEOUT).  syn_debug_set_spin_limit: the
+ * number of SM cycles after which a wait inside the projection kernels gives up (0 restores the default,
+ * about two seconds); applies to launches made afterwards, process-wide.  syn_debug_linear_counter:
+ * overwrite one of the arrival counters of syn_op_linear's own workspace (index in [0, 2 * SMs)), so
+ * that a wait for a count that can no longer be reached runs out; the counters are cleared again when
+ * the timeout is reported.  A wait that runs out unwinds normally: the kernel ends, the results of
+ * that call are invalid, the next call works. */
+int syn_debug_set_spin_limit(int64_t cycles);
+int syn_debug_linear_counter(int32_t index, int32_t value);
 
 /* The ragged paged attention of the step on its own (paper Sec. 3.2 attention equation over a
  * paged cache).  q: DEVICE bf16 [T][n_q_heads*head_dim] (rotated); out: DEVICE bf16, same
@@ -235,7 +265,7 @@ int syn_op_attention(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer
  * that loads the library, from load to exit).  The call itself allocates and frees nothing; the
  * model, cache and plan it is given were of course allocated earlier by their own calls.
  *   - A plan with more partial work items than SYN_STATIC_MAX_PARTS is refused with
- *     SYN_E_CAPACITY before anything is launched (syn_last_step_stats().attn_split_items tells).
+ *     SYN_E_CAPACITY before anything is launched (syn_plan_stats().attn_split_items tells).
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call outside any stream capture.
  *   - All calls on a device share the one array.  It keeps the previous call's contents; nothing
@@ -247,10 +277,10 @@ int syn_op_attention_static(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_
                             void *cuda_stream);
 
 /* The projection kernel's schedule without a device (tests): how a y[T][N] = x[T][K] w[N][K]^T
- * projection with the given epilogue (0 plain store, 1 QKV, 2 split-K partial, 3 SwiGLU, 4 lm_head)
+ * projection with the given epilogue (0 plain store, 1 QKV, 2 residual update, 3 SwiGLU, 4 lm_head)
  * is cut up on n_sm SMs.  syn_gemm_plan_host fills out[SYN_GEMM_PLAN_FIELDS] = {feature pairs of 256,
- * token tiles, tokens per tile, k-blocks of 64, CTAs, pair mode, split-K parts, k-blocks per part,
- * K parts of a leftover pair tile, k-blocks of a helper part}.  syn_gemm_work_host returns 1 and
+ * token tiles, tokens per tile, k-blocks of 64, CTAs, pair mode, CTAs that share a tile's K range
+ * (reduce-scatter), k-blocks of each, K parts of a leftover pair tile, k-blocks of a helper part}.  syn_gemm_work_host returns 1 and
  * fills out[SYN_GEMM_WORK_FIELDS] = {pair, token tile, first 128-feature tile, one past the last,
  * first k-block, one past the last, split-K part, role (0 whole K, 1 helper, 2 owner), leftover
  * tile, helper part} for work item i of CTA cta, 0 when that CTA has no item i.

@@ -46,17 +46,20 @@ class StepStats(C.Structure):
     _fields_ = [("n_req", C.c_int32), ("n_tokens", C.c_int32), ("ctx_tokens", C.c_int64),
                 ("weight_bytes", C.c_int64), ("kv_read_bytes", C.c_int64), ("kv_write_bytes", C.c_int64),
                 ("dense_flops", C.c_double), ("attn_flops", C.c_double), ("attn_items", C.c_int32),
-                ("attn_split_items", C.c_int32), ("kernel_launches", C.c_int32), ("h2d_bytes", C.c_int64)]
+                ("attn_split_items", C.c_int32), ("kernel_launches", C.c_int32), ("h2d_bytes", C.c_int64),
+                ("t_gpu_ms", C.c_double), ("t_wall_ms", C.c_double)]
 
 KERNEL_CLASSES = ("prep", "qkv_gemm", "attention", "attention_merge", "o_gemm", "gate_up_gemm", "down_gemm",
-                  "lm_head_gemm", "verify", "resid_norm")
+                  "lm_head_gemm", "verify", "unused")
 
 
 _LIB: Optional[C.CDLL] = None
 
 EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "syn_kv_import", "syn_kv_export",
            "syn_verify_batch", "syn_plan_create", "syn_plan_free", "syn_verify_run", "syn_model_status",
-           "syn_last_step_stats", "syn_plan_host", "syn_strerror", "syn_last_cuda_error", "syn_op_linear", "syn_op_attention", "syn_op_attention_static",
+           "syn_last_step_stats", "syn_plan_stats", "syn_plan_host", "syn_strerror", "syn_last_cuda_error", "syn_op_linear",
+           "syn_op_linear_as", "syn_op_linear_reset", "syn_debug_set_spin_limit", "syn_debug_linear_counter",
+           "syn_op_attention", "syn_op_attention_static",
            "syn_set_profile", "syn_get_profile", "syn_verify_batch_sampled", "syn_op_sample_verify",
            "syn_gemm_plan_host", "syn_gemm_work_host"]
 SCHED_EXPORTS = ["syn_sched_create", "syn_sched_free", "syn_sched_add_request", "syn_sched_add_verify", "syn_sched_finish",
@@ -150,6 +153,13 @@ class Model:
 
     def set_profile(self, on: bool) -> None:
         _check(self._lib.syn_set_profile(self._h, C.c_int(1 if on else 0)), "syn_set_profile")
+
+    def last_step_stats(self) -> "StepStats":
+        """syn_last_step_stats: counters of the last step launched on this model; with profiling on
+        also its device time and, for the blocking calls, the wall time."""
+        s = StepStats()
+        _check(self._lib.syn_last_step_stats(self._h, C.byref(s)), "syn_last_step_stats")
+        return s
 
     def get_profile(self):
         """{class name: (total ms, launches)} since the last call (synchronises the device)."""
@@ -269,7 +279,7 @@ def syn_op_sample_verify(logits: torch.Tensor, chunk_tokens, chunk_offsets, n_un
 
 
 class Plan:
-    """syn_plan_create / syn_verify_run / syn_op_attention / syn_last_step_stats / syn_plan_free."""
+    """syn_plan_create / syn_verify_run / syn_op_attention / syn_plan_stats / syn_plan_free."""
 
     def __init__(self, kv: KVCache, chunk_tokens, chunk_offsets, page_tables, ctx_lens, n_uncached=None):
         self._lib = load_library()
@@ -285,7 +295,7 @@ class Plan:
 
     def stats(self) -> StepStats:
         s = StepStats()
-        _check(self._lib.syn_last_step_stats(self._h, C.byref(s)), "syn_last_step_stats")
+        _check(self._lib.syn_plan_stats(self._h, C.byref(s)), "syn_plan_stats")
         return s
 
     def run(self, accept_len: torch.Tensor, correction: torch.Tensor, top1: Optional[torch.Tensor] = None,
@@ -484,7 +494,7 @@ class Scheduler:
 
 GEMM_PLAN_FIELDS = ("n_pairs", "n_tt", "TN", "num_kb", "n_cta", "pair_mode", "splits", "kb_per_split", "ksplit", "kper")
 GEMM_WORK_FIELDS = ("pair", "tt", "mt_lo", "mt_hi", "kb0", "kb1", "split", "role", "rtile", "hpart")
-GEMM_EPILOGUES = {"plain": 0, "qkv": 1, "part": 2, "swiglu": 3, "lmhead": 4}
+GEMM_EPILOGUES = {"plain": 0, "qkv": 1, "resid": 2, "swiglu": 3, "lmhead": 4}
 
 
 def gemm_plan_host(T: int, N: int, K: int, epilogue: str, n_sm: int = 148) -> Dict[str, int]:
@@ -505,13 +515,31 @@ def gemm_work_host(T: int, N: int, K: int, epilogue: str, cta: int, i: int, n_sm
     return dict(zip(GEMM_WORK_FIELDS, out)) if r == 1 else None
 
 
-def syn_op_linear(x: torch.Tensor, w: torch.Tensor, stream=None) -> torch.Tensor:
-    """y[T, N] fp32 = x[T, K] bf16 @ w[N, K]^T bf16 through the library's tcgen05 GEMM."""
+def syn_op_linear(x: torch.Tensor, w: torch.Tensor, stream=None, schedule_as: str = "plain",
+                  reuse_pack: bool = False) -> torch.Tensor:
+    """y[T, N] fp32 = x[T, K] bf16 @ w[N, K]^T bf16 through the library's tcgen05 GEMM, under the
+    schedule the step uses for the projection with epilogue `schedule_as`.  The library keeps a packed
+    copy of the last w keyed by address and shape; unless `reuse_pack` says the matrix is the one of the
+    previous call, the copy is dropped first (a new tensor may sit at a freed tensor's address)."""
     assert x.is_cuda and w.is_cuda and x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
     x, w = x.contiguous(), w.contiguous()
     T, K = x.shape
     N = w.shape[0]
     y = torch.empty(T, N, dtype=torch.float32, device="cuda")
-    _check(load_library().syn_op_linear(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
-                                        C.c_int32(T), C.c_int32(N), C.c_int32(K), _stream_ptr(stream)), "syn_op_linear")
+    lib = load_library()
+    if not reuse_pack:
+        _check(lib.syn_op_linear_reset(), "syn_op_linear_reset")
+    _check(lib.syn_op_linear_as(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
+                                C.c_int32(T), C.c_int32(N), C.c_int32(K), C.c_int32(GEMM_EPILOGUES[schedule_as]),
+                                _stream_ptr(stream)), "syn_op_linear_as")
     return y
+
+
+def debug_set_spin_limit(cycles: int) -> None:
+    """syn_debug_set_spin_limit: SM cycles after which a wait inside the projection kernels gives up (0: default)."""
+    _check(load_library().syn_debug_set_spin_limit(C.c_int64(cycles)), "syn_debug_set_spin_limit")
+
+
+def debug_linear_counter(index: int, value: int) -> None:
+    """syn_debug_linear_counter: overwrite one arrival counter of syn_op_linear's workspace."""
+    _check(load_library().syn_debug_linear_counter(C.c_int32(index), C.c_int32(value)), "syn_debug_linear_counter")

@@ -5,30 +5,43 @@
 // (N = 16..256 tokens), so a batch of T tokens pads to a multiple of 16 instead of 128.  Weights are
 // stored pre-tiled and pre-swizzled ([feature pair][k-block][2][128 x 64] images of the
 // 128-byte-swizzled shared-memory tile), so a stage's weights are ONE contiguous bulk copy;
-// activations come through a TMA tensor map.  One persistent CTA per SM walks a static schedule:
-// whole pair tiles in full waves; the pair tiles left over are cut along K into parts on different
-// CTAs (the "helper" parts run first and store their fp32 accumulators, the "owner" part runs last
-// on another CTA, adds them in part order and finishes the tile), or, where K is too short for
-// that, run as single 128-feature tiles; projections with few output tiles (o, down) split K over
-// CTAs and write fp32 partials that resid_norm_kernel adds to the residual stream in a fixed order.  Every CTA starts its k loop at a different k-block, so the CTAs
-// that share a token tile do not ask L2 for the same lines at the same moment.  Accumulation is
-// tcgen05.mma into TMEM, read back with tcgen05.ld by sixteen epilogue warps; a thread then holds one
-// output feature for sixteen tokens (thirty-two in the epilogues that need few other registers: the
-// fp32 stores and SwiGLU; an epilogue is bound by the round trips of its loads, not by their width),
-// and the epilogues work on those registers:
-//   EPI_QKV    : RoPE on q and k (the partner dimension sits 16 lanes away), q store, paged-KV append
-//   EPI_PART   : fp32 partial of a split-K projection (residual added by resid_norm_kernel)
-//   EPI_SWIGLU : silu(gate) * up (a gate feature and its up feature sit 16 lanes apart)
-//   EPI_LMHEAD : optional logits, vocabulary argmax (warp reduction, packed 64-bit atomicMax)
+// activations come through a TMA tensor map.  One persistent CTA per SM walks a static schedule.
+// Three variants of the kernel (template parameter):
+//   GEMM_WAVES  : whole pair tiles in full waves, leftovers as single 128-feature tiles;
+//   GEMM_KSPLIT : as above, but the pair tiles left over after the full waves are cut along K into
+//                 parts on different CTAs (the "helper" parts run first and store their fp32
+//                 accumulators, the "owner" part runs last on another CTA, adds them in part order
+//                 and finishes the tile);
+//   GEMM_RSPLIT : projections with fewer pair tiles than SMs (o, down, qkv at a few hundred tokens):
+//                 every tile's K range is split over S CTAs that run at the same time; each CTA
+//                 keeps a contiguous share of the tile's token columns, hands the accumulators of
+//                 the other columns to their keepers through global memory, adds what it receives
+//                 in split order (so the sum does not depend on timing) and runs the epilogue on
+//                 its own columns: a reduce-scatter, after which all S CTAs share the epilogue.
+// Every CTA starts its k loop at a different k-block, so the CTAs that share a token tile do not
+// ask L2 for the same lines at the same moment.  Accumulation is tcgen05.mma into TMEM, read back
+// with tcgen05.ld by sixteen epilogue warps; a thread then holds one output feature for sixteen
+// tokens (thirty-two in the epilogues that need few other registers), and the epilogues work on
+// those registers:
+//   EPI_QKV    : RMSNorm scale, RoPE on q and k (the partner dimension sits 16 lanes away), q store,
+//                paged-KV append
+//   EPI_RESID  : x += D (the residual stream, fp32), the next projection's operand bf16(x * gain) and
+//                the sums of x^2 over each group of 32 features that the next RMSNorm needs
+//   EPI_SWIGLU : RMSNorm scale, silu(gate) * up (a gate feature and its up feature sit 16 lanes apart)
+//   EPI_LMHEAD : RMSNorm scale, optional logits, vocabulary argmax (warp reduction, packed 64-bit atomicMax)
 //   EPI_PLAIN  : fp32 store (test hook)
-// The token operand of the QKV, gate/up and lm_head projections is the RMSNorm of the residual stream,
-// bf16(x * rstd * gain), written by resid_norm_kernel (prep_kernel for the first layer).
+// RMSNorm is split between producer and consumer: the kernel that writes the residual stream
+// (EPI_RESID, or prep_kernel for the first layer) stores bf16(x * gain) and partial sums of x^2; the
+// projection that consumes it multiplies its accumulators by the token's 1/sqrt(mean(x^2) + eps),
+// a per-column scalar in this orientation, which its epilogue warps work out from the partial sums
+// while the main loop runs.
 #pragma once
 #include "ptx.cuh"
 
 namespace syn {
 
-enum { EPI_PLAIN = 0, EPI_QKV = 1, EPI_PART = 2, EPI_SWIGLU = 3, EPI_LMHEAD = 4 };
+enum { EPI_PLAIN = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, EPI_LMHEAD = 4 };
+enum { GEMM_WAVES = 0, GEMM_KSPLIT = 1, GEMM_RSPLIT = 2 };
 
 struct EpiParams {
     int mode;
@@ -43,9 +56,15 @@ struct EpiParams {
     const float2* rope;  // [T][hd/2] (cos, sin)
     __nv_bfloat16* pool; // this layer's pool: [page][kvh][K|V][row][hd]
     const int* slot;     // [T] page * page_size + row
-    // PART
-    float* part;         // [splits][part_stride] fp32, row pitch d
-    size_t part_stride;
+    // RMSNorm scale of the token operand (QKV, SWIGLU, LMHEAD; NULL: the operand is used as it is)
+    const float* ssq_in; // [T][n_ssq] partial sums of x^2 of the operand's source rows
+    int n_ssq;           // a multiple of 4
+    float inv_d, eps;
+    // RESID
+    float* x;            // [T][d] residual stream, updated in place
+    const __nv_bfloat16* gain;   // [d] gain of the NEXT RMSNorm
+    __nv_bfloat16* xg;   // [T][d] bf16(x * gain): the next projection's operand
+    float* ssq_out;      // [T][d / 32]
     int d;
     // SWIGLU
     __nv_bfloat16* act;
@@ -79,25 +98,92 @@ __host__ __device__ __forceinline__ int rope_tile_feature(int l, int hd) {   // 
     return (q / groups) * hd + 16 * (q % groups) + (ll & 15) + ((ll & 16) ? half : 0);
 }
 
+constexpr int GEMM_EPI_WARPS = 16;               // four groups of four (one warp per TMEM lane quarter)
+
+// Sum over the 32 lanes of sixteen values per lane in sixteen shuffles: each round halves the values
+// a lane keeps (the lanes of a pair exchange the halves they give up).  Afterwards lane L holds the
+// total of value number L >> 1 (both lanes of a pair hold the same total).  The order of the
+// additions is fixed.
+__device__ __forceinline__ float warp_sum16(float (&v)[16], int lane) {
+    {
+        const bool up = (lane & 16) != 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float got = __shfl_xor_sync(0xFFFFFFFFu, up ? v[i] : v[8 + i], 16);
+            v[i] = (up ? v[8 + i] : v[i]) + got;
+        }
+    }
+    {
+        const bool up = (lane & 8) != 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float got = __shfl_xor_sync(0xFFFFFFFFu, up ? v[i] : v[4 + i], 8);
+            v[i] = (up ? v[4 + i] : v[i]) + got;
+        }
+    }
+    {
+        const bool up = (lane & 4) != 0;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const float got = __shfl_xor_sync(0xFFFFFFFFu, up ? v[i] : v[2 + i], 4);
+            v[i] = (up ? v[2 + i] : v[i]) + got;
+        }
+    }
+    {
+        const bool up = (lane & 2) != 0;
+        const float got = __shfl_xor_sync(0xFFFFFFFFu, up ? v[0] : v[1], 2);
+        v[0] = (up ? v[1] : v[0]) + got;
+    }
+    return v[0] + __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
+}
+
 // Epilogue of one 16-token chunk straight from registers: r[j] = D[feature of this thread][token
 // t0 + j]; tokens j >= ncols are padding.  `m0` = first packed row of the tile, `quarter` = warp's TMEM
-// lane quarter.  Warp shuffles, votes and reductions are never moved across stores by the compiler, and
+// lane quarter.  `rs` = NULL, or the RMSNorm scales of tokens t0 .. t0 + 15 (shared memory).
+// Warp shuffles, votes and reductions are never moved across stores by the compiler, and
 // loads not above stores that might alias them, so every mode first runs all its warp-wide exchanges
 // and loads back to back (their latencies overlap) and only then does the arithmetic and the stores.
 constexpr int EPI_COLS = 16;
 template <int MODE>
-__device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&r)[EPI_COLS], int m0, int t0, int ncols,
-                                           int split, int quarter, int lane) {
+__device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&r)[EPI_COLS], const float* rs, int m0, int t0,
+                                           int ncols, int quarter, int lane) {
     const int l = quarter * 32 + lane;
-    if (MODE == EPI_PLAIN || MODE == EPI_PART) {
+    float a[EPI_COLS];
+#pragma unroll
+    for (int j = 0; j < EPI_COLS; ++j) a[j] = __uint_as_float(r[j]);
+    if (MODE != EPI_PLAIN && MODE != EPI_RESID && rs != nullptr) {
+#pragma unroll
+        for (int j = 0; j < EPI_COLS; ++j) a[j] *= rs[j];
+    }
+    if (MODE == EPI_PLAIN) {
         const int f = m0 + l;
-        const size_t ld = MODE == EPI_PLAIN ? (size_t)p.ldy : (size_t)p.d;
-        float* base = (MODE == EPI_PLAIN ? p.y + f : p.part + (size_t)split * p.part_stride + f) + (size_t)t0 * ld;
+        float* base = p.y + f + (size_t)t0 * p.ldy;
         if (f < p.N) {
 #pragma unroll
             for (int j = 0; j < EPI_COLS; ++j)
-                if (j < ncols) base[(size_t)j * ld] = __uint_as_float(r[j]);
+                if (j < ncols) base[(size_t)j * p.ldy] = a[j];
         }
+    } else if (MODE == EPI_RESID) {
+        // x += D; operand of the next projection; sums of x^2 over this warp's 32 features
+        const int f = m0 + l;
+        const bool fv = f < p.N;
+        const size_t at = (size_t)t0 * p.d + (fv ? f : 0);
+        float xv[EPI_COLS];
+#pragma unroll
+        for (int j = 0; j < EPI_COLS; ++j) xv[j] = (fv && j < ncols) ? p.x[at + (size_t)j * p.d] : 0.f;
+        const float gn = fv ? __bfloat162float(p.gain[f]) : 0.f;
+#pragma unroll
+        for (int j = 0; j < EPI_COLS; ++j) {
+            xv[j] = (fv && j < ncols) ? xv[j] + a[j] : 0.f;
+            if (fv && j < ncols) {
+                p.x[at + (size_t)j * p.d] = xv[j];
+                p.xg[at + (size_t)j * p.d] = __float2bfloat16(xv[j] * gn);
+            }
+            xv[j] *= xv[j];
+        }
+        const float tot = warp_sum16(xv, lane);   // lane L: token L >> 1
+        if (!(lane & 1) && (lane >> 1) < ncols && m0 + quarter * 32 < p.N)
+            p.ssq_out[(size_t)(t0 + (lane >> 1)) * (p.d >> 5) + ((m0 >> 5) + quarter)] = tot;
     } else if (MODE == EPI_QKV) {
         const int which = m0 < p.q_dim ? 0 : (m0 < p.q_dim + p.kv_dim ? 1 : 2);
         const int region0 = which == 0 ? 0 : (which == 1 ? p.q_dim : p.q_dim + p.kv_dim);
@@ -106,26 +192,26 @@ __device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&
         const int dim = fr & (p.hd - 1);
         const bool lo = dim < half;
         const float2* cs = p.rope + (size_t)t0 * half + (lo ? dim : dim - half);
-        const int* slot = p.slot + t0;
         float o[EPI_COLS];   // rotate-half RoPE: the partner dimension is 16 lanes away
         float2 w[EPI_COLS];
-        int sl[EPI_COLS];
+        // KV slots (page * 16 + row) of the chunk's tokens: one coalesced load, handed round by shuffles
+        const int my_slot = (which > 0 && lane < ncols) ? __ldg(p.slot + t0 + lane) : 0;
 #pragma unroll
         for (int j = 0; j < EPI_COLS; ++j) {
-            o[j] = which < 2 ? __shfl_xor_sync(0xFFFFFFFFu, __uint_as_float(r[j]), 16) : 0.f;
+            o[j] = which < 2 ? __shfl_xor_sync(0xFFFFFFFFu, a[j], 16) : 0.f;
             w[j] = (which < 2 && j < ncols) ? __ldg(cs + (size_t)j * half) : make_float2(1.f, 0.f);
-            sl[j] = (which > 0 && j < ncols) ? __ldg(slot + j) : 0;   // page * 16 + row; same address in all lanes
         }
         __nv_bfloat16* const qdst = p.q + (size_t)t0 * p.q_dim + fr;
         __nv_bfloat16* const kvdst = p.pool + ((size_t)(fr / p.hd) * 2 + (which > 0 ? which - 1 : 0)) * 16 * p.hd + dim;
         const size_t page_stride = (size_t)p.n_kv_heads * 2 * 16 * p.hd;
 #pragma unroll
         for (int j = 0; j < EPI_COLS; ++j) {
+            const int sl = __shfl_sync(0xFFFFFFFFu, my_slot, j);
             if (j < ncols) {
-                float a = __uint_as_float(r[j]);
-                if (which < 2) a = lo ? (a * w[j].x - o[j] * w[j].y) : (a * w[j].x + o[j] * w[j].y);
-                if (which == 0) qdst[(size_t)j * p.q_dim] = __float2bfloat16(a);
-                else kvdst[(size_t)(sl[j] >> 4) * page_stride + (size_t)(sl[j] & 15) * p.hd] = __float2bfloat16(a);
+                float v = a[j];
+                if (which < 2) v = lo ? (v * w[j].x - o[j] * w[j].y) : (v * w[j].x + o[j] * w[j].y);
+                if (which == 0) qdst[(size_t)j * p.q_dim] = __float2bfloat16(v);
+                else kvdst[(size_t)(sl >> 4) * page_stride + (size_t)(sl & 15) * p.hd] = __float2bfloat16(v);
             }
         }
     } else if (MODE == EPI_SWIGLU) {
@@ -136,31 +222,31 @@ __device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&
         float got[EPI_COLS / 2];
 #pragma unroll
         for (int k = 0; k < EPI_COLS / 2; ++k)   // each half-warp sends what the other one needs
-            got[k] = __shfl_xor_sync(0xFFFFFFFFu, __uint_as_float(up_half ? r[2 * k] : r[2 * k + 1]), 16);
+            got[k] = __shfl_xor_sync(0xFFFFFFFFu, up_half ? a[2 * k] : a[2 * k + 1], 16);
         __nv_bfloat16* const dst = p.act + (size_t)(t0 + (up_half ? 1 : 0)) * p.f_pad + (m0 >> 1) + 16 * quarter + (lane & 15);
 #pragma unroll
         for (int k = 0; k < EPI_COLS / 2; ++k) {
-            const float gate = up_half ? got[k] : __uint_as_float(r[2 * k]);       // upper half: gate of token 2k + 1
-            const float upv = up_half ? __uint_as_float(r[2 * k + 1]) : got[k];    // lower half: up of token 2k
+            const float gate = up_half ? got[k] : a[2 * k];       // upper half: gate of token 2k + 1
+            const float upv = up_half ? a[2 * k + 1] : got[k];    // lower half: up of token 2k
             const float h = __fdividef(gate, 1.0f + __expf(-gate)) * upv;
             if (2 * k + (up_half ? 1 : 0) < ncols) dst[(size_t)(2 * k) * p.f_pad] = __float2bfloat16(h);
         }
-    } else {  // EPI_LMHEAD: the norm scale is positive, so the argmax needs nothing but the accumulators
+    } else {  // EPI_LMHEAD
         const int f = m0 + l;
         const bool valid = f < p.vocab;
         if (p.logits && valid) {
 #pragma unroll
             for (int j = 0; j < EPI_COLS; ++j)
-                if (j < ncols) p.logits[(size_t)(t0 + j) * p.vocab + f] = __uint_as_float(r[j]);
+                if (j < ncols) p.logits[(size_t)(t0 + j) * p.vocab + f] = a[j];
         }
         uint32_t mx[EPI_COLS];
 #pragma unroll
         for (int j = 0; j < EPI_COLS; ++j)
-            mx[j] = __reduce_max_sync(0xFFFFFFFFu, valid ? orderable_f32(__uint_as_float(r[j])) : 0u);
+            mx[j] = __reduce_max_sync(0xFFFFFFFFu, valid ? orderable_f32(a[j]) : 0u);
         unsigned long long mine = 0ull;   // lane j keeps the warp's best of token j
 #pragma unroll
         for (int j = 0; j < EPI_COLS; ++j) {
-            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, valid && orderable_f32(__uint_as_float(r[j])) == mx[j]);
+            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, valid && orderable_f32(a[j]) == mx[j]);
             if (lane == j && hit) mine = pack_argmax_key(mx[j], m0 + quarter * 32 + (__ffs(hit) - 1));
         }
         if (lane < ncols && mine) atomicMax(p.best + t0 + lane, mine);
@@ -174,45 +260,32 @@ __device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&
     }
 }
 
-// Residual update after a split-K projection, in a fixed order: x += part[0] + part[1] + ...;
-// then the next GEMM's operand, the RMSNorm of the row: bf16(x * rstd * gain).  One CTA per token.
-__global__ void __launch_bounds__(256)
-resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, size_t part_stride, int splits,
-                  const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ xn, int d, float inv_d, float eps) {
-    __shared__ float red[8];
-    __shared__ float rstd_s;
-    const int t = blockIdx.x;
-    float ss = 0.f;
-    pdl_launch_dependents();
-    pdl_wait();
-    for (int f = threadIdx.x * 4; f < d; f += blockDim.x * 4) {
-        float4 v = *reinterpret_cast<const float4*>(x + (size_t)t * d + f);
-        for (int s = 0; s < splits; ++s) {
-            const float4 q = *reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * d + f);
-            v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+__device__ __forceinline__ void epi_dispatch(int mode, const EpiParams& p, const uint32_t (&r)[EPI_COLS], const float* rs, int m0,
+                                             int t0, int ncols, int quarter, int lane) {
+    switch (mode) {
+        case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, rs, m0, t0, ncols, quarter, lane); break;
+        case EPI_QKV: epi_direct<EPI_QKV>(p, r, rs, m0, t0, ncols, quarter, lane); break;
+        case EPI_RESID: epi_direct<EPI_RESID>(p, r, rs, m0, t0, ncols, quarter, lane); break;
+        case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, rs, m0, t0, ncols, quarter, lane); break;
+        default: epi_direct<EPI_LMHEAD>(p, r, rs, m0, t0, ncols, quarter, lane); break;
+    }
+}
+
+// RMSNorm scales of the tokens n0 .. n0 + n_valid - 1 from the partial sums of x^2 their source rows
+// carry: one warp per token (warp `e` of GEMM_EPI_WARPS takes every sixteenth), a fixed reduction
+// order, so every CTA that needs a token's scale gets the same bits.
+__device__ __forceinline__ void epi_rms_scales(const EpiParams& p, float* dst, int n0, int n_valid, int e, int lane) {
+    const int nq = p.n_ssq >> 2;
+    for (int t = e; t < n_valid; t += GEMM_EPI_WARPS) {
+        const float4* row = reinterpret_cast<const float4*>(p.ssq_in + (size_t)(n0 + t) * p.n_ssq);
+        float sum = 0.f;
+        for (int i = lane; i < nq; i += 32) {
+            const float4 v = __ldcg(row + i);
+            sum += (v.x + v.y) + (v.z + v.w);
         }
-        *reinterpret_cast<float4*>(x + (size_t)t * d + f) = v;
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float tot = 0.f;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
-        rstd_s = rsqrtf(tot * inv_d + eps);
-    }
-    __syncthreads();
-    const float rs = rstd_s;
-    for (int f = threadIdx.x * 4; f < d; f += blockDim.x * 4) {   // each thread re-reads what it wrote
-        const float4 v = *reinterpret_cast<const float4*>(x + (size_t)t * d + f);
-        const uint2 gb = *reinterpret_cast<const uint2*>(gain + f);
-        const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gb.x);
-        const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gb.y);
-        *reinterpret_cast<uint2*>(xn + (size_t)t * d + f) =
-            make_uint2(pack_bf16(v.x * rs * __low2float(g01), v.y * rs * __high2float(g01)),
-                       pack_bf16(v.z * rs * __low2float(g23), v.w * rs * __high2float(g23)));
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+        if (lane == 0) dst[t] = rsqrtf(sum * p.inv_d + p.eps);
     }
 }
 
@@ -280,15 +353,17 @@ constexpr int GEMM_A_BYTES = 2 * GEMM_TILE_BYTES;  // stage room for a pair
 constexpr int GEMM_BOX_ROWS = 32;                  // token rows per B box
 constexpr int GEMM_BOX_BYTES = GEMM_BOX_ROWS * GEMM_BK * 2;
 constexpr int GEMM_MAX_STAGES = 8;
-constexpr int GEMM_EPI_WARPS = 16;               // four groups of four (one warp per TMEM lane quarter)
 constexpr int GEMM_THREADS = (2 + GEMM_EPI_WARPS) * 32;
 constexpr int GEMM_SMEM_MAX = 232448;
-constexpr int GEMM_PREFETCH_KB = 12;               // L2 prefetch distance in k-blocks
+constexpr int GEMM_BAR_BYTES = 256;                // mbarriers and the TMEM address word
 
 __host__ __device__ inline int gemm_stage_bytes(int TN) { return GEMM_A_BYTES + ((TN + 31) / 32) * GEMM_BOX_BYTES; }
-__host__ inline int gemm_fixed_smem() { return 1024 /*align*/ + 512 /*barriers*/; }
+// RMSNorm scales of an item's tokens, two buffers (items alternate); rounded up so that an epilogue
+// that takes 32 columns at a time stays inside the buffer
+__host__ __device__ inline int gemm_rs_stride(int TN) { return (TN + 31) & ~31; }
+__host__ inline int gemm_fixed_smem(int TN) { return 1024 /*align*/ + GEMM_BAR_BYTES + 2 * gemm_rs_stride(TN) * 4; }
 __host__ inline int gemm_stages(int TN) {
-    int s = (GEMM_SMEM_MAX - gemm_fixed_smem()) / gemm_stage_bytes(TN);
+    int s = (GEMM_SMEM_MAX - gemm_fixed_smem(TN)) / gemm_stage_bytes(TN);
     return s > GEMM_MAX_STAGES ? GEMM_MAX_STAGES : s;
 }
 
@@ -298,16 +373,19 @@ struct GemmParams {
     int n_pairs;                // 256-feature pairs
     int n_tt, TN;               // token tiles of TN columns (multiple of 16, <= 256)
     int n_stages;
-    int splits, kb_per_split;   // splits > 1: every CTA owns one (pair tile, k range)
+    int splits, kb_per_split;   // splits > 1 (GEMM_RSPLIT): every CTA owns one (pair tile, k range)
     int pair_mode;              // 1: pair tiles in full waves + remainder as singles; 0: all singles;
                                 // 2: one wave of n_cta items, pair tiles first, the rest as singles
     int ksplit;                 // pair mode, > 1: the remainder's pair tiles are cut along K into this many parts
     int kper;                   // ksplit: k-blocks of a helper part, (ksplit - 1) * kper < num_kb
-    float* fix_part;            // ksplit: fp32 partial accumulators of the helper parts, [slot][2][TN/16][4][32][16]
+    float* fix_part;            // ksplit: fp32 partial accumulators of the helper parts, [slot][2][TN/16][4][32][16];
+                                // splits > 1: the exchange slots of the CTAs, same layout, slot = CTA index
     int* fix_flag;              // ksplit: per remainder tile, epilogue warps of helpers that have stored; then
-                                // [n_sm + tile]: owner warps that are done reading (the last one clears both)
+                                // [n_sm + tile]: owner warps that are done reading (the last one clears both);
+                                // splits > 1: the same two counters per pair tile
     int n_sm;
     int* status;
+    long long spin_limit;       // SM cycles after which a wait gives up and sets *status
 };
 
 struct GemmWork {
@@ -416,14 +494,12 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                  ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
-__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(src)), "r"(bytes)
-                 : "memory");
-}
 
-template <bool KSPLIT>
+template <int VARIANT>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) {
+    constexpr bool KSPLIT = VARIANT == GEMM_KSPLIT;
+    constexpr bool RSPLIT = VARIANT == GEMM_RSPLIT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int stage_bytes = gemm_stage_bytes(g.TN);
@@ -431,10 +507,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
     uint64_t* empty_bar = full_bar + GEMM_MAX_STAGES;
     uint64_t* accf_bar = empty_bar + GEMM_MAX_STAGES;   // accumulators complete (MMA -> epilogue)
     uint64_t* acce_bar = accf_bar + 1;                  // accumulators drained (epilogue -> MMA)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acce_bar + 1);
+    uint64_t* rs_bar = acce_bar + 1;                    // RMSNorm scales of the item's tokens are in rs_s
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rs_bar + 1);
+    float* rs_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(full_bar) + GEMM_BAR_BYTES);   // [2][TN]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_cta = gridDim.x, cta = blockIdx.x;
+    const long long limit = g.spin_limit;
     pdl_launch_dependents();
     uint32_t acc_stride = 32;
     while ((int)acc_stride < g.TN) acc_stride <<= 1;
@@ -448,6 +527,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
         }
         mbar_init(accf_bar, 1);
         mbar_init(acce_bar, GEMM_EPI_WARPS);
+        mbar_init(rs_bar, GEMM_EPI_WARPS);
         mbar_fence_init();
     }
     if (warp == 1) {
@@ -485,7 +565,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                 for (int j = 0; j < nk; ++j, ++it) {
                     const int kb = w.kb0 + (j + rot) % nk;
                     const int s = it % g.n_stages;
-                    if (it >= (uint32_t)g.n_stages && !mbar_wait(&empty_bar[s], ((it / g.n_stages) - 1) & 1, g.status)) {
+                    if (it >= (uint32_t)g.n_stages && !mbar_wait(&empty_bar[s], ((it / g.n_stages) - 1) & 1, g.status, limit)) {
                         ok = false;
                         break;
                     }
@@ -511,14 +591,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                 const uint32_t nn = (uint32_t)((min(g.TN, p.T - w.tt * g.TN) + 15) & ~15);
                 const uint32_t idesc = umma_idesc_bf16(128, nn);
                 if (i > 0) {   // the epilogue must have drained the previous item's accumulators
-                    ok = mbar_wait(acce_bar, (i - 1) & 1, g.status);
+                    ok = mbar_wait(acce_bar, (i - 1) & 1, g.status, limit);
                     if (!ok) break;
                     tc_fence_after();
                 }
                 const int nk = w.kb1 - w.kb0;
                 for (int j = 0; j < nk; ++j, ++it) {
                     const int s = it % g.n_stages;
-                    ok = mbar_wait(&full_bar[s], (it / g.n_stages) & 1, g.status);
+                    ok = mbar_wait(&full_bar[s], (it / g.n_stages) & 1, g.status, limit);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
@@ -543,18 +623,106 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
         const int grp = e >> 2;               // the groups take the 16-token chunks round robin
         constexpr int NGRP = GEMM_EPI_WARPS / 4;
         const int quarter = warp & 3;         // TMEM lane quarter this warp may read
+        const bool scaled = p.ssq_in != nullptr;
         bool ok = true;
         GemmWork w;
-        pdl_wait();   // the epilogues write buffers that earlier kernels may still read
+        pdl_wait();   // the epilogues read and write buffers of earlier kernels
         for (int i = 0; ok && gemm_work<KSPLIT>(g, cta, n_cta, i, w); ++i) {
             const int n0 = w.tt * g.TN;
             const int n_valid = min(g.TN, p.T - n0);
             const int nchunks = (n_valid + EPI_COLS - 1) / EPI_COLS;
-            ok = mbar_wait(accf_bar, i & 1, g.status);
+            float* const rsi = rs_s + (i & 1) * gemm_rs_stride(g.TN);
+            if (scaled) {   // while the main loop runs: the scales of this item's tokens
+                epi_rms_scales(p, rsi, n0, n_valid, e, lane);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(rs_bar);
+            }
+            ok = mbar_wait(accf_bar, i & 1, g.status, limit);
+            if (ok && scaled) ok = mbar_wait(rs_bar, i & 1, g.status, limit);
             if (!ok) break;
             tc_fence_after();
             const int total_chunks = (w.mt_hi - w.mt_lo) * nchunks;
-            if ((!KSPLIT || w.role == 0) && (p.mode == EPI_PART || p.mode == EPI_PLAIN)) {
+            if (RSPLIT) {
+                // ---- reduce-scatter over the S CTAs that share this tile.  CTA `split` keeps the
+                // chunks [c_lo, c_hi) of both 128-feature tiles.  Exchange slot of a CTA:
+                // [tile of the pair][chunk][lane quarter][4][lane][4 floats], so that one 16-byte access
+                // per lane covers 512 contiguous bytes per warp.
+                const int S = g.splits, sp = w.split, tile = cta / S;
+                const int cpt = g.TN / EPI_COLS;
+                const size_t slot_elems = (size_t)2 * cpt * 128 * EPI_COLS;
+                const int c_lo = sp * nchunks / S, c_hi = (sp + 1) * nchunks / S;
+                float* const mine = g.fix_part + (size_t)cta * slot_elems;
+                int nth = 0;
+                for (int mt = 0; mt < 2; ++mt)
+                    for (int c = 0; c < nchunks; ++c) {
+                        if (c >= c_lo && c < c_hi) continue;
+                        if ((nth++ & (NGRP - 1)) != grp) continue;
+                        uint32_t r[EPI_COLS];
+                        tmem_ld16(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * EPI_COLS), r);
+                        tmem_ld_wait();
+                        uint4* dst = reinterpret_cast<uint4*>(mine + (((size_t)mt * cpt + c) * 4 + quarter) * 32 * EPI_COLS) + lane;
+#pragma unroll
+                        for (int v = 0; v < EPI_COLS / 4; ++v) dst[v * 32] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    }
+                __threadfence();        // this warp's share of the accumulators is in memory
+                __syncwarp();
+                if (lane == 0) atomicAdd(g.fix_flag + tile, 1);
+                // all warps of all S CTAs must have stored before anyone reads; the CTAs of a tile are
+                // neighbours in the grid and the grid is at most one CTA per SM, so they run together
+                if (lane == 0) {
+                    const int want = S * GEMM_EPI_WARPS;
+                    const long long t_end = clock64() + limit;
+                    while (ld_acquire_gpu(g.fix_flag + tile) < want) {
+                        if (clock64() > t_end) {
+                            atomicExch(g.status, 1);
+                            break;
+                        }
+                    }
+                }
+                __syncwarp();
+                nth = 0;
+                for (int mt = 0; mt < 2; ++mt)
+                    for (int c = c_lo; c < c_hi; ++c) {
+                        if ((nth++ & (NGRP - 1)) != grp) continue;
+                        const int m0 = w.pair * 256 + mt * 128;
+                        uint32_t own[EPI_COLS], r[EPI_COLS];
+                        tmem_ld16(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * EPI_COLS), own);
+                        tmem_ld_wait();
+                        const size_t at = (((size_t)mt * cpt + c) * 4 + quarter) * 32 * EPI_COLS;
+                        for (int q = 0; q < S; ++q) {   // fixed order: the parts in split order
+                            if (q == sp) {
+#pragma unroll
+                                for (int v = 0; v < EPI_COLS; ++v)
+                                    r[v] = q == 0 ? own[v] : __float_as_uint(__uint_as_float(r[v]) + __uint_as_float(own[v]));
+                            } else {
+                                const float4* src = reinterpret_cast<const float4*>(g.fix_part + (size_t)(tile * S + q) * slot_elems + at) + lane;
+#pragma unroll
+                                for (int v = 0; v < EPI_COLS / 4; ++v) {
+                                    const float4 q4 = __ldcg(src + v * 32);
+                                    if (q == 0) {
+                                        r[4 * v] = __float_as_uint(q4.x); r[4 * v + 1] = __float_as_uint(q4.y);
+                                        r[4 * v + 2] = __float_as_uint(q4.z); r[4 * v + 3] = __float_as_uint(q4.w);
+                                    } else {
+                                        r[4 * v] = __float_as_uint(__uint_as_float(r[4 * v]) + q4.x);
+                                        r[4 * v + 1] = __float_as_uint(__uint_as_float(r[4 * v + 1]) + q4.y);
+                                        r[4 * v + 2] = __float_as_uint(__uint_as_float(r[4 * v + 2]) + q4.z);
+                                        r[4 * v + 3] = __float_as_uint(__uint_as_float(r[4 * v + 3]) + q4.w);
+                                    }
+                                }
+                            }
+                        }
+                        const int tc0 = n0 + c * EPI_COLS, ncols = min(EPI_COLS, n_valid - c * EPI_COLS);
+                        if (m0 < p.N) epi_dispatch(p.mode, p, r, scaled ? rsi + c * EPI_COLS : nullptr, m0, tc0, ncols, quarter, lane);
+                    }
+                // the last warp of the tile's CTAs to finish reading clears the counters for the next launch
+                __syncwarp();
+                if (lane == 0 && atomicAdd(g.fix_flag + g.n_sm + tile, 1) == S * GEMM_EPI_WARPS - 1) {
+                    g.fix_flag[tile] = 0;
+                    g.fix_flag[g.n_sm + tile] = 0;
+                }
+                continue;
+            }
+            if ((!KSPLIT || w.role == 0) && p.mode == EPI_PLAIN) {
                 // fp32 stores only: 32 columns a TMEM load (the accumulator's columns beyond the
                 // tile's tokens are allocated, their contents are not stored)
                 const int nch2 = (nchunks + 1) >> 1;
@@ -572,11 +740,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                     const int f = m0 + quarter * 32 + lane;
                     const int tc0 = n0 + c2 * 32, ncols = min(32, n_valid - c2 * 32);
                     if (f < p.N) {
-                        const size_t ld = p.mode == EPI_PLAIN ? (size_t)p.ldy : (size_t)p.d;
-                        float* base = (p.mode == EPI_PLAIN ? p.y + f : p.part + (size_t)w.split * p.part_stride + f) + (size_t)tc0 * ld;
+                        float* base = p.y + f + (size_t)tc0 * p.ldy;
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (j < ncols) base[(size_t)j * ld] = __uint_as_float(r[j]);
+                            if (j < ncols) base[(size_t)j * p.ldy] = __uint_as_float(r[j]);
                     }
                 }
                 if (grp >= total2) {
@@ -603,6 +770,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                         if (lane == 0) mbar_arrive(acce_bar);
                     }
                     const int tc0 = n0 + c2 * 32, ncols = min(32, n_valid - c2 * 32);
+                    if (scaled) {   // columns beyond the tile's tokens hold stale scales: finite, never stored
+                        const float* rs = rsi + c2 * 32;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * rs[j]);
+                    }
                     float got[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k)   // each half-warp sends what the other one needs
@@ -636,15 +808,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                         if (lane == 0) mbar_arrive(acce_bar);
                     }
                     const int tc0 = n0 + c * EPI_COLS, ncols = min(EPI_COLS, n_valid - c * EPI_COLS);
-                    if (m0 < p.N) {
-                        switch (p.mode) {
-                            case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
-                            case EPI_QKV: epi_direct<EPI_QKV>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
-                            case EPI_PART: epi_direct<EPI_PART>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
-                            case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
-                            default: epi_direct<EPI_LMHEAD>(p, r, m0, tc0, ncols, w.split, quarter, lane); break;
-                        }
-                    }
+                    if (m0 < p.N) epi_dispatch(p.mode, p, r, scaled ? rsi + c * EPI_COLS : nullptr, m0, tc0, ncols, quarter, lane);
                 }
                 if (grp >= total_chunks) {   // a group without any chunk still releases the accumulators
                     tc_fence_before();
@@ -684,7 +848,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
             // owner: the helpers ran first; the wait is bounded all the same
             if (lane == 0) {
                 const int want = H * GEMM_EPI_WARPS;
-                const long long t_end = clock64() + SYN_SPIN_LIMIT_CYCLES;
+                const long long t_end = clock64() + limit;
                 while (ld_acquire_gpu(g.fix_flag + w.rtile) < want) {
                     if (clock64() > t_end) {
                         atomicExch(g.status, 1);
@@ -716,14 +880,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                     }
                 }
                 const int tc0 = n0 + c * EPI_COLS, ncols = min(EPI_COLS, n_valid - c * EPI_COLS);
-                if (m0 < p.N) {
-                    switch (p.mode) {
-                        case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, m0, tc0, ncols, 0, quarter, lane); break;
-                        case EPI_QKV: epi_direct<EPI_QKV>(p, r, m0, tc0, ncols, 0, quarter, lane); break;
-                        case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, m0, tc0, ncols, 0, quarter, lane); break;
-                        default: epi_direct<EPI_LMHEAD>(p, r, m0, tc0, ncols, 0, quarter, lane); break;
-                    }
-                }
+                if (m0 < p.N) epi_dispatch(p.mode, p, r, scaled ? rsi + c * EPI_COLS : nullptr, m0, tc0, ncols, quarter, lane);
             }
             if (grp >= total_chunks) {
                 tc_fence_before();

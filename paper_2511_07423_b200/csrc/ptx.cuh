@@ -1,7 +1,8 @@
 // Thin inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor), tcgen05
 // (TMEM allocation, UMMA issue, commit, TMEM loads), ldmatrix / mma.sync.
-// Every wait is bounded: after SYN_SPIN_LIMIT_CYCLES it records an error in a status word
-// and returns false so that the caller can unwind (free TMEM, reach the final barrier).
+// Every wait is bounded: after a limit in SM cycles (SYN_SPIN_LIMIT_CYCLES unless the launch says
+// otherwise) it records an error in a status word and returns false so that the caller can unwind
+// (free TMEM, reach the final barrier).
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -62,7 +63,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // Bounded wait on a phase parity.  On timeout: sets *status (if non-null) and returns false.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status,
+                                          long long limit = SYN_SPIN_LIMIT_CYCLES) {
     uint32_t addr = smem_u32(bar);
     long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -78,7 +80,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
         if ((it & 0x3FF) == 0x3FF) {
             long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > SYN_SPIN_LIMIT_CYCLES) {
+            else if (now - t0 > limit) {
                 if (status) atomicExch(status, 1);
                 return false;
             }
@@ -100,14 +102,6 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* m, uin
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* m, uint64_t* bar, int c0, int c1, int c2,
-                                            int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2),
-        "r"(c3)
         : "memory");
 }
 

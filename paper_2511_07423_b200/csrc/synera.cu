@@ -6,10 +6,11 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <chrono>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
-#include <queue>
 #include <vector>
 
 #include "attention.cuh"
@@ -20,7 +21,9 @@ using namespace syn;
 typedef __nv_bfloat16 bf16;
 // Slot of one helper part's stored accumulators: two tiles of 128 features x up to 256 tokens, fp32.
 constexpr size_t GEMM_FIX_SLOT_BYTES = (size_t)2 * 128 * 256 * 4;
-constexpr int GEMM_MAX_SPLITS = 8;   // split-K partial buffers of the o / down projections
+constexpr int GEMM_MAX_SPLITS = 8;   // most CTAs that share one pair tile's K range
+// Limit of the kernels' bounded waits in SM cycles (syn_debug_set_spin_limit; tests shorten it).
+static long long g_spin_limit = SYN_SPIN_LIMIT_CYCLES;
 
 // Name of the last CUDA error a call of this library met on this thread (for syn_last_cuda_error).
 static thread_local const char* g_last_cuda_error = "";
@@ -60,38 +63,28 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // ------------------------------------------------------------------------------------------ small kernels
 
 // Token embedding (paper Sec. 4.5: the flattened batch enters the transformer), the first layer's
-// GEMM operand bf16(rmsnorm(x) * gain), RoPE table, argmax reset.
+// GEMM operand bf16(x * gain) with the sums of x^2 per 32 features its RMSNorm scale is made of,
+// RoPE table, argmax reset.
 __global__ void __launch_bounds__(256)
 prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens, const int* __restrict__ pos,
             const bf16* __restrict__ gain, const double* __restrict__ inv_freq, float* __restrict__ x,
-            bf16* __restrict__ xn, float2* __restrict__ rope, unsigned long long* __restrict__ best, int d, int half,
-            float inv_d, float eps) {
-    __shared__ float red[8];
-    __shared__ float rstd_s;
-    const int t = blockIdx.x;
+            bf16* __restrict__ xg, float* __restrict__ ssq, float2* __restrict__ rope, unsigned long long* __restrict__ best,
+            int d, int half) {
+    const int t = blockIdx.x, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     pdl_wait();
     const bf16* e = embed + (size_t)tokens[t] * d;
-    float ss = 0.f;
-    for (int f = threadIdx.x; f < d; f += blockDim.x) {
+    for (int f0 = (threadIdx.x >> 5) * 32; f0 < d; f0 += blockDim.x) {   // one warp per group of 32 features
+        const int f = f0 + lane;
         const float v = __bfloat162float(e[f]);
         x[(size_t)t * d + f] = v;
-        ss += v * v;
-    }
+        xg[(size_t)t * d + f] = __float2bfloat16(v * __bfloat162float(gain[f]));
+        float ss = v * v;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float tot = 0.f;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += red[w];
-        rstd_s = rsqrtf(tot * inv_d + eps);
-        best[t] = 0ull;
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+        if (lane == 0) ssq[(size_t)t * (d >> 5) + (f0 >> 5)] = ss;
     }
-    __syncthreads();
-    const float rs = rstd_s;
-    for (int f = threadIdx.x; f < d; f += blockDim.x)
-        xn[(size_t)t * d + f] = __float2bfloat16(__bfloat162float(e[f]) * rs * __bfloat162float(gain[f]));
+    if (threadIdx.x == 0) best[t] = 0ull;
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
         double sn, cs;
         sincos((double)pos[t] * inv_freq[i], &sn, &cs);
@@ -173,8 +166,9 @@ struct syn_model {
     int* status_dev = nullptr;
     // workspace (grow-only)
     int t_cap = 0;
-    float *x = nullptr, *part = nullptr;   // residual stream, split-K partials
-    bf16 *xn = nullptr, *q = nullptr, *attn = nullptr, *act = nullptr;
+    float *x = nullptr, *ssq = nullptr;   // residual stream; sums of x^2 per token and 32 features
+    bf16 *xn = nullptr,   // bf16(x * gain of the next RMSNorm): the operand of the qkv, gate/up and lm_head projections
+          *q = nullptr, *attn = nullptr, *act = nullptr;
     float2* rope = nullptr;
     unsigned long long* best = nullptr;
     int *acc_dev = nullptr, *corr_dev = nullptr;
@@ -198,6 +192,13 @@ struct syn_model {
     } sw;
     int* pinned_out = nullptr;
     int pinned_out_cap = 0;
+    // what syn_last_step_stats reports: the counters of the last step launched on this model and,
+    // with profiling on, its device time (events around the whole step) and the wall time of the
+    // blocking call
+    syn_step_stats last_stats;
+    bool have_last = false, step_timed = false;
+    cudaEvent_t step_a = nullptr, step_b = nullptr;
+    double last_wall_ms = 0.0;
     // per-class event timing
     bool profile = false;
     struct Ev { cudaEvent_t a, b; int cls; };
@@ -237,15 +238,18 @@ struct syn_plan {
     size_t cap = 0, used = 0;
     // offsets into the buffer
     size_t o_tokens, o_pos, o_slot, o_offsets, o_uncached, o_tables, o_items, o_cta, o_groups;
-    bool uploaded_sync = false;
+    // the cache the page ids and slots were validated against
+    const syn_kv* kv = nullptr;
+    const void* kv_pool = nullptr;
+    uint32_t kv_pages = 0;
     template <class Tp> Tp* d(size_t off) const { return reinterpret_cast<Tp*>(dev + off); }
     template <class Tp> Tp* h(size_t off) const { return reinterpret_cast<Tp*>(host + off); }
 };
 
 static void free_workspace(syn_model* m) {
-    cudaFree(m->x); cudaFree(m->part); cudaFree(m->xn); cudaFree(m->q); cudaFree(m->attn); cudaFree(m->act);
+    cudaFree(m->x); cudaFree(m->ssq); cudaFree(m->xn); cudaFree(m->q); cudaFree(m->attn); cudaFree(m->act);
     cudaFree(m->rope); cudaFree(m->best);
-    m->x = m->part = nullptr; m->xn = m->q = m->attn = m->act = nullptr; m->rope = nullptr; m->best = nullptr;
+    m->x = m->ssq = nullptr; m->xn = m->q = m->attn = m->act = nullptr; m->rope = nullptr; m->best = nullptr;
     m->t_cap = 0;
 }
 
@@ -256,7 +260,7 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
         free_workspace(m);
         const int cap = (T + 255) / 256 * 256;
         CU_OK(cudaMalloc(&m->x, (size_t)cap * c.d_model * 4));
-        CU_OK(cudaMalloc(&m->part, (size_t)GEMM_MAX_SPLITS * cap * c.d_model * 4));
+        CU_OK(cudaMalloc(&m->ssq, (size_t)cap * (c.d_model / 32) * 4));
         CU_OK(cudaMalloc(&m->xn, (size_t)cap * c.d_model * 2));
         CU_OK(cudaMalloc(&m->q, (size_t)cap * q_dim * 2));
         CU_OK(cudaMalloc(&m->attn, (size_t)cap * q_dim * 2));
@@ -326,10 +330,12 @@ extern "C" void syn_model_free(syn_model* m) {
     if (m->scratch_plan) syn_plan_free(m->scratch_plan);
     for (auto* v : {&m->ev_used, &m->ev_free})
         for (auto& e : *v) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+    if (m->step_a) cudaEventDestroy(m->step_a);
+    if (m->step_b) cudaEventDestroy(m->step_b);
     delete m;
 }
 
-extern "C" int syn_model_load(const syn_model_desc* desc, const syn_weights* w, syn_model** out) {
+static int syn_model_load_impl(const syn_model_desc* desc, const syn_weights* w, syn_model** out) {
     if (!desc || !w || !out) return SYN_E_INVALID_ARG;
     const syn_model_desc c = *desc;
     if (c.flags != 0 || c.n_layers == 0 || c.vocab == 0 || c.d_ffn == 0) return SYN_E_INVALID_ARG;
@@ -480,8 +486,9 @@ extern "C" int syn_model_load(const syn_model_desc* desc, const syn_weights* w, 
     CU_M(cudaMemcpy(m->inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice));
     CU_M(cudaMalloc(&m->status_dev, 4));
     CU_M(cudaMemset(m->status_dev, 0, 4));
-    CU_M(cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
-    CU_M(cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_M(cudaFuncSetAttribute(gemm_kernel<GEMM_WAVES>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_M(cudaFuncSetAttribute(gemm_kernel<GEMM_KSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_M(cudaFuncSetAttribute(gemm_kernel<GEMM_RSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_M(cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::TOTAL));
     CU_M(cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::TOTAL));
     CU_M(cudaDeviceSynchronize());
@@ -562,11 +569,11 @@ static int kv_copy(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_
     return e == cudaSuccess ? SYN_OK : SYN_E_CUDA;
 }
 
-extern "C" int syn_kv_import(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_t pos0, int32_t n_pos,
+static int syn_kv_import_impl(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_t pos0, int32_t n_pos,
                              const void* k, const void* v, void* stream) {
     return kv_copy(kv, layer, page_table, pos0, n_pos, const_cast<void*>(k), const_cast<void*>(v), stream, 1);
 }
-extern "C" int syn_kv_export(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_t pos0, int32_t n_pos, void* k,
+static int syn_kv_export_impl(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_t pos0, int32_t n_pos, void* k,
                              void* v, void* stream) {
     return kv_copy(kv, layer, page_table, pos0, n_pos, k, v, stream, 0);
 }
@@ -830,7 +837,7 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
     s.dense_flops = 2.0 * T * params;
     s.attn_flops = 4.0 * qd * c.n_layers * (double)keys_seen;
     s.attn_items = n_items; s.attn_split_items = n_parts;
-    s.kernel_launches = 2 + c.n_layers * 7 + 1;
+    s.kernel_launches = 1 + c.n_layers * 5 + 2;
     return SYN_OK;
 }
 
@@ -879,12 +886,13 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     p->n_groups = (int)hp.groups.size(); p->n_parts = hp.n_parts;
     p->stats = hp.stats;
     p->stats.h2d_bytes = (int64_t)off;
+    p->kv = kv; p->kv_pool = kv->pool; p->kv_pages = kv->n_pages;
     return SYN_OK;
 }
 
 // The planner without a device: same validation and the same work list as syn_plan_create, returned
 // in caller-provided HOST arrays.
-extern "C" int syn_plan_host(const syn_model_desc* desc, uint32_t n_pages, uint32_t page_size, int32_t n_sm, int32_t n_req,
+static int syn_plan_host_impl(const syn_model_desc* desc, uint32_t n_pages, uint32_t page_size, int32_t n_sm, int32_t n_req,
                              const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables,
                              int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, int32_t* pos,
                              int32_t* slot, int32_t* items, int32_t items_cap, int32_t* n_items, int32_t* cta_begin,
@@ -914,7 +922,7 @@ extern "C" int syn_plan_host(const syn_model_desc* desc, uint32_t n_pages, uint3
     return SYN_OK;
 }
 
-extern "C" int syn_plan_create(syn_model* m, syn_kv* kv, int32_t n_req, const int32_t* chunk_tokens,
+static int syn_plan_create_impl(syn_model* m, syn_kv* kv, int32_t n_req, const int32_t* chunk_tokens,
                                const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages,
                                const int32_t* ctx_lens, const int32_t* n_uncached, syn_plan** out) {
     if (!out) return SYN_E_INVALID_ARG;
@@ -934,30 +942,52 @@ extern "C" int syn_plan_create(syn_model* m, syn_kv* kv, int32_t n_req, const in
     return SYN_OK;
 }
 
-extern "C" int syn_last_step_stats(const syn_plan* p, syn_step_stats* out) {
+extern "C" int syn_plan_stats(const syn_plan* p, syn_step_stats* out) {
     if (!p || !out) return SYN_E_INVALID_ARG;
     *out = p->stats;
     return SYN_OK;
 }
 
+extern "C" int syn_last_step_stats(syn_model* m, syn_step_stats* out) {
+    if (!m || !out || !m->have_last) return SYN_E_INVALID_ARG;
+    *out = m->last_stats;
+    if (m->step_timed) {
+        float ms = 0.f;
+        CU_OK(cudaEventSynchronize(m->step_b));
+        CU_OK(cudaEventElapsedTime(&ms, m->step_a, m->step_b));
+        out->t_gpu_ms = ms;
+        out->t_wall_ms = m->last_wall_ms;
+    }
+    return SYN_OK;
+}
+
+// A plan's page ids and KV slots were checked against one cache: only that cache may run it.
+static bool plan_matches(const syn_plan* p, const syn_kv* kv) {
+    return p->kv == kv && p->kv_pool == kv->pool && p->kv_pages == kv->n_pages;
+}
+
 // ------------------------------------------------------------------------------------------ launches
 
-// D[rows][T] = Wpacked[rows][K] * X[T][K]^T with the epilogue `ep`.  Chooses the schedule: split-K
-// for partial-sum epilogues with few output tiles, pair tiles when they fill the SMs, else singles.
-// Returns the number of splits through *splits_out (EPI_PART only).
-// The launch shape of one projection: token tiling, work decomposition, CTA count.  Host arithmetic only
-// (also exported as syn_gemm_plan_host so that the schedule can be checked without a device).
+// The launch shape of one projection D[rows][T] = Wpacked[rows][K] * X[T][K]^T: token tiling, work
+// decomposition, CTA count.  Host arithmetic only (also exported as syn_gemm_plan_host so that the
+// schedule can be checked without a device).  `mode` = the epilogue the schedule is made for.
 static int gemm_plan(int T, int packed_rows, int K, int n_sm, int mode, bool may_ksplit, GemmParams& g, int& n_cta) {
     g.num_kb = (K + 63) / 64;
     g.n_pairs = (packed_rows + 255) / 256;
     g.n_tt = (T + 255) / 256;
-    if (mode != EPI_PART) {
+    // A projection with fewer pair tiles than SMs can share a tile's K range between CTAs (reduce-
+    // scatter, GEMM_RSPLIT): always for the residual projections, whose K is long and whose output is
+    // narrow; for qkv from a few hundred tokens on, where single 128-feature tiles would ask L2 for
+    // the token tile twice as often; parts of at least 4 (residual) or 8 (qkv) k-blocks.
+    const int tiles_nat = g.n_pairs * g.n_tt;
+    const bool qkv_split = mode == EPI_QKV && T >= 256 && n_sm / tiles_nat >= 2 && g.num_kb >= 16;
+    if (mode != EPI_RESID) {
         // Few feature tiles and few tokens: narrower token tiles (32 tokens at least) put more SMs to
         // work; the weights are then read by several CTAs, which costs only L2 bandwidth.
         const int want = n_sm / std::max(1, 2 * g.n_pairs), most = (T + 31) / 32;
-        g.n_tt = std::max(g.n_tt, std::min(want, most));
+        if (!qkv_split) g.n_tt = std::max(g.n_tt, std::min(want, most));
     } else if (g.n_pairs * g.n_tt < n_sm && n_sm / (g.n_pairs * g.n_tt) < 2) {
-        // Split-K projection whose pair tiles cover more than half of the SMs but not all: K cannot be
+        // Residual projection whose pair tiles cover more than half of the SMs but not all: K cannot be
         // split, so narrower token tiles (64 tokens at least) fill the machine instead; every CTA still
         // walks the whole K, on a smaller item.
         const int fit = n_sm / g.n_pairs, most = (T + 63) / 64;
@@ -973,8 +1003,9 @@ static int gemm_plan(int T, int packed_rows, int K, int n_sm, int mode, bool may
     if (g.n_stages < 2 || g.TN < 16 || g.TN > 256 || (g.n_tt - 1) * g.TN >= T) return SYN_E_INVALID_ARG;
     const int tiles = g.n_pairs * g.n_tt;
     g.pair_mode = tiles >= n_sm;
-    if (mode == EPI_PART && tiles < n_sm) {
-        int sp = std::min(GEMM_MAX_SPLITS, std::min(n_sm / tiles, std::max(1, g.num_kb / 4)));
+    if ((mode == EPI_RESID || qkv_split) && tiles < n_sm) {
+        const int min_kb = mode == EPI_RESID ? 4 : 8;
+        int sp = std::min(GEMM_MAX_SPLITS, std::min(n_sm / tiles, std::max(1, g.num_kb / min_kb)));
         g.kb_per_split = (g.num_kb + sp - 1) / sp;
         g.splits = (g.num_kb + g.kb_per_split - 1) / g.kb_per_split;
         g.pair_mode = 1;
@@ -1003,21 +1034,28 @@ static int gemm_plan(int T, int packed_rows, int K, int n_sm, int mode, bool may
     return SYN_OK;
 }
 
+// One projection with the epilogue `ep`; `plan_mode` = the epilogue its schedule is made for (the
+// same, except in the test hook, which runs any schedule with the plain store epilogue).
 static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const bf16* w_packed, int packed_rows, int K,
-                       const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, int* splits_out = nullptr,
-                       float* fix_part = nullptr, int* fix_flag = nullptr) {
+                       const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, float* fix_part, int* fix_flag,
+                       int plan_mode = -1) {
     ProfScope prof(cls >= 0 ? prof_m : nullptr, cls, st);
     GemmParams g;
+    memset(&g, 0, sizeof(g));
     int n_cta = 0;
-    const int pr = gemm_plan(ep.T, packed_rows, K, n_sm, ep.mode, fix_part && fix_flag, g, n_cta);
+    if (plan_mode < 0) plan_mode = ep.mode;
+    if (!fix_part || !fix_flag) return SYN_E_INVALID_ARG;
+    const int pr = gemm_plan(ep.T, packed_rows, K, n_sm, plan_mode, plan_mode != EPI_RESID, g, n_cta);
     if (pr) return pr;
     g.w = w_packed;
     g.status = status;
     g.fix_part = fix_part; g.fix_flag = fix_flag;
-    if (splits_out) *splits_out = g.splits;
-    const int smem = gemm_fixed_smem() + g.n_stages * gemm_stage_bytes(g.TN);
-    const cudaError_t le = g.ksplit > 1 ? launch_pdl(gemm_kernel<true>, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep)
-                                        : launch_pdl(gemm_kernel<false>, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep);
+    g.spin_limit = g_spin_limit;
+    const int smem = gemm_fixed_smem(g.TN) + g.n_stages * gemm_stage_bytes(g.TN);
+    cudaError_t le;
+    if (g.splits > 1) le = launch_pdl(gemm_kernel<GEMM_RSPLIT>, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep);
+    else if (g.ksplit > 1) le = launch_pdl(gemm_kernel<GEMM_KSPLIT>, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep);
+    else le = launch_pdl(gemm_kernel<GEMM_WAVES>, dim3(n_cta), dim3(GEMM_THREADS), smem, st, tmB, g, ep);
     return le == cudaSuccess ? SYN_OK : SYN_E_CUDA;
 }
 
@@ -1068,50 +1106,57 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
     if (T > m->t_cap || p->n_req > m->b_cap || p->n_parts > m->part_cap) return SYN_E_INVALID_ARG;
     const int* tokens = p->d<int>(p->o_tokens);
     const float inv_d = 1.0f / (float)d;
+    m->last_stats = p->stats;
+    m->have_last = true;
+    m->step_timed = false;
+    m->last_wall_ms = 0.0;
+    if (m->profile) {
+        if (!m->step_a) CU_OK(cudaEventCreate(&m->step_a));
+        if (!m->step_b) CU_OK(cudaEventCreate(&m->step_b));
+        CU_OK(cudaEventRecord(m->step_a, st));
+    }
     {
         ProfScope prof(m, 0, st);
         if (launch_pdl(prep_kernel, dim3(T), dim3(256), 0, st, m->embed, tokens, p->d<int>(p->o_pos), m->norm1[0], m->inv_freq,
-                       m->x, m->xn, m->rope, m->best, d, (int)(c.head_dim / 2), inv_d, c.rms_eps) != cudaSuccess)
+                       m->x, m->xn, m->ssq, m->rope, m->best, d, (int)(c.head_dim / 2)) != cudaSuccess)
             return SYN_E_CUDA;
     }
     EpiParams base;
     memset(&base, 0, sizeof(base));
     base.T = T;
-    const size_t part_stride = (size_t)m->t_cap * d;
-    int r, splits = 1;
-    auto resid = [&](int cls, const bf16* gain) -> int {
-        ProfScope prof(m, cls, st);
-        return launch_pdl(resid_norm_kernel, dim3(T), dim3(256), 0, st, m->x, m->part, part_stride, splits, gain, m->xn, d,
-                          inv_d, c.rms_eps) == cudaSuccess ? SYN_OK : SYN_E_CUDA;
-    };
+    // the consumers of a normalised operand: RMSNorm scale from the partial sums of x^2
+    EpiParams scaled = base;
+    scaled.ssq_in = m->ssq; scaled.n_ssq = d / 32; scaled.inv_d = inv_d; scaled.eps = c.rms_eps;
+    // the writers of the residual stream: x += D, next operand bf16(x * gain), new partial sums
+    EpiParams resid = base;
+    resid.mode = EPI_RESID; resid.N = d; resid.d = d; resid.x = m->x; resid.xg = m->xn; resid.ssq_out = m->ssq;
+    int r;
     for (uint32_t l = 0; l < c.n_layers; ++l) {
-        EpiParams e = base;
+        EpiParams e = scaled;
         e.mode = EPI_QKV; e.N = m->qkv_rows;
         e.q = m->q; e.q_dim = q_dim; e.kv_dim = kv_dim; e.hd = c.head_dim; e.n_kv_heads = c.n_kv_heads;
         e.page_size = kv->page_size; e.rope = m->rope; e.pool = kv->pool + kv->layer_elems * l;
         e.slot = p->d<int>(p->o_slot);
-        if ((r = launch_gemm(m, 1, m->n_sm, m->status_dev, m->wqkv[l], m->qkv_rows, d, m->tm_xn, e, st, nullptr, m->fix_part,
-                             m->fix_flag)))
+        if ((r = launch_gemm(m, 1, m->n_sm, m->status_dev, m->wqkv[l], m->qkv_rows, d, m->tm_xn, e, st, m->fix_part, m->fix_flag)))
             return r;
         if ((r = launch_attention(m, kv, p, l, m->tm_q, m->attn, st))) return r;
-        e = base;
-        e.mode = EPI_PART; e.N = d; e.d = d; e.part = m->part; e.part_stride = part_stride;
-        if ((r = launch_gemm(m, 4, m->n_sm, m->status_dev, m->wo[l], d, q_dim, m->tm_attn, e, st, &splits))) return r;
-        if ((r = resid(9, m->norm2[l]))) return r;
-        e = base;
-        e.mode = EPI_SWIGLU; e.N = m->gu_rows; e.act = m->act; e.f_pad = m->f_pad;
-        if ((r = launch_gemm(m, 5, m->n_sm, m->status_dev, m->wgu[l], m->gu_rows, d, m->tm_xn, e, st, nullptr, m->fix_part,
-                             m->fix_flag)))
+        e = resid;
+        e.gain = m->norm2[l];
+        if ((r = launch_gemm(m, 4, m->n_sm, m->status_dev, m->wo[l], d, q_dim, m->tm_attn, e, st, m->fix_part, m->fix_flag)))
             return r;
-        e = base;
-        e.mode = EPI_PART; e.N = d; e.d = d; e.part = m->part; e.part_stride = part_stride;
-        if ((r = launch_gemm(m, 6, m->n_sm, m->status_dev, m->wd[l], d, m->f_pad, m->tm_act, e, st, &splits))) return r;
-        if ((r = resid(9, l + 1 < c.n_layers ? m->norm1[l + 1] : m->final_norm))) return r;
+        e = scaled;
+        e.mode = EPI_SWIGLU; e.N = m->gu_rows; e.act = m->act; e.f_pad = m->f_pad;
+        if ((r = launch_gemm(m, 5, m->n_sm, m->status_dev, m->wgu[l], m->gu_rows, d, m->tm_xn, e, st, m->fix_part, m->fix_flag)))
+            return r;
+        e = resid;
+        e.gain = l + 1 < c.n_layers ? m->norm1[l + 1] : m->final_norm;
+        if ((r = launch_gemm(m, 6, m->n_sm, m->status_dev, m->wd[l], d, m->f_pad, m->tm_act, e, st, m->fix_part, m->fix_flag)))
+            return r;
     }
-    EpiParams e = base;
+    EpiParams e = scaled;
     e.mode = EPI_LMHEAD; e.N = m->v_rows; e.vocab = c.vocab; e.logits = logits_out; e.best = m->best;
     e.warp_max = warp_max; e.n_warp_max = m->v_rows / 32;
-    if ((r = launch_gemm(m, 7, m->n_sm, m->status_dev, m->lm_head, m->v_rows, d, m->tm_xn, e, st, nullptr, m->fix_part, m->fix_flag)))
+    if ((r = launch_gemm(m, 7, m->n_sm, m->status_dev, m->lm_head, m->v_rows, d, m->tm_xn, e, st, m->fix_part, m->fix_flag)))
         return r;
     {
         ProfScope prof(m, 8, st);
@@ -1119,12 +1164,16 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
                        p->d<int>(p->o_uncached), p->n_req, acc_dev, corr_dev, top1_dev) != cudaSuccess)
             return SYN_E_CUDA;
     }
+    if (m->profile) {
+        CU_OK(cudaEventRecord(m->step_b, st));
+        m->step_timed = true;
+    }
     return SYN_OK;
 }
 
-extern "C" int syn_verify_run(syn_model* m, syn_kv* kv, const syn_plan* p, int32_t* accept_len_dev, int32_t* correction_dev,
+static int syn_verify_run_impl(syn_model* m, syn_kv* kv, const syn_plan* p, int32_t* accept_len_dev, int32_t* correction_dev,
                               int32_t* top1_dev, float* logits_out, void* cuda_stream) {
-    if (!m || !kv || !p || kv->model != m || !accept_len_dev || !correction_dev) return SYN_E_INVALID_ARG;
+    if (!m || !kv || !p || kv->model != m || !plan_matches(p, kv) || !accept_len_dev || !correction_dev) return SYN_E_INVALID_ARG;
     return run_step(m, kv, p, accept_len_dev, correction_dev, top1_dev, logits_out, reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -1134,7 +1183,7 @@ extern "C" int syn_set_profile(syn_model* m, int on) {
     return SYN_OK;
 }
 
-extern "C" int syn_get_profile(syn_model* m, double* ms, int32_t* launches) {
+static int syn_get_profile_impl(syn_model* m, double* ms, int32_t* launches) {
     if (!m || !ms || !launches) return SYN_E_INVALID_ARG;
     CU_OK(cudaDeviceSynchronize());
     for (int i = 0; i < SYN_N_KERNEL_CLASSES; ++i) { ms[i] = 0.0; launches[i] = 0; }
@@ -1163,7 +1212,7 @@ extern "C" int syn_model_status(syn_model* m) {
     return SYN_OK;
 }
 
-extern "C" int syn_verify_batch(syn_model* m, syn_kv* kv, int32_t n_req, const int64_t* req_ids, const int32_t* chunk_tokens,
+static int syn_verify_batch_impl(syn_model* m, syn_kv* kv, int32_t n_req, const int64_t* req_ids, const int32_t* chunk_tokens,
                                 const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages,
                                 const int32_t* ctx_lens, const int32_t* n_uncached, int32_t* accept_len,
                                 int32_t* correction_token, float* logits_out, void* cuda_stream) {
@@ -1277,7 +1326,7 @@ static int ensure_sample_ws(syn_model* m, int T, int B, int slm_k, bool own_logi
     return SYN_OK;
 }
 
-extern "C" int syn_verify_batch_sampled(syn_model* m, syn_kv* kv, int32_t n_req, const int64_t* req_ids,
+static int syn_verify_batch_sampled_impl(syn_model* m, syn_kv* kv, int32_t n_req, const int64_t* req_ids,
                                         const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables,
                                         int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached,
                                         const syn_sampling* cfg, const int32_t* slm_ids, const float* slm_probs,
@@ -1335,7 +1384,7 @@ extern "C" int syn_verify_batch_sampled(syn_model* m, syn_kv* kv, int32_t n_req,
 // ------------------------------------------------------------------------------------------ single ops
 
 // The sampling stage alone on logits the caller supplies (device, fp32 [T][vocab]).
-extern "C" int syn_op_sample_verify(const float* logits, int32_t T, int32_t vocab, int32_t n_req, const int32_t* chunk_tokens,
+static int syn_op_sample_verify_impl(const float* logits, int32_t T, int32_t vocab, int32_t n_req, const int32_t* chunk_tokens,
                                     const int32_t* chunk_offsets, const int32_t* n_uncached, const syn_sampling* cfg,
                                     const int32_t* slm_ids, const float* slm_probs, const float* rand_accept,
                                     const float* rand_sample, int32_t* accept_len, int32_t* correction_token,
@@ -1387,70 +1436,109 @@ extern "C" int syn_op_sample_verify(const float* logits, int32_t T, int32_t voca
     return SYN_OK;
 }
 
-extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, int32_t N, int32_t K, void* cuda_stream) {
-    if (!x || !w || !y || T <= 0 || N <= 0 || K <= 0 || K % 8 != 0) return SYN_E_INVALID_ARG;
+// Process-wide context of the single-projection test hook: status word, exchange workspace, and the
+// packed copy of the last weight matrix seen.
+struct LinearCtx {
+    int n_sm = 0;
+    int* status = nullptr;
+    float* fix_part = nullptr;
+    int* fix_flag = nullptr;
+    bf16* packed = nullptr;
+    const void* packed_src = nullptr;
+    int packed_n = 0, packed_k = 0;
+};
+static LinearCtx g_lin;
+
+static int linear_ctx_init() {
+    if (g_lin.status) return SYN_OK;
+    int dev = 0;
+    cudaDeviceProp prop;
+    CU_OK(cudaGetDevice(&dev));
+    CU_OK(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return SYN_E_ARCH;
+    g_lin.n_sm = prop.multiProcessorCount;
+    CU_OK(cudaFuncSetAttribute(gemm_kernel<GEMM_WAVES>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_OK(cudaFuncSetAttribute(gemm_kernel<GEMM_KSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_OK(cudaFuncSetAttribute(gemm_kernel<GEMM_RSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_OK(cudaMalloc(&g_lin.fix_part, (size_t)g_lin.n_sm * GEMM_FIX_SLOT_BYTES));
+    CU_OK(cudaMalloc(&g_lin.fix_flag, (size_t)2 * g_lin.n_sm * 4));
+    CU_OK(cudaMemset(g_lin.fix_flag, 0, (size_t)2 * g_lin.n_sm * 4));
+    CU_OK(cudaMalloc(&g_lin.status, 4));
+    CU_OK(cudaMemset(g_lin.status, 0, 4));
+    return SYN_OK;
+}
+
+extern "C" int syn_op_linear_reset(void) {
+    if (g_lin.packed) {
+        CU_OK(cudaDeviceSynchronize());
+        cudaFree(g_lin.packed);
+    }
+    g_lin.packed = nullptr; g_lin.packed_src = nullptr; g_lin.packed_n = g_lin.packed_k = 0;
+    return SYN_OK;
+}
+
+extern "C" int syn_op_linear_as(const void* x, const void* w, float* y, int32_t T, int32_t N, int32_t K, int32_t schedule_as,
+                                void* cuda_stream) {
+    if (!x || !w || !y || T <= 0 || N <= 0 || K <= 0 || K % 8 != 0 || schedule_as < EPI_PLAIN || schedule_as > EPI_LMHEAD)
+        return SYN_E_INVALID_ARG;
     int r = load_driver_entry();
     if (r) return r;
-    // process-wide context of the test hook: status word, stream-K workspace, and the packed copy of
-    // the last weight matrix seen (re-packed when the pointer or the shape changes)
-    static int n_sm = 0;
-    static int* status = nullptr;
-    static float* fix_part = nullptr;
-    static int* fix_flag = nullptr;
-    static bf16* packed = nullptr;
-    static const void* packed_src = nullptr;
-    static int packed_n = 0, packed_k = 0;
+    if ((r = linear_ctx_init())) return r;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-    if (!status) {
-        int dev = 0;
-        cudaDeviceProp prop;
-        CU_OK(cudaGetDevice(&dev));
-        CU_OK(cudaGetDeviceProperties(&prop, dev));
-        if (prop.major != 10) return SYN_E_ARCH;
-        n_sm = prop.multiProcessorCount;
-        CU_OK(cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
-        CU_OK(cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
-        CU_OK(cudaMalloc(&fix_part, (size_t)n_sm * GEMM_FIX_SLOT_BYTES));
-        CU_OK(cudaMalloc(&fix_flag, (size_t)2 * n_sm * 4));
-        CU_OK(cudaMemset(fix_flag, 0, (size_t)2 * n_sm * 4));
-        CU_OK(cudaMalloc(&status, 4));
-        CU_OK(cudaMemset(status, 0, 4));
-    }
     const int n_mt = (N + 255) / 256 * 2, nkb = (K + 63) / 64;
-    if (packed_src != w || packed_n != N || packed_k != K) {
-        CU_OK(cudaDeviceSynchronize());
-        cudaFree(packed);
-        packed = nullptr; packed_src = nullptr;
-        CU_OK(cudaMalloc(&packed, (size_t)n_mt * nkb * 128 * 64 * 2));
+    if (g_lin.packed_src != w || g_lin.packed_n != N || g_lin.packed_k != K) {
+        if ((r = syn_op_linear_reset())) return r;
+        CU_OK(cudaMalloc(&g_lin.packed, (size_t)n_mt * nkb * 128 * 64 * 2));
         PackSrc ps;
         memset(&ps, 0, sizeof(ps));
         ps.p[0] = (const bf16*)w; ps.rows[0] = N; ps.src_k = K;
-        pack_weight_kernel<<<dim3(n_mt, nkb), 256, 0, st>>>(ps, packed, nkb);
+        pack_weight_kernel<<<dim3(n_mt, nkb), 256, 0, st>>>(ps, g_lin.packed, nkb);
         if (!launch_ok()) return SYN_E_CUDA;
         CU_OK(cudaStreamSynchronize(st));   // the GEMM requests weight tiles before it waits for its predecessor
-        packed_src = w; packed_n = N; packed_k = K;
+        g_lin.packed_src = w; g_lin.packed_n = N; g_lin.packed_k = K;
     }
     CUtensorMap tmB;
     if ((r = make_map_2d(&tmB, x, T, K, K, GEMM_BOX_ROWS))) return r;
     EpiParams e;
     memset(&e, 0, sizeof(e));
     e.mode = EPI_PLAIN; e.T = T; e.N = N; e.y = y; e.ldy = N;
-    r = launch_gemm(nullptr, -1, n_sm, status, packed, n_mt * 128, K, tmB, e, st, nullptr, fix_part, fix_flag);
+    r = launch_gemm(nullptr, -1, g_lin.n_sm, g_lin.status, g_lin.packed, n_mt * 128, K, tmB, e, st, g_lin.fix_part, g_lin.fix_flag,
+                    schedule_as);
     if (r) return r;
     CU_OK(cudaStreamSynchronize(st));
-    int s = 0;
-    CU_OK(cudaMemcpy(&s, status, 4, cudaMemcpyDeviceToHost));
-    if (s) {
-        cudaMemset(status, 0, 4);
-        cudaMemset(fix_flag, 0, (size_t)2 * n_sm * 4);
+    int sflag = 0;
+    CU_OK(cudaMemcpy(&sflag, g_lin.status, 4, cudaMemcpyDeviceToHost));
+    if (sflag) {
+        cudaMemset(g_lin.status, 0, 4);
+        cudaMemset(g_lin.fix_flag, 0, (size_t)2 * g_lin.n_sm * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     return SYN_OK;
 }
 
-extern "C" int syn_op_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const void* q, void* out,
+extern "C" int syn_op_linear(const void* x, const void* w, float* y, int32_t T, int32_t N, int32_t K, void* cuda_stream) {
+    return syn_op_linear_as(x, w, y, T, N, K, EPI_PLAIN, cuda_stream);
+}
+
+extern "C" int syn_debug_set_spin_limit(int64_t cycles) {
+    if (cycles < 0) return SYN_E_INVALID_ARG;
+    g_spin_limit = cycles == 0 ? SYN_SPIN_LIMIT_CYCLES : (long long)cycles;
+    return SYN_OK;
+}
+
+extern "C" int syn_debug_linear_counter(int32_t index, int32_t value) {
+    int r = linear_ctx_init();
+    if (r) return r;
+    if (index < 0 || index >= 2 * g_lin.n_sm) return SYN_E_INVALID_ARG;
+    CU_OK(cudaDeviceSynchronize());
+    CU_OK(cudaMemcpy(g_lin.fix_flag + index, &value, 4, cudaMemcpyHostToDevice));
+    return SYN_OK;
+}
+
+static int syn_op_attention_impl(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const void* q, void* out,
                                 void* cuda_stream) {
-    if (!m || !kv || !p || kv->model != m || !q || !out || layer >= m->desc.n_layers) return SYN_E_INVALID_ARG;
+    if (!m || !kv || !p || kv->model != m || !plan_matches(p, kv) || !q || !out || layer >= m->desc.n_layers)
+        return SYN_E_INVALID_ARG;
     const syn_model_desc& c = m->desc;
     const int q_dim = c.n_q_heads * c.head_dim;
     if (p->T > m->t_cap || p->n_parts > m->part_cap) return SYN_E_INVALID_ARG;
@@ -1476,9 +1564,11 @@ static int static_scratch(float** part_o, float2** part_ml, int** group_count) {
     static float* o_of[MAX_DEV];
     static float2* ml_of[MAX_DEV];
     static int* cnt_of[MAX_DEV];
+    static std::mutex lock;   // two host threads may make the first call on a device together
     int dev = -1;
     CU_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= MAX_DEV) return SYN_E_INVALID_ARG;
+    std::lock_guard<std::mutex> hold(lock);
     if (!o_of[dev]) {   // first call on this device (which is current): resolve the symbols
         void *a = nullptr, *b = nullptr, *cn = nullptr;
         CU_OK(cudaGetSymbolAddress(&a, g_static_part_o));
@@ -1495,9 +1585,10 @@ static int static_scratch(float** part_o, float2** part_ml, int** group_count) {
     return SYN_OK;
 }
 
-extern "C" int syn_op_attention_static(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const void* q,
+static int syn_op_attention_static_impl(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const void* q,
                                        void* out, void* cuda_stream) {
-    if (!m || !kv || !p || kv->model != m || !q || !out || layer >= m->desc.n_layers) return SYN_E_INVALID_ARG;
+    if (!m || !kv || !p || kv->model != m || !plan_matches(p, kv) || !q || !out || layer >= m->desc.n_layers)
+        return SYN_E_INVALID_ARG;
     const syn_model_desc& c = m->desc;
     const int q_dim = c.n_q_heads * c.head_dim;
     if (p->T > m->t_cap) return SYN_E_INVALID_ARG;
@@ -1527,7 +1618,7 @@ extern "C" int syn_gemm_plan_host(int32_t T, int32_t N, int32_t K, int32_t n_sm,
     GemmParams g;
     memset(&g, 0, sizeof(g));
     int n_cta = 0;
-    const int r = gemm_plan(T, (N + 255) / 256 * 256, K, n_sm, epilogue, epilogue != EPI_PART, g, n_cta);
+    const int r = gemm_plan(T, (N + 255) / 256 * 256, K, n_sm, epilogue, epilogue != EPI_RESID, g, n_cta);
     if (r) return r;
     const int v[SYN_GEMM_PLAN_FIELDS] = {g.n_pairs, g.n_tt, g.TN, g.num_kb, n_cta, g.pair_mode, g.splits, g.kb_per_split, g.ksplit, g.kper};
     memcpy(out, v, sizeof(v));
@@ -1541,7 +1632,7 @@ extern "C" int syn_gemm_work_host(int32_t T, int32_t N, int32_t K, int32_t n_sm,
     GemmParams g;
     memset(&g, 0, sizeof(g));
     int n_cta = 0;
-    const int r = gemm_plan(T, (N + 255) / 256 * 256, K, n_sm, epilogue, epilogue != EPI_PART, g, n_cta);
+    const int r = gemm_plan(T, (N + 255) / 256 * 256, K, n_sm, epilogue, epilogue != EPI_RESID, g, n_cta);
     if (r) return r;
     if (cta < 0 || cta >= n_cta) return SYN_E_INVALID_ARG;
     GemmWork w;
@@ -1550,6 +1641,86 @@ extern "C" int syn_gemm_work_host(int32_t T, int32_t N, int32_t K, int32_t n_sm,
     const int v[SYN_GEMM_WORK_FIELDS] = {w.pair, w.tt, w.mt_lo, w.mt_hi, w.kb0, w.kb1, w.split, w.role, w.rtile, w.hpart};
     memcpy(out, v, sizeof(v));
     return 1;
+}
+
+
+// ------------------------------------------------------------------------------------------ exported wrappers
+// No C++ exception crosses the C ABI: the host code behind these entry points uses std::vector.
+#define SYN_GUARD(call)                  \
+    try {                                \
+        return (call);                   \
+    } catch (const std::bad_alloc&) {    \
+        return SYN_E_OOM;                \
+    } catch (...) {                      \
+        return SYN_E_INVALID_ARG;        \
+    }
+
+extern "C" int syn_model_load(const syn_model_desc* desc, const syn_weights* w, syn_model** out) {
+    SYN_GUARD(syn_model_load_impl(desc, w, out));
+}
+
+extern "C" int syn_kv_import(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_t pos0, int32_t n_pos, const void* k, const void* v, void* stream) {
+    SYN_GUARD(syn_kv_import_impl(kv, layer, page_table, pos0, n_pos, k, v, stream));
+}
+
+extern "C" int syn_kv_export(syn_kv* kv, uint32_t layer, const int32_t* page_table, int32_t pos0, int32_t n_pos, void* k, void* v, void* stream) {
+    SYN_GUARD(syn_kv_export_impl(kv, layer, page_table, pos0, n_pos, k, v, stream));
+}
+
+extern "C" int syn_plan_host(const syn_model_desc* desc, uint32_t n_pages, uint32_t page_size, int32_t n_sm, int32_t n_req, const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, int32_t* pos, int32_t* slot, int32_t* items, int32_t items_cap, int32_t* n_items, int32_t* cta_begin, int32_t* n_cta, syn_step_stats* stats) {
+    SYN_GUARD(syn_plan_host_impl(desc, n_pages, page_size, n_sm, n_req, chunk_tokens, chunk_offsets, page_tables, max_pages, ctx_lens, n_uncached, pos, slot, items, items_cap, n_items, cta_begin, n_cta, stats));
+}
+
+extern "C" int syn_plan_create(syn_model* m, syn_kv* kv, int32_t n_req, const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, syn_plan** out) {
+    SYN_GUARD(syn_plan_create_impl(m, kv, n_req, chunk_tokens, chunk_offsets, page_tables, max_pages, ctx_lens, n_uncached, out));
+}
+
+extern "C" int syn_verify_run(syn_model* m, syn_kv* kv, const syn_plan* p, int32_t* accept_len_dev, int32_t* correction_dev, int32_t* top1_dev, float* logits_out, void* cuda_stream) {
+    SYN_GUARD(syn_verify_run_impl(m, kv, p, accept_len_dev, correction_dev, top1_dev, logits_out, cuda_stream));
+}
+
+extern "C" int syn_get_profile(syn_model* m, double* ms, int32_t* launches) {
+    SYN_GUARD(syn_get_profile_impl(m, ms, launches));
+}
+
+extern "C" int syn_verify_batch(syn_model* m, syn_kv* kv, int32_t n_req, const int64_t* req_ids, const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, int32_t* accept_len, int32_t* correction_token, float* logits_out, void* cuda_stream) {
+    const auto t0 = std::chrono::steady_clock::now();
+    int r;
+    try {
+        r = syn_verify_batch_impl(m, kv, n_req, req_ids, chunk_tokens, chunk_offsets, page_tables, max_pages, ctx_lens, n_uncached, accept_len, correction_token, logits_out, cuda_stream);
+    } catch (const std::bad_alloc&) {
+        return SYN_E_OOM;
+    } catch (...) {
+        return SYN_E_INVALID_ARG;
+    }
+    if (m && m->profile) m->last_wall_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
+    return r;
+}
+
+extern "C" int syn_verify_batch_sampled(syn_model* m, syn_kv* kv, int32_t n_req, const int64_t* req_ids, const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables, int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, const syn_sampling* cfg, const int32_t* slm_ids, const float* slm_probs, const float* rand_accept, const float* rand_sample, int32_t* accept_len, int32_t* correction_token, float* logits_out, void* cuda_stream) {
+    const auto t0 = std::chrono::steady_clock::now();
+    int r;
+    try {
+        r = syn_verify_batch_sampled_impl(m, kv, n_req, req_ids, chunk_tokens, chunk_offsets, page_tables, max_pages, ctx_lens, n_uncached, cfg, slm_ids, slm_probs, rand_accept, rand_sample, accept_len, correction_token, logits_out, cuda_stream);
+    } catch (const std::bad_alloc&) {
+        return SYN_E_OOM;
+    } catch (...) {
+        return SYN_E_INVALID_ARG;
+    }
+    if (m && m->profile) m->last_wall_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t0).count();
+    return r;
+}
+
+extern "C" int syn_op_sample_verify(const float* logits, int32_t T, int32_t vocab, int32_t n_req, const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* n_uncached, const syn_sampling* cfg, const int32_t* slm_ids, const float* slm_probs, const float* rand_accept, const float* rand_sample, int32_t* accept_len, int32_t* correction_token, void* cuda_stream) {
+    SYN_GUARD(syn_op_sample_verify_impl(logits, T, vocab, n_req, chunk_tokens, chunk_offsets, n_uncached, cfg, slm_ids, slm_probs, rand_accept, rand_sample, accept_len, correction_token, cuda_stream));
+}
+
+extern "C" int syn_op_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const void* q, void* out, void* cuda_stream) {
+    SYN_GUARD(syn_op_attention_impl(m, kv, p, layer, q, out, cuda_stream));
+}
+
+extern "C" int syn_op_attention_static(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const void* q, void* out, void* cuda_stream) {
+    SYN_GUARD(syn_op_attention_static_impl(m, kv, p, layer, q, out, cuda_stream));
 }
 
 extern "C" const char* syn_last_cuda_error(void) { return g_last_cuda_error; }

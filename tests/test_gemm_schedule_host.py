@@ -38,11 +38,13 @@ def _check(T, N, K, epilogue, n_sm=148):
         assert parts[0][0] == 0 and parts[-1][1] == nkb
         for a, b in zip(parts, parts[1:]):
             assert a[1] == b[0]                                     # the k ranges tile [0, nkb) without gap or overlap
-        if p["splits"] > 1:                                         # split-K: every part its own CTA, parts numbered in order
-            assert epilogue == "part" and [x[2] for x in parts] == list(range(len(parts)))
-            assert len({x[4] for x in parts}) == len(parts)
+        if p["splits"] > 1:                                         # K shared by neighbouring CTAs, parts numbered in order
+            assert epilogue in ("resid", "qkv") and [x[2] for x in parts] == list(range(len(parts)))
+            ctas = [x[4] for x in parts]
+            assert ctas == list(range(ctas[0], ctas[0] + len(parts))) and ctas[0] % p["splits"] == 0
+            assert p["n_cta"] <= n_sm                                   # all of them run at the same time
         elif len(parts) > 1:                                        # a leftover tile cut along K
-            assert p["ksplit"] == len(parts) and epilogue != "part"
+            assert p["ksplit"] == len(parts) and epilogue != "resid"
             assert [x[3] for x in parts] == [1] * (len(parts) - 1) + [2]
             assert len({x[4] for x in parts}) == len(parts)         # helpers and the owner are different CTAs
             assert all(x[5] == 0 for x in parts[:-1])               # helper parts are their CTAs' first items
@@ -58,8 +60,8 @@ def test_projections_of_the_configurations(cfg):
     s = wl.shape
     T = gen.gen_batch(wl).n_tokens
     f_pad = -(-s.d_ffn // 64) * 64
-    for N, K, epi in ((s.q_dim + 2 * s.kv_dim, s.d_model, "qkv"), (s.d_model, s.q_dim, "part"),
-                      (2 * f_pad, s.d_model, "swiglu"), (s.d_model, f_pad, "part"), (s.vocab, s.d_model, "lmhead")):
+    for N, K, epi in ((s.q_dim + 2 * s.kv_dim, s.d_model, "qkv"), (s.d_model, s.q_dim, "resid"),
+                      (2 * f_pad, s.d_model, "swiglu"), (s.d_model, f_pad, "resid"), (s.vocab, s.d_model, "lmhead")):
         _check(T, N, K, epi)
 
 
@@ -73,13 +75,16 @@ def test_the_launch_rules_show_up_where_they_should():
     p = _check(129, 3072, 2048, "qkv")
     assert p["TN"] == 32 and p["n_cta"] == 120
     # the 32B shape's down projection: 100 pair tiles cannot split K, seven token tiles fill the machine
-    p = _check(1194, 5120, 27648, "part")
+    p = _check(1194, 5120, 27648, "resid")
     assert p["n_tt"] == 7 and p["splits"] == 1 and p["n_cta"] == 140
-    # the 8B shape's o projection at 544 tokens: 48 pair tiles, K in three parts
-    assert _check(544, 4096, 4096, "part")["splits"] == 3
+    # the 8B shape's o projection at 544 tokens: 48 pair tiles, K shared by three CTAs each
+    assert _check(544, 4096, 4096, "resid")["splits"] == 3
+    # its QKV projection at 544 tokens: 72 pair tiles, K shared by two CTAs each instead of 144 single tiles
+    p = _check(544, 6144, 4096, "qkv")
+    assert (p["splits"], p["n_cta"], p["TN"]) == (2, 144, 192)
 
 
-@pytest.mark.parametrize("epilogue", ["plain", "qkv", "part", "swiglu", "lmhead"])
+@pytest.mark.parametrize("epilogue", ["plain", "qkv", "resid", "swiglu", "lmhead"])
 def test_sweep_of_awkward_sizes(epilogue):
     sizes = [(1, 128, 64), (16, 128, 688), (17, 384, 2048), (33, 256, 128), (129, 3072, 2048), (137, 4096, 512),
              (255, 640, 320), (256, 25600, 256), (257, 128, 128), (300, 38144, 1024), (544, 640, 4096), (921, 6144, 512),

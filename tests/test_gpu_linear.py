@@ -43,3 +43,66 @@ def test_linear_matches_oracle(T, N, K):
     scale = np.abs(ref).max()
     err = np.abs(y - ref).max()
     assert err <= 2e-5 * scale * max(1.0, (K / 256) ** 0.5), (err, scale)
+
+
+@pytest.mark.parametrize("T,N,K,sched", [
+    (544, 4096, 4096, "resid"),    # the 8B o projection: 48 pair tiles, K shared by three CTAs each (reduce-scatter)
+    (544, 4096, 14336, "resid"),   # its down projection: 224 k-blocks in three parts of 75, 75, 74
+    (544, 6144, 4096, "qkv"),      # its qkv projection: 72 pair tiles, K shared by two CTAs each
+    (129, 2048, 2048, "resid"),    # the 1B o projection: 8 tiles, K shared by eight CTAs, nine chunks among them
+    (144, 2048, 8192, "resid"),    # the 1B down projection
+    (300, 5120, 1024, "resid"),    # 40 tiles of 160 tokens (the last with 140), three parts
+    (50, 300, 1024, "resid"),      # ragged tokens and features, four parts of four k-blocks
+    (17, 256, 2048, "resid"),      # two chunks among eight CTAs: most of them keep no column
+    (1194, 5120, 1024, "resid"),   # 100 pair tiles: K not shared, seven narrower token tiles instead
+    (544, 28672, 4096, "swiglu"),  # schedule of the gate/up projection (leftover tiles cut along K)
+    (300, 38144, 1024, "lmhead"),
+])
+def test_every_schedule_of_the_step_gives_the_plain_product(T, N, K, sched):
+    """The work decompositions the step uses for its projections (K shared between CTAs with a
+    reduce-scatter of the accumulators, leftover tiles cut along K, mixed waves), each run with the
+    plain store epilogue and held to the same tolerance as the plain schedule."""
+    import paper_2511_07423_b200 as syn
+    x, w = _case(T, N, K, T + N + K + 1)
+    xc, wc = x.cuda(), w.cuda()
+    y = syn.syn_op_linear(xc, wc, schedule_as=sched)
+    y2 = syn.syn_op_linear(xc, wc, schedule_as=sched, reuse_pack=True)
+    assert torch.equal(y, y2)                      # fixed summation order, counters back at zero
+    ref = Oracle(TINY).linear(x.double().numpy(), w)
+    y = y.cpu().double().numpy()
+    scale = np.abs(ref).max()
+    err = np.abs(y - ref).max()
+    assert err <= 2e-5 * scale * max(1.0, (K / 256) ** 0.5), (err, scale)
+
+
+def test_a_new_matrix_at_an_old_address_is_packed_again():
+    import paper_2511_07423_b200 as syn
+    x, w = _case(32, 256, 256, 5)
+    xc, wc = x.cuda(), w.cuda()
+    y1 = syn.syn_op_linear(xc, wc)
+    wc.mul_(2)                                     # same address, same shape, new contents
+    y2 = syn.syn_op_linear(xc, wc)
+    assert torch.allclose(y2, 2 * y1)
+
+
+def test_a_wait_that_cannot_end_runs_out_and_the_next_call_works():
+    """SYN_E_DEVICE_TIMEOUT end to end: an arrival counter of the reduce-scatter is set so far below
+    zero that the count its readers wait for cannot be reached; with the waits' limit shortened to a
+    fraction of a millisecond they give up, the kernel ends normally, the call reports the timeout and
+    clears the counters, and the same call then succeeds with the right result."""
+    import paper_2511_07423_b200 as syn
+    T, N, K = 544, 4096, 4096
+    assert syn.gemm_plan_host(T, N, K, "resid")["splits"] == 3
+    x, w = _case(T, N, K, 77)
+    xc, wc = x.cuda(), w.cuda()
+    good = syn.syn_op_linear(xc, wc, schedule_as="resid")
+    try:
+        syn.debug_set_spin_limit(400_000)
+        syn.debug_linear_counter(0, -1_000_000)    # tile 0: its three CTAs wait for 48 arrivals
+        with pytest.raises(syn.SynError) as ei:
+            syn.syn_op_linear(xc, wc, schedule_as="resid", reuse_pack=True)
+        assert ei.value.code == -11
+    finally:
+        syn.debug_set_spin_limit(0)
+    again = syn.syn_op_linear(xc, wc, schedule_as="resid", reuse_pack=True)
+    assert torch.equal(again, good)
