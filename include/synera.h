@@ -231,7 +231,9 @@ const char *syn_last_cuda_error(void);
  * be a multiple of 16; N arbitrary.  Blocks until the result is there.
  * syn_op_linear_as runs the same product under the schedule the step uses for the projection with
  * epilogue `schedule_as` (0 plain, 1 qkv, 2 residual, 3 SwiGLU, 4 lm_head; see syn_gemm_plan_host), so
- * that every schedule can be checked against a plain matrix product.
+ * that every schedule can be checked against a plain matrix product; 5 and 6 take the CTA-pair kernel
+ * with items of 512 and of 256 features whatever the shape, 7 and 8 the same as residual projections
+ * (K shared between clusters where the shape allows it).
  * Errors: SYN_E_INVALID_ARG, SYN_E_CUDA, SYN_E_DEVICE_TIMEOUT. */
 int syn_op_linear(const void *x, const void *w, float *y, int32_t T, int32_t N, int32_t K, void *cuda_stream);
 int syn_op_linear_as(const void *x, const void *w, float *y, int32_t T, int32_t N, int32_t K, int32_t schedule_as,
@@ -244,9 +246,13 @@ int syn_op_linear_reset(void);
  * overwrite one of the arrival counters of syn_op_linear's own workspace (index in [0, 2 * SMs)), so
  * that a wait for a count that can no longer be reached runs out; the counters are cleared again when
  * the timeout is reported.  A wait that runs out unwinds normally: the kernel ends, the results of
- * that call are invalid, the next call works. */
+ * that call are invalid, the next call works.
+ * syn_debug_set_schedule: 0 (default) lets every projection take the kernel its shape calls for (CTA
+ * pairs from 256 tokens on); 1 keeps all of them on the one-CTA kernel, so that both can be measured
+ * and checked on the same batch.  Process-wide. */
 int syn_debug_set_spin_limit(int64_t cycles);
 int syn_debug_linear_counter(int32_t index, int32_t value);
+int syn_debug_set_schedule(int32_t which);
 
 /* The ragged paged attention of the step on its own (paper Sec. 3.2 attention equation over a
  * paged cache).  q: DEVICE bf16 [T][n_q_heads*head_dim] (rotated); out: DEVICE bf16, same

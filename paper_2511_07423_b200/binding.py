@@ -58,7 +58,7 @@ _LIB: Optional[C.CDLL] = None
 EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "syn_kv_import", "syn_kv_export",
            "syn_verify_batch", "syn_plan_create", "syn_plan_free", "syn_verify_run", "syn_model_status",
            "syn_last_step_stats", "syn_plan_stats", "syn_plan_host", "syn_strerror", "syn_last_cuda_error", "syn_op_linear",
-           "syn_op_linear_as", "syn_op_linear_reset", "syn_debug_set_spin_limit", "syn_debug_linear_counter",
+           "syn_op_linear_as", "syn_op_linear_reset", "syn_debug_set_spin_limit", "syn_debug_linear_counter", "syn_debug_set_schedule",
            "syn_op_attention", "syn_op_attention_static",
            "syn_set_profile", "syn_get_profile", "syn_verify_batch_sampled", "syn_op_sample_verify",
            "syn_gemm_plan_host", "syn_gemm_work_host"]
@@ -495,6 +495,9 @@ class Scheduler:
 GEMM_PLAN_FIELDS = ("n_pairs", "n_tt", "TN", "num_kb", "n_cta", "pair_mode", "splits", "kb_per_split", "ksplit", "kper")
 GEMM_WORK_FIELDS = ("pair", "tt", "mt_lo", "mt_hi", "kb0", "kb1", "split", "role", "rtile", "hpart")
 GEMM_EPILOGUES = {"plain": 0, "qkv": 1, "resid": 2, "swiglu": 3, "lmhead": 4}
+# syn_op_linear_as only: the CTA-pair kernel with 512-feature (quad) or 256-feature (duo) items, as a
+# plain projection or as a residual projection (K shared between clusters where the shape allows it)
+LINEAR_SCHEDULES = dict(GEMM_EPILOGUES, pair_quad=5, pair_duo=6, pair_quad_resid=7, pair_duo_resid=8)
 
 
 def gemm_plan_host(T: int, N: int, K: int, epilogue: str, n_sm: int = 148) -> Dict[str, int]:
@@ -530,7 +533,7 @@ def syn_op_linear(x: torch.Tensor, w: torch.Tensor, stream=None, schedule_as: st
     if not reuse_pack:
         _check(lib.syn_op_linear_reset(), "syn_op_linear_reset")
     _check(lib.syn_op_linear_as(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
-                                C.c_int32(T), C.c_int32(N), C.c_int32(K), C.c_int32(GEMM_EPILOGUES[schedule_as]),
+                                C.c_int32(T), C.c_int32(N), C.c_int32(K), C.c_int32(LINEAR_SCHEDULES[schedule_as]),
                                 _stream_ptr(stream)), "syn_op_linear_as")
     return y
 
@@ -538,6 +541,11 @@ def syn_op_linear(x: torch.Tensor, w: torch.Tensor, stream=None, schedule_as: st
 def debug_set_spin_limit(cycles: int) -> None:
     """syn_debug_set_spin_limit: SM cycles after which a wait inside the projection kernels gives up (0: default)."""
     _check(load_library().syn_debug_set_spin_limit(C.c_int64(cycles)), "syn_debug_set_spin_limit")
+
+
+def debug_set_schedule(which: int) -> None:
+    """syn_debug_set_schedule: 0 automatic, 1 every projection on the one-CTA kernel."""
+    _check(load_library().syn_debug_set_schedule(C.c_int32(which)), "syn_debug_set_schedule")
 
 
 def debug_linear_counter(index: int, value: int) -> None:

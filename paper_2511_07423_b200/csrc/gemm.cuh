@@ -21,8 +21,8 @@
 // Every CTA starts its k loop at a different k-block, so the CTAs that share a token tile do not
 // ask L2 for the same lines at the same moment.  Accumulation is tcgen05.mma into TMEM, read back
 // with tcgen05.ld by sixteen epilogue warps; a thread then holds one output feature for sixteen
-// tokens (thirty-two in the epilogues that need few other registers), and the epilogues work on
-// those registers:
+// tokens; a warp turns its 32 x 16 block round in shared memory, so that every lane reads and writes
+// 16-byte pieces of token-major rows:
 //   EPI_QKV    : RMSNorm scale, RoPE on q and k (the partner dimension sits 16 lanes away), q store,
 //                paged-KV append
 //   EPI_RESID  : x += D (the residual stream, fp32), the next projection's operand bf16(x * gain) and
@@ -100,174 +100,199 @@ __host__ __device__ __forceinline__ int rope_tile_feature(int l, int hd) {   // 
 
 constexpr int GEMM_EPI_WARPS = 16;               // four groups of four (one warp per TMEM lane quarter)
 
-// Sum over the 32 lanes of sixteen values per lane in sixteen shuffles: each round halves the values
-// a lane keeps (the lanes of a pair exchange the halves they give up).  Afterwards lane L holds the
-// total of value number L >> 1 (both lanes of a pair hold the same total).  The order of the
-// additions is fixed.
-__device__ __forceinline__ float warp_sum16(float (&v)[16], int lane) {
-    {
-        const bool up = (lane & 16) != 0;
+// Epilogue of one 16-token chunk of one warp: a[j] = D[feature of this lane][token t0 + j] (tokens
+// j >= ncols are padding), already summed and scaled.  In this orientation a lane holds ONE output
+// feature for sixteen tokens, while every output is token-major in memory, so the 32 x 16 block is
+// first turned round in a shared-memory scratch of the warp (16 rows of 33 floats: no bank conflicts
+// either way).  Afterwards the lanes walk the block row by row: eight neighbouring lanes cover the 32
+// columns of one token with four columns each, so that a warp-wide access touches whole 32-byte
+// sectors of four tokens' rows (the cost of these epilogues is the number of sectors and of memory
+// instructions they issue, not their arithmetic).
+// `m0` = first packed row of the tile, `quarter` = warp's TMEM lane quarter.
+constexpr int EPI_COLS = 16;
+constexpr int EPI_SCR_STRIDE = 33;
+constexpr int EPI_SCR_FLOATS = EPI_COLS * EPI_SCR_STRIDE;   // per epilogue warp
+
+__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) { return make_uint2(pack_bf16(a, b), pack_bf16(c, d)); }
+
+template <int MODE>
+__device__ __forceinline__ void epi_unit(const EpiParams& p, const float (&a)[EPI_COLS], float* scr, int m0, int t0, int ncols,
+                                         int quarter, int lane) {
+    __syncwarp();   // the previous chunk's rows have been read
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float got = __shfl_xor_sync(0xFFFFFFFFu, up ? v[i] : v[8 + i], 16);
-            v[i] = (up ? v[8 + i] : v[i]) + got;
-        }
-    }
-    {
-        const bool up = (lane & 8) != 0;
+    for (int j = 0; j < EPI_COLS; ++j) scr[j * EPI_SCR_STRIDE + lane] = a[j];
+    __syncwarp();
+    const int tq = lane >> 3, c0 = (lane & 7) * 4;   // token (+ 4 i) and first of four columns of this lane
+    if (MODE == EPI_PLAIN) {
+        const int f = m0 + quarter * 32 + c0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float got = __shfl_xor_sync(0xFFFFFFFFu, up ? v[i] : v[4 + i], 8);
-            v[i] = (up ? v[4 + i] : v[i]) + got;
-        }
-    }
-    {
-        const bool up = (lane & 4) != 0;
+            const int t = tq + 4 * i;
+            const float* row = scr + t * EPI_SCR_STRIDE + c0;
+            if (t < ncols) {
+                float* dst = p.y + (size_t)(t0 + t) * p.ldy + f;
+                if ((p.ldy & 3) == 0 && f + 4 <= p.N) {
+                    *reinterpret_cast<float4*>(dst) = make_float4(row[0], row[1], row[2], row[3]);
+                } else {
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const float got = __shfl_xor_sync(0xFFFFFFFFu, up ? v[i] : v[2 + i], 4);
-            v[i] = (up ? v[2 + i] : v[i]) + got;
-        }
-    }
-    {
-        const bool up = (lane & 2) != 0;
-        const float got = __shfl_xor_sync(0xFFFFFFFFu, up ? v[0] : v[1], 2);
-        v[0] = (up ? v[1] : v[0]) + got;
-    }
-    return v[0] + __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
-}
-
-// Epilogue of one 16-token chunk straight from registers: r[j] = D[feature of this thread][token
-// t0 + j]; tokens j >= ncols are padding.  `m0` = first packed row of the tile, `quarter` = warp's TMEM
-// lane quarter.  `rs` = NULL, or the RMSNorm scales of tokens t0 .. t0 + 15 (shared memory).
-// Warp shuffles, votes and reductions are never moved across stores by the compiler, and
-// loads not above stores that might alias them, so every mode first runs all its warp-wide exchanges
-// and loads back to back (their latencies overlap) and only then does the arithmetic and the stores.
-constexpr int EPI_COLS = 16;
-template <int MODE>
-__device__ __forceinline__ void epi_direct(const EpiParams& p, const uint32_t (&r)[EPI_COLS], const float* rs, int m0, int t0,
-                                           int ncols, int quarter, int lane) {
-    const int l = quarter * 32 + lane;
-    float a[EPI_COLS];
-#pragma unroll
-    for (int j = 0; j < EPI_COLS; ++j) a[j] = __uint_as_float(r[j]);
-    if (MODE != EPI_PLAIN && MODE != EPI_RESID && rs != nullptr) {
-#pragma unroll
-        for (int j = 0; j < EPI_COLS; ++j) a[j] *= rs[j];
-    }
-    if (MODE == EPI_PLAIN) {
-        const int f = m0 + l;
-        float* base = p.y + f + (size_t)t0 * p.ldy;
-        if (f < p.N) {
-#pragma unroll
-            for (int j = 0; j < EPI_COLS; ++j)
-                if (j < ncols) base[(size_t)j * p.ldy] = a[j];
+                    for (int k = 0; k < 4; ++k)
+                        if (f + k < p.N) dst[k] = row[k];
+                }
+            }
         }
     } else if (MODE == EPI_RESID) {
-        // x += D; operand of the next projection; sums of x^2 over this warp's 32 features
-        const int f = m0 + l;
-        const bool fv = f < p.N;
-        const size_t at = (size_t)t0 * p.d + (fv ? f : 0);
-        float xv[EPI_COLS];
+        // x += D; operand of the next projection bf16(x * gain); sum of x^2 over this warp's 32 features
+        const int f = m0 + quarter * 32 + c0;
+        const uint2 gb = __ldg(reinterpret_cast<const uint2*>(p.gain + f));
+        const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gb.x);
+        const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gb.y);
+        float4 xv[4];
 #pragma unroll
-        for (int j = 0; j < EPI_COLS; ++j) xv[j] = (fv && j < ncols) ? p.x[at + (size_t)j * p.d] : 0.f;
-        const float gn = fv ? __bfloat162float(p.gain[f]) : 0.f;
+        for (int i = 0; i < 4; ++i)
+            xv[i] = tq + 4 * i < ncols ? *reinterpret_cast<const float4*>(p.x + (size_t)(t0 + tq + 4 * i) * p.d + f)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int j = 0; j < EPI_COLS; ++j) {
-            xv[j] = (fv && j < ncols) ? xv[j] + a[j] : 0.f;
-            if (fv && j < ncols) {
-                p.x[at + (size_t)j * p.d] = xv[j];
-                p.xg[at + (size_t)j * p.d] = __float2bfloat16(xv[j] * gn);
+        for (int i = 0; i < 4; ++i) {
+            const int t = tq + 4 * i;
+            const bool tv = t < ncols;
+            const float* row = scr + t * EPI_SCR_STRIDE + c0;
+            const float4 nx = make_float4(xv[i].x + row[0], xv[i].y + row[1], xv[i].z + row[2], xv[i].w + row[3]);
+            float ss = tv ? (nx.x * nx.x + nx.y * nx.y) + (nx.z * nx.z + nx.w * nx.w) : 0.f;
+            if (tv) {
+                const size_t at = (size_t)(t0 + t) * p.d + f;
+                *reinterpret_cast<float4*>(p.x + at) = nx;
+                *reinterpret_cast<uint2*>(p.xg + at) = pack4_bf16(nx.x * __low2float(g01), nx.y * __high2float(g01),
+                                                                  nx.z * __low2float(g23), nx.w * __high2float(g23));
             }
-            xv[j] *= xv[j];
+            ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);   // the eight lanes of the token, a fixed order
+            ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+            ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 4);
+            if (tv && (lane & 7) == 0) p.ssq_out[(size_t)(t0 + t) * (p.d >> 5) + ((m0 >> 5) + quarter)] = ss;
         }
-        const float tot = warp_sum16(xv, lane);   // lane L: token L >> 1
-        if (!(lane & 1) && (lane >> 1) < ncols && m0 + quarter * 32 < p.N)
-            p.ssq_out[(size_t)(t0 + (lane >> 1)) * (p.d >> 5) + ((m0 >> 5) + quarter)] = tot;
     } else if (MODE == EPI_QKV) {
         const int which = m0 < p.q_dim ? 0 : (m0 < p.q_dim + p.kv_dim ? 1 : 2);
         const int region0 = which == 0 ? 0 : (which == 1 ? p.q_dim : p.q_dim + p.kv_dim);
-        const int fr = m0 - region0 + (which < 2 ? rope_tile_feature(l, p.hd) : l);   // feature inside q, k or v
         const int half = p.hd >> 1;
-        const int dim = fr & (p.hd - 1);
-        const bool lo = dim < half;
-        const float2* cs = p.rope + (size_t)t0 * half + (lo ? dim : dim - half);
-        float o[EPI_COLS];   // rotate-half RoPE: the partner dimension is 16 lanes away
-        float2 w[EPI_COLS];
-        // KV slots (page * 16 + row) of the chunk's tokens: one coalesced load, handed round by shuffles
-        const int my_slot = (which > 0 && lane < ncols) ? __ldg(p.slot + t0 + lane) : 0;
-#pragma unroll
-        for (int j = 0; j < EPI_COLS; ++j) {
-            o[j] = which < 2 ? __shfl_xor_sync(0xFFFFFFFFu, a[j], 16) : 0.f;
-            w[j] = (which < 2 && j < ncols) ? __ldg(cs + (size_t)j * half) : make_float2(1.f, 0.f);
-        }
-        __nv_bfloat16* const qdst = p.q + (size_t)t0 * p.q_dim + fr;
-        __nv_bfloat16* const kvdst = p.pool + ((size_t)(fr / p.hd) * 2 + (which > 0 ? which - 1 : 0)) * 16 * p.hd + dim;
         const size_t page_stride = (size_t)p.n_kv_heads * 2 * 16 * p.hd;
+        // KV slot (page * 16 + row) of token lane & 15, handed round by shuffles
+        const int my_slot = (which > 0 && (lane & 15) < ncols) ? __ldg(p.slot + t0 + (lane & 15)) : 0;
+        if (which < 2) {
+            // q and k tiles: columns 0..15 of the block are the dims [d0, d0 + 16) of one head, columns 16..31
+            // the same dims + hd/2 (rope_tile_feature); a lane rotates its four columns with their partners
+            const int groups = half >> 4;
+            const int fhead = (m0 - region0) + (quarter / groups) * p.hd;   // first feature of the head, inside q or k
+            const bool hi = c0 >= 16;
+            const int dim = 16 * (quarter % groups) + (c0 & 15);            // lower dim of the pair
+            float4 w[4][2];
 #pragma unroll
-        for (int j = 0; j < EPI_COLS; ++j) {
-            const int sl = __shfl_sync(0xFFFFFFFFu, my_slot, j);
-            if (j < ncols) {
-                float v = a[j];
-                if (which < 2) v = lo ? (v * w[j].x - o[j] * w[j].y) : (v * w[j].x + o[j] * w[j].y);
-                if (which == 0) qdst[(size_t)j * p.q_dim] = __float2bfloat16(v);
-                else kvdst[(size_t)(sl >> 4) * page_stride + (size_t)(sl & 15) * p.hd] = __float2bfloat16(v);
+            for (int i = 0; i < 4; ++i) {
+                const float4* cs = reinterpret_cast<const float4*>(p.rope + (size_t)(t0 + tq + 4 * i) * half + dim);   // 4 x (cos, sin)
+                const bool tv = tq + 4 * i < ncols;
+                w[i][0] = tv ? __ldg(cs) : make_float4(1.f, 0.f, 1.f, 0.f);
+                w[i][1] = tv ? __ldg(cs + 1) : make_float4(1.f, 0.f, 1.f, 0.f);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int t = tq + 4 * i;
+                const float* mine = scr + t * EPI_SCR_STRIDE + c0;
+                const float* part = scr + t * EPI_SCR_STRIDE + (c0 ^ 16);
+                const float sg = hi ? 1.f : -1.f;   // dim i: x cos - y sin; dim i + hd/2: y cos + x sin
+                const float o0 = mine[0] * w[i][0].x + sg * part[0] * w[i][0].y;
+                const float o1 = mine[1] * w[i][0].z + sg * part[1] * w[i][0].w;
+                const float o2 = mine[2] * w[i][1].x + sg * part[2] * w[i][1].y;
+                const float o3 = mine[3] * w[i][1].z + sg * part[3] * w[i][1].w;
+                const int sl = __shfl_sync(0xFFFFFFFFu, my_slot, t);
+                if (t < ncols) {
+                    __nv_bfloat16* dst;
+                    if (which == 0) dst = p.q + (size_t)(t0 + t) * p.q_dim + fhead;
+                    else dst = p.pool + (size_t)(sl >> 4) * page_stride + ((size_t)(fhead / p.hd) * 2) * 16 * p.hd + (size_t)(sl & 15) * p.hd;
+                    *reinterpret_cast<uint2*>(dst + dim + (hi ? half : 0)) = pack4_bf16(o0, o1, o2, o3);
+                }
+            }
+        } else {
+            // v tiles: features in natural order
+            const int fr = (m0 - region0) + quarter * 32 + c0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int t = tq + 4 * i;
+                const float* row = scr + t * EPI_SCR_STRIDE + c0;
+                const int sl = __shfl_sync(0xFFFFFFFFu, my_slot, t);
+                if (t < ncols) {
+                    __nv_bfloat16* dst = p.pool + (size_t)(sl >> 4) * page_stride + ((size_t)(fr / p.hd) * 2 + 1) * 16 * p.hd +
+                                         (size_t)(sl & 15) * p.hd + (fr & (p.hd - 1));
+                    *reinterpret_cast<uint2*>(dst) = pack4_bf16(row[0], row[1], row[2], row[3]);
+                }
             }
         }
     } else if (MODE == EPI_SWIGLU) {
-        // Two tokens per step: the lower half-warp finishes token j, the upper one token j + 1, so all
-        // lanes evaluate silu and one store covers two rows of 16 features.
-        // Lanes 0..15 hold gate, lanes 16..31 the matching up features.
-        const bool up_half = lane >= 16;
-        float got[EPI_COLS / 2];
+        // columns 0..15 of the block hold gate features, columns 16..31 the matching up features: 16
+        // outputs per token; four neighbouring lanes cover them, eight tokens per pass
+        const int tq8 = lane >> 2, g0 = (lane & 3) * 4;
 #pragma unroll
-        for (int k = 0; k < EPI_COLS / 2; ++k)   // each half-warp sends what the other one needs
-            got[k] = __shfl_xor_sync(0xFFFFFFFFu, up_half ? a[2 * k] : a[2 * k + 1], 16);
-        __nv_bfloat16* const dst = p.act + (size_t)(t0 + (up_half ? 1 : 0)) * p.f_pad + (m0 >> 1) + 16 * quarter + (lane & 15);
+        for (int i = 0; i < 2; ++i) {
+            const int t = tq8 + 8 * i;
+            const float* row = scr + t * EPI_SCR_STRIDE + g0;
+            float h[4];
 #pragma unroll
-        for (int k = 0; k < EPI_COLS / 2; ++k) {
-            const float gate = up_half ? got[k] : a[2 * k];       // upper half: gate of token 2k + 1
-            const float upv = up_half ? a[2 * k + 1] : got[k];    // lower half: up of token 2k
-            const float h = __fdividef(gate, 1.0f + __expf(-gate)) * upv;
-            if (2 * k + (up_half ? 1 : 0) < ncols) dst[(size_t)(2 * k) * p.f_pad] = __float2bfloat16(h);
+            for (int k = 0; k < 4; ++k) h[k] = __fdividef(row[k], 1.0f + __expf(-row[k])) * row[16 + k];
+            if (t < ncols)
+                *reinterpret_cast<uint2*>(p.act + (size_t)(t0 + t) * p.f_pad + (m0 >> 1) + 16 * quarter + g0) = pack4_bf16(h[0], h[1], h[2], h[3]);
         }
     } else {  // EPI_LMHEAD
-        const int f = m0 + l;
-        const bool valid = f < p.vocab;
-        if (p.logits && valid) {
+        const int f = m0 + quarter * 32 + c0;
 #pragma unroll
-            for (int j = 0; j < EPI_COLS; ++j)
-                if (j < ncols) p.logits[(size_t)(t0 + j) * p.vocab + f] = a[j];
-        }
-        uint32_t mx[EPI_COLS];
+        for (int i = 0; i < 4; ++i) {
+            const int t = tq + 4 * i;
+            const bool tv = t < ncols;
+            const float* row = scr + t * EPI_SCR_STRIDE + c0;
+            const float v[4] = {row[0], row[1], row[2], row[3]};
+            if (p.logits && tv) {
+                float* dst = p.logits + (size_t)(t0 + t) * p.vocab + f;
+                if ((p.vocab & 3) == 0 && f + 4 <= p.vocab) {
+                    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+                } else {
 #pragma unroll
-        for (int j = 0; j < EPI_COLS; ++j)
-            mx[j] = __reduce_max_sync(0xFFFFFFFFu, valid ? orderable_f32(a[j]) : 0u);
-        unsigned long long mine = 0ull;   // lane j keeps the warp's best of token j
+                    for (int k = 0; k < 4; ++k)
+                        if (f + k < p.vocab) dst[k] = v[k];
+                }
+            }
+            // largest logit of the token among this lane's features, lowest id on ties; then over the
+            // token's eight lanes (the packed key orders by logit, then by lower id)
+            unsigned long long mine = 0ull;
 #pragma unroll
-        for (int j = 0; j < EPI_COLS; ++j) {
-            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, valid && orderable_f32(a[j]) == mx[j]);
-            if (lane == j && hit) mine = pack_argmax_key(mx[j], m0 + quarter * 32 + (__ffs(hit) - 1));
-        }
-        if (lane < ncols && mine) atomicMax(p.best + t0 + lane, mine);
-        if (p.warp_max) {   // lane j keeps the group's maximum of token j: a threshold source for a later top-k
-            uint32_t gm = 0u;
+            for (int k = 0; k < 4; ++k) {
+                const unsigned long long key = f + k < p.vocab ? pack_argmax_key(orderable_f32(v[k]), f + k) : 0ull;
+                if (key > mine) mine = key;
+            }
 #pragma unroll
-            for (int j = 0; j < EPI_COLS; ++j)
-                if (lane == j) gm = mx[j];
-            if (lane < ncols) p.warp_max[(size_t)(t0 + lane) * p.n_warp_max + (m0 >> 5) + quarter] = gm;
+            for (int o = 1; o < 8; o <<= 1) {
+                const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, mine, o);
+                if (other > mine) mine = other;
+            }
+            if (tv && (lane & 7) == 0) {
+                if (mine) atomicMax(p.best + t0 + t, mine);
+                // the group's maximum of the token (0: no valid feature): a threshold source for a later top-k
+                if (p.warp_max) p.warp_max[(size_t)(t0 + t) * p.n_warp_max + (m0 >> 5) + quarter] = (uint32_t)(mine >> 32);
+            }
         }
     }
 }
 
-__device__ __forceinline__ void epi_dispatch(int mode, const EpiParams& p, const uint32_t (&r)[EPI_COLS], const float* rs, int m0,
-                                             int t0, int ncols, int quarter, int lane) {
+__device__ __forceinline__ void epi_dispatch(int mode, const EpiParams& p, const uint32_t (&r)[EPI_COLS], const float* rs, float* scr,
+                                             int m0, int t0, int ncols, int quarter, int lane) {
+    float a[EPI_COLS];
+#pragma unroll
+    for (int j = 0; j < EPI_COLS; ++j) a[j] = __uint_as_float(r[j]);
+    if (rs != nullptr) {
+#pragma unroll
+        for (int j = 0; j < EPI_COLS; ++j) a[j] *= rs[j];
+    }
     switch (mode) {
-        case EPI_PLAIN: epi_direct<EPI_PLAIN>(p, r, rs, m0, t0, ncols, quarter, lane); break;
-        case EPI_QKV: epi_direct<EPI_QKV>(p, r, rs, m0, t0, ncols, quarter, lane); break;
-        case EPI_RESID: epi_direct<EPI_RESID>(p, r, rs, m0, t0, ncols, quarter, lane); break;
-        case EPI_SWIGLU: epi_direct<EPI_SWIGLU>(p, r, rs, m0, t0, ncols, quarter, lane); break;
-        default: epi_direct<EPI_LMHEAD>(p, r, rs, m0, t0, ncols, quarter, lane); break;
+        case EPI_PLAIN: epi_unit<EPI_PLAIN>(p, a, scr, m0, t0, ncols, quarter, lane); break;
+        case EPI_QKV: epi_unit<EPI_QKV>(p, a, scr, m0, t0, ncols, quarter, lane); break;
+        case EPI_RESID: epi_unit<EPI_RESID>(p, a, scr, m0, t0, ncols, quarter, lane); break;
+        case EPI_SWIGLU: epi_unit<EPI_SWIGLU>(p, a, scr, m0, t0, ncols, quarter, lane); break;
+        default: epi_unit<EPI_LMHEAD>(p, a, scr, m0, t0, ncols, quarter, lane); break;
     }
 }
 
@@ -294,7 +319,7 @@ __device__ __forceinline__ void epi_rms_scales(const EpiParams& p, float* dst, i
 // stored as the 128-byte-swizzled shared-memory image (16-byte chunk c of row r at chunk c ^ (r & 7)).
 // mode 0: packed row pr = row pr of the concatenation of up to three matrices.
 // mode 1: gate/up: tile b holds gate and up features [64 b, 64 b + 64) in the lane order of
-//         epi_direct (quarter q: lanes 0..15 gate 64 b + 16 q + lane, lanes 16..31 the same up rows).
+//         epi_unit (quarter q: lanes 0..15 gate 64 b + 16 q + lane, lanes 16..31 the same up rows).
 // mode 2: q | k | v concatenation; q and k tiles in the RoPE lane order (rope_tile_feature), v plain.
 // ------------------------------------------------------------------------------------------
 struct PackSrc {
@@ -361,7 +386,8 @@ __host__ __device__ inline int gemm_stage_bytes(int TN) { return GEMM_A_BYTES + 
 // RMSNorm scales of an item's tokens, two buffers (items alternate); rounded up so that an epilogue
 // that takes 32 columns at a time stays inside the buffer
 __host__ __device__ inline int gemm_rs_stride(int TN) { return (TN + 31) & ~31; }
-__host__ inline int gemm_fixed_smem(int TN) { return 1024 /*align*/ + GEMM_BAR_BYTES + 2 * gemm_rs_stride(TN) * 4; }
+__host__ __device__ inline int gemm_scr_offset(int TN) { return GEMM_BAR_BYTES + 2 * gemm_rs_stride(TN) * 4; }   // from the barriers
+__host__ inline int gemm_fixed_smem(int TN) { return 1024 /*align*/ + gemm_scr_offset(TN) + GEMM_EPI_WARPS * EPI_SCR_FLOATS * 4; }
 __host__ inline int gemm_stages(int TN) {
     int s = (GEMM_SMEM_MAX - gemm_fixed_smem(TN)) / gemm_stage_bytes(TN);
     return s > GEMM_MAX_STAGES ? GEMM_MAX_STAGES : s;
@@ -509,7 +535,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
     uint64_t* acce_bar = accf_bar + 1;                  // accumulators drained (epilogue -> MMA)
     uint64_t* rs_bar = acce_bar + 1;                    // RMSNorm scales of the item's tokens are in rs_s
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rs_bar + 1);
-    float* rs_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(full_bar) + GEMM_BAR_BYTES);   // [2][TN]
+    float* rs_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(full_bar) + GEMM_BAR_BYTES);   // [2][rs stride]
+    float* scr_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(full_bar) + gemm_scr_offset(g.TN));   // [epilogue warp][16][33]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_cta = gridDim.x, cta = blockIdx.x;
@@ -624,6 +651,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
         constexpr int NGRP = GEMM_EPI_WARPS / 4;
         const int quarter = warp & 3;         // TMEM lane quarter this warp may read
         const bool scaled = p.ssq_in != nullptr;
+        float* const scr = scr_s + e * EPI_SCR_FLOATS;
         bool ok = true;
         GemmWork w;
         pdl_wait();   // the epilogues read and write buffers of earlier kernels
@@ -712,87 +740,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                             }
                         }
                         const int tc0 = n0 + c * EPI_COLS, ncols = min(EPI_COLS, n_valid - c * EPI_COLS);
-                        if (m0 < p.N) epi_dispatch(p.mode, p, r, scaled ? rsi + c * EPI_COLS : nullptr, m0, tc0, ncols, quarter, lane);
+                        if (m0 < p.N) epi_dispatch(p.mode, p, r, scaled ? rsi + c * EPI_COLS : nullptr, scr, m0, tc0, ncols, quarter, lane);
                     }
                 // the last warp of the tile's CTAs to finish reading clears the counters for the next launch
                 __syncwarp();
                 if (lane == 0 && atomicAdd(g.fix_flag + g.n_sm + tile, 1) == S * GEMM_EPI_WARPS - 1) {
                     g.fix_flag[tile] = 0;
                     g.fix_flag[g.n_sm + tile] = 0;
-                }
-                continue;
-            }
-            if ((!KSPLIT || w.role == 0) && p.mode == EPI_PLAIN) {
-                // fp32 stores only: 32 columns a TMEM load (the accumulator's columns beyond the
-                // tile's tokens are allocated, their contents are not stored)
-                const int nch2 = (nchunks + 1) >> 1;
-                const int total2 = (w.mt_hi - w.mt_lo) * nch2;
-                for (int ci = grp; ci < total2; ci += NGRP) {
-                    const int mt = w.mt_lo + ci / nch2, c2 = ci % nch2;
-                    const int m0 = w.pair * 256 + mt * 128;
-                    uint32_t r[32];
-                    tmem_ld32(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c2 * 32), r);
-                    tmem_ld_wait();
-                    if (ci + NGRP >= total2) {
-                        tc_fence_before();
-                        if (lane == 0) mbar_arrive(acce_bar);
-                    }
-                    const int f = m0 + quarter * 32 + lane;
-                    const int tc0 = n0 + c2 * 32, ncols = min(32, n_valid - c2 * 32);
-                    if (f < p.N) {
-                        float* base = p.y + f + (size_t)tc0 * p.ldy;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j < ncols) base[(size_t)j * p.ldy] = __uint_as_float(r[j]);
-                    }
-                }
-                if (grp >= total2) {
-                    tc_fence_before();
-                    if (lane == 0) mbar_arrive(acce_bar);
-                }
-                continue;
-            }
-            if ((!KSPLIT || w.role == 0) && p.mode == EPI_SWIGLU) {
-                // silu(gate) * up on 32 columns a TMEM load.  Lanes 0..15 hold gate, lanes 16..31 the
-                // matching up features; the lower half-warp finishes the even tokens, the upper one the
-                // odd tokens, so all lanes evaluate silu and one store covers two rows of 16 features.
-                const int nch2 = (nchunks + 1) >> 1;
-                const int total2 = (w.mt_hi - w.mt_lo) * nch2;
-                const bool up_half = lane >= 16;
-                for (int ci = grp; ci < total2; ci += NGRP) {
-                    const int mt = w.mt_lo + ci / nch2, c2 = ci % nch2;
-                    const int m0 = w.pair * 256 + mt * 128;
-                    uint32_t r[32];
-                    tmem_ld32(tmem_base + mt * acc_stride + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c2 * 32), r);
-                    tmem_ld_wait();
-                    if (ci + NGRP >= total2) {
-                        tc_fence_before();
-                        if (lane == 0) mbar_arrive(acce_bar);
-                    }
-                    const int tc0 = n0 + c2 * 32, ncols = min(32, n_valid - c2 * 32);
-                    if (scaled) {   // columns beyond the tile's tokens hold stale scales: finite, never stored
-                        const float* rs = rsi + c2 * 32;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * rs[j]);
-                    }
-                    float got[16];
-#pragma unroll
-                    for (int k = 0; k < 16; ++k)   // each half-warp sends what the other one needs
-                        got[k] = __shfl_xor_sync(0xFFFFFFFFu, __uint_as_float(up_half ? r[2 * k] : r[2 * k + 1]), 16);
-                    if (m0 < p.N) {
-                        __nv_bfloat16* const dst = p.act + (size_t)(tc0 + (up_half ? 1 : 0)) * p.f_pad + (m0 >> 1) + 16 * quarter + (lane & 15);
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const float gate = up_half ? got[k] : __uint_as_float(r[2 * k]);       // upper half: gate of token 2k + 1
-                            const float upv = up_half ? __uint_as_float(r[2 * k + 1]) : got[k];    // lower half: up of token 2k
-                            const float h = __fdividef(gate, 1.0f + __expf(-gate)) * upv;
-                            if (2 * k + (up_half ? 1 : 0) < ncols) dst[(size_t)(2 * k) * p.f_pad] = __float2bfloat16(h);
-                        }
-                    }
-                }
-                if (grp >= total2) {
-                    tc_fence_before();
-                    if (lane == 0) mbar_arrive(acce_bar);
                 }
                 continue;
             }
@@ -808,7 +762,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                         if (lane == 0) mbar_arrive(acce_bar);
                     }
                     const int tc0 = n0 + c * EPI_COLS, ncols = min(EPI_COLS, n_valid - c * EPI_COLS);
-                    if (m0 < p.N) epi_dispatch(p.mode, p, r, scaled ? rsi + c * EPI_COLS : nullptr, m0, tc0, ncols, quarter, lane);
+                    if (m0 < p.N) epi_dispatch(p.mode, p, r, scaled ? rsi + c * EPI_COLS : nullptr, scr, m0, tc0, ncols, quarter, lane);
                 }
                 if (grp >= total_chunks) {   // a group without any chunk still releases the accumulators
                     tc_fence_before();
@@ -880,7 +834,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                     }
                 }
                 const int tc0 = n0 + c * EPI_COLS, ncols = min(EPI_COLS, n_valid - c * EPI_COLS);
-                if (m0 < p.N) epi_dispatch(p.mode, p, r, scaled ? rsi + c * EPI_COLS : nullptr, m0, tc0, ncols, quarter, lane);
+                if (m0 < p.N) epi_dispatch(p.mode, p, r, scaled ? rsi + c * EPI_COLS : nullptr, scr, m0, tc0, ncols, quarter, lane);
             }
             if (grp >= total_chunks) {
                 tc_fence_before();

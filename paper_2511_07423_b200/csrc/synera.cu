@@ -15,15 +15,19 @@
 
 #include "attention.cuh"
 #include "gemm.cuh"
+#include "gemm2.cuh"
 #include "sampling.cuh"
 
 using namespace syn;
 typedef __nv_bfloat16 bf16;
 // Slot of one helper part's stored accumulators: two tiles of 128 features x up to 256 tokens, fp32.
 constexpr size_t GEMM_FIX_SLOT_BYTES = (size_t)2 * 128 * 256 * 4;
+constexpr int GEMM_FLAG_INTS = 4;   // arrival / release counters of the exchanges: ints per SM
 constexpr int GEMM_MAX_SPLITS = 8;   // most CTAs that share one pair tile's K range
 // Limit of the kernels' bounded waits in SM cycles (syn_debug_set_spin_limit; tests shorten it).
 static long long g_spin_limit = SYN_SPIN_LIMIT_CYCLES;
+// 0: every projection takes the kernel its shape calls for; 1: the one-CTA kernel always (syn_debug_set_schedule).
+static int g_schedule = 0;
 
 // Name of the last CUDA error a call of this library met on this thread (for syn_last_cuda_error).
 static thread_local const char* g_last_cuda_error = "";
@@ -57,6 +61,23 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
+    return note_cuda(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+}
+
+// The same for a kernel whose CTAs form clusters of two.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    memset(attr, 0, sizeof(attr));
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     return note_cuda(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
 }
 
@@ -157,11 +178,34 @@ static int make_map_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_
     return r == CUDA_SUCCESS ? SYN_OK : SYN_E_CUDA;
 }
 
+// 2-D view of a packed weight matrix for the CTA-pair kernel: rows of 128 bytes (64 bf16), no
+// swizzle (the tiles already are shared-memory images); one box = the two 128-row tiles of a
+// feature pair for one k-block (QUAD items) or one of them (DUO items).
+struct WMaps {
+    CUtensorMap quad, duo;
+};
+static int make_wmaps(const void* packed, int packed_rows, int K, WMaps* out) {
+    const uint64_t n_pairs = (uint64_t)((packed_rows + 511) / 512 * 2), nkb = (uint64_t)((K + 63) / 64);
+    cuuint64_t dims[2] = {64, n_pairs * nkb * 256};
+    cuuint64_t strides[1] = {128};
+    cuuint32_t estr[2] = {1, 1};
+    for (int k = 0; k < 2; ++k) {
+        cuuint32_t box[2] = {64, k == 0 ? 256u : 128u};
+        if (g_encode(k == 0 ? &out->quad : &out->duo, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(packed), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return SYN_E_CUDA;
+    }
+    return SYN_OK;
+}
+
 struct syn_model {
     syn_model_desc desc;
     int f_pad, n_sm, gu_rows, qkv_rows, v_rows;
     bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
     std::vector<bf16*> wqkv, wo, wgu, wd, norm1, norm2;   // projections in the packed tile layout
+    std::vector<WMaps> tm_wqkv, tm_wo, tm_wgu, tm_wd;      // their tensor maps
+    WMaps tm_lm_head;
     double* inv_freq = nullptr;
     int* status_dev = nullptr;
     // workspace (grow-only)
@@ -175,7 +219,7 @@ struct syn_model {
     int b_cap = 0;
     CUtensorMap tm_xn, tm_attn, tm_act, tm_q;
     float* fix_part = nullptr;      // stored accumulators of K-split remainder tiles (one slot per SM)
-    int* fix_flag = nullptr;        // their arrival / release counters, [2 * n_sm], zero between launches
+    int* fix_flag = nullptr;        // their arrival / release counters, [GEMM_FLAG_INTS * n_sm], zero between launches
     float* part_o = nullptr;
     float2* part_ml = nullptr;
     int* group_count = nullptr;     // per merge group: partial items completed (zero between launches)
@@ -290,8 +334,8 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
     }
     if (!m->fix_part) {
         CU_OK(cudaMalloc(&m->fix_part, (size_t)m->n_sm * GEMM_FIX_SLOT_BYTES));
-        CU_OK(cudaMalloc(&m->fix_flag, (size_t)2 * m->n_sm * 4));
-        CU_OK(cudaMemset(m->fix_flag, 0, (size_t)2 * m->n_sm * 4));
+        CU_OK(cudaMalloc(&m->fix_flag, (size_t)GEMM_FLAG_INTS * m->n_sm * 4));
+        CU_OK(cudaMemset(m->fix_flag, 0, (size_t)GEMM_FLAG_INTS * m->n_sm * 4));
     }
     if (B > m->b_cap) {
         cudaFree(m->acc_dev); cudaFree(m->corr_dev);
@@ -406,7 +450,7 @@ static int syn_model_load_impl(const syn_model_desc* desc, const syn_weights* w,
     // pack `n` row-major sources (rows[i] x src_k each) into a new tile-layout buffer of `packed_rows` x K
     auto pack = [&](const void* const* srcs, const int* rows, int n, int mode, int src_k, int packed_rows,
                     bf16** out_ptr) -> int {
-        const int n_mt = (packed_rows + 255) / 256 * 2, nkb = (src_k + 63) / 64;
+        const int n_mt = (packed_rows + 511) / 512 * 4, nkb = (src_k + 63) / 64;   // an even number of feature pairs (zero rows at the end)
         bf16* outp = nullptr;
         cudaError_t e = cudaMalloc(&outp, (size_t)n_mt * nkb * 128 * 64 * 2);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return SYN_E_OOM; }
@@ -446,6 +490,7 @@ static int syn_model_load_impl(const syn_model_desc* desc, const syn_weights* w,
         const void* srcs[1] = {w->lm_head};
         const int rows[1] = {(int)c.vocab};
         PACK_OR_FAIL(pack(srcs, rows, 1, 0, d, c.vocab, &m->lm_head));
+        PACK_OR_FAIL(make_wmaps(m->lm_head, m->v_rows, d, &m->tm_lm_head));
     }
     for (uint32_t l = 0; l < c.n_layers; ++l) {
         bf16 *n1 = nullptr, *n2 = nullptr, *pk = nullptr;
@@ -454,24 +499,36 @@ static int syn_model_load_impl(const syn_model_desc* desc, const syn_weights* w,
             const int rows[3] = {q_dim, kv_dim, kv_dim};
             PACK_OR_FAIL(pack(srcs, rows, 3, 2, d, m->qkv_rows, &pk));
             m->wqkv.push_back(pk);
+            WMaps wm;
+            PACK_OR_FAIL(make_wmaps(pk, m->qkv_rows, d, &wm));
+            m->tm_wqkv.push_back(wm);
         }
         {
             const void* srcs[1] = {w->wo[l]};
             const int rows[1] = {d};
             PACK_OR_FAIL(pack(srcs, rows, 1, 0, q_dim, d, &pk));
             m->wo.push_back(pk);
+            WMaps wm;
+            PACK_OR_FAIL(make_wmaps(pk, d, q_dim, &wm));
+            m->tm_wo.push_back(wm);
         }
         {   // a tile holds the gate and the up rows of the same 64 features; rows of the padded tail are zero
             const void* srcs[2] = {w->wg[l], w->wu[l]};
             const int rows[2] = {f, f};
             PACK_OR_FAIL(pack(srcs, rows, 2, 1, d, m->gu_rows, &pk));
             m->wgu.push_back(pk);
+            WMaps wm;
+            PACK_OR_FAIL(make_wmaps(pk, m->gu_rows, d, &wm));
+            m->tm_wgu.push_back(wm);
         }
         {   // down projection: K = d_ffn, zero-padded to f_pad by the k-block tail
             const void* srcs[1] = {w->wd[l]};
             const int rows[1] = {d};
             PACK_OR_FAIL(pack(srcs, rows, 1, 0, f, d, &pk));
             m->wd.push_back(pk);
+            WMaps wm;
+            PACK_OR_FAIL(make_wmaps(pk, d, m->f_pad, &wm));
+            m->tm_wd.push_back(wm);
         }
         CU_M(cudaMalloc(&n1, (size_t)d * 2)); m->norm1.push_back(n1);
         CU_M(cudaMalloc(&n2, (size_t)d * 2)); m->norm2.push_back(n2);
@@ -489,6 +546,8 @@ static int syn_model_load_impl(const syn_model_desc* desc, const syn_weights* w,
     CU_M(cudaFuncSetAttribute(gemm_kernel<GEMM_WAVES>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_M(cudaFuncSetAttribute(gemm_kernel<GEMM_KSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_M(cudaFuncSetAttribute(gemm_kernel<GEMM_RSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_M(cudaFuncSetAttribute(gemm2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_M(cudaFuncSetAttribute(gemm2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_M(cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::TOTAL));
     CU_M(cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::TOTAL));
     CU_M(cudaDeviceSynchronize());
@@ -1059,6 +1118,75 @@ static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const 
     return le == cudaSuccess ? SYN_OK : SYN_E_CUDA;
 }
 
+// Schedules of the CTA-pair kernel (gemm2.cuh).
+enum { PAIR_NONE = 0, PAIR_QUAD = 1, PAIR_DUO = 2 };
+
+// Launch shape of a projection on CTA pairs, or PAIR_NONE when the one-CTA kernel serves it better
+// (few tokens: the pair kernel's token tiles are the natural 256-token cut, it has no narrow tiles).
+// Host arithmetic only.  `force`: PAIR_QUAD / PAIR_DUO to take that item shape regardless (test hook).
+static int gemm2_plan(int T, int packed_rows, int K, int n_sm, int mode, int force, Gemm2Params& g, int& n_cl) {
+    memset(&g, 0, sizeof(g));
+    const int n_pairs = (packed_rows + 255) / 256, n_cl_max = n_sm / 2;
+    g.num_kb = (K + 63) / 64;
+    g.n_tt = (T + 255) / 256;
+    g.TN = (((T + g.n_tt - 1) / g.n_tt) + 15) / 16 * 16;
+    g.n_tt = (T + g.TN - 1) / g.TN;
+    g.splits = 1; g.kb_per_split = g.num_kb; g.n_sm = n_sm;
+    if (n_cl_max < 1 || (force == PAIR_NONE && T < 256)) return PAIR_NONE;
+    const int quad_items = (n_pairs + 1) / 2 * g.n_tt, duo_items = n_pairs * g.n_tt;
+    int kind = force;
+    if (kind == PAIR_NONE) {
+        if (quad_items >= n_cl_max) kind = PAIR_QUAD;                                   // full waves of 512-feature items
+        else if (mode == EPI_RESID && g.num_kb >= 96 && n_cl_max / quad_items >= 2) kind = PAIR_QUAD;   // long K: shared between clusters
+        else if (2 * duo_items >= n_cl_max) kind = PAIR_DUO;
+        else return PAIR_NONE;
+    }
+    const int items = kind == PAIR_QUAD ? quad_items : duo_items;
+    g.n_groups = kind == PAIR_QUAD ? (n_pairs + 1) / 2 : n_pairs;
+    if (mode == EPI_RESID && items < n_cl_max && n_cl_max / items >= 2) {
+        const int sp = std::min(GEMM_MAX_SPLITS, std::min(n_cl_max / items, std::max(1, g.num_kb / 8)));
+        g.kb_per_split = (g.num_kb + sp - 1) / sp;
+        g.splits = (g.num_kb + g.kb_per_split - 1) / g.kb_per_split;
+    }
+    n_cl = g.splits > 1 ? items * g.splits : std::min(n_cl_max, items);
+    if (g.splits == 1 && items > n_cl) {
+        // items left after the full waves: cut along K into one part per cluster (parts of at least 8 k-blocks,
+        // at most GEMM_MAX_SPLITS of them), so that the last round takes a fraction of an item's time
+        const int rem = items % n_cl;
+        if (rem > 0 && n_cl / rem >= 2) {
+            int base = n_cl / rem, extra = n_cl % rem;
+            const int most = std::min(GEMM_MAX_SPLITS, g.num_kb / 8);
+            if (base + (extra > 0 ? 1 : 0) > most) { base = most; extra = 0; }
+            if (base >= 2) { g.rem_base = base; g.rem_extra = extra; }
+        }
+    }
+    g.n_stages = gemm2_stages(g.TN, kind == PAIR_DUO);
+    if (g.n_stages < 2 || g.TN < 16 || g.TN > 256 || (g.n_tt - 1) * g.TN >= T) return PAIR_NONE;
+    return kind;
+}
+
+// One projection with the epilogue `ep` on whichever kernel its shape calls for.  `plan_mode` = the
+// epilogue the schedule is made for (the same, except in the test hook); `force_pair`: test hook.
+static int launch_proj(syn_model* prof_m, int cls, int n_sm, int* status, const bf16* w_packed, const WMaps* wm, int packed_rows,
+                       int K, const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, float* fix_part, int* fix_flag,
+                       int plan_mode = -1, int force_pair = PAIR_NONE) {
+    if (plan_mode < 0) plan_mode = ep.mode;
+    Gemm2Params g2;
+    int n_cl = 0;
+    const int kind = (wm && (g_schedule == 0 || force_pair != PAIR_NONE)) ? gemm2_plan(ep.T, packed_rows, K, n_sm, plan_mode, force_pair, g2, n_cl)
+                                                                            : PAIR_NONE;
+    if (kind == PAIR_NONE) return launch_gemm(prof_m, cls, n_sm, status, w_packed, packed_rows, K, tmB, ep, st, fix_part, fix_flag, plan_mode);
+    if (!fix_part || !fix_flag) return SYN_E_INVALID_ARG;
+    ProfScope prof(cls >= 0 ? prof_m : nullptr, cls, st);
+    g2.status = status; g2.spin_limit = g_spin_limit;
+    g2.fix_part = fix_part; g2.fix_flag = fix_flag;
+    const bool duo = kind == PAIR_DUO;
+    const int smem = gemm_fixed_smem(g2.TN) + g2.n_stages * gemm2_stage_bytes(g2.TN, duo);
+    const cudaError_t le = duo ? launch_pdl_pairs(gemm2_kernel<true>, dim3(2 * n_cl), dim3(GEMM_THREADS), smem, st, wm->duo, tmB, g2, ep)
+                               : launch_pdl_pairs(gemm2_kernel<false>, dim3(2 * n_cl), dim3(GEMM_THREADS), smem, st, wm->quad, tmB, g2, ep);
+    return le == cudaSuccess ? SYN_OK : SYN_E_CUDA;
+}
+
 static void attn_params(AttnParams& ap, const syn_model* m, const syn_kv* kv, const syn_plan* p, uint32_t layer, bf16* out,
                         float* part_o, float2* part_ml, int* group_count) {
     const syn_model_desc& c = m->desc;
@@ -1137,26 +1265,26 @@ static int run_step(syn_model* m, syn_kv* kv, const syn_plan* p, int* acc_dev, i
         e.q = m->q; e.q_dim = q_dim; e.kv_dim = kv_dim; e.hd = c.head_dim; e.n_kv_heads = c.n_kv_heads;
         e.page_size = kv->page_size; e.rope = m->rope; e.pool = kv->pool + kv->layer_elems * l;
         e.slot = p->d<int>(p->o_slot);
-        if ((r = launch_gemm(m, 1, m->n_sm, m->status_dev, m->wqkv[l], m->qkv_rows, d, m->tm_xn, e, st, m->fix_part, m->fix_flag)))
+        if ((r = launch_proj(m, 1, m->n_sm, m->status_dev, m->wqkv[l], &m->tm_wqkv[l], m->qkv_rows, d, m->tm_xn, e, st, m->fix_part, m->fix_flag)))
             return r;
         if ((r = launch_attention(m, kv, p, l, m->tm_q, m->attn, st))) return r;
         e = resid;
         e.gain = m->norm2[l];
-        if ((r = launch_gemm(m, 4, m->n_sm, m->status_dev, m->wo[l], d, q_dim, m->tm_attn, e, st, m->fix_part, m->fix_flag)))
+        if ((r = launch_proj(m, 4, m->n_sm, m->status_dev, m->wo[l], &m->tm_wo[l], d, q_dim, m->tm_attn, e, st, m->fix_part, m->fix_flag)))
             return r;
         e = scaled;
         e.mode = EPI_SWIGLU; e.N = m->gu_rows; e.act = m->act; e.f_pad = m->f_pad;
-        if ((r = launch_gemm(m, 5, m->n_sm, m->status_dev, m->wgu[l], m->gu_rows, d, m->tm_xn, e, st, m->fix_part, m->fix_flag)))
+        if ((r = launch_proj(m, 5, m->n_sm, m->status_dev, m->wgu[l], &m->tm_wgu[l], m->gu_rows, d, m->tm_xn, e, st, m->fix_part, m->fix_flag)))
             return r;
         e = resid;
         e.gain = l + 1 < c.n_layers ? m->norm1[l + 1] : m->final_norm;
-        if ((r = launch_gemm(m, 6, m->n_sm, m->status_dev, m->wd[l], d, m->f_pad, m->tm_act, e, st, m->fix_part, m->fix_flag)))
+        if ((r = launch_proj(m, 6, m->n_sm, m->status_dev, m->wd[l], &m->tm_wd[l], d, m->f_pad, m->tm_act, e, st, m->fix_part, m->fix_flag)))
             return r;
     }
     EpiParams e = scaled;
     e.mode = EPI_LMHEAD; e.N = m->v_rows; e.vocab = c.vocab; e.logits = logits_out; e.best = m->best;
     e.warp_max = warp_max; e.n_warp_max = m->v_rows / 32;
-    if ((r = launch_gemm(m, 7, m->n_sm, m->status_dev, m->lm_head, m->v_rows, d, m->tm_xn, e, st, m->fix_part, m->fix_flag)))
+    if ((r = launch_proj(m, 7, m->n_sm, m->status_dev, m->lm_head, &m->tm_lm_head, m->v_rows, d, m->tm_xn, e, st, m->fix_part, m->fix_flag)))
         return r;
     {
         ProfScope prof(m, 8, st);
@@ -1206,7 +1334,7 @@ extern "C" int syn_model_status(syn_model* m) {
     if (s) {
         cudaMemset(m->status_dev, 0, 4);
         if (m->group_count) cudaMemset(m->group_count, 0, (size_t)m->part_cap * 4);   // an aborted step may leave counts
-        if (m->fix_flag) cudaMemset(m->fix_flag, 0, (size_t)2 * m->n_sm * 4);
+        if (m->fix_flag) cudaMemset(m->fix_flag, 0, (size_t)GEMM_FLAG_INTS * m->n_sm * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     return SYN_OK;
@@ -1244,7 +1372,7 @@ static int syn_verify_batch_impl(syn_model* m, syn_kv* kv, int32_t n_req, const 
     if (po[2 * m->pinned_out_cap]) {
         cudaMemset(m->status_dev, 0, 4);
         if (m->group_count) cudaMemset(m->group_count, 0, (size_t)m->part_cap * 4);
-        if (m->fix_flag) cudaMemset(m->fix_flag, 0, (size_t)2 * m->n_sm * 4);
+        if (m->fix_flag) cudaMemset(m->fix_flag, 0, (size_t)GEMM_FLAG_INTS * m->n_sm * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     memcpy(accept_len, po, (size_t)n_req * 4);
@@ -1373,7 +1501,7 @@ static int syn_verify_batch_sampled_impl(syn_model* m, syn_kv* kv, int32_t n_req
     if (po[2 * m->pinned_out_cap]) {
         cudaMemset(m->status_dev, 0, 4);
         if (m->group_count) cudaMemset(m->group_count, 0, (size_t)m->part_cap * 4);
-        if (m->fix_flag) cudaMemset(m->fix_flag, 0, (size_t)2 * m->n_sm * 4);
+        if (m->fix_flag) cudaMemset(m->fix_flag, 0, (size_t)GEMM_FLAG_INTS * m->n_sm * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     memcpy(accept_len, po, (size_t)n_req * 4);
@@ -1446,6 +1574,7 @@ struct LinearCtx {
     bf16* packed = nullptr;
     const void* packed_src = nullptr;
     int packed_n = 0, packed_k = 0;
+    WMaps wm;
 };
 static LinearCtx g_lin;
 
@@ -1460,9 +1589,11 @@ static int linear_ctx_init() {
     CU_OK(cudaFuncSetAttribute(gemm_kernel<GEMM_WAVES>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_OK(cudaFuncSetAttribute(gemm_kernel<GEMM_KSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_OK(cudaFuncSetAttribute(gemm_kernel<GEMM_RSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_OK(cudaFuncSetAttribute(gemm2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
+    CU_OK(cudaFuncSetAttribute(gemm2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_OK(cudaMalloc(&g_lin.fix_part, (size_t)g_lin.n_sm * GEMM_FIX_SLOT_BYTES));
-    CU_OK(cudaMalloc(&g_lin.fix_flag, (size_t)2 * g_lin.n_sm * 4));
-    CU_OK(cudaMemset(g_lin.fix_flag, 0, (size_t)2 * g_lin.n_sm * 4));
+    CU_OK(cudaMalloc(&g_lin.fix_flag, (size_t)GEMM_FLAG_INTS * g_lin.n_sm * 4));
+    CU_OK(cudaMemset(g_lin.fix_flag, 0, (size_t)GEMM_FLAG_INTS * g_lin.n_sm * 4));
     CU_OK(cudaMalloc(&g_lin.status, 4));
     CU_OK(cudaMemset(g_lin.status, 0, 4));
     return SYN_OK;
@@ -1479,13 +1610,13 @@ extern "C" int syn_op_linear_reset(void) {
 
 extern "C" int syn_op_linear_as(const void* x, const void* w, float* y, int32_t T, int32_t N, int32_t K, int32_t schedule_as,
                                 void* cuda_stream) {
-    if (!x || !w || !y || T <= 0 || N <= 0 || K <= 0 || K % 8 != 0 || schedule_as < EPI_PLAIN || schedule_as > EPI_LMHEAD)
+    if (!x || !w || !y || T <= 0 || N <= 0 || K <= 0 || K % 8 != 0 || schedule_as < EPI_PLAIN || schedule_as > EPI_LMHEAD + 4)
         return SYN_E_INVALID_ARG;
     int r = load_driver_entry();
     if (r) return r;
     if ((r = linear_ctx_init())) return r;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-    const int n_mt = (N + 255) / 256 * 2, nkb = (K + 63) / 64;
+    const int n_mt = (N + 511) / 512 * 4, nkb = (K + 63) / 64;
     if (g_lin.packed_src != w || g_lin.packed_n != N || g_lin.packed_k != K) {
         if ((r = syn_op_linear_reset())) return r;
         CU_OK(cudaMalloc(&g_lin.packed, (size_t)n_mt * nkb * 128 * 64 * 2));
@@ -1496,21 +1627,26 @@ extern "C" int syn_op_linear_as(const void* x, const void* w, float* y, int32_t 
         if (!launch_ok()) return SYN_E_CUDA;
         CU_OK(cudaStreamSynchronize(st));   // the GEMM requests weight tiles before it waits for its predecessor
         g_lin.packed_src = w; g_lin.packed_n = N; g_lin.packed_k = K;
+        if ((r = make_wmaps(g_lin.packed, n_mt * 128, K, &g_lin.wm))) return r;
     }
     CUtensorMap tmB;
     if ((r = make_map_2d(&tmB, x, T, K, K, GEMM_BOX_ROWS))) return r;
     EpiParams e;
     memset(&e, 0, sizeof(e));
     e.mode = EPI_PLAIN; e.T = T; e.N = N; e.y = y; e.ldy = N;
-    r = launch_gemm(nullptr, -1, g_lin.n_sm, g_lin.status, g_lin.packed, n_mt * 128, K, tmB, e, st, g_lin.fix_part, g_lin.fix_flag,
-                    schedule_as);
+    // 0..4: the schedule the step would take for that epilogue; 5, 6: CTA pairs with QUAD / DUO items; 7, 8: the
+    // same as residual projections (K shared between clusters where the shape allows it)
+    const int force = schedule_as <= EPI_LMHEAD ? PAIR_NONE : (schedule_as == 5 || schedule_as == 7 ? PAIR_QUAD : PAIR_DUO);
+    const int plan_mode = schedule_as <= EPI_LMHEAD ? schedule_as : (schedule_as >= 7 ? EPI_RESID : EPI_PLAIN);
+    r = launch_proj(nullptr, -1, g_lin.n_sm, g_lin.status, g_lin.packed, &g_lin.wm, (N + 127) / 128 * 128, K, tmB, e, st, g_lin.fix_part,
+                    g_lin.fix_flag, plan_mode, force);
     if (r) return r;
     CU_OK(cudaStreamSynchronize(st));
     int sflag = 0;
     CU_OK(cudaMemcpy(&sflag, g_lin.status, 4, cudaMemcpyDeviceToHost));
     if (sflag) {
         cudaMemset(g_lin.status, 0, 4);
-        cudaMemset(g_lin.fix_flag, 0, (size_t)2 * g_lin.n_sm * 4);
+        cudaMemset(g_lin.fix_flag, 0, (size_t)GEMM_FLAG_INTS * g_lin.n_sm * 4);
         return SYN_E_DEVICE_TIMEOUT;
     }
     return SYN_OK;
@@ -1526,10 +1662,16 @@ extern "C" int syn_debug_set_spin_limit(int64_t cycles) {
     return SYN_OK;
 }
 
+extern "C" int syn_debug_set_schedule(int32_t which) {
+    if (which < 0 || which > 1) return SYN_E_INVALID_ARG;
+    g_schedule = which;
+    return SYN_OK;
+}
+
 extern "C" int syn_debug_linear_counter(int32_t index, int32_t value) {
     int r = linear_ctx_init();
     if (r) return r;
-    if (index < 0 || index >= 2 * g_lin.n_sm) return SYN_E_INVALID_ARG;
+    if (index < 0 || index >= GEMM_FLAG_INTS * g_lin.n_sm) return SYN_E_INVALID_ARG;
     CU_OK(cudaDeviceSynchronize());
     CU_OK(cudaMemcpy(g_lin.fix_flag + index, &value, 4, cudaMemcpyHostToDevice));
     return SYN_OK;

@@ -54,9 +54,10 @@ def bench_linear(a):
     key = rng.stream_key(0, 1234)
     x = rng.normal_f32(key, 0, a.T * a.K, 1.0, device="cuda").view(a.T, a.K).to(torch.bfloat16)
     w = rng.normal_f32(key, a.T * a.K, a.N * a.K, 0.02, device="cuda").view(a.N, a.K).to(torch.bfloat16)
-    med, best = _time(lambda: syn.syn_op_linear(x, w), a.iters)
+    syn.syn_op_linear(x, w, schedule_as=a.sched)
+    med, best = _time(lambda: syn.syn_op_linear(x, w, schedule_as=a.sched, reuse_pack=True), a.iters)
     fl = 2.0 * a.T * a.N * a.K
-    print(json.dumps({"op": "linear", "T": a.T, "N": a.N, "K": a.K, "ms_median": med, "ms_best": best,
+    print(json.dumps({"op": "linear", "sched": a.sched, "T": a.T, "N": a.N, "K": a.K, "ms_median": med, "ms_best": best,
                       "tflops": fl / med / 1e9, "weight_gbs": 2.0 * a.N * a.K / med / 1e6,
                       "note": "includes the fp32 [T][N] store of the test epilogue and a stream sync per call"}))
 
@@ -290,6 +291,7 @@ def main():
     l.add_argument("--N", type=int, default=28672)
     l.add_argument("--K", type=int, default=4096)
     l.add_argument("--iters", type=int, default=10)
+    l.add_argument("--sched", default="plain", help="schedule: plain, qkv, resid, swiglu, lmhead, pair_quad, pair_duo, pair_quad_resid, pair_duo_resid")
     t = sub.add_parser("attention")
     t.add_argument("--config", type=int, default=3)
     t.add_argument("--pool-tokens", type=int, default=None)

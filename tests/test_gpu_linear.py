@@ -55,8 +55,18 @@ def test_linear_matches_oracle(T, N, K):
     (50, 300, 1024, "resid"),      # ragged tokens and features, four parts of four k-blocks
     (17, 256, 2048, "resid"),      # two chunks among eight CTAs: most of them keep no column
     (1194, 5120, 1024, "resid"),   # 100 pair tiles: K not shared, seven narrower token tiles instead
-    (544, 28672, 4096, "swiglu"),  # schedule of the gate/up projection (leftover tiles cut along K)
+    (544, 28672, 4096, "swiglu"),  # schedule of the gate/up projection
     (300, 38144, 1024, "lmhead"),
+    # the CTA-pair kernel (clusters of two share a token tile)
+    (544, 28672, 4096, "pair_quad"),       # 56 x 3 items of 512 features on 74 clusters: 2.3 waves
+    (544, 6144, 4096, "pair_duo"),         # 24 x 3 items of 256 features, two k-interleaved accumulators per CTA
+    (544, 4096, 4096, "pair_duo"),         # 48 clusters
+    (544, 4096, 14336, "pair_quad_resid"), # 24 items, K shared by three clusters each: exchange between CTAs of equal rank
+    (300, 1280, 1024, "pair_quad"),        # five feature pairs: the last cluster's second pair is all padding; 160-token tiles
+    (1194, 7168, 5120, "pair_quad"),       # five token tiles of 240, the last with 234 tokens
+    (921, 4096, 512, "pair_duo_resid"),    # 64 items, no room to share K
+    (257, 640, 2048, "pair_duo_resid"),    # token tiles of 144 and 113; 6 items, K shared by four clusters each
+    (40, 512, 256, "pair_quad"),           # one item, a 48-token tile: halves of 24 rows
 ])
 def test_every_schedule_of_the_step_gives_the_plain_product(T, N, K, sched):
     """The work decompositions the step uses for its projections (K shared between CTAs with a
@@ -85,24 +95,26 @@ def test_a_new_matrix_at_an_old_address_is_packed_again():
     assert torch.allclose(y2, 2 * y1)
 
 
-def test_a_wait_that_cannot_end_runs_out_and_the_next_call_works():
+@pytest.mark.parametrize("T,N,K,sched", [
+    (129, 2048, 2048, "resid"),              # one-CTA kernel: tile 0's eight CTAs wait for 128 arrivals
+    (544, 4096, 14336, "pair_quad_resid"),   # CTA-pair kernel: the rank-0 CTAs of tile 0's three clusters wait for 48
+])
+def test_a_wait_that_cannot_end_runs_out_and_the_next_call_works(T, N, K, sched):
     """SYN_E_DEVICE_TIMEOUT end to end: an arrival counter of the reduce-scatter is set so far below
     zero that the count its readers wait for cannot be reached; with the waits' limit shortened to a
     fraction of a millisecond they give up, the kernel ends normally, the call reports the timeout and
     clears the counters, and the same call then succeeds with the right result."""
     import paper_2511_07423_b200 as syn
-    T, N, K = 544, 4096, 4096
-    assert syn.gemm_plan_host(T, N, K, "resid")["splits"] == 3
     x, w = _case(T, N, K, 77)
     xc, wc = x.cuda(), w.cuda()
-    good = syn.syn_op_linear(xc, wc, schedule_as="resid")
+    good = syn.syn_op_linear(xc, wc, schedule_as=sched)
     try:
         syn.debug_set_spin_limit(400_000)
-        syn.debug_linear_counter(0, -1_000_000)    # tile 0: its three CTAs wait for 48 arrivals
+        syn.debug_linear_counter(0, -1_000_000)
         with pytest.raises(syn.SynError) as ei:
-            syn.syn_op_linear(xc, wc, schedule_as="resid", reuse_pack=True)
+            syn.syn_op_linear(xc, wc, schedule_as=sched, reuse_pack=True)
         assert ei.value.code == -11
     finally:
         syn.debug_set_spin_limit(0)
-    again = syn.syn_op_linear(xc, wc, schedule_as="resid", reuse_pack=True)
+    again = syn.syn_op_linear(xc, wc, schedule_as=sched, reuse_pack=True)
     assert torch.equal(again, good)
