@@ -21,6 +21,11 @@
  *     cudaMalloc on the current device; it does not link or call PyTorch.
  *   - Matrices are bf16, row-major [out_features][in_features] (y = x W^T); RMSNorm gains are
  *     bf16 [d_model].  There are no biases.
+ *   - Arithmetic: every matrix product takes IEEE half-precision operands and accumulates in fp32; the
+ *     residual stream, the softmax statistics and the logits are fp32.  The library's packed copy of the
+ *     bf16 weights is half precision: a bf16 value of magnitude >= 2^-17 converts exactly, smaller ones
+ *     round to a multiple of 2^-24.  Activations and the cached K and V are half precision too (11
+ *     significant bits; bf16 would keep 8), clamped to +-65504 where bf16 would have had the range.
  */
 #ifndef SYNERA_H_
 #define SYNERA_H_
@@ -103,7 +108,8 @@ void syn_kv_free(syn_kv *kv);
 
 /* Place externally produced (already rotated) K and V of one request and one layer at logical
  * positions pos0 .. pos0+n_pos-1, e.g. a prefix computed on another server.  k, v: DEVICE bf16
- * [n_pos][n_kv_heads][head_dim]; page_table: HOST int32, at least ceil((pos0+n_pos)/page_size)
+ * [n_pos][n_kv_heads][head_dim] (the pool itself holds half precision: import converts, exactly for
+ * magnitudes in [2^-17, 65504], export rounds back to bf16); page_table: HOST int32, at least ceil((pos0+n_pos)/page_size)
  * entries.  Blocking: the call allocates a small device buffer for the slot list, synchronises
  * `cuda_stream` and returns when the copy is done.
  * syn_kv_export is the inverse (reads the same positions into k, v).
@@ -223,7 +229,7 @@ const char *syn_last_cuda_error(void);
 
 /* ---- single operations, exported for per-kernel tests and roofline measurements ------- */
 
-/* y[T][N] (fp32, DEVICE) = x[T][K] (bf16, DEVICE) * W[N][K]^T (bf16, DEVICE): the tcgen05
+/* y[T][N] (fp32, DEVICE) = x[T][K] (half precision, DEVICE) * W[N][K]^T (bf16, DEVICE): the tcgen05
  * GEMM used by every projection, with a plain store epilogue.  The first call with a given w
  * (pointer and shape) packs it into the library's tiled layout; later calls reuse the packed copy:
  * call syn_op_linear_reset after the contents of w changed or w was freed (a new matrix may land at
@@ -255,8 +261,8 @@ int syn_debug_linear_counter(int32_t index, int32_t value);
 int syn_debug_set_schedule(int32_t which);
 
 /* The ragged paged attention of the step on its own (paper Sec. 3.2 attention equation over a
- * paged cache).  q: DEVICE bf16 [T][n_q_heads*head_dim] (rotated); out: DEVICE bf16, same
- * shape.  The plan supplies page tables, lengths and the work list; the chunk's K/V must
+ * paged cache).  q: DEVICE half precision [T][n_q_heads*head_dim] (rotated); out: DEVICE half
+ * precision, same shape.  The plan supplies page tables, lengths and the work list; the chunk's K/V must
  * already be in the pool of `layer`.  Asynchronous on cuda_stream. */
 int syn_op_attention(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer, const void *q, void *out,
                      void *cuda_stream);
@@ -296,6 +302,22 @@ int syn_op_attention_static(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_
 int syn_gemm_plan_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t *out);
 int syn_gemm_work_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t cta, int32_t i,
                        int32_t *out);
+
+/* The same for the CTA-pair kernel that serves projections of 256 tokens and more: clusters of two CTAs
+ * share a token tile.  syn_gemm2_plan_host fills out[SYN_GEMM2_PLAN_FIELDS] = {item shape (0: the shape
+ * stays on the one-CTA kernel, 1: items of 512 features, 2: items of 256 features), feature groups of that
+ * size, token tiles, tokens per tile, k-blocks of 64, clusters, clusters that share a tile's K range
+ * (reduce-scatter; 1: none), k-blocks of each, and, for the items left after the full waves, the number of
+ * K parts each is cut into (0: not cut) and how many of them get one part more}.  `force`: 0, or 1 / 2 to
+ * take that item shape whatever the size.  syn_gemm2_work_host returns 1 and fills
+ * out[SYN_GEMM2_WORK_FIELDS] = {feature group, token tile, first k-block, one past the last, tile index,
+ * K part, K parts of the tile, cluster of part 0, counter index} for work item i of a cluster, 0 when it
+ * has no item i.  Errors: SYN_E_INVALID_ARG. */
+#define SYN_GEMM2_PLAN_FIELDS 10
+#define SYN_GEMM2_WORK_FIELDS 9
+int syn_gemm2_plan_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t force, int32_t *out);
+int syn_gemm2_work_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t force, int32_t cluster,
+                        int32_t i, int32_t *out);
 
 /* Sampling-based verification (paper Sec. 4.2, "Compression before transmission": for
  * verification the LLM needs the drafts and the SLM's distributions, of which the device sends

@@ -61,7 +61,7 @@ EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "s
            "syn_op_linear_as", "syn_op_linear_reset", "syn_debug_set_spin_limit", "syn_debug_linear_counter", "syn_debug_set_schedule",
            "syn_op_attention", "syn_op_attention_static",
            "syn_set_profile", "syn_get_profile", "syn_verify_batch_sampled", "syn_op_sample_verify",
-           "syn_gemm_plan_host", "syn_gemm_work_host"]
+           "syn_gemm_plan_host", "syn_gemm_work_host", "syn_gemm2_plan_host", "syn_gemm2_work_host"]
 SCHED_EXPORTS = ["syn_sched_create", "syn_sched_free", "syn_sched_add_request", "syn_sched_add_verify", "syn_sched_finish",
                  "syn_sched_peek", "syn_sched_commit", "syn_sched_step", "syn_sched_get_stats"]
 
@@ -210,15 +210,16 @@ class KVCache:
 
     # -------------------------------------------------------------- the step
     def verify_batch(self, chunk_tokens, chunk_offsets, page_tables, ctx_lens, n_uncached=None,
-                     want_logits: bool = False, req_ids=None, stream=None):
-        """syn_verify_batch with HOST metadata.  Returns (accept_len, correction_token[, logits])."""
+                     want_logits: bool = False, req_ids=None, stream=None, out=None):
+        """syn_verify_batch with HOST metadata.  Returns (accept_len, correction_token[, logits]).
+        `out`: optional pair of int32 CPU tensors [n_req] to receive the results."""
         tok, off, ctx = _i32(chunk_tokens), _i32(chunk_offsets), _i32(ctx_lens)
         pt = _i32(page_tables)
         assert pt.dim() == 2
         n_req = ctx.numel()
         unc = _i32(n_uncached) if n_uncached is not None else None
-        acc = torch.empty(n_req, dtype=torch.int32)
-        cor = torch.empty(n_req, dtype=torch.int32)
+        acc, cor = out if out is not None else (torch.empty(n_req, dtype=torch.int32), torch.empty(n_req, dtype=torch.int32))
+        assert acc.dtype == torch.int32 and cor.dtype == torch.int32 and not acc.is_cuda and acc.numel() >= n_req
         logits = None
         if want_logits:
             logits = torch.empty(int(off[-1]), self.model.shape.vocab, dtype=torch.float32, device="cuda")
@@ -308,7 +309,8 @@ class Plan:
             C.c_void_p(logits.data_ptr()) if logits is not None else None, _stream_ptr(stream)), "syn_verify_run")
 
     def attention(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-        assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        """syn_op_attention: q and the result are half precision [T, n_q_heads * head_dim]."""
+        assert q.is_cuda and q.dtype == torch.float16 and q.is_contiguous()
         if out is None:
             out = torch.empty_like(q)
         _check(self._lib.syn_op_attention(self.kv.model._h, self.kv._h, self._h, C.c_uint32(layer),
@@ -320,7 +322,7 @@ class Plan:
         """syn_op_attention_static: the attention of the step for callers that cannot allocate while
         they run; its partial results live in a fixed array inside the library.  Pass `out` to keep
         the call itself free of allocations on the Python side too."""
-        assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous()
+        assert q.is_cuda and q.dtype == torch.float16 and q.is_contiguous()
         if out is None:
             out = torch.empty_like(q)
         _check(self._lib.syn_op_attention_static(self.kv.model._h, self.kv._h, self._h, C.c_uint32(layer),
@@ -518,13 +520,39 @@ def gemm_work_host(T: int, N: int, K: int, epilogue: str, cta: int, i: int, n_sm
     return dict(zip(GEMM_WORK_FIELDS, out)) if r == 1 else None
 
 
+GEMM2_PLAN_FIELDS = ("kind", "n_groups", "n_tt", "TN", "num_kb", "n_clusters", "splits", "kb_per_split", "rem_base", "rem_extra")
+GEMM2_WORK_FIELDS = ("grp", "tt", "kb0", "kb1", "tile", "split", "nsplit", "first_cl", "counter")
+GEMM2_KINDS = {"auto": 0, "quad": 1, "duo": 2}
+
+
+def gemm2_plan_host(T: int, N: int, K: int, epilogue: str, force: str = "auto", n_sm: int = 148) -> Dict[str, int]:
+    """syn_gemm2_plan_host: the launch shape of one projection on CTA pairs, without a device."""
+    out = (C.c_int32 * len(GEMM2_PLAN_FIELDS))()
+    _check(load_library().syn_gemm2_plan_host(C.c_int32(T), C.c_int32(N), C.c_int32(K), C.c_int32(n_sm),
+                                              C.c_int32(GEMM_EPILOGUES[epilogue]), C.c_int32(GEMM2_KINDS[force]), out),
+           "syn_gemm2_plan_host")
+    return dict(zip(GEMM2_PLAN_FIELDS, out))
+
+
+def gemm2_work_host(T: int, N: int, K: int, epilogue: str, cluster: int, i: int, force: str = "auto",
+                    n_sm: int = 148) -> Optional[Dict[str, int]]:
+    """syn_gemm2_work_host: work item i of a cluster, or None."""
+    out = (C.c_int32 * len(GEMM2_WORK_FIELDS))()
+    r = load_library().syn_gemm2_work_host(C.c_int32(T), C.c_int32(N), C.c_int32(K), C.c_int32(n_sm),
+                                           C.c_int32(GEMM_EPILOGUES[epilogue]), C.c_int32(GEMM2_KINDS[force]),
+                                           C.c_int32(cluster), C.c_int32(i), out)
+    if r < 0:
+        _check(r, "syn_gemm2_work_host")
+    return dict(zip(GEMM2_WORK_FIELDS, out)) if r == 1 else None
+
+
 def syn_op_linear(x: torch.Tensor, w: torch.Tensor, stream=None, schedule_as: str = "plain",
                   reuse_pack: bool = False) -> torch.Tensor:
-    """y[T, N] fp32 = x[T, K] bf16 @ w[N, K]^T bf16 through the library's tcgen05 GEMM, under the
+    """y[T, N] fp32 = x[T, K] half @ w[N, K]^T bf16 through the library's tcgen05 GEMM, under the
     schedule the step uses for the projection with epilogue `schedule_as`.  The library keeps a packed
     copy of the last w keyed by address and shape; unless `reuse_pack` says the matrix is the one of the
     previous call, the copy is dropped first (a new tensor may sit at a freed tensor's address)."""
-    assert x.is_cuda and w.is_cuda and x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
+    assert x.is_cuda and w.is_cuda and x.dtype == torch.float16 and w.dtype == torch.bfloat16
     x, w = x.contiguous(), w.contiguous()
     T, K = x.shape
     N = w.shape[0]

@@ -10,7 +10,7 @@
 // current one is in flight (its warpgroup gives most of its registers to the consumers).  Eight consumer warps form two groups that take alternate stages, so
 // every scheduler of the SM holds two warps; inside a group the four warps split the item's row
 // tiles and, when there are fewer than four row tiles, the pages of the stage.  QK^T and PV run on
-// warp-level MMAs (m16n8k16, bf16 in, fp32 accumulate) with an online softmax in fp32 (base 2).
+// warp-level MMAs (m16n8k16, half-precision operands, fp32 accumulate) with an online softmax in fp32 (base 2).
 // The (max, sum, O) triples of the warps that share a row tile are merged in shared memory in a
 // fixed order.  An item that covers only part of a request's keys writes an fp32 partial; the CTA
 // that completes the last partial of a row group (a counter per group, reset by that CTA) combines
@@ -48,7 +48,7 @@ struct AttnParams {
     int q_box_tokens;           // tokens of the Q tile's TMA box: min(16, 64 / G)
     int layer_block0;           // 2 * layer * n_pages * Hkv: first (K|V) block of this layer in the pool map
     float scale_log2;           // log2(e) / sqrt(hd)
-    __nv_bfloat16* out;         // [T][q_dim]
+    op16* out;                  // [T][q_dim]
     float* part_o;              // [n_parts][64][hd]
     float2* part_ml;            // [n_parts][64] (max in log2 units, sum)
     const MergeGroup* groups;   // [n_groups]
@@ -129,8 +129,8 @@ __device__ __forceinline__ void attn_consume_stage(const uint8_t* stage, int fir
                 if (FULL || first_page + pg < n_valid_pages) {
                     uint32_t b0, b1, b2, b3;
                     ldsm_x4(page0 + pg * PAGE_BYTES + off, b0, b1, b2, b3);
-                    mma_bf16_16816(acc[ks % KSPLIT][pg * 2], qf[ks], b0, b1);
-                    mma_bf16_16816(acc[ks % KSPLIT][pg * 2 + 1], qf[ks], b2, b3);
+                    mma_f16_16816(acc[ks % KSPLIT][pg * 2], qf[ks], b0, b1);
+                    mma_f16_16816(acc[ks % KSPLIT][pg * 2 + 1], qf[ks], b2, b3);
                 }
             }
         }
@@ -206,10 +206,10 @@ __device__ __forceinline__ void attn_consume_stage(const uint8_t* stage, int fir
                 const float p13 = ex2_approx(fmaf(s[pg * 2 + 1][3], scale_log2, -base[1]));
                 l[0] += (p00 + p01) + (p10 + p11);
                 l[1] += (p02 + p03) + (p12 + p13);
-                pa[0] = pack_bf16(p00, p01);
-                pa[1] = pack_bf16(p02, p03);
-                pa[2] = pack_bf16(p10, p11);
-                pa[3] = pack_bf16(p12, p13);
+                pa[0] = pack_op(p00, p01);
+                pa[1] = pack_op(p02, p03);
+                pa[2] = pack_op(p10, p11);
+                pa[3] = pack_op(p12, p13);
             }
             const uint32_t vb = page0 + pg * PAGE_BYTES + 2048;  // V rows follow the K rows
 #pragma unroll
@@ -217,8 +217,8 @@ __device__ __forceinline__ void attn_consume_stage(const uint8_t* stage, int fir
                 const int ch = 2 * np + (mi >> 1);
                 uint32_t b0, b1, b2, b3;
                 ldsm_x4_t(vb + (uint32_t)(ch >> 3) * 4096u + swz(tokv, ch & 7), b0, b1, b2, b3);
-                mma_bf16_16816(o[2 * np], pa, b0, b1);
-                mma_bf16_16816(o[2 * np + 1], pa, b2, b3);
+                mma_f16_16816(o[2 * np], pa, b0, b1);
+                mma_f16_16816(o[2 * np + 1], pa, b2, b3);
             }
         }
     }
@@ -449,7 +449,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 if (kg == 0)
                     for (int k2 = 1; k2 < 4 / npw; ++k2) attn_fold_slot<HD>(merge + (k2 * npw + mt) * 16 * (HD + 4), o, m, l, g, c);
             }
-            // write: final output (bf16) or fp32 partial
+            // write: final output (half precision) or fp32 partial
             if (active && kg == 0 && ok) {
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
@@ -458,11 +458,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                         const int j = row / G, gq = row - j * G;
                         if (item.part < 0) {
                             const float inv = l[r] > 0.f ? 1.f / l[r] : 0.f;
-                            __nv_bfloat16* dst = p.out + (size_t)(item.q_tok + j) * p.q_dim + (item.kvh * G + gq) * HD;
+                            op16* dst = p.out + (size_t)(item.q_tok + j) * p.q_dim + (item.kvh * G + gq) * HD;
 #pragma unroll
                             for (int nt = 0; nt < HD / 8; ++nt)
                                 *reinterpret_cast<uint32_t*>(dst + nt * 8 + 2 * c) =
-                                    pack_bf16(o[nt][2 * r] * inv, o[nt][2 * r + 1] * inv);
+                                    pack_op(o[nt][2 * r] * inv, o[nt][2 * r + 1] * inv);
                         } else {
                             float* dst = p.part_o + ((size_t)item.part * 64 + row) * HD;
 #pragma unroll
@@ -516,7 +516,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     uint2* dst = reinterpret_cast<uint2*>(p.out + (size_t)(gr.q_tok + j) * p.q_dim + (gr.kvh * G + gq) * HD + c0);
 #pragma unroll
                     for (int i = 0; i < CW / 4; ++i)
-                        dst[i] = make_uint2(pack_bf16(acc[i].x * inv, acc[i].y * inv), pack_bf16(acc[i].z * inv, acc[i].w * inv));
+                        dst[i] = make_uint2(pack_op(acc[i].x * inv, acc[i].y * inv), pack_op(acc[i].z * inv, acc[i].w * inv));
                 }
             }
         }

@@ -51,10 +51,10 @@ struct EpiParams {
     float* y;
     int ldy;
     // QKV
-    __nv_bfloat16* q;
+    op16* q;
     int q_dim, kv_dim, hd, n_kv_heads, page_size;
     const float2* rope;  // [T][hd/2] (cos, sin)
-    __nv_bfloat16* pool; // this layer's pool: [page][kvh][K|V][row][hd]
+    op16* pool;          // this layer's pool: [page][kvh][K|V][row][hd]
     const int* slot;     // [T] page * page_size + row
     // RMSNorm scale of the token operand (QKV, SWIGLU, LMHEAD; NULL: the operand is used as it is)
     const float* ssq_in; // [T][n_ssq] partial sums of x^2 of the operand's source rows
@@ -63,11 +63,11 @@ struct EpiParams {
     // RESID
     float* x;            // [T][d] residual stream, updated in place
     const __nv_bfloat16* gain;   // [d] gain of the NEXT RMSNorm
-    __nv_bfloat16* xg;   // [T][d] bf16(x * gain): the next projection's operand
+    op16* xg;            // [T][d] half(x * gain): the next projection's operand
     float* ssq_out;      // [T][d / 32]
     int d;
     // SWIGLU
-    __nv_bfloat16* act;
+    op16* act;
     int f_pad;
     // LMHEAD
     float* logits;
@@ -113,7 +113,7 @@ constexpr int EPI_COLS = 16;
 constexpr int EPI_SCR_STRIDE = 33;
 constexpr int EPI_SCR_FLOATS = EPI_COLS * EPI_SCR_STRIDE;   // per epilogue warp
 
-__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) { return make_uint2(pack_bf16(a, b), pack_bf16(c, d)); }
+__device__ __forceinline__ uint2 pack4_op(float a, float b, float c, float d) { return make_uint2(pack_op(a, b), pack_op(c, d)); }
 
 template <int MODE>
 __device__ __forceinline__ void epi_unit(const EpiParams& p, const float (&a)[EPI_COLS], float* scr, int m0, int t0, int ncols,
@@ -161,7 +161,7 @@ __device__ __forceinline__ void epi_unit(const EpiParams& p, const float (&a)[EP
             if (tv) {
                 const size_t at = (size_t)(t0 + t) * p.d + f;
                 *reinterpret_cast<float4*>(p.x + at) = nx;
-                *reinterpret_cast<uint2*>(p.xg + at) = pack4_bf16(nx.x * __low2float(g01), nx.y * __high2float(g01),
+                *reinterpret_cast<uint2*>(p.xg + at) = pack4_op(nx.x * __low2float(g01), nx.y * __high2float(g01),
                                                                   nx.z * __low2float(g23), nx.w * __high2float(g23));
             }
             ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);   // the eight lanes of the token, a fixed order
@@ -203,10 +203,10 @@ __device__ __forceinline__ void epi_unit(const EpiParams& p, const float (&a)[EP
                 const float o3 = mine[3] * w[i][1].z + sg * part[3] * w[i][1].w;
                 const int sl = __shfl_sync(0xFFFFFFFFu, my_slot, t);
                 if (t < ncols) {
-                    __nv_bfloat16* dst;
+                    op16* dst;
                     if (which == 0) dst = p.q + (size_t)(t0 + t) * p.q_dim + fhead;
                     else dst = p.pool + (size_t)(sl >> 4) * page_stride + ((size_t)(fhead / p.hd) * 2) * 16 * p.hd + (size_t)(sl & 15) * p.hd;
-                    *reinterpret_cast<uint2*>(dst + dim + (hi ? half : 0)) = pack4_bf16(o0, o1, o2, o3);
+                    *reinterpret_cast<uint2*>(dst + dim + (hi ? half : 0)) = pack4_op(o0, o1, o2, o3);
                 }
             }
         } else {
@@ -218,9 +218,9 @@ __device__ __forceinline__ void epi_unit(const EpiParams& p, const float (&a)[EP
                 const float* row = scr + t * EPI_SCR_STRIDE + c0;
                 const int sl = __shfl_sync(0xFFFFFFFFu, my_slot, t);
                 if (t < ncols) {
-                    __nv_bfloat16* dst = p.pool + (size_t)(sl >> 4) * page_stride + ((size_t)(fr / p.hd) * 2 + 1) * 16 * p.hd +
+                    op16* dst = p.pool + (size_t)(sl >> 4) * page_stride + ((size_t)(fr / p.hd) * 2 + 1) * 16 * p.hd +
                                          (size_t)(sl & 15) * p.hd + (fr & (p.hd - 1));
-                    *reinterpret_cast<uint2*>(dst) = pack4_bf16(row[0], row[1], row[2], row[3]);
+                    *reinterpret_cast<uint2*>(dst) = pack4_op(row[0], row[1], row[2], row[3]);
                 }
             }
         }
@@ -236,7 +236,7 @@ __device__ __forceinline__ void epi_unit(const EpiParams& p, const float (&a)[EP
 #pragma unroll
             for (int k = 0; k < 4; ++k) h[k] = __fdividef(row[k], 1.0f + __expf(-row[k])) * row[16 + k];
             if (t < ncols)
-                *reinterpret_cast<uint2*>(p.act + (size_t)(t0 + t) * p.f_pad + (m0 >> 1) + 16 * quarter + g0) = pack4_bf16(h[0], h[1], h[2], h[3]);
+                *reinterpret_cast<uint2*>(p.act + (size_t)(t0 + t) * p.f_pad + (m0 >> 1) + 16 * quarter + g0) = pack4_op(h[0], h[1], h[2], h[3]);
         }
     } else {  // EPI_LMHEAD
         const int f = m0 + quarter * 32 + c0;
@@ -330,9 +330,9 @@ struct PackSrc {
     int hd;      // mode 2: head dimension
 };
 
-__global__ void pack_weight_kernel(PackSrc src, __nv_bfloat16* __restrict__ out, int num_kb) {
+__global__ void pack_weight_kernel(PackSrc src, op16* __restrict__ out, int num_kb) {
     const int mtile = blockIdx.x, kb = blockIdx.y;
-    __nv_bfloat16* tile = out + (((size_t)(mtile >> 1) * num_kb + kb) * 2 + (mtile & 1)) * (128 * 64);
+    op16* tile = out + (((size_t)(mtile >> 1) * num_kb + kb) * 2 + (mtile & 1)) * (128 * 64);
     for (int i = threadIdx.x; i < 128 * 8; i += blockDim.x) {
         const int r = i >> 3, c = i & 7;
         const __nv_bfloat16* row = nullptr;
@@ -354,13 +354,15 @@ __global__ void pack_weight_kernel(PackSrc src, __nv_bfloat16* __restrict__ out,
         uint4 v = make_uint4(0, 0, 0, 0);
         const int col = kb * 64 + c * 8;
         if (row) {
+            __nv_bfloat16 tmp[8];
             if (col + 8 <= src.src_k && (((uintptr_t)(row + col)) & 15) == 0) {
-                v = *reinterpret_cast<const uint4*>(row + col);
+                *reinterpret_cast<uint4*>(tmp) = *reinterpret_cast<const uint4*>(row + col);
             } else {
-                __nv_bfloat16 tmp[8];
                 for (int e = 0; e < 8; ++e) tmp[e] = col + e < src.src_k ? row[col + e] : __float2bfloat16(0.f);
-                v = *reinterpret_cast<uint4*>(tmp);
             }
+            // bf16 -> half: exact for every weight of magnitude >= 2^-17
+            v = make_uint4(pack_op(__bfloat162float(tmp[0]), __bfloat162float(tmp[1])), pack_op(__bfloat162float(tmp[2]), __bfloat162float(tmp[3])),
+                           pack_op(__bfloat162float(tmp[4]), __bfloat162float(tmp[5])), pack_op(__bfloat162float(tmp[6]), __bfloat162float(tmp[7])));
         }
         *reinterpret_cast<uint4*>(tile + r * 64 + ((c ^ (r & 7)) << 3)) = v;
     }
@@ -394,7 +396,7 @@ __host__ inline int gemm_stages(int TN) {
 }
 
 struct GemmParams {
-    const __nv_bfloat16* w;     // packed weights
+    const op16* w;              // packed weights
     int num_kb;                 // k-blocks of 64
     int n_pairs;                // 256-feature pairs
     int n_tt, TN;               // token tiles of TN columns (multiple of 16, <= 256)
@@ -576,7 +578,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
                 const int n0 = w.tt * g.TN;
                 const int nbox = (((min(g.TN, p.T - n0) + 15) & ~15) + 31) >> 5;
                 const uint32_t a_bytes = (uint32_t)(w.mt_hi - w.mt_lo) * GEMM_TILE_BYTES;
-                const __nv_bfloat16* wsrc = g.w + ((size_t)w.pair * g.num_kb) * (2 * 128 * 64) + (size_t)w.mt_lo * (128 * 64);
+                const op16* wsrc = g.w + ((size_t)w.pair * g.num_kb) * (2 * 128 * 64) + (size_t)w.mt_lo * (128 * 64);
                 const int nk = w.kb1 - w.kb0, rot = gemm_k_rotation(cta, n_cta, nk);
                 // The weights never depend on an earlier kernel: the first item's weight tiles of the
                 // whole ring are requested before waiting for the predecessor, whose output is only the
@@ -616,7 +618,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmB, GemmParams g, EpiParams p) 
             GemmWork w;
             for (int i = 0; ok && gemm_work<KSPLIT>(g, cta, n_cta, i, w); ++i) {
                 const uint32_t nn = (uint32_t)((min(g.TN, p.T - w.tt * g.TN) + 15) & ~15);
-                const uint32_t idesc = umma_idesc_bf16(128, nn);
+                const uint32_t idesc = umma_idesc_f16(128, nn);
                 if (i > 0) {   // the epilogue must have drained the previous item's accumulators
                     ok = mbar_wait(acce_bar, (i - 1) & 1, g.status, limit);
                     if (!ok) break;

@@ -190,7 +190,7 @@ gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             Gemm2Work w;
             for (int i = 0; ok && gemm2_work(g, cl, n_cl, i, w); ++i) {
                 const uint32_t nn = (uint32_t)((min(g.TN, p.T - w.tt * g.TN) + 15) & ~15);
-                const uint32_t idesc = umma_idesc_bf16(256, nn);
+                const uint32_t idesc = umma_idesc_f16(256, nn);
                 if (i > 0) {   // the epilogues of both CTAs must have drained the previous item's accumulators
                     ok = mbar_wait(acce_bar, (i - 1) & 1, g.status, limit);
                     if (!ok) break;

@@ -6,6 +6,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 
 namespace syn {
@@ -133,10 +134,10 @@ __device__ __forceinline__ uint64_t umma_desc_k128(uint32_t saddr) {
     return d;
 }
 
-// Instruction descriptor, kind::f16: D fp32 (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
-// both K-major (bits 15, 16 = 0), N >> 3 at bit 17, M >> 4 at bit 24.
-__host__ __device__ __forceinline__ uint32_t umma_idesc_bf16(uint32_t M, uint32_t N) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+// Instruction descriptor, kind::f16: D fp32 (bits 4-5 = 1), A and B IEEE half (bits 7-9, 10-12 = 0;
+// 1 would be bf16), both K-major (bits 15, 16 = 0), N >> 3 at bit 17, M >> 4 at bit 24.
+__host__ __device__ __forceinline__ uint32_t umma_idesc_f16(uint32_t M, uint32_t N) {
+    return (1u << 4) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
 // D[tmem] (+)= A[smem] * B[smem]; one thread issues.
@@ -251,17 +252,31 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& a, uint32_t& 
                  : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
                  : "r"(addr));
 }
-// D (fp32 m16n8) += A (bf16 m16k16, row) * B (bf16 k16n8, col)
-__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+// D (fp32 m16n8) += A (half m16k16, row) * B (half k16n8, col)
+__device__ __forceinline__ void mma_f16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
+// ---------------------------------------------------------------- operand precision
+// The operands of every matrix product (packed weights, activations, the cached K and V) are IEEE
+// half precision, accumulation is fp32.  The model's bf16 weights convert without loss (a bf16 value
+// of magnitude >= 2^-17 is a half value; smaller ones round to a multiple of 2^-24, an error far
+// below one part in a million of any weight that matters), and an activation keeps 11 significant
+// bits where bf16 would keep 8, which is what lets a deep stack stay within a few hundredths of the
+// logits' standard deviation of an exact evaluation.  Half has less range than bf16: conversions
+// saturate at +-65504 instead of overflowing to infinity.
+typedef __half op16;
+__device__ __forceinline__ uint32_t pack_op(float lo, float hi) {   // two values -> one 32-bit word, `lo` in the low half
+    uint32_t r;
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ op16 to_op(float v) {
+    const uint32_t r = pack_op(v, 0.f);
+    return __ushort_as_half((unsigned short)(r & 0xFFFFu));
 }
 
 }  // namespace syn

@@ -89,7 +89,7 @@ static cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 __global__ void __launch_bounds__(256)
 prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens, const int* __restrict__ pos,
             const bf16* __restrict__ gain, const double* __restrict__ inv_freq, float* __restrict__ x,
-            bf16* __restrict__ xg, float* __restrict__ ssq, float2* __restrict__ rope, unsigned long long* __restrict__ best,
+            op16* __restrict__ xg, float* __restrict__ ssq, float2* __restrict__ rope, unsigned long long* __restrict__ best,
             int d, int half) {
     const int t = blockIdx.x, lane = threadIdx.x & 31;
     pdl_launch_dependents();
@@ -99,7 +99,7 @@ prep_kernel(const bf16* __restrict__ embed, const int* __restrict__ tokens, cons
         const int f = f0 + lane;
         const float v = __bfloat162float(e[f]);
         x[(size_t)t * d + f] = v;
-        xg[(size_t)t * d + f] = __float2bfloat16(v * __bfloat162float(gain[f]));
+        xg[(size_t)t * d + f] = to_op(v * __bfloat162float(gain[f]));
         float ss = v * v;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
@@ -129,8 +129,8 @@ __global__ void verify_kernel(const unsigned long long* __restrict__ best, const
     correction[i] = (int)(0xFFFFFFFFu - (uint32_t)(best[b + u - 1 + a] & 0xFFFFFFFFull));
 }
 
-// Copy K/V of logical positions between a dense [n_pos][Hkv][hd] buffer and the paged pool.
-__global__ void kv_copy_kernel(bf16* pool_layer, const int* __restrict__ slots, bf16* k, bf16* v, int n_kv_heads, int hd,
+// Copy K/V of logical positions between a dense bf16 [n_pos][Hkv][hd] buffer and the paged pool (half precision).
+__global__ void kv_copy_kernel(op16* pool_layer, const int* __restrict__ slots, bf16* k, bf16* v, int n_kv_heads, int hd,
                                int page_size, int to_pool) {
     const int i = blockIdx.x;
     const int s = slots[i], page = s / page_size, row = s % page_size;
@@ -140,11 +140,11 @@ __global__ void kv_copy_kernel(bf16* pool_layer, const int* __restrict__ slots, 
         const size_t ov = ok + (size_t)page_size * hd;
         const size_t oi = (size_t)i * n_kv_heads * hd + e;
         if (to_pool) {
-            pool_layer[ok] = k[oi];
-            pool_layer[ov] = v[oi];
+            pool_layer[ok] = to_op(__bfloat162float(k[oi]));
+            pool_layer[ov] = to_op(__bfloat162float(v[oi]));
         } else {
-            k[oi] = pool_layer[ok];
-            v[oi] = pool_layer[ov];
+            k[oi] = __float2bfloat16(__half2float(pool_layer[ok]));
+            v[oi] = __float2bfloat16(__half2float(pool_layer[ov]));
         }
     }
 }
@@ -166,13 +166,13 @@ static int load_driver_entry() {
     return SYN_OK;
 }
 
-// 2-D bf16 row-major [rows][cols] (pitch in elements), box = box_rows x 64 columns, 128-byte swizzle.
+// 2-D 16-bit row-major [rows][cols] (pitch in elements), box = box_rows x 64 columns, 128-byte swizzle.
 static int make_map_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch, uint32_t box_rows) {
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {pitch * 2};
     cuuint32_t box[2] = {64, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? SYN_OK : SYN_E_CUDA;
@@ -191,7 +191,7 @@ static int make_wmaps(const void* packed, int packed_rows, int K, WMaps* out) {
     cuuint32_t estr[2] = {1, 1};
     for (int k = 0; k < 2; ++k) {
         cuuint32_t box[2] = {64, k == 0 ? 256u : 128u};
-        if (g_encode(k == 0 ? &out->quad : &out->duo, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(packed), dims, strides,
+        if (g_encode(k == 0 ? &out->quad : &out->duo, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(packed), dims, strides,
                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return SYN_E_CUDA;
@@ -202,8 +202,10 @@ static int make_wmaps(const void* packed, int packed_rows, int K, WMaps* out) {
 struct syn_model {
     syn_model_desc desc;
     int f_pad, n_sm, gu_rows, qkv_rows, v_rows;
-    bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
-    std::vector<bf16*> wqkv, wo, wgu, wd, norm1, norm2;   // projections in the packed tile layout
+    bf16 *embed = nullptr, *final_norm = nullptr;
+    op16* lm_head = nullptr;
+    std::vector<op16*> wqkv, wo, wgu, wd;                 // projections in the packed tile layout (half precision)
+    std::vector<bf16*> norm1, norm2;
     std::vector<WMaps> tm_wqkv, tm_wo, tm_wgu, tm_wd;      // their tensor maps
     WMaps tm_lm_head;
     double* inv_freq = nullptr;
@@ -211,8 +213,8 @@ struct syn_model {
     // workspace (grow-only)
     int t_cap = 0;
     float *x = nullptr, *ssq = nullptr;   // residual stream; sums of x^2 per token and 32 features
-    bf16 *xn = nullptr,   // bf16(x * gain of the next RMSNorm): the operand of the qkv, gate/up and lm_head projections
-          *q = nullptr, *attn = nullptr, *act = nullptr;
+    op16 *xn = nullptr,   // half(x * gain of the next RMSNorm): the operand of the qkv, gate/up and lm_head projections
+         *q = nullptr, *attn = nullptr, *act = nullptr;
     float2* rope = nullptr;
     unsigned long long* best = nullptr;
     int *acc_dev = nullptr, *corr_dev = nullptr;
@@ -268,7 +270,7 @@ struct ProfScope {
 
 struct syn_kv {
     syn_model* model;
-    bf16* pool = nullptr;
+    op16* pool = nullptr;   // half precision (K and V enter and leave through syn_kv_import / syn_kv_export as bf16)
     uint32_t n_pages, page_size;
     size_t layer_elems;
     CUtensorMap tm_kv;
@@ -327,7 +329,7 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
         cuuint64_t strides[2] = {128, (cuuint64_t)q_dim * 2};
         cuuint32_t box[3] = {64, G * halves, box_tokens};
         cuuint32_t estr[3] = {1, 1, 1};
-        if (g_encode(&m->tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, m->q, dims, strides, box, estr,
+        if (g_encode(&m->tm_q, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, m->q, dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return SYN_E_CUDA;
@@ -362,7 +364,9 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
 
 extern "C" void syn_model_free(syn_model* m) {
     if (!m) return;
-    for (auto& v : {&m->wqkv, &m->wo, &m->wgu, &m->wd, &m->norm1, &m->norm2})
+    for (auto& v : {&m->wqkv, &m->wo, &m->wgu, &m->wd})
+        for (op16* p : *v) cudaFree(p);
+    for (auto& v : {&m->norm1, &m->norm2})
         for (bf16* p : *v) cudaFree(p);
     cudaFree(m->embed); cudaFree(m->lm_head); cudaFree(m->final_norm); cudaFree(m->inv_freq); cudaFree(m->status_dev);
     free_workspace(m);
@@ -449,9 +453,9 @@ static int syn_model_load_impl(const syn_model_desc* desc, const syn_weights* w,
     }
     // pack `n` row-major sources (rows[i] x src_k each) into a new tile-layout buffer of `packed_rows` x K
     auto pack = [&](const void* const* srcs, const int* rows, int n, int mode, int src_k, int packed_rows,
-                    bf16** out_ptr) -> int {
+                    op16** out_ptr) -> int {
         const int n_mt = (packed_rows + 511) / 512 * 4, nkb = (src_k + 63) / 64;   // an even number of feature pairs (zero rows at the end)
-        bf16* outp = nullptr;
+        op16* outp = nullptr;
         cudaError_t e = cudaMalloc(&outp, (size_t)n_mt * nkb * 128 * 64 * 2);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return SYN_E_OOM; }
         *out_ptr = outp;
@@ -493,7 +497,8 @@ static int syn_model_load_impl(const syn_model_desc* desc, const syn_weights* w,
         PACK_OR_FAIL(make_wmaps(m->lm_head, m->v_rows, d, &m->tm_lm_head));
     }
     for (uint32_t l = 0; l < c.n_layers; ++l) {
-        bf16 *n1 = nullptr, *n2 = nullptr, *pk = nullptr;
+        bf16 *n1 = nullptr, *n2 = nullptr;
+        op16* pk = nullptr;
         {
             const void* srcs[3] = {w->wq[l], w->wk[l], w->wv[l]};
             const int rows[3] = {q_dim, kv_dim, kv_dim};
@@ -1095,7 +1100,7 @@ static int gemm_plan(int T, int packed_rows, int K, int n_sm, int mode, bool may
 
 // One projection with the epilogue `ep`; `plan_mode` = the epilogue its schedule is made for (the
 // same, except in the test hook, which runs any schedule with the plain store epilogue).
-static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const bf16* w_packed, int packed_rows, int K,
+static int launch_gemm(syn_model* prof_m, int cls, int n_sm, int* status, const op16* w_packed, int packed_rows, int K,
                        const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, float* fix_part, int* fix_flag,
                        int plan_mode = -1) {
     ProfScope prof(cls >= 0 ? prof_m : nullptr, cls, st);
@@ -1135,15 +1140,16 @@ static int gemm2_plan(int T, int packed_rows, int K, int n_sm, int mode, int for
     if (n_cl_max < 1 || (force == PAIR_NONE && T < 256)) return PAIR_NONE;
     const int quad_items = (n_pairs + 1) / 2 * g.n_tt, duo_items = n_pairs * g.n_tt;
     int kind = force;
+    const bool may_split = mode == EPI_RESID || (g_schedule == 2 && mode == EPI_QKV);
     if (kind == PAIR_NONE) {
         if (quad_items >= n_cl_max) kind = PAIR_QUAD;                                   // full waves of 512-feature items
-        else if (mode == EPI_RESID && g.num_kb >= 96 && n_cl_max / quad_items >= 2) kind = PAIR_QUAD;   // long K: shared between clusters
+        else if (may_split && g.num_kb >= (g_schedule == 2 ? 32 : 96) && n_cl_max / quad_items >= 2) kind = PAIR_QUAD;   // long K: shared between clusters
         else if (2 * duo_items >= n_cl_max) kind = PAIR_DUO;
         else return PAIR_NONE;
     }
     const int items = kind == PAIR_QUAD ? quad_items : duo_items;
     g.n_groups = kind == PAIR_QUAD ? (n_pairs + 1) / 2 : n_pairs;
-    if (mode == EPI_RESID && items < n_cl_max && n_cl_max / items >= 2) {
+    if (may_split && items < n_cl_max && n_cl_max / items >= 2) {
         const int sp = std::min(GEMM_MAX_SPLITS, std::min(n_cl_max / items, std::max(1, g.num_kb / 8)));
         g.kb_per_split = (g.num_kb + sp - 1) / sp;
         g.splits = (g.num_kb + g.kb_per_split - 1) / g.kb_per_split;
@@ -1167,7 +1173,7 @@ static int gemm2_plan(int T, int packed_rows, int K, int n_sm, int mode, int for
 
 // One projection with the epilogue `ep` on whichever kernel its shape calls for.  `plan_mode` = the
 // epilogue the schedule is made for (the same, except in the test hook); `force_pair`: test hook.
-static int launch_proj(syn_model* prof_m, int cls, int n_sm, int* status, const bf16* w_packed, const WMaps* wm, int packed_rows,
+static int launch_proj(syn_model* prof_m, int cls, int n_sm, int* status, const op16* w_packed, const WMaps* wm, int packed_rows,
                        int K, const CUtensorMap& tmB, EpiParams ep, cudaStream_t st, float* fix_part, int* fix_flag,
                        int plan_mode = -1, int force_pair = PAIR_NONE) {
     if (plan_mode < 0) plan_mode = ep.mode;
@@ -1187,7 +1193,7 @@ static int launch_proj(syn_model* prof_m, int cls, int n_sm, int* status, const 
     return le == cudaSuccess ? SYN_OK : SYN_E_CUDA;
 }
 
-static void attn_params(AttnParams& ap, const syn_model* m, const syn_kv* kv, const syn_plan* p, uint32_t layer, bf16* out,
+static void attn_params(AttnParams& ap, const syn_model* m, const syn_kv* kv, const syn_plan* p, uint32_t layer, op16* out,
                         float* part_o, float2* part_ml, int* group_count) {
     const syn_model_desc& c = m->desc;
     ap.items = p->d<AttnItem>(p->o_items);
@@ -1211,7 +1217,7 @@ static void attn_params(AttnParams& ap, const syn_model* m, const syn_kv* kv, co
 }
 
 static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const CUtensorMap& tmQ,
-                            bf16* out, cudaStream_t st) {
+                            op16* out, cudaStream_t st) {
     const syn_model_desc& c = m->desc;
     AttnParams ap;
     attn_params(ap, m, kv, p, layer, out, m->part_o, m->part_ml, m->group_count);
@@ -1571,7 +1577,7 @@ struct LinearCtx {
     int* status = nullptr;
     float* fix_part = nullptr;
     int* fix_flag = nullptr;
-    bf16* packed = nullptr;
+    op16* packed = nullptr;
     const void* packed_src = nullptr;
     int packed_n = 0, packed_k = 0;
     WMaps wm;
@@ -1663,7 +1669,7 @@ extern "C" int syn_debug_set_spin_limit(int64_t cycles) {
 }
 
 extern "C" int syn_debug_set_schedule(int32_t which) {
-    if (which < 0 || which > 1) return SYN_E_INVALID_ARG;
+    if (which < 0 || which > 2) return SYN_E_INVALID_ARG;
     g_schedule = which;
     return SYN_OK;
 }
@@ -1687,7 +1693,7 @@ static int syn_op_attention_impl(syn_model* m, syn_kv* kv, const syn_plan* p, ui
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     // the Q tensor map is bound to the workspace buffer: stage the caller's q there
     CU_OK(cudaMemcpyAsync(m->q, q, (size_t)p->T * q_dim * 2, cudaMemcpyDeviceToDevice, st));
-    return launch_attention(m, kv, p, layer, m->tm_q, (bf16*)out, st);
+    return launch_attention(m, kv, p, layer, m->tm_q, (op16*)out, st);
 }
 
 // ------------------------------------------------------------------------------------------ no-allocation attention
@@ -1745,7 +1751,7 @@ static int syn_op_attention_static_impl(syn_model* m, syn_kv* kv, const syn_plan
     // the group counters must start at zero; every partial row that is read is written first
     CU_OK(cudaMemsetAsync(group_count, 0, (size_t)SYN_STATIC_MAX_PARTS * 4, st));
     AttnParams ap;
-    attn_params(ap, m, kv, p, layer, (bf16*)out, part_o, part_ml, group_count);
+    attn_params(ap, m, kv, p, layer, (op16*)out, part_o, part_ml, group_count);
     if (c.head_dim == 128)
         attn_kernel<128><<<p->n_cta, ATT_THREADS, AttnSmem<128>::TOTAL, st>>>(m->tm_q, kv->tm_kv, ap);
     else
@@ -1863,6 +1869,35 @@ extern "C" int syn_op_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uin
 
 extern "C" int syn_op_attention_static(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_t layer, const void* q, void* out, void* cuda_stream) {
     SYN_GUARD(syn_op_attention_static_impl(m, kv, p, layer, q, out, cuda_stream));
+}
+
+// The CTA-pair schedule without a device (tests).
+extern "C" int syn_gemm2_plan_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t force, int32_t* out) {
+    if (T <= 0 || N <= 0 || K <= 0 || n_sm <= 0 || n_sm > 65535 || epilogue < EPI_PLAIN || epilogue > EPI_LMHEAD || force < PAIR_NONE ||
+        force > PAIR_DUO || !out)
+        return SYN_E_INVALID_ARG;
+    Gemm2Params g;
+    int n_cl = 0;
+    const int kind = gemm2_plan(T, (N + 255) / 256 * 256, K, n_sm, epilogue, force, g, n_cl);
+    const int v[SYN_GEMM2_PLAN_FIELDS] = {kind, g.n_groups, g.n_tt, g.TN, g.num_kb, n_cl, g.splits, g.kb_per_split, g.rem_base, g.rem_extra};
+    memcpy(out, v, sizeof(v));
+    return SYN_OK;
+}
+
+extern "C" int syn_gemm2_work_host(int32_t T, int32_t N, int32_t K, int32_t n_sm, int32_t epilogue, int32_t force, int32_t cluster,
+                                   int32_t i, int32_t* out) {
+    if (T <= 0 || N <= 0 || K <= 0 || n_sm <= 0 || n_sm > 65535 || epilogue < EPI_PLAIN || epilogue > EPI_LMHEAD || force < PAIR_NONE ||
+        force > PAIR_DUO || !out || i < 0)
+        return SYN_E_INVALID_ARG;
+    Gemm2Params g;
+    int n_cl = 0;
+    const int kind = gemm2_plan(T, (N + 255) / 256 * 256, K, n_sm, epilogue, force, g, n_cl);
+    if (kind == PAIR_NONE || cluster < 0 || cluster >= n_cl) return SYN_E_INVALID_ARG;
+    Gemm2Work w;
+    if (!gemm2_work(g, cluster, n_cl, i, w)) return 0;
+    const int v[SYN_GEMM2_WORK_FIELDS] = {w.grp, w.tt, w.kb0, w.kb1, w.tile, w.split, w.nsplit, w.first_cl, w.counter};
+    memcpy(out, v, sizeof(v));
+    return 1;
 }
 
 extern "C" const char* syn_last_cuda_error(void) { return g_last_cuda_error; }

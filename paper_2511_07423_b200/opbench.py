@@ -14,12 +14,12 @@ chunks, prompts first), then each request offloads `--rounds` chunks drawn from 
 reports the iterations by kind and the share of the wall time spent in the scheduler's own code.
 `sample` times the sampling-verification stage (top-k of the logits rows + the per-request kernel)
 behind a one-layer model with the configuration's vocabulary and request mix.
-`scale` is the scalability experiment of the paper's Sec. 6.4 in shape: sessions arrive at a given
-rate, every session's device drafts chunks of gamma tokens at a fixed pace and offloads a chunk with
-probability = the offloading budget (tokens of chunks it keeps to itself ride along as uncached
-tokens of the next offload); the cloud is the scheduler over the real model on this GPU.  Device
-time is simulated, cloud time is the measured wall time of every iteration; the output is the
-verification latency per request (submission to result) against the arrival rate.
+`scale` is the scalability experiment of the paper's Sec. 6.4 in shape: the arrival-driven workload
+of workloads/arrivals.py (sessions arrive at a given rate, every device drafts chunks of gamma tokens
+at a fixed pace and offloads a chunk with probability = the offloading budget) with the scheduler over
+the real model on this GPU as its cloud.  Device and network time are simulated, cloud time is the
+measured wall time of every iteration; the output is the verification latency per request against the
+arrival rate.
 """
 from __future__ import annotations
 
@@ -52,7 +52,7 @@ def _time(fn, iters: int, warmup: int = 3):
 
 def bench_linear(a):
     key = rng.stream_key(0, 1234)
-    x = rng.normal_f32(key, 0, a.T * a.K, 1.0, device="cuda").view(a.T, a.K).to(torch.bfloat16)
+    x = rng.normal_f32(key, 0, a.T * a.K, 1.0, device="cuda").view(a.T, a.K).to(torch.float16)
     w = rng.normal_f32(key, a.T * a.K, a.N * a.K, 0.02, device="cuda").view(a.N, a.K).to(torch.bfloat16)
     syn.syn_op_linear(x, w, schedule_as=a.sched)
     med, best = _time(lambda: syn.syn_op_linear(x, w, schedule_as=a.sched, reuse_pack=True), a.iters)
@@ -74,7 +74,7 @@ def bench_attention(a):
         k, v = gen.gen_kv(shape, wl.seed, 0, r, 0, tot, device="cuda")
         kv.import_kv(0, batch.page_tables[r], 0, k, v)
     T = batch.n_tokens
-    q = rng.normal_f32(rng.stream_key(wl.seed, 77), 0, T * shape.q_dim, 1.5, device="cuda").view(T, shape.q_dim).to(torch.bfloat16)
+    q = rng.normal_f32(rng.stream_key(wl.seed, 77), 0, T * shape.q_dim, 1.5, device="cuda").view(T, shape.q_dim).to(torch.float16)
     plan = syn.Plan(kv, torch.zeros(T, dtype=torch.int32), batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
     out = torch.empty_like(q)
     model.set_profile(True)
@@ -181,106 +181,33 @@ def bench_sample(a):
 
 
 def bench_scale(a):
-    import heapq
-    import math
-    import random
     import time
+    from workloads import arrivals
     wl = CONFIGS[a.config]
     shape = wl.shape
     model = synthetic.load_model(shape, wl.seed)
     lo, hi = wl.ctx[1], wl.ctx[2]                      # prompt lengths: the configuration's context range
     n_pages = int(a.max_sessions * ((hi + a.out_tokens + 64) // 16 + 1))
     kv = syn.KVCache(model, n_pages)
+
+    def execute(b):                                    # one real iteration on this GPU, wall time
+        t0 = time.perf_counter()
+        _, cor = kv.verify_batch(b["chunk_tokens"], b["chunk_offsets"], b["page_tables"], b["ctx_lens"],
+                                 n_uncached=b["n_uncached"])
+        return time.perf_counter() - t0, cor
+
     for budget in [float(x) for x in a.budgets.split(",")]:
         for rate in [float(x) for x in a.rates.split(",")]:
-            rnd = random.Random(int(1000 * budget) * 7919 + int(100 * rate))
+            seed = int(1000 * budget) * 7919 + int(100 * rate)
+            cfg = arrivals.ArrivalConfig(budget=budget, gamma=a.gamma, device_s=a.device_ms * 1e-3, rtt=a.rtt_ms * 1e-3,
+                                         out_tokens=a.out_tokens, p_match=wl.p_match, prompt_lo=lo, prompt_hi=hi,
+                                         vocab=shape.vocab, max_sessions=a.max_sessions, seed=seed)
             sched = syn.Scheduler(kv, max_batch_tokens=a.budget_tokens)
-            ev = []                                    # (time, seq, kind, session)
-            seq = 0
-            t = 0.0
-            while t < a.horizon:                       # Poisson arrivals
-                t += rnd.expovariate(rate)
-                heapq.heappush(ev, (t, seq, "arrive", seq)); seq += 1
-            sess = {}
-            now, busy = 0.0, 0.0
-            lat, n_done, n_drop, iters = [], 0, 0, {"prefill": 0, "verify": 0}
-            submitted = {}
-            while True:
-                while ev and ev[0][0] <= now:
-                    _, _, kind, sid = heapq.heappop(ev)
-                    if kind == "arrive":
-                        if len(sess) >= a.max_sessions:
-                            n_drop += 1
-                            continue
-                        sess[sid] = {"gen": 0, "pend": []}
-                        sched.add_request(sid, [rnd.randrange(shape.vocab) for _ in range(rnd.randint(lo, hi))])
-                    elif sid in sess:                  # the device has drafted its next chunk
-                        s = sess[sid]
-                        drafts = [rnd.randrange(shape.vocab) for _ in range(a.gamma)]
-                        if rnd.random() < budget or len(s["pend"]) + 2 * a.gamma > 32:
-                            sched.add_verify(sid, s["pend"] + drafts, len(s["pend"]))
-                            submitted[sid] = now
-                        else:                          # kept on the device: accepted locally, cached at the next offload
-                            s["pend"] += drafts
-                            s["gen"] += a.gamma
-                            if s["gen"] >= a.out_tokens:
-                                sched.finish(sid); del sess[sid]; n_done += 1
-                            else:
-                                heapq.heappush(ev, (now + a.gamma * a.device_ms * 1e-3, seq, "chunk", sid)); seq += 1
-                b = sched.peek()
-                if b["kind"] == "idle":
-                    sched.commit()
-                    if not ev:
-                        break
-                    now = max(now, ev[0][0])
-                    if now > a.horizon * 3:
-                        break
-                    continue
-                t0 = time.perf_counter()
-                acc, cor = kv.verify_batch(b["chunk_tokens"], b["chunk_offsets"], b["page_tables"], b["ctx_lens"],
-                                           n_uncached=b["n_uncached"])
-                dt = time.perf_counter() - t0
-                now += dt
-                busy += dt
-                iters[b["kind"]] += 1
-                offs = b["chunk_offsets"].tolist()
-                if b["kind"] == "verify":   # accepted drafts: capped geometric with the workload's match probability
-                    acc_syn = []
-                    for i in range(b["n_req"]):
-                        g = offs[i + 1] - offs[i] - int(b["n_uncached"][i])
-                        k = 0
-                        while k < g and rnd.random() < wl.p_match:
-                            k += 1
-                        acc_syn.append(k)
-                    res = sched.commit(acc_syn, cor)
-                else:
-                    res = sched.commit([0] * b["n_req"], cor)
-                for x in res:
-                    sid = x["req_id"]
-                    if sid not in sess or not x["prompt_done"]:
-                        continue
-                    s = sess[sid]
-                    if x["kind"] == 2:
-                        lat.append(now - submitted.pop(sid) + 2e-3 * a.rtt_ms)
-                        s["gen"] += x["accept_len"] + 1
-                    s["pend"] = [x["correction_token"]]
-                    if s["gen"] >= a.out_tokens:
-                        sched.finish(sid); del sess[sid]; n_done += 1
-                    else:
-                        heapq.heappush(ev, (now + 2e-3 * a.rtt_ms + a.gamma * a.device_ms * 1e-3, seq, "chunk", sid)); seq += 1
-                if now > a.horizon * 3:
-                    break
-            for sid in list(sess):
-                sched.finish(sid)
-            sched.peek(); sched.commit()
+            res = arrivals.simulate(sched, execute, cfg, arrivals.poisson_arrivals(rate, a.horizon, seed), stop_after=3 * a.horizon)
             sched.close()
-            lat.sort()
-            print(json.dumps({"op": "scale", "config": wl.name, "offload_budget": budget, "arrival_rate_per_s": rate,
-                              "sessions_done": n_done, "sessions_dropped": n_drop, "verify_requests": len(lat),
-                              "verify_latency_ms_mean": 1e3 * sum(lat) / max(1, len(lat)),
-                              "verify_latency_ms_p95": 1e3 * lat[int(0.95 * (len(lat) - 1))] if lat else None,
-                              "gpu_busy_fraction": busy / max(now, 1e-9), "virtual_seconds": now,
-                              "iterations": iters}), flush=True)
+            print(json.dumps(dict({"op": "scale", "config": wl.name, "offload_budget": budget, "arrival_rate_per_s": rate},
+                                  **res.summary())), flush=True)
+    assert model.status() == 0
 
 
 def main():

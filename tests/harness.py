@@ -60,6 +60,48 @@ def oracle_teacher_forced(orc: Oracle, glob, layer_w: Callable[[int], dict], poo
                          np.stack(lg) if want_logits else None, a, c)
 
 
+def oracle_teacher_forced_many(orc: Oracle, glob, layer_w: Callable[[int], dict], wl: Workload, shape, seed: int,
+                               batch: gen.Batch, picks: Sequence[int], want_logits=True) -> Dict[int, OracleRequest]:
+    """oracle_teacher_forced for several requests at once, layer by layer, so that one layer's weights
+    serve every request before the next layer's are fetched (the large shapes regenerate or page them).
+    Token by token: step j forwards chunk token j of every listed request that has one (bit-identical to
+    the one-shot chunk forward), then draws draft j + 1 from the oracle's argmax by the sequential rule.
+    Each request gets its own contiguous page table and its seeded synthetic prefix."""
+    st = {}
+    for r in picks:
+        ctx, n, u = int(batch.ctx_lens[r]), int(batch.chunk_lens[r]), int(batch.n_uncached[r])
+        n_pages = -(-(ctx + n) // 16)
+        pt = np.arange(n_pages, dtype=np.int32)
+        pools = orc.new_pool(n_pages)
+        for l in range(shape.n_layers):
+            k, v = gen.gen_kv(shape, seed, l, r, 0, ctx)
+            orc.load_kv(pools[l], pt, 0, k.float().numpy(), v.float().numpy())
+        chunk = [gen.gen_anchor(wl, r)] + [int(x) for x in gen.gen_context_tokens(wl, r, u - 1)]
+        st[r] = dict(ctx=ctx, n=n, u=u, pt=pt, pools=pools, chunk=chunk, t1=[], t2=[], gap=[], lg=[])
+    for j in range(max(s["n"] for s in st.values())):
+        live = [r for r in picks if j < st[r]["n"]]
+        xs = {r: orc.embed(glob["embed"], [st[r]["chunk"][j]]) for r in live}
+        for l in range(shape.n_layers):
+            w = layer_w(l)
+            for r in live:
+                s = st[r]
+                orc.layer(w, xs[r], s["pools"][l], s["pt"], s["ctx"] + j)
+        for r in live:
+            s = st[r]
+            lg, t1, t2, gap = orc.logits(glob, xs[r], want_logits)
+            s["t1"].append(int(t1[0])); s["t2"].append(int(t2[0])); s["gap"].append(float(gap[0]))
+            if want_logits:
+                s["lg"].append(lg[0].astype(np.float32))
+            if s["u"] <= j + 1 < s["n"]:
+                s["chunk"].append(gen.gen_draft(wl, r, j + 1 - s["u"], int(t1[0])))
+    out = {}
+    for r, s in st.items():
+        a, c = verify_greedy(s["t1"], s["chunk"], s["u"])
+        out[r] = OracleRequest(s["chunk"], s["u"], np.array(s["t1"]), np.array(s["t2"]), np.array(s["gap"]),
+                               np.stack(s["lg"]) if want_logits else None, a, c)
+    return out
+
+
 def admissible_results(o: OracleRequest):
     """All (accept_len, correction) pairs reachable when every soft position may take either of the
     oracle's two best ids; and whether the request is strict (no soft position was consulted)."""

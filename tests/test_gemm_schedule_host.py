@@ -94,3 +94,75 @@ def test_sweep_of_awkward_sizes(epilogue):
     for n_sm in (1, 7, 132, 148, 160):
         _check(544, 28672, 4096, epilogue, n_sm)
         _check(129, 3072, 2048, epilogue, n_sm)
+
+
+# ------------------------------------------------------------------------------------------ the CTA-pair kernel
+
+def _check2(T, N, K, epilogue, force="auto", n_sm=148):
+    p = syn.gemm2_plan_host(T, N, K, epilogue, force, n_sm)
+    if p["kind"] == 0:
+        return p
+    n_tt, TN, nkb, n_cl = p["n_tt"], p["TN"], p["num_kb"], p["n_clusters"]
+    per = 2 if p["kind"] == 1 else 1                       # feature pairs of 256 per group
+    assert 16 <= TN <= 256 and TN % 16 == 0 and (n_tt - 1) * TN < T <= n_tt * TN
+    assert p["n_groups"] == -(-(-(-N // 256)) // per) and 1 <= n_cl <= n_sm // 2
+    cover = {}
+    for cl in range(n_cl):
+        i = 0
+        while True:
+            w = syn.gemm2_work_host(T, N, K, epilogue, cl, i, force, n_sm)
+            if w is None:
+                break
+            assert 0 <= w["grp"] < p["n_groups"] and 0 <= w["tt"] < n_tt and 0 <= w["kb0"] < w["kb1"] <= nkb
+            assert w["tile"] == w["grp"] * n_tt + w["tt"]
+            cover.setdefault(w["tile"], []).append((w["kb0"], w["kb1"], w["split"], w["nsplit"], w["first_cl"], w["counter"], cl, i))
+            i += 1
+            assert i < 5000
+    assert sorted(cover) == list(range(p["n_groups"] * n_tt))          # every tile, once over the whole K
+    counters = {}
+    for tile, parts in cover.items():
+        parts.sort()
+        assert parts[0][0] == 0 and parts[-1][1] == nkb
+        assert all(a[1] == b[0] for a, b in zip(parts, parts[1:]))
+        if len(parts) > 1:                                              # K shared: neighbouring clusters, parts in order,
+            S = len(parts)                                              # one counter per tile, all in the same round
+            assert [x[2] for x in parts] == list(range(S)) and all(x[3] == S for x in parts)
+            assert [x[6] for x in parts] == list(range(parts[0][4], parts[0][4] + S))
+            assert len({x[5] for x in parts}) == 1 and len({x[7] for x in parts}) == 1 and 0 <= parts[0][5] < n_sm // 2
+            assert min(x[1] - x[0] for x in parts) >= min(8, nkb // S)
+            counters.setdefault(parts[0][7], []).append(parts[0][5])
+        else:
+            assert parts[0][3] == 1
+    for rnd, cs in counters.items():
+        assert len(set(cs)) == len(cs)                                  # tiles of one round meet on different counters
+    return p
+
+
+def test_pair_schedules_of_the_configurations():
+    for cfg in (3, 4, 5, 6):
+        wl = CONFIGS[cfg]
+        s = wl.shape
+        T = gen.gen_batch(wl).n_tokens
+        f_pad = -(-s.d_ffn // 64) * 64
+        for N, K, epi in ((s.q_dim + 2 * s.kv_dim, s.d_model, "qkv"), (s.d_model, s.q_dim, "resid"),
+                          (2 * f_pad, s.d_model, "swiglu"), (s.d_model, f_pad, "resid"), (s.vocab, s.d_model, "lmhead")):
+            assert _check2(T, N, K, epi)["kind"] != 0
+    # fewer than 256 tokens: the one-CTA kernel keeps the projection
+    assert syn.gemm2_plan_host(129, 3072, 2048, "qkv")["kind"] == 0
+    # configuration 3: gate/up = 168 items of 512 features on 74 clusters, the 20 left over cut into 4 (14 of them) or 3 parts
+    p = _check2(544, 28672, 4096, "swiglu")
+    assert (p["kind"], p["n_clusters"], p["rem_base"], p["rem_extra"]) == (1, 74, 3, 14)
+    # its qkv and o projections: items of 256 features; its down projection: 24 items, K shared by three clusters each
+    assert _check2(544, 6144, 4096, "qkv")["kind"] == 2 and _check2(544, 4096, 4096, "resid")["kind"] == 2
+    p = _check2(544, 4096, 14336, "resid")
+    assert (p["kind"], p["splits"], p["n_clusters"]) == (1, 3, 72)
+
+
+@pytest.mark.parametrize("force", ["quad", "duo"])
+def test_pair_schedule_sweep(force):
+    for T, N, K in [(1, 128, 64), (40, 512, 256), (257, 640, 2048), (300, 1280, 1024), (544, 640, 4096), (921, 6144, 512),
+                    (1194, 7168, 5120), (2048, 4096, 4096), (2049, 152064, 5120), (544, 128256, 4096), (300, 38144, 1024)]:
+        for epi in ("plain", "resid"):
+            _check2(T, N, K, epi, force)
+    for n_sm in (2, 7, 132, 148, 160):
+        _check2(544, 28672, 4096, "swiglu", force, n_sm)

@@ -46,7 +46,7 @@ def test_attention_matches_oracle(hd, Hq, Hkv, ctx, chunk):
     pools = orc.new_pool(batch.n_pages)
     layer = 1
     T = batch.n_tokens
-    q = rng.normal_f32(rng.stream_key(seed, 77), 0, T * shape.q_dim, 1.5).view(T, shape.q_dim).to(torch.bfloat16)
+    q = rng.normal_f32(rng.stream_key(seed, 77), 0, T * shape.q_dim, 1.5).view(T, shape.q_dim).to(torch.float16)
     # cached prefix + the chunk's own keys/values: all positions < ctx + n come from the seeded stream
     for r in range(batch.n_req):
         tot = int(batch.ctx_lens[r] + batch.chunk_lens[r])
@@ -69,7 +69,7 @@ def test_attention_matches_oracle(hd, Hq, Hkv, ctx, chunk):
         ref = orc.attention(q[b:b + n].double().numpy(), pools[layer], batch.page_tables[r].numpy(), int(batch.ctx_lens[r]))
         scale = np.abs(ref).max()
         err = np.abs(got[b:b + n] - ref).max()
-        assert err <= 0.02 * scale, (r, err, scale)   # bf16 P and bf16 output rounding
+        assert err <= 2e-3 * scale, (r, err, scale)   # half-precision softmax weights and output (11 significant bits)
     st = plan.stats()
     if max(ctx) > 1000:
         assert st.attn_split_items > 0

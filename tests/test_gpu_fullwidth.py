@@ -1,10 +1,12 @@
-"""The full-width code paths held to the stated logit tolerance: 2-layer models at the FULL width of
-the 8B and 32B shapes (d_model, d_ffn, vocabulary, head geometry) with the FULL batches of
-configurations 3 and 5.  These reach what the reduced shapes cannot: pair tiles in full waves with
-leftover tiles cut along K under the SwiGLU and lm_head epilogues, K shared between CTAs under the
-qkv and residual epilogues, mixed waves of pair and single tiles, four row tiles and split key
-ranges in the attention; at a depth where the rounding of the bf16 operands still allows
-max |dlogit| <= 0.03 sigma.  The oracle judges a seeded choice of requests; their drafts come from the
+"""The full-width code paths held to a TIGHT logit tolerance: 2-layer models at the FULL width of the
+8B and 32B shapes (d_model, d_ffn, vocabulary, head geometry) with the FULL batches of configurations 3
+and 5, once on the kernels their shapes call for (CTA pairs: 512- and 256-feature items, K shared
+between clusters, leftover items cut along K) and once with every projection on the one-CTA kernel
+(pair tiles in full waves with leftover tiles cut along K under the SwiGLU and lm_head epilogues, K
+shared between CTAs under the qkv and residual epilogues, mixed waves of pair and single tiles); four
+row tiles and split key ranges in the attention.  At two layers the half-precision operands leave about
+0.001 sigma rms, so a slip in any epilogue, schedule or exchange shows: the bound asserted is a third of
+the stated 0.03 sigma.  The oracle judges a seeded choice of requests; their drafts come from the
 ORACLE's argmax (sequential rule), the other requests' from the library's."""
 import dataclasses
 
@@ -35,8 +37,18 @@ def judged_requests(wl, batch, count):
     return sorted(set(picks))
 
 
-@pytest.mark.parametrize("cfg,n_judged", [(3, 6), (5, 4)])
-def test_two_layers_at_full_width_meet_the_stated_tolerance(cfg, n_judged):
+@pytest.mark.parametrize("cfg,n_judged,schedule", [(3, 6, 0), (3, 6, 1), (5, 4, 0), (5, 4, 1)])
+def test_two_layers_at_full_width_meet_a_third_of_the_stated_tolerance(cfg, n_judged, schedule):
+    import paper_2511_07423_b200 as syn
+    from paper_2511_07423_b200 import synthetic
+    syn.debug_set_schedule(schedule)
+    try:
+        _run(cfg, n_judged)
+    finally:
+        syn.debug_set_schedule(0)
+
+
+def _run(cfg, n_judged):
     import paper_2511_07423_b200 as syn
     from paper_2511_07423_b200 import synthetic
     base = CONFIGS[cfg]
@@ -83,8 +95,8 @@ def test_two_layers_at_full_width_meet_the_stated_tolerance(cfg, n_judged):
         else:
             assert got in ok, (cfg, r, got, sorted(ok))
     print(f"config {cfg} width, 2 layers: judged {picks}, strict {n_strict}/{len(picks)}, "
-          f"max |dlogit|/sigma {worst:.4f} (rms {worst_rms:.5f}), tolerance {LOGIT_TOL}")
-    assert worst <= LOGIT_TOL, f"max |dlogit| / sigma = {worst:.4f} > {LOGIT_TOL}"
+          f"max |dlogit|/sigma {worst:.4f} (rms {worst_rms:.5f}), bound {LOGIT_TOL / 3:.3f}")
+    assert worst <= LOGIT_TOL / 3, f"max |dlogit| / sigma = {worst:.4f} > {LOGIT_TOL / 3}"
     kv.close()
     model.close()
     torch.cuda.empty_cache()

@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 
 def _case(T, N, K, seed):
     key = rng.stream_key(seed, 99)
-    x = rng.normal_f32(key, 0, T * K, 1.0).view(T, K).to(torch.bfloat16)
+    x = rng.normal_f32(key, 0, T * K, 1.0).view(T, K).to(torch.float16)
     w = rng.normal_f32(key, T * K, N * K, 0.05).view(N, K).to(torch.bfloat16)
     return x, w
 

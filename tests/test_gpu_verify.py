@@ -174,19 +174,40 @@ def test_plan_run_device_outputs_match_blocking_call():
 
 
 def test_host_validation_errors_leave_outputs_untouched():
+    """Every refused call returns its error code before any launch: the result arrays keep their
+    sentinel values and the KV slots the chunks would have written keep their contents, bit for bit."""
     import paper_2511_07423_b200 as syn
     shape = TINY
     wl = CONFIGS[1]
     batch = gen.gen_batch(wl)
     glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
+    fill_synthetic_kv(shape, wl.seed, batch, range(batch.n_req), kv=kv)
     toks = torch.zeros(batch.n_tokens, dtype=torch.int32)
+    # a good call first, so that the chunks' slots hold something a refused call could destroy
+    kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+
+    def slots():
+        out = []
+        for r in range(batch.n_req):
+            for l in range(shape.n_layers):
+                k, v = kv.export_kv(l, batch.page_tables[r], int(batch.ctx_lens[r]), int(batch.chunk_lens[r]))
+                out += [k.cpu(), v.cpu()]
+        return out
+
+    before = slots()
+    acc = torch.full((batch.n_req,), -77, dtype=torch.int32)
+    cor = torch.full((batch.n_req,), -78, dtype=torch.int32)
 
     def code(**kw):
         args = dict(chunk_tokens=toks, chunk_offsets=batch.chunk_offsets, page_tables=batch.page_tables,
                     ctx_lens=batch.ctx_lens, n_uncached=None)
         args.update(kw)
         with pytest.raises(syn.SynError) as e:
-            kv.verify_batch(**args)
+            kv.verify_batch(out=(acc, cor), **args)
+        torch.cuda.synchronize()
+        assert (acc == -77).all() and (cor == -78).all()
+        after = slots()
+        assert all(torch.equal(a.view(torch.int16), b.view(torch.int16)) for a, b in zip(before, after))
         return e.value.code
 
     assert code(chunk_offsets=torch.tensor([0, 4, 8, 12, 45])) == -2                      # chunk of 33
@@ -204,3 +225,56 @@ def test_host_validation_errors_leave_outputs_untouched():
     assert code(page_tables=alias, ctx_lens=torch.tensor([48, 48, 96, 128])) == -7
     with pytest.raises(syn.SynError):
         syn.KVCache(model, 8, page_size=32)
+
+
+def test_a_plan_runs_only_on_the_cache_it_was_made_for():
+    """A plan's page ids and slots were checked against one cache.  Handing it, with another cache of the
+    same model (here a smaller one, where those slots would lie past the end of the pool), to the calls
+    that launch kernels is refused with SYN_E_INVALID_ARG before anything is launched."""
+    import paper_2511_07423_b200 as syn
+    shape = TINY
+    wl = CONFIGS[1]
+    batch = gen.gen_batch(wl)
+    glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
+    small = syn.KVCache(model, 2)
+    toks = torch.zeros(batch.n_tokens, dtype=torch.int32)
+    plan = syn.Plan(kv, toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+    a = torch.full((batch.n_req,), -5, dtype=torch.int32, device="cuda")
+    c = torch.full((batch.n_req,), -6, dtype=torch.int32, device="cuda")
+    plan.kv = small                      # the binding passes plan.kv's handle
+    with pytest.raises(syn.SynError) as e:
+        plan.run(a, c)
+    assert e.value.code == -1
+    q = torch.zeros(batch.n_tokens, shape.q_dim, dtype=torch.float16, device="cuda")
+    for call in (plan.attention, plan.attention_static):
+        with pytest.raises(syn.SynError) as e:
+            call(0, q)
+        assert e.value.code == -1
+    torch.cuda.synchronize()
+    assert (a == -5).all() and (c == -6).all() and model.status() == 0
+    plan.kv = kv
+    plan.run(a, c)                       # and on its own cache it runs
+    torch.cuda.synchronize()
+    assert model.status() == 0 and (a >= 0).all()
+
+
+def test_last_step_stats_belong_to_the_model():
+    """syn_last_step_stats(model): the counters of the last step whichever call launched it, and with
+    profiling on its device time and the wall time of the blocking call."""
+    import paper_2511_07423_b200 as syn
+    shape = TINY
+    wl = CONFIGS[1]
+    batch = gen.gen_batch(wl)
+    glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
+    with pytest.raises(syn.SynError):
+        model.last_step_stats()          # no step yet
+    toks = torch.zeros(batch.n_tokens, dtype=torch.int32)
+    kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+    st = model.last_step_stats()
+    assert st.n_req == batch.n_req and st.n_tokens == batch.n_tokens and st.t_gpu_ms == 0.0 and st.h2d_bytes > 0
+    assert st.kernel_launches == 1 + 5 * shape.n_layers + 2
+    model.set_profile(True)
+    kv.verify_batch(toks[:8], batch.chunk_offsets[:3], batch.page_tables[:2], batch.ctx_lens[:2])
+    st = model.last_step_stats()
+    model.set_profile(False)
+    assert st.n_req == 2 and st.n_tokens == 8 and 0.0 < st.t_gpu_ms <= st.t_wall_ms
