@@ -196,7 +196,7 @@ def run_ours(args):
     wl = CONFIGS[args.config]
     shape = wl.shape
     peaks = _peaks()
-    syn.debug_set_schedule({"auto": 0, "one-cta": 1, "split": 2}[args.schedule])
+    syn.debug_set_schedule({"auto": 0, "one-cta": 1}[args.schedule])
 
     via_host = shape.dense_params() * 2 > 40e9
     model = synthetic.load_model(shape, wl.seed, via_host=via_host)
@@ -427,7 +427,7 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="1..6; 3 = the 8B-shape step the metric is quoted on; 6 = 32-token chunked partial prefill")
     ap.add_argument("--pool-tokens", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--schedule", default="auto", choices=["auto", "one-cta", "split"],
+    ap.add_argument("--schedule", default="auto", choices=["auto", "one-cta"],
                     help="auto: every projection takes the kernel its shape calls for; one-cta: none takes the CTA-pair kernel")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsynera.so")
 SOURCES = ["synera.cu", "scheduler.cpp"]
-HEADERS = ["ptx.cuh", "gemm.cuh", "attention.cuh", "sampling.cuh", os.path.join("..", "..", "include", "synera.h"),
+HEADERS = ["ptx.cuh", "gemm.cuh", "gemm2.cuh", "attention.cuh", "sampling.cuh", os.path.join("..", "..", "include", "synera.h"),
            os.path.join("..", "..", "include", "synera_sched.h")]
 
 
@@ -34,6 +34,18 @@ def build(force: bool = False, verbose: bool = False, extra=(), out: str = LIB) 
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)
     return out
+
+
+PROBE = os.path.join(HERE, "probe_mma_rate")
+
+
+def build_probe(force: bool = False) -> str:
+    """The stand-alone tcgen05.mma issue-rate measurement (csrc/probe_mma_rate.cu), built beside the library."""
+    src = os.path.join(CSRC, "probe_mma_rate.cu")
+    if not force and os.path.exists(PROBE) and os.path.getmtime(PROBE) >= max(os.path.getmtime(src), os.path.getmtime(os.path.join(CSRC, "ptx.cuh"))):
+        return PROBE
+    subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-o", PROBE, src])
+    return PROBE
 
 
 if __name__ == "__main__":

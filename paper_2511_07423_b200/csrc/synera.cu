@@ -1140,10 +1140,10 @@ static int gemm2_plan(int T, int packed_rows, int K, int n_sm, int mode, int for
     if (n_cl_max < 1 || (force == PAIR_NONE && T < 256)) return PAIR_NONE;
     const int quad_items = (n_pairs + 1) / 2 * g.n_tt, duo_items = n_pairs * g.n_tt;
     int kind = force;
-    const bool may_split = mode == EPI_RESID || (g_schedule == 2 && mode == EPI_QKV);
+    const bool may_split = mode == EPI_RESID;
     if (kind == PAIR_NONE) {
         if (quad_items >= n_cl_max) kind = PAIR_QUAD;                                   // full waves of 512-feature items
-        else if (may_split && g.num_kb >= (g_schedule == 2 ? 32 : 96) && n_cl_max / quad_items >= 2) kind = PAIR_QUAD;   // long K: shared between clusters
+        else if (may_split && g.num_kb >= 96 && n_cl_max / quad_items >= 2) kind = PAIR_QUAD;   // long K: shared between clusters
         else if (2 * duo_items >= n_cl_max) kind = PAIR_DUO;
         else return PAIR_NONE;
     }
@@ -1155,9 +1155,17 @@ static int gemm2_plan(int T, int packed_rows, int K, int n_sm, int mode, int for
         g.splits = (g.num_kb + g.kb_per_split - 1) / g.kb_per_split;
     }
     n_cl = g.splits > 1 ? items * g.splits : std::min(n_cl_max, items);
+    // Fewer than three full waves and a last round that fills less than half of the clusters: the one-CTA kernel,
+    // whose leftover tiles cost less (helper parts first, short owner parts last), is the faster one there
+    // (gate/up at 544 tokens: 168 items on 74 clusters, 2.27 waves: 130 us here against 118 us).
+    if (force == PAIR_NONE && g.splits == 1 && items > n_cl && items / n_cl < 3 && items % n_cl != 0 && 2 * (items % n_cl) < n_cl)
+        return PAIR_NONE;
     if (g.splits == 1 && items > n_cl) {
         // items left after the full waves: cut along K into one part per cluster (parts of at least 8 k-blocks,
-        // at most GEMM_MAX_SPLITS of them), so that the last round takes a fraction of an item's time
+        // at most GEMM_MAX_SPLITS of them), so that the last round takes a fraction of an item's time.  (Helper
+        // parts that run first and an owner part that runs last, as in the one-CTA kernel, measured slower here:
+        // gate/up 138 against 130 us at 544 tokens, 241 against 201 us at 921: the owner adds up to seven stored
+        // parts alone, where the reduce-scatter shares that work between all the tile's clusters.)
         const int rem = items % n_cl;
         if (rem > 0 && n_cl / rem >= 2) {
             int base = n_cl / rem, extra = n_cl % rem;
@@ -1179,7 +1187,7 @@ static int launch_proj(syn_model* prof_m, int cls, int n_sm, int* status, const 
     if (plan_mode < 0) plan_mode = ep.mode;
     Gemm2Params g2;
     int n_cl = 0;
-    const int kind = (wm && (g_schedule == 0 || force_pair != PAIR_NONE)) ? gemm2_plan(ep.T, packed_rows, K, n_sm, plan_mode, force_pair, g2, n_cl)
+    const int kind = (wm && (g_schedule != 1 || force_pair != PAIR_NONE)) ? gemm2_plan(ep.T, packed_rows, K, n_sm, plan_mode, force_pair, g2, n_cl)
                                                                             : PAIR_NONE;
     if (kind == PAIR_NONE) return launch_gemm(prof_m, cls, n_sm, status, w_packed, packed_rows, K, tmB, ep, st, fix_part, fix_flag, plan_mode);
     if (!fix_part || !fix_flag) return SYN_E_INVALID_ARG;
@@ -1669,7 +1677,7 @@ extern "C" int syn_debug_set_spin_limit(int64_t cycles) {
 }
 
 extern "C" int syn_debug_set_schedule(int32_t which) {
-    if (which < 0 || which > 2) return SYN_E_INVALID_ARG;
+    if (which < 0 || which > 1) return SYN_E_INVALID_ARG;
     g_schedule = which;
     return SYN_OK;
 }

@@ -146,12 +146,17 @@ def test_pair_schedules_of_the_configurations():
         f_pad = -(-s.d_ffn // 64) * 64
         for N, K, epi in ((s.q_dim + 2 * s.kv_dim, s.d_model, "qkv"), (s.d_model, s.q_dim, "resid"),
                           (2 * f_pad, s.d_model, "swiglu"), (s.d_model, f_pad, "resid"), (s.vocab, s.d_model, "lmhead")):
-            assert _check2(T, N, K, epi)["kind"] != 0
+            _check2(T, N, K, epi)
     # fewer than 256 tokens: the one-CTA kernel keeps the projection
     assert syn.gemm2_plan_host(129, 3072, 2048, "qkv")["kind"] == 0
-    # configuration 3: gate/up = 168 items of 512 features on 74 clusters, the 20 left over cut into 4 (14 of them) or 3 parts
-    p = _check2(544, 28672, 4096, "swiglu")
+    # configuration 3: gate/up = 168 items of 512 features on 74 clusters, 2.27 waves: left to the one-CTA kernel; taken
+    # all the same (forced), the 20 items left over are cut into 4 (14 of them) or 3 parts
+    assert syn.gemm2_plan_host(544, 28672, 4096, "swiglu")["kind"] == 0
+    p = _check2(544, 28672, 4096, "swiglu", "quad")
     assert (p["kind"], p["n_clusters"], p["rem_base"], p["rem_extra"]) == (1, 74, 3, 14)
+    # configuration 4 (921 tokens): 224 items, three full waves and two items over, cut in eight
+    p = _check2(921, 28672, 4096, "swiglu")
+    assert (p["kind"], p["rem_base"], p["rem_extra"]) == (1, 8, 0)
     # its qkv and o projections: items of 256 features; its down projection: 24 items, K shared by three clusters each
     assert _check2(544, 6144, 4096, "qkv")["kind"] == 2 and _check2(544, 4096, 4096, "resid")["kind"] == 2
     p = _check2(544, 4096, 14336, "resid")
