@@ -28,26 +28,32 @@ from workloads.configs import CONFIGS  # noqa: E402
 METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from an ncu capture of two timed
-# steps of the workload (mean over all launches of the kernel function), with the hash of the kernel's
-# source file at capture time: the figure is reported only while that source is unchanged.  Summaries of
-# the captures: profiles/.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from an ncu capture of two timed steps of the
+# workload (mean over all launches of the kernel function), with the hash of the kernel's source files at capture
+# time: the figure is reported only while those sources are unchanged.  Summaries of the captures: profiles/.
+KERNEL_SOURCES = {"attn_kernel": ("attention.cuh", "ptx.cuh"), "gemm_kernel": ("gemm.cuh", "ptx.cuh"),
+                  "gemm2_kernel": ("gemm2.cuh", "gemm.cuh", "ptx.cuh")}
 NCU_TRAFFIC = {
-    # workload: {kernel: (bytes per launch, sha256 of the kernel's source file)}
+    # workload: {kernel function: (bytes per launch, sha256 of its source files, concatenated in KERNEL_SOURCES order)}
     "cfg3-8b": {
-        "attention": (615966076, "5558da2a6e4259bcd3fa1795bf3a507c8bb196b6d6ecc740399ecad306e5f1c2"),
-        "gemm": (140141518, "4caa57856b234a4a49c91d04f4f6f1c774d7a1598602fd63507e1b776e9f5f84"),
+        "attn_kernel": (616014112, "682f0116cfa8499d6b1c49c45b87bc8d9a30401ec6fa024850de59b7260f6846"),
+        "gemm_kernel": (285482664, "e8082fa3de83d7301bd5963a42f663d57750315c78ce009c4a2db741ec3d142f"),
+        "gemm2_kernel": (99062525, "67deb0babfce543e60d48b918e7bc89a8ad159385d0cf19562b496aaba0ddf2a"),
     },
 }
 
 
-def _traffic(workload: str, kernel: str):
+def _source_hash(kernel: str) -> str:
     import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES[kernel]:
+        h.update(open(os.path.join(ROOT, "paper_2511_07423_b200", "csrc", f), "rb").read())
+    return h.hexdigest()
+
+
+def _traffic(workload: str, kernel: str):
     ent = NCU_TRAFFIC.get(workload, {}).get(kernel)
-    if not ent:
-        return None
-    src = os.path.join(ROOT, "paper_2511_07423_b200", "csrc", "attention.cuh" if kernel == "attention" else "gemm.cuh")
-    if hashlib.sha256(open(src, "rb").read()).hexdigest() != ent[1]:
+    if not ent or _source_hash(kernel) != ent[1]:
         return None
     return ent[0]
 
@@ -284,31 +290,51 @@ def run_ours(args):
         if name == "attention":
             k["kv_gbs"] = kv_bytes_layer / (avg * 1e-3) / 1e9
         kernels[name] = k
-    # The five projection classes are launches of ONE kernel (gemm_kernel); shares by kernel function
+    # The projection classes are launches of two kernel functions: gemm2_kernel (CTA pairs, from 256 tokens on) and
+    # gemm_kernel (one CTA per item); which one a class takes is the library's launch rule, asked of its schedule export.
+    shapes = {"qkv_gemm": (qd + 2 * kd, d, "qkv"), "o_gemm": (d, qd, "resid"), "gate_up_gemm": (2 * ((f + 63) // 64 * 64), d, "swiglu"),
+              "down_gemm": (d, (f + 63) // 64 * 64, "resid"), "lm_head_gemm": (V, d, "lmhead")}
+    func_of = {}
+    for name, (N_, K_, epi) in shapes.items():
+        pair = args.schedule == "auto" and syn.gemm2_plan_host(T, N_, K_, epi)["kind"] != 0
+        func_of[name] = "gemm2_kernel" if pair else "gemm_kernel"
+        if name in kernels:
+            kernels[name]["kernel"] = func_of[name]
+    ridge = peaks["tf_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+
+    def func_roof(func):
+        """Roofline of one kernel function: the algorithmic work of its launches / the summed CUDA-event time of
+        its launches (per launch: both divided by the number of launches)."""
+        if func == "attn_kernel":
+            return {"kernel": func, "bound": "hbm", "achieved": kernels["attention"]["kv_gbs"], "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "traffic": _traffic(wl.name, func), "share_of_step": kernels["attention"]["share"],
+                    "launches_per_step": kernels["attention"]["launches_per_step"]}
+        cls = [n for n in kernels if func_of.get(n) == func]
+        if not cls:
+            return None
+        ms_step = sum(kernels[n]["avg_ms"] * kernels[n]["launches_per_step"] for n in cls)
+        launches = sum(kernels[n]["launches_per_step"] for n in cls)
+        fl = sum(flops[n] * kernels[n]["launches_per_step"] for n in cls)
+        wb = sum(wbytes[n] * kernels[n]["launches_per_step"] for n in cls)
+        out = {"kernel": func, "classes": cls, "share_of_step": sum(kernels[n]["share"] for n in cls), "launches_per_step": launches,
+               "traffic": _traffic(wl.name, func)}
+        if T >= ridge:
+            out.update({"bound": "tensor", "achieved": fl / (ms_step * 1e-3) / 1e12, "peak": peaks["tf_sustained"], "unit": "TFLOP/s"})
+        else:
+            out.update({"bound": "hbm", "achieved": wb / (ms_step * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"})
+        return out
+
+    roofs = [r_ for r_ in (func_roof(fn) for fn in ("gemm2_kernel", "gemm_kernel", "attn_kernel")) if r_]
+    for r_ in roofs:
+        r_["frac"] = r_["achieved"] / r_["peak"]
+        r_["peak_source"] = peaks["source"] + (" sustained" if r_["bound"] == "tensor" else "")
+    roofs.sort(key=lambda r_: -r_["share_of_step"])
+    roof, other = roofs[0], roofs[1:]
+    # all projections together (both kernel functions), for comparison across versions
     gemm_classes = [n for n in kernels if n in flops]
     gemm_ms_step = sum(kernels[n]["avg_ms"] * kernels[n]["launches_per_step"] for n in gemm_classes)
-    gemm_launches = sum(kernels[n]["launches_per_step"] for n in gemm_classes)
-    gemm_share = sum(kernels[n]["share"] for n in gemm_classes)
-    ridge = peaks["tf_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
-    # the projections run on the CTA-pair kernel from 256 tokens on (unless --schedule one-cta), else on the one-CTA kernel
-    gemm_name = "gemm2_kernel" if (T >= 256 and args.schedule != "one-cta") else "gemm_kernel"
-    def gemm_roof():
-        # per launch: algorithmic work of the average launch / average launch duration
-        avg_s = gemm_ms_step * 1e-3 / gemm_launches
-        if T >= ridge:
-            return {"kernel": gemm_name, "bound": "tensor", "achieved": st.dense_flops / gemm_launches / avg_s / 1e12,
-                    "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "traffic": _traffic(wl.name, "gemm")}
-        return {"kernel": gemm_name, "bound": "hbm", "achieved": st.weight_bytes / gemm_launches / avg_s / 1e9,
-                "peak": peaks["hbm_gbs"], "unit": "GB/s", "traffic": _traffic(wl.name, "gemm")}
-    def attn_roof():
-        return {"kernel": "attn_kernel", "bound": "hbm", "achieved": kernels["attention"]["kv_gbs"], "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "traffic": _traffic(wl.name, "attention")}
-    roof = gemm_roof() if gemm_share >= kernels["attention"]["share"] else attn_roof()
-    other = attn_roof() if roof["kernel"] != "attn_kernel" else gemm_roof()
-    for r_ in (roof, other):
-        r_["frac"] = r_["achieved"] / r_["peak"]
-        r_["share_of_step"] = gemm_share if r_["kernel"] != "attn_kernel" else kernels["attention"]["share"]
-        r_["peak_source"] = peaks["source"] + (" sustained" if r_["bound"] == "tensor" else "")
+    projections = {"tflops": st.dense_flops / (gemm_ms_step * 1e-3) / 1e12, "share_of_step": sum(kernels[n]["share"] for n in gemm_classes),
+                   "frac_of_sustained": st.dense_flops / (gemm_ms_step * 1e-3) / 1e12 / peaks["tf_sustained"]}
     step_bytes = st.weight_bytes + st.kv_read_bytes + st.kv_write_bytes
     step_flops = st.dense_flops + st.attn_flops
     t_roof = max(step_flops / (peaks["tf_sustained"] * 1e12), step_bytes / (peaks["hbm_gbs"] * 1e9))
@@ -338,7 +364,8 @@ def run_ours(args):
         "gpu_launches": int(st.kernel_launches) * args.steps,
         "clocks": clocks,
         "roofline": roof,
-        "roofline_second_kernel": other,
+        "roofline_other_kernels": other,
+        "projections": projections,
         "step_roofline": {"bytes": step_bytes, "flops": step_flops, "t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms,
                           "peaks": peaks, "t_roof_ms_nominal": t_roof_spec * 1e3, "frac_of_nominal": t_roof_spec * 1e3 / ms},
         "kernels": kernels,
@@ -386,7 +413,8 @@ def cpu_baseline(wl, batch, toks, acc_gpu, cor_gpu, min_seconds: float = 12.0, m
             cache[l] = {k: v.cpu() for k, v in gen.gen_layer(shape, wl.seed, l, device="cuda").items()}
         return cache[l]
 
-    if shape.dense_params() * 2 < 40e9:   # smaller shapes: hold all layers, generation stays out of the timing
+    import psutil
+    if shape.dense_params() * 2 < 0.4 * psutil.virtual_memory().available:   # hold all layers: generation stays out of the timing
         layers = [{k: v.cpu() for k, v in gen.gen_layer(shape, wl.seed, l, device="cuda").items()} for l in range(shape.n_layers)]
         layer_w = lambda l: layers[l]
     done, tokens, seconds, agree, allowed, gap = [], 0, 0.0, True, True, float("inf")
