@@ -48,10 +48,24 @@ def test_two_layers_at_full_width_meet_a_third_of_the_stated_tolerance(cfg, n_ju
         syn.debug_set_schedule(0)
 
 
-def _run(cfg, n_judged):
+def test_wide_batch_at_the_1b_width_puts_64_wide_heads_through_the_pair_kernels():
+    """Configuration 2's own batch (129 tokens) stays on the one-CTA kernel.  A wider mix at the same width
+    (64 requests, chunks of 9-16 tokens: about 800 tokens) sends the qkv projection (64-wide heads, two per
+    128-feature tile), gate/up, down (K shared between clusters) and the lm_head through the CTA-pair kernel."""
+    import paper_2511_07423_b200 as syn
+    base = CONFIGS[2]
+    wl = dataclasses.replace(base, name="1b-wide", n_req=64, ctx=("uniform", 64, 768), chunk=("uniform", 9, 16))
+    T = int(gen.gen_batch(dataclasses.replace(wl, shape=dataclasses.replace(base.shape, n_layers=2))).chunk_offsets[-1])
+    s = base.shape
+    assert syn.gemm2_plan_host(T, s.q_dim + 2 * s.kv_dim, s.d_model, "qkv")["kind"] != 0
+    assert syn.gemm2_plan_host(T, s.d_model, s.d_ffn, "resid")["splits"] > 1
+    _run(2, 4, wl)
+
+
+def _run(cfg, n_judged, base=None):
     import paper_2511_07423_b200 as syn
     from paper_2511_07423_b200 import synthetic
-    base = CONFIGS[cfg]
+    base = base or CONFIGS[cfg]
     shape = dataclasses.replace(base.shape, n_layers=2, name=base.shape.name + "-2l")
     wl = dataclasses.replace(base, shape=shape, fit_to_pool=False)
     model = synthetic.load_model(shape, wl.seed)
