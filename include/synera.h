@@ -255,10 +255,14 @@ int syn_op_linear_reset(void);
  * that call are invalid, the next call works.
  * syn_debug_set_schedule: 0 (default) lets every projection take the kernel its shape calls for (CTA
  * pairs from 256 tokens on); 1 keeps all of them on the one-CTA kernel, so that both can be measured
- * and checked on the same batch.  Process-wide. */
+ * and checked on the same batch.  Process-wide.
+ * syn_debug_set_attention: which attention kernel the plans made AFTERWARDS are laid out for (a plan
+ * keeps its kernel): 0 default, 1 the warp-level-MMA kernel (row tiles of 64), 2 the tcgen05 kernel (row
+ * tiles of 128: a whole chunk of up to 128 / G tokens is one work item per kv head).  Process-wide. */
 int syn_debug_set_spin_limit(int64_t cycles);
 int syn_debug_linear_counter(int32_t index, int32_t value);
 int syn_debug_set_schedule(int32_t which);
+int syn_debug_set_attention(int32_t which);
 
 /* The ragged paged attention of the step on its own (paper Sec. 3.2 attention equation over a
  * paged cache).  q: DEVICE half precision [T][n_q_heads*head_dim] (rotated); out: DEVICE half

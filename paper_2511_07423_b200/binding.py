@@ -59,6 +59,7 @@ EXPORTS = ["syn_model_load", "syn_model_free", "syn_kv_alloc", "syn_kv_free", "s
            "syn_verify_batch", "syn_plan_create", "syn_plan_free", "syn_verify_run", "syn_model_status",
            "syn_last_step_stats", "syn_plan_stats", "syn_plan_host", "syn_strerror", "syn_last_cuda_error", "syn_op_linear",
            "syn_op_linear_as", "syn_op_linear_reset", "syn_debug_set_spin_limit", "syn_debug_linear_counter", "syn_debug_set_schedule",
+           "syn_debug_set_attention",
            "syn_op_attention", "syn_op_attention_static",
            "syn_set_profile", "syn_get_profile", "syn_verify_batch_sampled", "syn_op_sample_verify",
            "syn_gemm_plan_host", "syn_gemm_work_host", "syn_gemm2_plan_host", "syn_gemm2_work_host"]
@@ -574,6 +575,11 @@ def debug_set_spin_limit(cycles: int) -> None:
 def debug_set_schedule(which: int) -> None:
     """syn_debug_set_schedule: 0 automatic, 1 every projection on the one-CTA kernel."""
     _check(load_library().syn_debug_set_schedule(C.c_int32(which)), "syn_debug_set_schedule")
+
+
+def debug_set_attention(which: int) -> None:
+    """syn_debug_set_attention: 0 default, 1 warp-level-MMA kernel, 2 tcgen05 kernel; applies to plans made afterwards."""
+    _check(load_library().syn_debug_set_attention(C.c_int32(which)), "syn_debug_set_attention")
 
 
 def debug_linear_counter(index: int, value: int) -> None:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsynera.so")
 SOURCES = ["synera.cu", "scheduler.cpp"]
-HEADERS = ["ptx.cuh", "gemm.cuh", "gemm2.cuh", "attention.cuh", "sampling.cuh", os.path.join("..", "..", "include", "synera.h"),
+HEADERS = ["ptx.cuh", "gemm.cuh", "gemm2.cuh", "attention.cuh", "attention2.cuh", "sampling.cuh", os.path.join("..", "..", "include", "synera.h"),
            os.path.join("..", "..", "include", "synera_sched.h")]
 
 

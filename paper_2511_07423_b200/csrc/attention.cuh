@@ -22,7 +22,7 @@ namespace syn {
 
 struct AttnItem {
     int q_tok;      // index of the first query token of this item in the flattened batch
-    int nj;         // query tokens in this item (rows = nj * G <= 64)
+    int nj;         // query tokens in this item (rows = nj * G <= AttnParams::row_cap)
     int kvh;        // kv head
     int req;        // request (page table row)
     int kv_begin;   // first key position (multiple of 64)
@@ -45,12 +45,13 @@ struct AttnParams {
     int max_pages;
     int n_kv_heads, group;      // G = Hq / Hkv
     int q_dim;                  // Hq * hd
-    int q_box_tokens;           // tokens of the Q tile's TMA box: min(16, 64 / G)
+    int q_box_tokens;           // tokens of the Q tile's TMA box: min(16, 64 / G) (tensor-memory kernel: min(32, 128 / G))
+    int row_cap;                // rows of an item's tile: 64 (128 in the tensor-memory kernel); row stride of the partials
     int layer_block0;           // 2 * layer * n_pages * Hkv: first (K|V) block of this layer in the pool map
     float scale_log2;           // log2(e) / sqrt(hd)
     op16* out;                  // [T][q_dim]
-    float* part_o;              // [n_parts][64][hd]
-    float2* part_ml;            // [n_parts][64] (max in log2 units, sum)
+    float* part_o;              // [n_parts][row_cap][hd]
+    float2* part_ml;            // [n_parts][row_cap] (max in log2 units, sum)
     const MergeGroup* groups;   // [n_groups]
     int* group_count;           // [n_groups] partials completed so far; zero between launches
     int* status;                // 0 ok, 1 a bounded wait ran out, 2 the work list failed a bounds check
@@ -60,7 +61,7 @@ struct AttnParams {
 
 // The work list is host-made; the kernel still refuses an item that would index out of bounds.
 __device__ __forceinline__ bool attn_item_ok(const AttnItem& it, const AttnParams& p) {
-    const bool ok = it.q_tok >= 0 && it.nj >= 1 && it.q_tok + it.nj <= p.n_tokens && it.nj * p.group <= 64 &&
+    const bool ok = it.q_tok >= 0 && it.nj >= 1 && it.q_tok + it.nj <= p.n_tokens && it.nj * p.group <= p.row_cap &&
                     it.kvh >= 0 && it.kvh < p.n_kv_heads && it.req >= 0 && it.req < p.n_req && it.kv_begin >= 0 &&
                     (it.kv_begin & 63) == 0 && it.kv_begin < it.kv_end && ((it.kv_end - 1) >> 4) < p.max_pages &&
                     (it.part < 0 || (it.part < p.n_parts && it.grp >= 0 && it.grp < p.n_groups));
@@ -464,11 +465,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                                 *reinterpret_cast<uint32_t*>(dst + nt * 8 + 2 * c) =
                                     pack_op(o[nt][2 * r] * inv, o[nt][2 * r + 1] * inv);
                         } else {
-                            float* dst = p.part_o + ((size_t)item.part * 64 + row) * HD;
+                            float* dst = p.part_o + ((size_t)item.part * p.row_cap + row) * HD;
 #pragma unroll
                             for (int nt = 0; nt < HD / 8; ++nt)
                                 *reinterpret_cast<float2*>(dst + nt * 8 + 2 * c) = make_float2(o[nt][2 * r], o[nt][2 * r + 1]);
-                            if (c == 0) p.part_ml[(size_t)item.part * 64 + row] = make_float2(m[r], l[r]);
+                            if (c == 0) p.part_ml[(size_t)item.part * p.row_cap + row] = make_float2(m[r], l[r]);
                         }
                     }
                 }
@@ -494,17 +495,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                 const int row = threadIdx.x >> 2, c0 = (threadIdx.x & 3) * CW;
                 if (row < rows) {
                     float mx = -INFINITY;
-                    for (int k = 0; k < gr.n_parts; ++k) mx = fmaxf(mx, __ldcg(&p.part_ml[(size_t)(gr.part0 + k) * 64 + row]).x);
+                    for (int k = 0; k < gr.n_parts; ++k) mx = fmaxf(mx, __ldcg(&p.part_ml[(size_t)(gr.part0 + k) * p.row_cap + row]).x);
                     const float bs = mx == -INFINITY ? 0.f : mx;
                     float lsum = 0.f;
                     float4 acc[CW / 4];
 #pragma unroll
                     for (int i = 0; i < CW / 4; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
                     for (int k = 0; k < gr.n_parts; ++k) {
-                        const float2 ml = __ldcg(&p.part_ml[(size_t)(gr.part0 + k) * 64 + row]);
+                        const float2 ml = __ldcg(&p.part_ml[(size_t)(gr.part0 + k) * p.row_cap + row]);
                         const float w = ex2_approx(ml.x - bs);
                         lsum += ml.y * w;
-                        const float4* src = reinterpret_cast<const float4*>(p.part_o + ((size_t)(gr.part0 + k) * 64 + row) * HD + c0);
+                        const float4* src = reinterpret_cast<const float4*>(p.part_o + ((size_t)(gr.part0 + k) * p.row_cap + row) * HD + c0);
 #pragma unroll
                         for (int i = 0; i < CW / 4; ++i) {
                             const float4 v = __ldcg(src + i);

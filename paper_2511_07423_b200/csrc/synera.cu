@@ -13,7 +13,7 @@
 #include <new>
 #include <vector>
 
-#include "attention.cuh"
+#include "attention2.cuh"
 #include "gemm.cuh"
 #include "gemm2.cuh"
 #include "sampling.cuh"
@@ -28,6 +28,9 @@ constexpr int GEMM_MAX_SPLITS = 8;   // most CTAs that share one pair tile's K r
 static long long g_spin_limit = SYN_SPIN_LIMIT_CYCLES;
 // 0: every projection takes the kernel its shape calls for; 1: the one-CTA kernel always (syn_debug_set_schedule).
 static int g_schedule = 0;
+// Attention kernel: 0 = the default of attn_row_cap(), 1 = warp-level MMAs (64-row tiles), 2 = tcgen05 (128-row tiles).
+static int g_attention = 0;
+static int attn_row_cap() { return g_attention == 2 ? 128 : 64; }
 
 // Name of the last CUDA error a call of this library met on this thread (for syn_last_cuda_error).
 static thread_local const char* g_last_cuda_error = "";
@@ -219,7 +222,7 @@ struct syn_model {
     unsigned long long* best = nullptr;
     int *acc_dev = nullptr, *corr_dev = nullptr;
     int b_cap = 0;
-    CUtensorMap tm_xn, tm_attn, tm_act, tm_q;
+    CUtensorMap tm_xn, tm_attn, tm_act, tm_q, tm_q4;
     float* fix_part = nullptr;      // stored accumulators of K-split remainder tiles (one slot per SM)
     int* fix_flag = nullptr;        // their arrival / release counters, [GEMM_FLAG_INTS * n_sm], zero between launches
     float* part_o = nullptr;
@@ -273,12 +276,13 @@ struct syn_kv {
     op16* pool = nullptr;   // half precision (K and V enter and leave through syn_kv_import / syn_kv_export as bf16)
     uint32_t n_pages, page_size;
     size_t layer_elems;
-    CUtensorMap tm_kv;
+    CUtensorMap tm_kv, tm_kv16;   // boxes of 32 rows (K and V of a page and head) and of 16 rows (K or V)
 };
 
 struct syn_plan {
     syn_step_stats stats;
     int n_req = 0, T = 0, max_pages = 0, n_items = 0, n_cta = 0, n_groups = 0, n_parts = 0;
+    int row_cap = 64;   // rows of an attention item's tile: which attention kernel the work list was made for
     // one device buffer and its pinned host mirror
     uint8_t *dev = nullptr, *host = nullptr;
     size_t cap = 0, used = 0;
@@ -333,6 +337,16 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return SYN_E_CUDA;
+        // Q tile of the tensor-memory attention kernel: [token][head][64-dim half][64]; one box = one half of the
+        // G heads of a kv head for min(32, 128 / G) tokens, i.e. rows (token, head) of 128 bytes
+        cuuint64_t dims4[4] = {64, halves, c.n_q_heads, (cuuint64_t)cap};
+        cuuint64_t strides4[3] = {128, (cuuint64_t)c.head_dim * 2, (cuuint64_t)q_dim * 2};
+        cuuint32_t box4[4] = {64, 1, G, std::min((uint32_t)SYN_MAX_CHUNK, 128u / G)};
+        cuuint32_t estr4[4] = {1, 1, 1, 1};
+        if (g_encode(&m->tm_q4, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, m->q, dims4, strides4, box4, estr4,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return SYN_E_CUDA;
     }
     if (!m->fix_part) {
         CU_OK(cudaMalloc(&m->fix_part, (size_t)m->n_sm * GEMM_FIX_SLOT_BYTES));
@@ -351,8 +365,8 @@ static int ensure_workspace(syn_model* m, int T, int B, int n_parts) {
         cudaFree(m->part_o); cudaFree(m->part_ml); cudaFree(m->group_count);
         m->part_o = nullptr; m->part_ml = nullptr; m->group_count = nullptr; m->part_cap = 0;
         const int cap = (n_parts + 255) / 256 * 256;
-        CU_OK(cudaMalloc(&m->part_o, (size_t)cap * 64 * c.head_dim * 4));
-        CU_OK(cudaMalloc(&m->part_ml, (size_t)cap * 64 * 8));
+        CU_OK(cudaMalloc(&m->part_o, (size_t)cap * 128 * c.head_dim * 4));   // rows of the larger tile
+        CU_OK(cudaMalloc(&m->part_ml, (size_t)cap * 128 * 8));
         CU_OK(cudaMalloc(&m->group_count, (size_t)cap * 4));   // a group has >= 2 parts: cap/2 would do
         CU_OK(cudaMemset(m->group_count, 0, (size_t)cap * 4));
         m->part_cap = cap;
@@ -555,6 +569,8 @@ static int syn_model_load_impl(const syn_model_desc* desc, const syn_weights* w,
     CU_M(cudaFuncSetAttribute(gemm2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_MAX));
     CU_M(cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::TOTAL));
     CU_M(cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::TOTAL));
+    CU_M(cudaFuncSetAttribute(attn2_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Attn2Smem<128>::TOTAL));
+    CU_M(cudaFuncSetAttribute(attn2_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Attn2Smem<64>::TOTAL));
     CU_M(cudaDeviceSynchronize());
     *out = m;
     return SYN_OK;
@@ -595,6 +611,10 @@ extern "C" int syn_kv_alloc(syn_model* m, uint32_t n_pages, uint32_t page_size, 
     // pool as a 2-D tensor [blocks * 16 rows][head_dim]; a box of 32 rows x 64 columns is one
     // 64-element half of the K rows and the V rows of one (page, kv head)
     if (make_map_2d(&kv->tm_kv, kv->pool, blocks * page_size, c.head_dim, c.head_dim, 2 * page_size) != SYN_OK) {
+        syn_kv_free(kv);
+        return SYN_E_CUDA;
+    }
+    if (make_map_2d(&kv->tm_kv16, kv->pool, blocks * page_size, c.head_dim, c.head_dim, page_size) != SYN_OK) {
         syn_kv_free(kv);
         return SYN_E_CUDA;
     }
@@ -666,7 +686,7 @@ struct HostPlan {
 // (the "flatten" of paper Sec. 4.5).  Pure host code.
 static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_sm, int32_t n_req,
                         const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables,
-                        int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, HostPlan& hp) {
+                        int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, int row_cap, HostPlan& hp) {
     if (n_req <= 0 || !chunk_tokens || !chunk_offsets || !page_tables || !ctx_lens || max_pages <= 0 || n_sm <= 0)
         return SYN_E_INVALID_ARG;
     const int G = c.n_q_heads / c.n_kv_heads, Hkv = c.n_kv_heads;
@@ -726,10 +746,15 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
     // when one unit alone would exceed a CTA's fair share: every split costs an fp32 partial and a
     // merge.
     const int n_cta_max = n_sm;
-    const int tok_per_group = std::min(16, 64 / G);
+    // The tensor-memory kernel (row_cap 128) spends the same time on a stage whatever the number of rows.
+    const bool wide = row_cap == 128;
+    const int tok_per_group = wide ? std::min(SYN_MAX_CHUNK, 128 / G) : std::min(16, 64 / G);
     static const int STAGE_COST[5] = {0, 1040, 1200, 1500, 1540};
-    const int ITEM_COST = 5500, PART_COST = 3000;
-    auto unit_cost = [&](int L, int nj) { return (int64_t)((L + 63) / 64) * STAGE_COST[(nj * G + 15) / 16] + ITEM_COST; };
+    const int WIDE_STAGE_COST = 1300;
+    const int ITEM_COST = wide ? 6000 : 5500, PART_COST = wide ? 4000 : 3000;
+    auto unit_cost = [&](int L, int nj) {
+        return (int64_t)((L + 63) / 64) * (wide ? WIDE_STAGE_COST : STAGE_COST[(nj * G + 15) / 16]) + ITEM_COST;
+    };
     int64_t total_cost = 0;
     for (int i = 0; i < n_req; ++i) {
         const int b = chunk_offsets[i], n = chunk_offsets[i + 1] - b;
@@ -738,7 +763,7 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
             total_cost += unit_cost(ctx_lens[i] + j0 + nj, nj) * Hkv;
         }
     }
-    const int64_t share = std::max<int64_t>(8 * STAGE_COST[4] + ITEM_COST, (total_cost + n_cta_max - 1) / n_cta_max);
+    const int64_t share = std::max<int64_t>(8 * (wide ? WIDE_STAGE_COST : STAGE_COST[4]) + ITEM_COST, (total_cost + n_cta_max - 1) / n_cta_max);
     std::vector<AttnItem> items;
     std::vector<int> item_cost;
     std::vector<MergeGroup>& groups = hp.groups;
@@ -912,7 +937,7 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     if (!m || !kv || kv->model != m) return SYN_E_INVALID_ARG;
     HostPlan hp;
     int r = plan_compute(m->desc, (int)kv->page_size, kv->n_pages, m->n_sm, n_req, chunk_tokens, chunk_offsets, page_tables,
-                         max_pages, ctx_lens, n_uncached, hp);
+                         max_pages, ctx_lens, n_uncached, attn_row_cap(), hp);
     if (r) return r;
     const int T = hp.T, n_items = (int)hp.items.size(), n_cta = hp.n_cta;
     size_t off = 0;
@@ -948,6 +973,7 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     if (!hp.groups.empty()) memcpy(p->h<MergeGroup>(p->o_groups), hp.groups.data(), hp.groups.size() * sizeof(MergeGroup));
     p->n_req = n_req; p->T = T; p->max_pages = max_pages; p->n_items = n_items; p->n_cta = n_cta;
     p->n_groups = (int)hp.groups.size(); p->n_parts = hp.n_parts;
+    p->row_cap = attn_row_cap();
     p->stats = hp.stats;
     p->stats.h2d_bytes = (int64_t)off;
     p->kv = kv; p->kv_pool = kv->pool; p->kv_pages = kv->n_pages;
@@ -966,7 +992,7 @@ static int syn_plan_host_impl(const syn_model_desc* desc, uint32_t n_pages, uint
         return SYN_E_INVALID_ARG;
     HostPlan hp;
     int r = plan_compute(*desc, (int)page_size, n_pages, n_sm, n_req, chunk_tokens, chunk_offsets, page_tables, max_pages,
-                         ctx_lens, n_uncached, hp);
+                         ctx_lens, n_uncached, attn_row_cap(), hp);
     if (r) return r;
     *n_items = (int)hp.items.size();
     *n_cta = hp.n_cta;
@@ -1211,7 +1237,8 @@ static void attn_params(AttnParams& ap, const syn_model* m, const syn_kv* kv, co
     ap.n_kv_heads = c.n_kv_heads;
     ap.group = c.n_q_heads / c.n_kv_heads;
     ap.q_dim = c.n_q_heads * c.head_dim;
-    ap.q_box_tokens = std::min(16, 64 / ap.group);
+    ap.row_cap = p->row_cap;
+    ap.q_box_tokens = p->row_cap == 128 ? std::min(SYN_MAX_CHUNK, 128 / ap.group) : std::min(16, 64 / ap.group);
     ap.layer_block0 = (int)(2ull * layer * kv->n_pages * c.n_kv_heads);
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
     ap.out = out;
@@ -1232,7 +1259,11 @@ static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_
     {
         ProfScope prof(m, 2, st);
         cudaError_t e;
-        if (c.head_dim == 128)
+        if (p->row_cap == 128 && c.head_dim == 128)
+            e = launch_pdl(attn2_kernel<128>, dim3(p->n_cta), dim3(ATT2_THREADS), Attn2Smem<128>::TOTAL, st, m->tm_q4, kv->tm_kv16, ap);
+        else if (p->row_cap == 128)
+            e = launch_pdl(attn2_kernel<64>, dim3(p->n_cta), dim3(ATT2_THREADS), Attn2Smem<64>::TOTAL, st, m->tm_q4, kv->tm_kv16, ap);
+        else if (c.head_dim == 128)
             e = launch_pdl(attn_kernel<128>, dim3(p->n_cta), dim3(ATT_THREADS), AttnSmem<128>::TOTAL, st, tmQ, kv->tm_kv, ap);
         else
             e = launch_pdl(attn_kernel<64>, dim3(p->n_cta), dim3(ATT_THREADS), AttnSmem<64>::TOTAL, st, tmQ, kv->tm_kv, ap);
@@ -1682,6 +1713,12 @@ extern "C" int syn_debug_set_schedule(int32_t which) {
     return SYN_OK;
 }
 
+extern "C" int syn_debug_set_attention(int32_t which) {
+    if (which < 0 || which > 2) return SYN_E_INVALID_ARG;
+    g_attention = which;
+    return SYN_OK;
+}
+
 extern "C" int syn_debug_linear_counter(int32_t index, int32_t value) {
     int r = linear_ctx_init();
     if (r) return r;
@@ -1748,7 +1785,7 @@ static int syn_op_attention_static_impl(syn_model* m, syn_kv* kv, const syn_plan
     const syn_model_desc& c = m->desc;
     const int q_dim = c.n_q_heads * c.head_dim;
     if (p->T > m->t_cap) return SYN_E_INVALID_ARG;
-    if (p->n_parts > SYN_STATIC_MAX_PARTS) return SYN_E_CAPACITY;
+    if ((int64_t)p->n_parts * p->row_cap > (int64_t)SYN_STATIC_MAX_PARTS * 64) return SYN_E_CAPACITY;
     float* part_o = nullptr;
     float2* part_ml = nullptr;
     int* group_count = nullptr;
@@ -1760,7 +1797,11 @@ static int syn_op_attention_static_impl(syn_model* m, syn_kv* kv, const syn_plan
     CU_OK(cudaMemsetAsync(group_count, 0, (size_t)SYN_STATIC_MAX_PARTS * 4, st));
     AttnParams ap;
     attn_params(ap, m, kv, p, layer, (op16*)out, part_o, part_ml, group_count);
-    if (c.head_dim == 128)
+    if (p->row_cap == 128 && c.head_dim == 128)
+        attn2_kernel<128><<<p->n_cta, ATT2_THREADS, Attn2Smem<128>::TOTAL, st>>>(m->tm_q4, kv->tm_kv16, ap);
+    else if (p->row_cap == 128)
+        attn2_kernel<64><<<p->n_cta, ATT2_THREADS, Attn2Smem<64>::TOTAL, st>>>(m->tm_q4, kv->tm_kv16, ap);
+    else if (c.head_dim == 128)
         attn_kernel<128><<<p->n_cta, ATT_THREADS, AttnSmem<128>::TOTAL, st>>>(m->tm_q, kv->tm_kv, ap);
     else
         attn_kernel<64><<<p->n_cta, ATT_THREADS, AttnSmem<64>::TOTAL, st>>>(m->tm_q, kv->tm_kv, ap);

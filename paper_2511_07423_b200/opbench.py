@@ -63,6 +63,7 @@ def bench_linear(a):
 
 
 def bench_attention(a):
+    syn.debug_set_attention(a.kind)
     wl = CONFIGS[a.config]
     s = wl.shape
     shape = ModelShape(f"attn-{s.name}", 1, s.d_model, s.n_q_heads, s.n_kv_heads, s.head_dim, 1024, 1024)
@@ -88,7 +89,7 @@ def bench_attention(a):
     kvb = st.kv_read_bytes  # one layer
     ms_att = prof["attention"][0] / prof["attention"][1]
     ms_mrg = prof["attention_merge"][0] / max(1, prof["attention_merge"][1])
-    print(json.dumps({"op": "attention", "config": wl.name, "n_req": batch.n_req, "T": T, "kv_bytes": kvb,
+    print(json.dumps({"op": "attention", "kind": a.kind, "config": wl.name, "n_req": batch.n_req, "T": T, "kv_bytes": kvb,
                       "items": st.attn_items, "split_items": st.attn_split_items, "ms_attention": ms_att,
                       "ms_merge": ms_mrg, "kv_gbs": kvb / ms_att / 1e6, "kv_gbs_with_merge": kvb / (ms_att + ms_mrg) / 1e6,
                       "attn_tflops": st.attn_flops / ms_att / 1e9}))
@@ -222,6 +223,7 @@ def main():
     t = sub.add_parser("attention")
     t.add_argument("--config", type=int, default=3)
     t.add_argument("--pool-tokens", type=int, default=None)
+    t.add_argument("--kind", type=int, default=0, help="attention kernel: 0 default, 1 warp-level MMAs, 2 tcgen05")
     t.add_argument("--iters", type=int, default=10)
     m = sub.add_parser("sample")
     m.add_argument("--config", type=int, default=3)

@@ -32,8 +32,18 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("kind", [1, 2], ids=["warp_mma", "tcgen05"])
 @pytest.mark.parametrize("hd,Hq,Hkv,ctx,chunk", CASES)
-def test_attention_matches_oracle(hd, Hq, Hkv, ctx, chunk):
+def test_attention_matches_oracle(hd, Hq, Hkv, ctx, chunk, kind):
+    import paper_2511_07423_b200 as syn
+    syn.debug_set_attention(kind)
+    try:
+        _run(hd, Hq, Hkv, ctx, chunk)
+    finally:
+        syn.debug_set_attention(0)
+
+
+def _run(hd, Hq, Hkv, ctx, chunk):
     import paper_2511_07423_b200 as syn
     shape = ModelShape("att", 2, 256, Hq, Hkv, hd, 256, 512)
     seed = 7
