@@ -4,17 +4,18 @@
 // Same work items as attention.cuh (request, kv head, token sub-range, key range), but the row tile
 // of an item is 128 rows (row = j * G + g): a chunk of up to 128 / G tokens is ONE item per kv head,
 // so every K/V byte of a request is read once per kv head however long the chunk is.  Both products
-// run on tcgen05.mma with M = 128:
+// run on tcgen05.mma with M = 128, in stages of 64 keys:
 //   S = Q K^T : A = the Q tile (K-major, 128-byte swizzle), B = 64 keys of K (K-major), D = S in tensor
-//               memory (two buffers of 64 columns, so the next stage's scores are computed while the
-//               softmax of the current one runs);
+//               memory, as TWO partial sums over halves of the head dimension (see the MMA issuer);
 //   O += P V  : A = P (half precision, written by the softmax warps into shared memory in the
 //               K-major swizzled layout), B = V as it lies in the cache, [key][dim], i.e. an MN-major
 //               operand, D = O in tensor memory for the whole item.
-// Warp roles: warp 0 streams K and V pages (TMA, boxes of 16 rows x 128 bytes) and the Q tiles
-// through mbarrier rings; one thread of warp 1 issues every MMA; warps 4..7 (one thread per row) do
-// the online softmax in fp32 (base 2) and the item's epilogue.  The running maximum used for P is
-// only raised when a stage's maximum exceeds it by more than 2^8 (P stays well inside half
+// Warp roles: warp 0 streams K and V pages (TMA, boxes of 16 rows x 128 bytes, separate rings for K
+// and V because a stage's K is free two steps before its V) and the Q tile through mbarriers; one
+// thread of warp 1 issues every MMA; warps 4..7 (one thread per row) do the online softmax in fp32
+// (base 2) and the item's epilogue.  Pipeline: while the softmax warps work on stage k - 1, the
+// tensor pipe computes the scores of stage k and O += P V of stage k - 2.  The running maximum used
+// for P is only raised when a stage's maximum exceeds it by more than 2^8 (P stays well inside half
 // precision); O in tensor memory is rescaled at those moments only, and the final division by the
 // row sum uses the same maximum, so the result is the exact softmax whatever the moments were.
 // Items that cover part of a request's keys store fp32 partials (m, l, O) that the CTA completing a
@@ -33,14 +34,14 @@ template <int HD>
 struct Attn2Smem {
     static constexpr int HALVES = HD / 64;
     static constexpr int KBOX_BYTES = 16 * 128;                       // 16 keys x 64 dims
-    static constexpr int K_BYTES = HALVES * ATT2_STAGE_KEYS * 128;    // [half][64 keys][128 bytes]
-    static constexpr int STAGE_BYTES = 2 * K_BYTES;                   // K then V
+    static constexpr int K_BYTES = HALVES * ATT2_STAGE_KEYS * 128;    // K (or V) of a stage: [half][64 keys][128 bytes]
     static constexpr int Q_BYTES = HALVES * ATT2_ROWS * 128;          // [half][128 rows][128 bytes]
     static constexpr int P_BYTES = ATT2_ROWS * 128;                   // [128 rows][64 keys]
-    static constexpr int STAGES = HD == 128 ? 4 : 8;
+    static constexpr int K_SLOTS = HD == 128 ? 4 : 6;                 // K is released when the stage's scores are done,
+    static constexpr int V_SLOTS = HD == 128 ? 6 : 8;                 // V two steps later
     static constexpr int BAR_BYTES = 512;
-    static constexpr int TOTAL = 1024 + STAGES * STAGE_BYTES + 2 * Q_BYTES + 2 * P_BYTES + BAR_BYTES;
-    static constexpr int TMEM_COLS = 256;                             // O: HD columns at 0; S buffers at 128 and 192
+    static constexpr int TOTAL = 1024 + (K_SLOTS + V_SLOTS) * K_BYTES + Q_BYTES + 2 * P_BYTES + BAR_BYTES;
+    static constexpr int TMEM_COLS = 512;   // O: HD columns at 0; two score buffers of 2 x 64 columns at 128 and 256
 };
 
 __device__ __forceinline__ void att2_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -49,24 +50,28 @@ template <int HD>
 __global__ void __launch_bounds__(ATT2_THREADS, 1)
 attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
     using SM = Attn2Smem<HD>;
-    constexpr int HALVES = SM::HALVES;
+    constexpr int HALVES = SM::HALVES, KS = SM::K_SLOTS, VS = SM::V_SLOTS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* stages = smem;
-    uint8_t* qbuf = smem + SM::STAGES * SM::STAGE_BYTES;
-    uint8_t* pbuf = qbuf + 2 * SM::Q_BYTES;
-    uint64_t* kv_full = reinterpret_cast<uint64_t*>(pbuf + 2 * SM::P_BYTES);
-    uint64_t* kv_empty = kv_full + SM::STAGES;
-    uint64_t* q_full = kv_empty + SM::STAGES;    // [2]
-    uint64_t* q_empty = q_full + 2;              // [2] the item's last QK^T has read the tile
-    uint64_t* s_full = q_empty + 2;              // [2] scores of a stage are in tensor memory
-    uint64_t* s_empty = s_full + 2;              // [2] the softmax warps have read them
-    uint64_t* p_full = s_empty + 2;              // [2] P of a stage is in shared memory (and O rescaled if need be)
-    uint64_t* p_empty = p_full + 2;              // [2] the stage's P V has completed
-    uint64_t* o_full = p_empty + 2;              // the item's last P V has completed
-    uint64_t* o_empty = o_full + 1;              // the softmax warps have read O
+    uint8_t* kring = smem;
+    uint8_t* vring = kring + KS * SM::K_BYTES;
+    uint8_t* qbuf = vring + VS * SM::K_BYTES;
+    uint8_t* pbuf = qbuf + SM::Q_BYTES;
+    uint64_t* k_full = reinterpret_cast<uint64_t*>(pbuf + 2 * SM::P_BYTES);
+    uint64_t* k_empty = k_full + KS;     // the stage's scores are complete
+    uint64_t* v_full = k_empty + KS;
+    uint64_t* v_empty = v_full + VS;     // the stage's P V is complete
+    uint64_t* q_full = v_empty + VS;
+    uint64_t* q_empty = q_full + 1;      // the item's last QK^T has read the tile
+    uint64_t* s_full = q_empty + 1;      // [2] scores of a stage are in tensor memory
+    uint64_t* s_empty = s_full + 2;      // [2] the softmax warps have read them
+    uint64_t* p_full = s_empty + 2;      // [2] P of a stage is in shared memory (and O rescaled if need be)
+    uint64_t* p_empty = p_full + 2;      // [2] the stage's P V is complete
+    uint64_t* o_full = p_empty + 2;      // the item's last P V is complete
+    uint64_t* o_empty = o_full + 1;      // the softmax warps have read O
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 1);
     int* last_flag = reinterpret_cast<int*>(tmem_slot + 1);
+    static_assert((2 * KS + 2 * VS + 12) * 8 + 8 <= SM::BAR_BYTES, "barrier area");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int it_begin = p.cta_begin[blockIdx.x], it_end = p.cta_begin[blockIdx.x + 1];
@@ -76,13 +81,17 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&tmQ);
         tma_prefetch_desc(&tmKV);
-        for (int s = 0; s < SM::STAGES; ++s) {
-            mbar_init(&kv_full[s], 1);
-            mbar_init(&kv_empty[s], 1);
+        for (int s = 0; s < KS; ++s) {
+            mbar_init(&k_full[s], 1);
+            mbar_init(&k_empty[s], 1);
         }
+        for (int s = 0; s < VS; ++s) {
+            mbar_init(&v_full[s], 1);
+            mbar_init(&v_empty[s], 1);
+        }
+        mbar_init(q_full, 1);
+        mbar_init(q_empty, 1);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&q_full[s], 1);
-            mbar_init(&q_empty[s], 1);
             mbar_init(&s_full[s], 1);
             mbar_init(&s_empty[s], 4);
             mbar_init(&p_full[s], 4);
@@ -113,13 +122,13 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         for (int it = it_begin; list_ok && it < it_end && ok; ++it) {
             const AttnItem item = p.items[it];
             if (!attn_item_ok(item, p)) break;   // the other roles flag it and stop as well
-            const int qi = it - it_begin, qb = qi & 1;
+            const int qi = it - it_begin;
             if (lane == 0) {
-                if (qi >= 2) ok = mbar_wait(&q_empty[qb], ((qi >> 1) - 1) & 1, p.status);
+                if (qi >= 1) ok = mbar_wait(q_empty, (uint32_t)(qi - 1) & 1u, p.status);
                 if (ok) {
-                    mbar_expect_tx(&q_full[qb], (uint32_t)p.q_box_tokens * G * HD * 2u);
+                    mbar_expect_tx(q_full, (uint32_t)p.q_box_tokens * G * HD * 2u);
                     for (int h = 0; h < HALVES; ++h)
-                        tma_load_4d(qbuf + qb * SM::Q_BYTES + h * (ATT2_ROWS * 128), &tmQ, &q_full[qb], 0, h, item.kvh * G, item.q_tok);
+                        tma_load_4d(qbuf + h * (ATT2_ROWS * 128), &tmQ, q_full, 0, h, item.kvh * G, item.q_tok);
                 }
             }
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
@@ -129,13 +138,17 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             int pidx = (item.kv_begin >> 4) + my_pg;
             int page = (my_pg < ATT_STAGE_PAGES && pidx <= last_page) ? pt[pidx] : 0;
             for (int kv0 = item.kv_begin; kv0 < item.kv_end; kv0 += ATT2_STAGE_KEYS, ++st) {
-                const int s = st % SM::STAGES;
+                const int ks = st % KS, vs = st % VS;
                 const int nidx = pidx + ATT_STAGE_PAGES;
                 const int page_next = (my_pg < ATT_STAGE_PAGES && nidx <= last_page) ? pt[nidx] : 0;
                 const int npg = min(ATT_STAGE_PAGES, (item.kv_end - kv0 + 15) >> 4);
                 if (lane == 0) {
-                    if (st >= (uint32_t)SM::STAGES) ok = mbar_wait(&kv_empty[s], ((st / SM::STAGES) - 1) & 1, p.status);
-                    if (ok) mbar_expect_tx(&kv_full[s], (uint32_t)npg * 2u * HALVES * SM::KBOX_BYTES);
+                    if (st >= (uint32_t)KS) ok = mbar_wait(&k_empty[ks], ((st / KS) - 1) & 1u, p.status);
+                    if (ok && st >= (uint32_t)VS) ok = mbar_wait(&v_empty[vs], ((st / VS) - 1) & 1u, p.status);
+                    if (ok) {
+                        mbar_expect_tx(&k_full[ks], (uint32_t)npg * HALVES * SM::KBOX_BYTES);
+                        mbar_expect_tx(&v_full[vs], (uint32_t)npg * HALVES * SM::KBOX_BYTES);
+                    }
                 }
                 ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
@@ -145,9 +158,9 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
                 if (my_pg < npg) {
                     const int row0 = (p.layer_block0 + 2 * (page * p.n_kv_heads + item.kvh) + my_v) * 16;
-                    tma_load_2d(stages + s * SM::STAGE_BYTES + my_v * SM::K_BYTES + my_half * (ATT2_STAGE_KEYS * 128) +
-                                    my_pg * SM::KBOX_BYTES,
-                                &tmKV, &kv_full[s], my_half * 64, row0);
+                    uint8_t* dst = (my_v ? vring + vs * SM::K_BYTES : kring + ks * SM::K_BYTES) +
+                                   my_half * (ATT2_STAGE_KEYS * 128) + my_pg * SM::KBOX_BYTES;
+                    tma_load_2d(dst, &tmKV, my_v ? &v_full[vs] : &k_full[ks], my_half * 64, row0);
                 }
                 page = page_next;
                 pidx = nidx;
@@ -155,60 +168,73 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (one thread)
+        // An MMA into the accumulator of its predecessor waits about 144 cycles for it, more than
+        // these small MMAs take, so three accumulators are in flight and consecutive MMAs go to
+        // different ones: the scores of stage k as two partial sums over halves of the head
+        // dimension (the softmax warps add them), and O += P V of stage k - 2.
         if (elect_one()) {
-            uint32_t st = 0;
+            uint32_t st = 0;   // global stage counter of the item's first stage
             bool ok = true;
             const uint32_t idesc_pv = umma_idesc_f16_bmn(ATT2_ROWS, HD);
-            // P V of stage `t` (global stage counter) with `npg` pages of keys; `first`: the item's first stage
-            auto issue_pv = [&](uint32_t t, int npg, bool first, int qi) -> bool {
-                const uint32_t sb = t & 1u;
-                if (!mbar_wait(&p_full[sb], (t >> 1) & 1u, p.status)) return false;
-                if (first && qi >= 1 && !mbar_wait(o_empty, (uint32_t)(qi - 1) & 1u, p.status)) return false;
-                tc_fence_after();
-                const uint32_t p_addr = smem_u32(pbuf + sb * SM::P_BYTES);
-                const uint32_t v_addr = smem_u32(stages + (t % SM::STAGES) * SM::STAGE_BYTES + SM::K_BYTES);
-                for (int k = 0; k < npg; ++k)
-                    umma_bf16(tmem_base, umma_desc_k128(p_addr) + 2 * k,
-                              umma_desc_mn128(v_addr + k * 2048, ATT2_STAGE_KEYS * 128, 1024), idesc_pv, !(first && k == 0));
-                umma_commit(&kv_empty[t % SM::STAGES]);
-                umma_commit(&p_empty[sb]);
-                return true;
-            };
+            constexpr int QK_STEPS = HD / 32;   // k-steps of 16 dims per partial sum
             for (int it = it_begin; list_ok && it < it_end && ok; ++it) {
                 const AttnItem item = p.items[it];
                 if (!attn_item_ok(item, p)) break;
-                const int qi = it - it_begin, qb = qi & 1;
-                ok = mbar_wait(&q_full[qb], (qi >> 1) & 1, p.status);
+                const int qi = it - it_begin;
+                ok = mbar_wait(q_full, (uint32_t)qi & 1u, p.status);
                 if (!ok) break;
-                const uint32_t q_addr = smem_u32(qbuf + qb * SM::Q_BYTES);
-                int prev_npg = 0;
-                for (int kv0 = item.kv_begin; kv0 < item.kv_end; kv0 += ATT2_STAGE_KEYS, ++st) {
-                    const int s = st % SM::STAGES;
-                    const uint32_t sb = st & 1u;
-                    const int npg = min(ATT_STAGE_PAGES, (item.kv_end - kv0 + 15) >> 4);
-                    ok = mbar_wait(&kv_full[s], (st / SM::STAGES) & 1u, p.status);
-                    if (ok && (st >> 1) >= 1) ok = mbar_wait(&s_empty[sb], ((st >> 1) - 1) & 1u, p.status);
+                const uint32_t q_addr = smem_u32(qbuf);
+                const int n_st = (item.kv_end - item.kv_begin + ATT2_STAGE_KEYS - 1) / ATT2_STAGE_KEYS;
+                auto pages_of = [&](int k) { return min(ATT_STAGE_PAGES, (item.kv_end - item.kv_begin - k * ATT2_STAGE_KEYS + 15) >> 4); };
+                // step k: scores of stage k (k < n_st) interleaved with P V of stage k - 2 (k >= 2)
+                for (int k = 0; k < n_st + 2 && ok; ++k) {
+                    const bool qk = k < n_st, pv = k >= 2;
+                    const uint32_t tq = st + k, tp = st + k - 2;
+                    uint32_t k_addr = 0, idesc_qk = 0, s_tmem = 0, p_addr = 0, v_addr = 0;
+                    int npv = 0;
+                    if (qk) {
+                        ok = mbar_wait(&k_full[tq % KS], (tq / KS) & 1u, p.status);
+                        if (ok && (tq >> 1) >= 1) ok = mbar_wait(&s_empty[tq & 1u], ((tq >> 1) - 1) & 1u, p.status);
+                        k_addr = smem_u32(kring + (tq % KS) * SM::K_BYTES);
+                        idesc_qk = umma_idesc_f16(ATT2_ROWS, 16 * pages_of(k));
+                        s_tmem = tmem_base + 128 + (tq & 1u) * 128;
+                    }
+                    if (pv && ok) {
+                        ok = mbar_wait(&p_full[tp & 1u], (tp >> 1) & 1u, p.status);
+                        if (ok) ok = mbar_wait(&v_full[tp % VS], (tp / VS) & 1u, p.status);
+                        if (ok && k == 2 && qi >= 1) ok = mbar_wait(o_empty, (uint32_t)(qi - 1) & 1u, p.status);
+                        p_addr = smem_u32(pbuf + (tp & 1u) * SM::P_BYTES);
+                        v_addr = smem_u32(vring + (tp % VS) * SM::K_BYTES);
+                        npv = pages_of(k - 2);
+                    }
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t k_addr = smem_u32(stages + s * SM::STAGE_BYTES);
-                    const uint32_t idesc_qk = umma_idesc_f16(ATT2_ROWS, 16 * npg);
 #pragma unroll
-                    for (int h = 0; h < HALVES; ++h)
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            umma_bf16(tmem_base + 128 + sb * 64, umma_desc_k128(q_addr + h * (ATT2_ROWS * 128)) + 2 * k,
-                                      umma_desc_k128(k_addr + h * (ATT2_STAGE_KEYS * 128)) + 2 * k, idesc_qk, (h | k) != 0);
-                    umma_commit(&s_full[sb]);
-                    if (kv0 + ATT2_STAGE_KEYS >= item.kv_end) umma_commit(&q_empty[qb]);
-                    if (kv0 > item.kv_begin) {
-                        ok = issue_pv(st - 1, prev_npg, kv0 - ATT2_STAGE_KEYS == item.kv_begin, qi);
-                        if (!ok) break;
+                    for (int i = 0; i < 4; ++i) {
+                        if (qk && i < QK_STEPS) {
+                            // partial sum A: dims [0, HD/2) -> columns 0..63 of the buffer; B: dims [HD/2, HD) -> 64..127
+                            const uint32_t qa = 2 * i, ka = 2 * i;
+                            const uint32_t qb = HD == 128 ? ((ATT2_ROWS * 128) >> 4) + 2 * i : 2 * (i + QK_STEPS);
+                            const uint32_t kb = HD == 128 ? ((ATT2_STAGE_KEYS * 128) >> 4) + 2 * i : 2 * (i + QK_STEPS);
+                            umma_bf16(s_tmem, umma_desc_k128(q_addr) + qa, umma_desc_k128(k_addr) + ka, idesc_qk, i != 0);
+                            umma_bf16(s_tmem + 64, umma_desc_k128(q_addr) + qb, umma_desc_k128(k_addr) + kb, idesc_qk, i != 0);
+                        }
+                        if (pv && i < npv)
+                            umma_bf16(tmem_base, umma_desc_k128(p_addr) + 2 * i,
+                                      umma_desc_mn128(v_addr + i * 2048, ATT2_STAGE_KEYS * 128, 1024), idesc_pv, !(k == 2 && i == 0));
                     }
-                    prev_npg = npg;
+                    if (qk) {
+                        umma_commit(&s_full[tq & 1u]);
+                        umma_commit(&k_empty[tq % KS]);
+                        if (k == n_st - 1) umma_commit(q_empty);
+                    }
+                    if (pv) {
+                        umma_commit(&v_empty[tp % VS]);
+                        umma_commit(&p_empty[tp & 1u]);
+                        if (k == n_st + 1) umma_commit(o_full);
+                    }
                 }
-                if (!ok) break;
-                ok = issue_pv(st - 1, prev_npg, item.kv_end - item.kv_begin <= ATT2_STAGE_KEYS, qi);
-                if (ok) umma_commit(o_full);
+                st += (uint32_t)n_st;
             }
         }
         __syncwarp();
@@ -241,10 +267,19 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 uint32_t s0[32], s1[32];
                 if (ok) ok = wait_all(&s_full[sb], us & 1u);
                 if (ok) {
+                    // the two partial sums of the scores (halves of the head dimension)
+                    uint32_t b0[32];
                     tc_fence_after();
-                    tmem_ld32(t_lane + 128 + sb * 64, s0);
-                    tmem_ld32(t_lane + 128 + sb * 64 + 32, s1);
+                    tmem_ld32(t_lane + 128 + sb * 128, s0);
+                    tmem_ld32(t_lane + 128 + sb * 128 + 64, b0);
                     tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) s0[c] = __float_as_uint(__uint_as_float(s0[c]) + __uint_as_float(b0[c]));
+                    tmem_ld32(t_lane + 128 + sb * 128 + 32, s1);
+                    tmem_ld32(t_lane + 128 + sb * 128 + 96, b0);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) s1[c] = __float_as_uint(__uint_as_float(s1[c]) + __uint_as_float(b0[c]));
                     tc_fence_before();
                 } else {
 #pragma unroll
