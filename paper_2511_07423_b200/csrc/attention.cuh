@@ -6,8 +6,9 @@
 // at most 64), so every K/V byte of the item is read from HBM once.  A persistent CTA walks a
 // host-planned list of items.  One producer warp streams pages (TMA, 128-byte swizzle, one box of
 // 32 rows x 128 bytes per page and 64-element half: K and V of 16 tokens) and the item's Q tile
-// through mbarrier rings; its lanes fetch the page-table entries of the next stage while the
-// current one is in flight (its warpgroup gives most of its registers to the consumers).  Eight consumer warps form two groups that take alternate stages, so
+// through mbarrier rings; its lanes hold the page-table entries of eight stages and fetch the next
+// eight stages' entries meanwhile (its warpgroup gives most of its registers to the consumers).
+// Eight consumer warps form two groups that take alternate stages, so
 // every scheduler of the SM holds two warps; inside a group the four warps split the item's row
 // tiles and, when there are fewer than four row tiles, the pages of the stage.  QK^T and PV run on
 // warp-level MMAs (m16n8k16, half-precision operands, fp32 accumulate) with an online softmax in fp32 (base 2).
@@ -323,15 +324,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             }
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
+            // Page-table entries: the warp holds the entries of 8 stages (32 pages, one per lane) and fetches the
+            // next 32 while those are in use, so no load's latency sits between two stages' requests.
             const int* pt = p.page_tables + (size_t)item.req * p.max_pages;
-            const int last_page = (item.kv_end - 1) >> 4;
-            // this lane's page of the first stage; the next stage's entry is fetched one stage ahead
-            int pidx = (item.kv_begin >> 4) + my_pg;
-            int page = (my_pg < ATT_STAGE_PAGES && pidx <= last_page) ? pt[pidx] : 0;
-            for (int kv0 = item.kv_begin; kv0 < item.kv_end; kv0 += 16 * ATT_STAGE_PAGES, ++st) {
+            const int first_page = item.kv_begin >> 4, last_page = (item.kv_end - 1) >> 4;
+            int ent_cur = first_page + lane <= last_page ? pt[first_page + lane] : 0;
+            int ent_next = first_page + 32 + lane <= last_page ? pt[first_page + 32 + lane] : 0;
+            int k = 0;   // stage of the item
+            for (int kv0 = item.kv_begin; kv0 < item.kv_end; kv0 += 16 * ATT_STAGE_PAGES, ++st, ++k) {
                 const int s = st % SM::STAGES;
-                const int nidx = pidx + ATT_STAGE_PAGES;
-                const int page_next = (my_pg < ATT_STAGE_PAGES && nidx <= last_page) ? pt[nidx] : 0;
+                if (k > 0 && (k & 7) == 0) {
+                    ent_cur = ent_next;
+                    const int nidx = first_page + (k >> 3) * 32 + 32 + lane;
+                    ent_next = nidx <= last_page ? pt[nidx] : 0;
+                }
+                int page = __shfl_sync(0xFFFFFFFFu, ent_cur, ((k & 7) * ATT_STAGE_PAGES + my_pg) & 31);
                 const int npg = min(ATT_STAGE_PAGES, (item.kv_end - kv0 + 15) >> 4);
                 uint64_t* fb = &full_bar[(st & 1u) * SM::STAGES + s];   // the consuming group's barrier
                 if (lane == 0) {
@@ -349,8 +356,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
                     tma_load_2d(stages + s * SM::STAGE_BYTES + my_pg * SM::PAGE_BYTES + my_half * 4096, &tmKV, fb,
                                 my_half * 64, row0);
                 }
-                page = page_next;
-                pidx = nidx;
             }
         }
         return;

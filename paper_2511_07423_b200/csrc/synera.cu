@@ -276,7 +276,7 @@ struct syn_kv {
     op16* pool = nullptr;   // half precision (K and V enter and leave through syn_kv_import / syn_kv_export as bf16)
     uint32_t n_pages, page_size;
     size_t layer_elems;
-    CUtensorMap tm_kv, tm_kv16;   // boxes of 32 rows (K and V of a page and head) and of 16 rows (K or V)
+    CUtensorMap tm_kv, tm_kv5;   // boxes of 32 rows (K and V of a page and head), in two row orders
 };
 
 struct syn_plan {
@@ -614,9 +614,21 @@ extern "C" int syn_kv_alloc(syn_model* m, uint32_t n_pages, uint32_t page_size, 
         syn_kv_free(kv);
         return SYN_E_CUDA;
     }
-    if (make_map_2d(&kv->tm_kv16, kv->pool, blocks * page_size, c.head_dim, c.head_dim, page_size) != SYN_OK) {
-        syn_kv_free(kv);
-        return SYN_E_CUDA;
+    {
+        // The same box for the tensor-memory attention kernel, landing in shared memory as
+        // [K rows 0-7][V rows 0-7][K rows 8-15][V rows 8-15]: the 8-row groups of K (and of V) of consecutive
+        // boxes are then evenly spaced, which a tcgen05 operand descriptor needs.  Dimensions: dim, row in a
+        // group, K or V, group, (page, head) block.
+        const cuuint64_t hd2 = (cuuint64_t)c.head_dim * 2;
+        cuuint64_t dims[5] = {c.head_dim, 8, 2, 2, (cuuint64_t)blocks / 2};
+        cuuint64_t strides[4] = {hd2, 16 * hd2, 8 * hd2, 32 * hd2};
+        cuuint32_t box[5] = {64, 8, 2, 2, 1};
+        cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        if (g_encode(&kv->tm_kv5, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, kv->pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+            syn_kv_free(kv);
+            return SYN_E_CUDA;
+        }
     }
     if (cudaDeviceSynchronize() != cudaSuccess) {
         syn_kv_free(kv);
@@ -1260,9 +1272,9 @@ static int launch_attention(syn_model* m, syn_kv* kv, const syn_plan* p, uint32_
         ProfScope prof(m, 2, st);
         cudaError_t e;
         if (p->row_cap == 128 && c.head_dim == 128)
-            e = launch_pdl(attn2_kernel<128>, dim3(p->n_cta), dim3(ATT2_THREADS), Attn2Smem<128>::TOTAL, st, m->tm_q4, kv->tm_kv16, ap);
+            e = launch_pdl(attn2_kernel<128>, dim3(p->n_cta), dim3(ATT2_THREADS), Attn2Smem<128>::TOTAL, st, m->tm_q4, kv->tm_kv5, ap);
         else if (p->row_cap == 128)
-            e = launch_pdl(attn2_kernel<64>, dim3(p->n_cta), dim3(ATT2_THREADS), Attn2Smem<64>::TOTAL, st, m->tm_q4, kv->tm_kv16, ap);
+            e = launch_pdl(attn2_kernel<64>, dim3(p->n_cta), dim3(ATT2_THREADS), Attn2Smem<64>::TOTAL, st, m->tm_q4, kv->tm_kv5, ap);
         else if (c.head_dim == 128)
             e = launch_pdl(attn_kernel<128>, dim3(p->n_cta), dim3(ATT_THREADS), AttnSmem<128>::TOTAL, st, tmQ, kv->tm_kv, ap);
         else
@@ -1798,9 +1810,9 @@ static int syn_op_attention_static_impl(syn_model* m, syn_kv* kv, const syn_plan
     AttnParams ap;
     attn_params(ap, m, kv, p, layer, (op16*)out, part_o, part_ml, group_count);
     if (p->row_cap == 128 && c.head_dim == 128)
-        attn2_kernel<128><<<p->n_cta, ATT2_THREADS, Attn2Smem<128>::TOTAL, st>>>(m->tm_q4, kv->tm_kv16, ap);
+        attn2_kernel<128><<<p->n_cta, ATT2_THREADS, Attn2Smem<128>::TOTAL, st>>>(m->tm_q4, kv->tm_kv5, ap);
     else if (p->row_cap == 128)
-        attn2_kernel<64><<<p->n_cta, ATT2_THREADS, Attn2Smem<64>::TOTAL, st>>>(m->tm_q4, kv->tm_kv16, ap);
+        attn2_kernel<64><<<p->n_cta, ATT2_THREADS, Attn2Smem<64>::TOTAL, st>>>(m->tm_q4, kv->tm_kv5, ap);
     else if (c.head_dim == 128)
         attn_kernel<128><<<p->n_cta, ATT_THREADS, AttnSmem<128>::TOTAL, st>>>(m->tm_q, kv->tm_kv, ap);
     else
