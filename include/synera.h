@@ -183,6 +183,7 @@ typedef struct {
     double attn_flops;             /* 4 * Hq*hd * n_layers * sum over tokens of keys seen    */
     int32_t attn_items, attn_split_items; /* attention work items per layer / those that are partial */
     int32_t kernel_launches;       /* kernels launched by one syn_verify_run                */
+    int32_t attn_rows;             /* row tile of the attention kernel the batch was planned for: 64 (warp-level MMAs) or 128 (tcgen05) */
     int64_t h2d_bytes;             /* batch description uploaded per step by syn_verify_batch */
     double t_gpu_ms;               /* device time of the step, first kernel to last (CUDA events); 0 unless profiling is on */
     double t_wall_ms;              /* host wall time of the blocking call that ran it; 0 unless profiling is on  */
@@ -257,8 +258,9 @@ int syn_op_linear_reset(void);
  * pairs from 256 tokens on); 1 keeps all of them on the one-CTA kernel, so that both can be measured
  * and checked on the same batch.  Process-wide.
  * syn_debug_set_attention: which attention kernel the plans made AFTERWARDS are laid out for (a plan
- * keeps its kernel): 0 default, 1 the warp-level-MMA kernel (row tiles of 64), 2 the tcgen05 kernel (row
- * tiles of 128: a whole chunk of up to 128 / G tokens is one work item per kv head).  Process-wide. */
+ * keeps its kernel): 0 (default) the cheaper of the two for the batch by the planner's cost model, 1 the
+ * warp-level-MMA kernel (row tiles of 64), 2 the tcgen05 kernel (row tiles of 128: a whole chunk of up to
+ * 128 / G tokens is one work item per kv head).  Process-wide. */
 int syn_debug_set_spin_limit(int64_t cycles);
 int syn_debug_linear_counter(int32_t index, int32_t value);
 int syn_debug_set_schedule(int32_t which);

@@ -46,7 +46,7 @@ class StepStats(C.Structure):
     _fields_ = [("n_req", C.c_int32), ("n_tokens", C.c_int32), ("ctx_tokens", C.c_int64),
                 ("weight_bytes", C.c_int64), ("kv_read_bytes", C.c_int64), ("kv_write_bytes", C.c_int64),
                 ("dense_flops", C.c_double), ("attn_flops", C.c_double), ("attn_items", C.c_int32),
-                ("attn_split_items", C.c_int32), ("kernel_launches", C.c_int32), ("h2d_bytes", C.c_int64),
+                ("attn_split_items", C.c_int32), ("kernel_launches", C.c_int32), ("attn_rows", C.c_int32), ("h2d_bytes", C.c_int64),
                 ("t_gpu_ms", C.c_double), ("t_wall_ms", C.c_double)]
 
 KERNEL_CLASSES = ("prep", "qkv_gemm", "attention", "attention_merge", "o_gemm", "gate_up_gemm", "down_gemm",

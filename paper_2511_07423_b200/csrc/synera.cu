@@ -28,9 +28,9 @@ constexpr int GEMM_MAX_SPLITS = 8;   // most CTAs that share one pair tile's K r
 static long long g_spin_limit = SYN_SPIN_LIMIT_CYCLES;
 // 0: every projection takes the kernel its shape calls for; 1: the one-CTA kernel always (syn_debug_set_schedule).
 static int g_schedule = 0;
-// Attention kernel: 0 = the default of attn_row_cap(), 1 = warp-level MMAs (64-row tiles), 2 = tcgen05 (128-row tiles).
+// Attention kernel: 0 = whichever the planner's cost model makes cheaper for the batch, 1 = warp-level MMAs
+// (64-row tiles), 2 = tcgen05 (128-row tiles).
 static int g_attention = 0;
-static int attn_row_cap() { return g_attention == 2 ? 128 : 64; }
 
 // Name of the last CUDA error a call of this library met on this thread (for syn_last_cuda_error).
 static thread_local const char* g_last_cuda_error = "";
@@ -687,7 +687,7 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Host-side result of planning one batch (no device involved).
 struct HostPlan {
-    int T = 0, n_cta = 0, n_parts = 0;
+    int T = 0, n_cta = 0, n_parts = 0, row_cap = 64;
     std::vector<int> pos, slot, cta_begin;
     std::vector<AttnItem> items;          // sorted by CTA
     std::vector<MergeGroup> groups;
@@ -698,7 +698,7 @@ struct HostPlan {
 // (the "flatten" of paper Sec. 4.5).  Pure host code.
 static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_sm, int32_t n_req,
                         const int32_t* chunk_tokens, const int32_t* chunk_offsets, const int32_t* page_tables,
-                        int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, int row_cap, HostPlan& hp) {
+                        int32_t max_pages, const int32_t* ctx_lens, const int32_t* n_uncached, int attention, HostPlan& hp) {
     if (n_req <= 0 || !chunk_tokens || !chunk_offsets || !page_tables || !ctx_lens || max_pages <= 0 || n_sm <= 0)
         return SYN_E_INVALID_ARG;
     const int G = c.n_q_heads / c.n_kv_heads, Hkv = c.n_kv_heads;
@@ -758,23 +758,32 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
     // when one unit alone would exceed a CTA's fair share: every split costs an fp32 partial and a
     // merge.
     const int n_cta_max = n_sm;
-    // The tensor-memory kernel (row_cap 128) spends the same time on a stage whatever the number of rows.
-    const bool wide = row_cap == 128;
-    const int tok_per_group = wide ? std::min(SYN_MAX_CHUNK, 128 / G) : std::min(16, 64 / G);
+    // Two kernels: the warp-level-MMA one (row tiles of 64: a stage costs more the more 16-row tiles the
+    // item has, and a chunk of more than 64 / G tokens is several items that each read the request's keys)
+    // and the tensor-memory one (row tiles of 128: the same time per stage whatever the number of rows,
+    // a larger fixed cost per item).  Unless one is asked for, the batch takes the cheaper by this model.
     static const int STAGE_COST[5] = {0, 1040, 1200, 1500, 1540};
-    const int WIDE_STAGE_COST = 1300;
-    const int ITEM_COST = wide ? 6000 : 5500, PART_COST = wide ? 4000 : 3000;
+    const int WIDE_STAGE_COST = 1500;
+    auto total_of = [&](bool w) {
+        const int tpg = w ? std::min(SYN_MAX_CHUNK, 128 / G) : std::min(16, 64 / G);
+        int64_t sum = 0;
+        for (int i = 0; i < n_req; ++i) {
+            const int n = chunk_offsets[i + 1] - chunk_offsets[i];
+            for (int j0 = 0; j0 < n; j0 += tpg) {
+                const int nj = std::min(tpg, n - j0);
+                sum += ((int64_t)((ctx_lens[i] + j0 + nj + 63) / 64) * (w ? WIDE_STAGE_COST : STAGE_COST[(nj * G + 15) / 16]) + (w ? 8000 : 5500)) * Hkv;
+            }
+        }
+        return sum;
+    };
+    const bool wide = attention == 2 || (attention == 0 && total_of(true) < total_of(false));
+    hp.row_cap = wide ? 128 : 64;
+    const int tok_per_group = wide ? std::min(SYN_MAX_CHUNK, 128 / G) : std::min(16, 64 / G);
+    const int ITEM_COST = wide ? 8000 : 5500, PART_COST = wide ? 4000 : 3000;
     auto unit_cost = [&](int L, int nj) {
         return (int64_t)((L + 63) / 64) * (wide ? WIDE_STAGE_COST : STAGE_COST[(nj * G + 15) / 16]) + ITEM_COST;
     };
-    int64_t total_cost = 0;
-    for (int i = 0; i < n_req; ++i) {
-        const int b = chunk_offsets[i], n = chunk_offsets[i + 1] - b;
-        for (int j0 = 0; j0 < n; j0 += tok_per_group) {
-            const int nj = std::min(tok_per_group, n - j0);
-            total_cost += unit_cost(ctx_lens[i] + j0 + nj, nj) * Hkv;
-        }
-    }
+    const int64_t total_cost = total_of(wide);
     const int64_t share = std::max<int64_t>(8 * (wide ? WIDE_STAGE_COST : STAGE_COST[4]) + ITEM_COST, (total_cost + n_cta_max - 1) / n_cta_max);
     std::vector<AttnItem> items;
     std::vector<int> item_cost;
@@ -939,6 +948,7 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
     s.attn_flops = 4.0 * qd * c.n_layers * (double)keys_seen;
     s.attn_items = n_items; s.attn_split_items = n_parts;
     s.kernel_launches = 1 + c.n_layers * 5 + 2;
+    s.attn_rows = hp.row_cap;
     return SYN_OK;
 }
 
@@ -949,7 +959,7 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     if (!m || !kv || kv->model != m) return SYN_E_INVALID_ARG;
     HostPlan hp;
     int r = plan_compute(m->desc, (int)kv->page_size, kv->n_pages, m->n_sm, n_req, chunk_tokens, chunk_offsets, page_tables,
-                         max_pages, ctx_lens, n_uncached, attn_row_cap(), hp);
+                         max_pages, ctx_lens, n_uncached, g_attention, hp);
     if (r) return r;
     const int T = hp.T, n_items = (int)hp.items.size(), n_cta = hp.n_cta;
     size_t off = 0;
@@ -985,7 +995,7 @@ static int plan_build(syn_plan* p, syn_model* m, syn_kv* kv, int32_t n_req, cons
     if (!hp.groups.empty()) memcpy(p->h<MergeGroup>(p->o_groups), hp.groups.data(), hp.groups.size() * sizeof(MergeGroup));
     p->n_req = n_req; p->T = T; p->max_pages = max_pages; p->n_items = n_items; p->n_cta = n_cta;
     p->n_groups = (int)hp.groups.size(); p->n_parts = hp.n_parts;
-    p->row_cap = attn_row_cap();
+    p->row_cap = hp.row_cap;
     p->stats = hp.stats;
     p->stats.h2d_bytes = (int64_t)off;
     p->kv = kv; p->kv_pool = kv->pool; p->kv_pages = kv->n_pages;
@@ -1004,7 +1014,7 @@ static int syn_plan_host_impl(const syn_model_desc* desc, uint32_t n_pages, uint
         return SYN_E_INVALID_ARG;
     HostPlan hp;
     int r = plan_compute(*desc, (int)page_size, n_pages, n_sm, n_req, chunk_tokens, chunk_offsets, page_tables, max_pages,
-                         ctx_lens, n_uncached, attn_row_cap(), hp);
+                         ctx_lens, n_uncached, g_attention, hp);
     if (r) return r;
     *n_items = (int)hp.items.size();
     *n_cta = hp.n_cta;

@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(params=[1, 2], ids=["warp_mma_attention", "tcgen05_attention"])
+def attention_kind(request):
+    """Plans made inside the test are laid out for the named attention kernel (the default leaves the
+    choice to the planner's cost model)."""
+    import paper_2511_07423_b200 as syn
+    syn.debug_set_attention(request.param)
+    yield request.param
+    syn.debug_set_attention(0)

@@ -91,7 +91,7 @@ def test_config1_tiny_real_prefill():
     (MINI_8B, [17, 64, 300, 1200], [16, 2, 9, 13]),                    # head_dim 128, G = 4
     (ModelShape("g5", 2, 640, 10, 2, 128, 1376, 3000), [100, 40], [16, 13]),   # G = 5, ffn and vocab with ragged tails
 ])
-def test_mini_shapes_synthetic_cache(shape, ctx, chunk):
+def test_mini_shapes_synthetic_cache(shape, ctx, chunk, attention_kind):
     wl = Workload("mini", shape, 11, len(ctx), ("list", tuple(ctx)), ("list", tuple(chunk)), 0.7)
     batch = gen.gen_batch(wl)
     glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)
@@ -106,7 +106,7 @@ def test_mini_shapes_synthetic_cache(shape, ctx, chunk):
     (MINI_1B, [7, 260], [32, 29], [1, 29]),                                             # head_dim 64
     (ModelShape("g5c", 2, 640, 10, 2, 128, 1376, 3000), [100, 33], [32, 27], [16, 3]),  # G = 5: groups of 12
 ])
-def test_chunks_up_to_32_and_long_uncached_runs(shape, ctx, chunk, unc):
+def test_chunks_up_to_32_and_long_uncached_runs(shape, ctx, chunk, unc, attention_kind):
     wl = Workload("chunk32", shape, 13, len(ctx), ("list", tuple(ctx)), ("list", tuple(chunk)), 0.7)
     batch = gen.gen_batch(wl)
     glob, layers, model, kv, orc, pools = _setup(shape, wl.seed, batch)

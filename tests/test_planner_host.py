@@ -28,12 +28,20 @@ def test_positions_and_slots_follow_the_page_table():
     assert r["slot"].tolist() == [4 * 16 + 12, 4 * 16 + 13, 4 * 16 + 14, 4 * 16 + 15, 0, 1, 2, 3, 16, 17, 18]
 
 
+@pytest.mark.parametrize("attention", [0, 1, 2], ids=["auto", "warp_mma", "tcgen05"])
 @pytest.mark.parametrize("cfg", [1, 2, 3, 4, 6])
-def test_work_list_covers_every_key_of_every_row_group_exactly_once(cfg):
+def test_work_list_covers_every_key_of_every_row_group_exactly_once(cfg, attention):
     wl = CONFIGS[cfg]
     shape = wl.shape
     batch = gen.gen_batch(wl)
-    r = _plan(shape, batch)
+    syn.debug_set_attention(attention)
+    try:
+        r = _plan(shape, batch)
+    finally:
+        syn.debug_set_attention(0)
+    rows = r["stats"].attn_rows
+    # the planner's own choice: 128-row tiles where a chunk would otherwise be several items per kv head
+    assert rows == {0: 128 if cfg == 6 else 64, 1: 64, 2: 128}[attention]
     items = r["items"].numpy()
     cb = r["cta_begin"].numpy()
     G, Hkv = shape.group, shape.n_kv_heads
@@ -41,7 +49,7 @@ def test_work_list_covers_every_key_of_every_row_group_exactly_once(cfg):
     offs = batch.chunk_offsets.numpy()
     cover = {}
     for q_tok, nj, kvh, req, kb, ke, qp0, part, grp in items:
-        assert offs[req] <= q_tok and q_tok + nj <= offs[req + 1] and 1 <= nj and nj * G <= 64
+        assert offs[req] <= q_tok and q_tok + nj <= offs[req + 1] and 1 <= nj and nj * G <= rows
         assert 0 <= kvh < Hkv and kb % 64 == 0 and kb < ke
         assert qp0 == batch.ctx_lens[req] + (q_tok - offs[req])
         assert ke <= qp0 + nj                       # never past the last key the group's last row may see
@@ -51,7 +59,7 @@ def test_work_list_covers_every_key_of_every_row_group_exactly_once(cfg):
     n_groups = 0
     for i in range(batch.n_req):
         n = offs[i + 1] - offs[i]
-        tpg = min(16, 64 // G)
+        tpg = min(16, 64 // G) if rows == 64 else min(32, 128 // G)
         for j0 in range(0, n, tpg):
             nj = min(tpg, n - j0)
             for h in range(Hkv):
