@@ -31,7 +31,8 @@ UNIT = "tokens/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from an ncu capture of two timed steps of the
 # workload (mean over all launches of the kernel function), with the hash of the kernel's source files at capture
 # time: the figure is reported only while those sources are unchanged.  Summaries of the captures: profiles/.
-KERNEL_SOURCES = {"attn_kernel": ("attention.cuh", "ptx.cuh"), "gemm_kernel": ("gemm.cuh", "ptx.cuh"),
+KERNEL_SOURCES = {"attn_kernel": ("attention.cuh", "ptx.cuh"), "attn2_kernel": ("attention2.cuh", "attention.cuh", "ptx.cuh"),
+                  "gemm_kernel": ("gemm.cuh", "ptx.cuh"),
                   "gemm2_kernel": ("gemm2.cuh", "gemm.cuh", "ptx.cuh")}
 NCU_TRAFFIC = {
     # workload: {kernel function: (bytes per launch, sha256 of its source files, concatenated in KERNEL_SOURCES order)}
@@ -203,6 +204,7 @@ def run_ours(args):
     shape = wl.shape
     peaks = _peaks()
     syn.debug_set_schedule({"auto": 0, "one-cta": 1}[args.schedule])
+    syn.debug_set_attention({"auto": 0, "warp-mma": 1, "tcgen05": 2}[args.attention])
 
     via_host = shape.dense_params() * 2 > 40e9
     model = synthetic.load_model(shape, wl.seed, via_host=via_host)
@@ -301,11 +303,14 @@ def run_ours(args):
         if name in kernels:
             kernels[name]["kernel"] = func_of[name]
     ridge = peaks["tf_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    # the attention kernel the planner chose for this batch: row tiles of 64 (warp-level MMAs) or 128 (tcgen05)
+    attn_func = "attn2_kernel" if st.attn_rows == 128 else "attn_kernel"
+    kernels["attention"]["kernel"] = attn_func
 
     def func_roof(func):
         """Roofline of one kernel function: the algorithmic work of its launches / the summed CUDA-event time of
         its launches (per launch: both divided by the number of launches)."""
-        if func == "attn_kernel":
+        if func == attn_func:
             return {"kernel": func, "bound": "hbm", "achieved": kernels["attention"]["kv_gbs"], "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "traffic": _traffic(wl.name, func), "share_of_step": kernels["attention"]["share"],
                     "launches_per_step": kernels["attention"]["launches_per_step"]}
@@ -324,7 +329,7 @@ def run_ours(args):
             out.update({"bound": "hbm", "achieved": wb / (ms_step * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"})
         return out
 
-    roofs = [r_ for r_ in (func_roof(fn) for fn in ("gemm2_kernel", "gemm_kernel", "attn_kernel")) if r_]
+    roofs = [r_ for r_ in (func_roof(fn) for fn in ("gemm2_kernel", "gemm_kernel", attn_func)) if r_]
     for r_ in roofs:
         r_["frac"] = r_["achieved"] / r_["peak"]
         r_["peak_source"] = peaks["source"] + (" sustained" if r_["bound"] == "tensor" else "")
@@ -356,7 +361,7 @@ def run_ours(args):
                         "results D2H, host clock",
         "arithmetic": "half-precision (fp16) operands holding the bf16 weights exactly, fp32 accumulation, fp32 residual stream",
         "config": {"workload": wl.name, "shape": shape.name, "n_req": B, "chunk_tokens": T, "ctx_tokens": int(st.ctx_tokens),
-                   "p_match": wl.p_match, "page_size": 16, "ctx_scale": batch.scale,
+                   "p_match": wl.p_match, "page_size": 16, "ctx_scale": batch.scale, "attention_kernel": attn_func,
                    "l2": "every step streams weights + KV far larger than L2; no flush needed",
                    "replicas": world},
         "e2e": {"value": whole_job_value(T, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e, "ms_per_step_median": ms_e2e_median,
@@ -455,6 +460,8 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="1..6; 3 = the 8B-shape step the metric is quoted on; 6 = 32-token chunked partial prefill")
     ap.add_argument("--pool-tokens", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--attention", default="auto", choices=["auto", "warp-mma", "tcgen05"],
+                    help="auto: the planner's cost model picks the attention kernel for the batch")
     ap.add_argument("--schedule", default="auto", choices=["auto", "one-cta"],
                     help="auto: every projection takes the kernel its shape calls for; one-cta: none takes the CTA-pair kernel")
     args = ap.parse_args()
