@@ -37,9 +37,13 @@ KERNEL_SOURCES = {"attn_kernel": ("attention.cuh", "ptx.cuh"), "attn2_kernel": (
 NCU_TRAFFIC = {
     # workload: {kernel function: (bytes per launch, sha256 of its source files, concatenated in KERNEL_SOURCES order)}
     "cfg3-8b": {
-        "attn_kernel": (616014112, "682f0116cfa8499d6b1c49c45b87bc8d9a30401ec6fa024850de59b7260f6846"),
-        "gemm_kernel": (285482664, "e8082fa3de83d7301bd5963a42f663d57750315c78ce009c4a2db741ec3d142f"),
-        "gemm2_kernel": (99062525, "67deb0babfce543e60d48b918e7bc89a8ad159385d0cf19562b496aaba0ddf2a"),
+        "attn_kernel": (616005760, "e7eab610c1c0e32bcd8a2b1b08bccefa5523b7c068fd3c6ca6349d9a5a0c9722"),
+        "gemm_kernel": (284994688, "415a44815d425fce6e0ffc40b6e9788e53f3b2c3d4b3acc83ceb62134c7a078c"),
+        "gemm2_kernel": (99183492, "61a52084542c4d41ffc56e91dceb9efb0846429310e9840952db0981acfd97ec"),
+    },
+    # one layer's launch of the same work list, captured through `opbench attention --config 6 --kind 2`
+    "cfg6-8b-chunk32": {
+        "attn2_kernel": (645844992, "5a02e9018c744d79ec1a3ae14e0b2f9cf236331e6d2ca9c578a435c7a48791da"),
     },
 }
 
