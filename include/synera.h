@@ -279,11 +279,12 @@ int syn_op_attention(syn_model *m, syn_kv *kv, const syn_plan *p, uint32_t layer
  * no counterpart; this is a service of the library.)  Same arguments, same result and same
  * asynchronous behaviour as syn_op_attention, but the partial results of work items that cover
  * only part of a request's keys live in a fixed array inside the library instead of a workspace
- * that grows on demand.  The array holds SYN_STATIC_MAX_PARTS partials (about 8.5 MB of every GPU
- * that loads the library, from load to exit).  The call itself allocates and frees nothing; the
+ * that grows on demand.  The array holds SYN_STATIC_MAX_PARTS partials of 64 rows, or half as many of
+ * the 128-row kind of a plan made for the tcgen05 kernel (about 8.5 MB of every GPU that loads the
+ * library, from load to exit).  The call itself allocates and frees nothing; the
  * model, cache and plan it is given were of course allocated earlier by their own calls.
- *   - A plan with more partial work items than SYN_STATIC_MAX_PARTS is refused with
- *     SYN_E_CAPACITY before anything is launched (syn_plan_stats().attn_split_items tells).
+ *   - A plan with more partial work items than that (attn_split_items x attn_rows of syn_plan_stats()
+ *     above SYN_STATIC_MAX_PARTS x 64) is refused with SYN_E_CAPACITY before anything is launched.
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call outside any stream capture.
  *   - All calls on a device share the one array.  It keeps the previous call's contents; nothing

@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("hd", [128, 64])
-def test_static_scratch_attention_equals_the_allocating_one_twice_in_a_row(hd):
+def test_static_scratch_attention_equals_the_allocating_one_twice_in_a_row(hd, attention_kind):
     import paper_2511_07423_b200 as syn
     shape = ModelShape("att-static", 1, 256, 8, 2, hd, 256, 512)
     seed = 21
