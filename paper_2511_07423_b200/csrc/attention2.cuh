@@ -10,10 +10,12 @@
 //   O += P V  : A = P (half precision, written by the softmax warps into shared memory in the
 //               K-major swizzled layout), B = V as it lies in the cache, [key][dim], i.e. an MN-major
 //               operand, D = O in tensor memory for the whole item.
-// Warp roles: warp 0 streams pages (TMA: one request per page and 64-dim half brings its 16 K rows and
-// 16 V rows as [K 0-7][V 0-7][K 8-15][V 8-15], so that the 8-row groups of K, and of V, of a stage's
-// four pages are evenly spaced; requests are the scarce resource of this loop, about 80 cycles each)
-// and the Q tile through mbarriers; one
+// Warp roles: warp 0 streams pages (TMA: one request brings the 16 K rows of a page, another its 16 V
+// rows, each as [rows 0-7: dims 0-63][rows 0-7: dims 64-127][rows 8-15: ...], so that the 8-row groups
+// of a stage's four pages are evenly spaced for either half of the head dimension; requests are the
+// scarce resource of this loop, about 80 cycles each; K and V have rings of their own because a
+// stage's K is free as soon as its scores are done, its V only after P V) and the Q tile through
+// mbarriers; one
 // thread of warp 1 issues every MMA; warps 4..7 and 8..11 are two softmax groups (one thread per row
 // each) that take alternate stages, each with its own score buffer, P buffer, running (max, sum) and
 // O accumulator in tensor memory; the first group combines the two at the end of the item and writes
@@ -37,14 +39,15 @@ constexpr float ATT2_RESCALE_GAP = 8.0f;   // log2 units
 template <int HD>
 struct Attn2Smem {
     static constexpr int HALVES = HD / 64;
-    static constexpr int BOX_BYTES = 32 * 128;                        // K and V rows of a page, one 64-dim half
-    static constexpr int HALF_BYTES = ATT_STAGE_PAGES * BOX_BYTES;    // the four pages of a stage, one half
-    static constexpr int STAGE_BYTES = HALVES * HALF_BYTES;           // [half][page][group of 8 keys][K | V][8 rows][128 bytes]
+    static constexpr int GROUP_BYTES = HALVES * 1024;                 // 8 rows: [64-dim half][8 rows][128 bytes]
+    static constexpr int BOX_BYTES = 2 * GROUP_BYTES;                 // the K rows (or the V rows) of a page
+    static constexpr int K_BYTES = ATT_STAGE_PAGES * BOX_BYTES;       // K (or V) of a stage: [page][group][half][8 rows][128 bytes]
     static constexpr int Q_BYTES = HALVES * ATT2_ROWS * 128;          // [half][128 rows][128 bytes]
     static constexpr int P_BYTES = ATT2_ROWS * 128;                   // [128 rows][64 keys]
-    static constexpr int STAGES = HD == 128 ? 5 : 10;
+    static constexpr int K_SLOTS = HD == 128 ? 4 : 8;                 // K is released when the stage's scores are done,
+    static constexpr int V_SLOTS = HD == 128 ? 6 : 12;                // V when its P V is
     static constexpr int BAR_BYTES = 512 + ATT2_ROWS * 8;             // barriers, then (max, sum) of the second group's rows
-    static constexpr int TOTAL = 1024 + STAGES * STAGE_BYTES + Q_BYTES + 2 * P_BYTES + BAR_BYTES;
+    static constexpr int TOTAL = 1024 + (K_SLOTS + V_SLOTS) * K_BYTES + Q_BYTES + 2 * P_BYTES + BAR_BYTES;
     static_assert(TOTAL <= 232448, "shared memory of one CTA");
     static constexpr int TMEM_COLS = 512;   // O of the two groups at 0 and 128; their score buffers (2 x 64 columns) at 256 and 384
 };
@@ -56,15 +59,18 @@ template <int HD>
 __global__ void __launch_bounds__(ATT2_THREADS, 1)
 attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, AttnParams p) {
     using SM = Attn2Smem<HD>;
-    constexpr int HALVES = SM::HALVES, NS = SM::STAGES;
+    constexpr int HALVES = SM::HALVES, KS = SM::K_SLOTS, VS = SM::V_SLOTS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* ring = smem;
-    uint8_t* qbuf = ring + NS * SM::STAGE_BYTES;
+    uint8_t* kring = smem;
+    uint8_t* vring = kring + KS * SM::K_BYTES;
+    uint8_t* qbuf = vring + VS * SM::K_BYTES;
     uint8_t* pbuf = qbuf + SM::Q_BYTES;
-    uint64_t* kv_full = reinterpret_cast<uint64_t*>(pbuf + 2 * SM::P_BYTES);
-    uint64_t* kv_empty = kv_full + NS;   // the stage's P V is complete
-    uint64_t* q_full = kv_empty + NS;
+    uint64_t* k_full = reinterpret_cast<uint64_t*>(pbuf + 2 * SM::P_BYTES);
+    uint64_t* k_empty = k_full + KS;     // the stage's scores are complete
+    uint64_t* v_full = k_empty + KS;
+    uint64_t* v_empty = v_full + VS;     // the stage's P V is complete
+    uint64_t* q_full = v_empty + VS;
     uint64_t* q_empty = q_full + 1;      // the item's last QK^T has read the tile
     uint64_t* s_full = q_empty + 1;      // [group] scores of a stage are in tensor memory
     uint64_t* s_empty = s_full + 2;      // [group] its warps have read them
@@ -74,8 +80,8 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     uint64_t* o_empty = o_full + 1;      // the first group has read both O
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 1);
     int* last_flag = reinterpret_cast<int*>(tmem_slot + 1);
-    static_assert((2 * NS + 12) * 8 + 8 <= 512, "barrier area");
-    float2* ml_x = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(kv_full) + 512);   // [128]
+    static_assert((2 * KS + 2 * VS + 12) * 8 + 8 <= 512, "barrier area");
+    float2* ml_x = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(k_full) + 512);   // [128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int it_begin = p.cta_begin[blockIdx.x], it_end = p.cta_begin[blockIdx.x + 1];
@@ -85,9 +91,13 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&tmQ);
         tma_prefetch_desc(&tmKV);
-        for (int s = 0; s < NS; ++s) {
-            mbar_init(&kv_full[s], 1);
-            mbar_init(&kv_empty[s], 1);
+        for (int s = 0; s < KS; ++s) {
+            mbar_init(&k_full[s], 1);
+            mbar_init(&k_empty[s], 1);
+        }
+        for (int s = 0; s < VS; ++s) {
+            mbar_init(&v_full[s], 1);
+            mbar_init(&v_empty[s], 1);
         }
         mbar_init(q_full, 1);
         mbar_init(q_empty, 1);
@@ -115,8 +125,8 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        // lane -> (page of the stage, 64-dim half): one request each
-        const int my_pg = lane / HALVES, my_half = lane % HALVES;
+        // lane -> (page of the stage, K or V): one request each
+        const int my_pg = lane >> 1, my_v = lane & 1;
         uint32_t st = 0;
         bool ok = true;
         for (int it = it_begin; list_ok && it < it_end && ok; ++it) {
@@ -141,7 +151,7 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             int ent_next = first_page + 32 + lane <= last_page ? pt[first_page + 32 + lane] : 0;
             int k = 0;   // stage of the item
             for (int kv0 = item.kv_begin; kv0 < item.kv_end; kv0 += ATT2_STAGE_KEYS, ++st, ++k) {
-                const int s = st % NS;
+                const int ks = st % KS, vs = st % VS;
                 if (k > 0 && (k & 7) == 0) {
                     ent_cur = ent_next;
                     const int nidx = first_page + (k >> 3) * 32 + 32 + lane;
@@ -150,8 +160,12 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 int page = __shfl_sync(0xFFFFFFFFu, ent_cur, ((k & 7) * ATT_STAGE_PAGES + my_pg) & 31);
                 const int npg = min(ATT_STAGE_PAGES, (item.kv_end - kv0 + 15) >> 4);
                 if (lane == 0) {
-                    if (st >= (uint32_t)NS) ok = mbar_wait(&kv_empty[s], ((st / NS) - 1) & 1u, p.status);
-                    if (ok) mbar_expect_tx(&kv_full[s], (uint32_t)npg * HALVES * SM::BOX_BYTES);
+                    if (st >= (uint32_t)KS) ok = mbar_wait(&k_empty[ks], ((st / KS) - 1) & 1u, p.status);
+                    if (ok && st >= (uint32_t)VS) ok = mbar_wait(&v_empty[vs], ((st / VS) - 1) & 1u, p.status);
+                    if (ok) {
+                        mbar_expect_tx(&k_full[ks], (uint32_t)npg * SM::BOX_BYTES);
+                        mbar_expect_tx(&v_full[vs], (uint32_t)npg * SM::BOX_BYTES);
+                    }
                 }
                 ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
@@ -160,8 +174,9 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     page = 0;
                 }
                 if (my_pg < npg) {
-                    tma_load_5d(ring + s * SM::STAGE_BYTES + my_half * SM::HALF_BYTES + my_pg * SM::BOX_BYTES, &tmKV, &kv_full[s],
-                                my_half * 64, 0, 0, 0, (p.layer_block0 >> 1) + page * p.n_kv_heads + item.kvh);
+                    tma_load_5d((my_v ? vring + vs * SM::K_BYTES : kring + ks * SM::K_BYTES) + my_pg * SM::BOX_BYTES, &tmKV,
+                                my_v ? &v_full[vs] : &k_full[ks], 0, 0, 0, 0,
+                                p.layer_block0 + 2 * (page * p.n_kv_heads + item.kvh) + my_v);
                 }
             }
         }
@@ -193,9 +208,9 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 uint32_t idle = 0;
                 while (np < n_st) {
                     const uint32_t tq = st + nq, tp = st + np;
-                    bool qk = nq < n_st && mbar_test(&kv_full[tq % NS], (tq / NS) & 1u) &&
+                    bool qk = nq < n_st && mbar_test(&k_full[tq % KS], (tq / KS) & 1u) &&
                               ((tq >> 1) == 0 || mbar_test(&s_empty[tq & 1u], ((tq >> 1) - 1) & 1u));
-                    bool pv = np < nq && mbar_test(&p_full[tp & 1u], (tp >> 1) & 1u) &&
+                    bool pv = np < nq && mbar_test(&p_full[tp & 1u], (tp >> 1) & 1u) && mbar_test(&v_full[tp % VS], (tp / VS) & 1u) &&
                               (np >= 2 || qi == 0 || mbar_test(o_empty, (uint32_t)(qi - 1) & 1u));
                     if (!qk && !pv) {
                         if ((++idle & 0x3FFu) == 0) {
@@ -212,11 +227,11 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     idle = 0;
                     t0 = 0;
                     tc_fence_after();
-                    const uint32_t k_addr = smem_u32(ring + (tq % NS) * SM::STAGE_BYTES);
+                    const uint32_t k_addr = smem_u32(kring + (tq % KS) * SM::K_BYTES);
                     const uint32_t idesc_qk = umma_idesc_f16(ATT2_ROWS, 16 * (qk ? pages_of(nq) : 1));
                     const uint32_t s_tmem = tmem_base + 256 + (tq & 1u) * 128;
                     const uint32_t p_addr = smem_u32(pbuf + (tp & 1u) * SM::P_BYTES);
-                    const uint32_t v_addr = smem_u32(ring + (tp % NS) * SM::STAGE_BYTES) + 1024;   // the V rows follow the K rows of a group
+                    const uint32_t v_addr = smem_u32(vring + (tp % VS) * SM::K_BYTES);
                     const uint32_t o_tmem = tmem_base + (tp & 1u) * 128;
                     const int npv = pv ? pages_of(np) : 0;
 #pragma unroll
@@ -225,21 +240,22 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                             // partial sum A: dims [0, HD/2) -> columns 0..63 of the buffer; B: dims [HD/2, HD) -> 64..127
                             const uint32_t qa = 2 * i, ka = 2 * i;
                             const uint32_t qb = HD == 128 ? ((ATT2_ROWS * 128) >> 4) + 2 * i : 2 * (i + QK_STEPS);
-                            const uint32_t kb = HD == 128 ? (SM::HALF_BYTES >> 4) + 2 * i : 2 * (i + QK_STEPS);
-                            umma_bf16(s_tmem, umma_desc_k128(q_addr) + qa, umma_desc_k128s(k_addr, 2048) + ka, idesc_qk, i != 0);
-                            umma_bf16(s_tmem + 64, umma_desc_k128(q_addr) + qb, umma_desc_k128s(k_addr, 2048) + kb, idesc_qk, i != 0);
+                            const uint32_t kb = HD == 128 ? (1024 >> 4) + 2 * i : 2 * (i + QK_STEPS);   // the second half's 8 rows follow the first's
+                            umma_bf16(s_tmem, umma_desc_k128(q_addr) + qa, umma_desc_k128s(k_addr, SM::GROUP_BYTES) + ka, idesc_qk, i != 0);
+                            umma_bf16(s_tmem + 64, umma_desc_k128(q_addr) + qb, umma_desc_k128s(k_addr, SM::GROUP_BYTES) + kb, idesc_qk, i != 0);
                         }
                         if (i < npv)   // the group's first stage of the item starts its O afresh
                             umma_bf16(o_tmem, umma_desc_k128(p_addr) + 2 * i,
-                                      umma_desc_mn128(v_addr + i * SM::BOX_BYTES, SM::HALF_BYTES, 2048), idesc_pv, !(np < 2 && i == 0));
+                                      umma_desc_mn128(v_addr + i * SM::BOX_BYTES, 1024, SM::GROUP_BYTES), idesc_pv, !(np < 2 && i == 0));
                     }
                     if (qk) {
                         umma_commit(&s_full[tq & 1u]);
+                        umma_commit(&k_empty[tq % KS]);
                         if (nq == n_st - 1) umma_commit(q_empty);
                         ++nq;
                     }
                     if (pv) {
-                        umma_commit(&kv_empty[tp % NS]);
+                        umma_commit(&v_empty[tp % VS]);
                         umma_commit(&p_empty[tp & 1u]);
                         if (np == n_st - 1) umma_commit(o_full);
                         ++np;

@@ -276,7 +276,7 @@ struct syn_kv {
     op16* pool = nullptr;   // half precision (K and V enter and leave through syn_kv_import / syn_kv_export as bf16)
     uint32_t n_pages, page_size;
     size_t layer_elems;
-    CUtensorMap tm_kv, tm_kv5;   // boxes of 32 rows (K and V of a page and head), in two row orders
+    CUtensorMap tm_kv, tm_kv5;   // boxes of 32 rows (K and V of a page and head); of 16 rows (K or V) with both 64-dim halves
 };
 
 struct syn_plan {
@@ -615,14 +615,14 @@ extern "C" int syn_kv_alloc(syn_model* m, uint32_t n_pages, uint32_t page_size, 
         return SYN_E_CUDA;
     }
     {
-        // The same box for the tensor-memory attention kernel, landing in shared memory as
-        // [K rows 0-7][V rows 0-7][K rows 8-15][V rows 8-15]: the 8-row groups of K (and of V) of consecutive
-        // boxes are then evenly spaced, which a tcgen05 operand descriptor needs.  Dimensions: dim, row in a
-        // group, K or V, group, (page, head) block.
+        // The 16 K rows (or the 16 V rows) of a page and head as one box for the tensor-memory attention
+        // kernel, landing in shared memory as [rows 0-7: dims 0-63][rows 0-7: dims 64-127][rows 8-15: ...]:
+        // the 8-row groups of consecutive boxes are then evenly spaced for either 64-dim half, which a tcgen05
+        // operand descriptor needs.  Dimensions: dim in a half, row in a group, half, group, 16-row block.
         const cuuint64_t hd2 = (cuuint64_t)c.head_dim * 2;
-        cuuint64_t dims[5] = {c.head_dim, 8, 2, 2, (cuuint64_t)blocks / 2};
-        cuuint64_t strides[4] = {hd2, 16 * hd2, 8 * hd2, 32 * hd2};
-        cuuint32_t box[5] = {64, 8, 2, 2, 1};
+        cuuint64_t dims[5] = {64, 8, c.head_dim / 64, 2, (cuuint64_t)blocks};
+        cuuint64_t strides[4] = {hd2, 128, 8 * hd2, 16 * hd2};
+        cuuint32_t box[5] = {64, 8, c.head_dim / 64, 2, 1};
         cuuint32_t estr[5] = {1, 1, 1, 1, 1};
         if (g_encode(&kv->tm_kv5, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 5, kv->pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
