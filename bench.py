@@ -43,7 +43,7 @@ NCU_TRAFFIC = {
     },
     # one layer's launch of the same work list, captured through `opbench attention --config 6 --kind 2`
     "cfg6-8b-chunk32": {
-        "attn2_kernel": (645844992, "5a02e9018c744d79ec1a3ae14e0b2f9cf236331e6d2ca9c578a435c7a48791da"),
+        "attn2_kernel": (645016064, "7f440a1370868a22f7065d27b06b79b8288df0935aa0c214a3e102ab8922fed7"),
     },
 }
 

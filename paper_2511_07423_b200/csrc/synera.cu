@@ -763,7 +763,7 @@ static int plan_compute(const syn_model_desc& c, int P, uint32_t n_pages, int n_
     // and the tensor-memory one (row tiles of 128: the same time per stage whatever the number of rows,
     // a larger fixed cost per item).  Unless one is asked for, the batch takes the cheaper by this model.
     static const int STAGE_COST[5] = {0, 1040, 1200, 1500, 1540};
-    const int WIDE_STAGE_COST = 1500;
+    const int WIDE_STAGE_COST = 1450;
     auto total_of = [&](bool w) {
         const int tpg = w ? std::min(SYN_MAX_CHUNK, 128 / G) : std::min(16, 64 / G);
         int64_t sum = 0;
