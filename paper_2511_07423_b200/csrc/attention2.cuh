@@ -15,15 +15,14 @@
 // of a stage's four pages are evenly spaced for either half of the head dimension; requests are the
 // scarce resource of this loop, about 80 cycles each; K and V have rings of their own because a
 // stage's K is free as soon as its scores are done, its V only after P V) and the Q tile through
-// mbarriers; one
-// thread of warp 1 issues every MMA; warps 4..7 and 8..11 are two softmax groups (one thread per row
-// each) that take alternate stages, each with its own score buffer, P buffer, running (max, sum) and
-// O accumulator in tensor memory; the first group combines the two at the end of the item and writes
-// the result.  A group's softmax of a stage (fp32, base 2) therefore has two stage times, and the
-// scores of its next stage are computed as soon as it has read the current ones.  The running
-// maximum used for P is only raised when a stage's maximum exceeds it by more than 2^8 (P stays well
-// inside half precision); O in tensor memory is rescaled at those moments only, and the final
-// division by the row sum uses the same maximum, so the result is the exact softmax.
+// mbarriers; one thread of warp 1 issues every MMA; warps 4..7 and 8..11 are two softmax groups (one
+// thread per row each) that take alternate stages, each with its own score buffer, P buffer, running
+// (max, sum) and O accumulator in tensor memory; the first group combines the two at the end of the
+// item and writes the result.  A group's softmax of a stage (fp32, base 2) therefore has two stage
+// times, and the scores of its next stage are computed as soon as it has read the current ones.  The
+// running maximum used for P is only raised when a stage's maximum exceeds it by more than 2^8 (P
+// stays well inside half precision); O in tensor memory is rescaled at those moments only, and the
+// final division by the row sum uses the same maximum, so the result is the exact softmax.
 // Items that cover part of a request's keys store fp32 partials (m, l, O) that the CTA completing a
 // row group combines in part order, as in attention.cuh.  Every wait is bounded.
 #pragma once
