@@ -10,12 +10,12 @@
 //   O += P V  : A = P (half precision, written by the softmax warps into shared memory in the
 //               K-major swizzled layout), B = V as it lies in the cache, [key][dim], i.e. an MN-major
 //               operand, D = O in tensor memory for the whole item.
-// Warp roles: warp 0 streams pages (TMA: one request brings the 16 K rows of a page, another its 16 V
+// Warp roles: warp 3 streams pages (TMA: one request brings the 16 K rows of a page, another its 16 V
 // rows, each as [rows 0-7: dims 0-63][rows 0-7: dims 64-127][rows 8-15: ...], so that the 8-row groups
 // of a stage's four pages are evenly spaced for either half of the head dimension; requests are the
 // scarce resource of this loop, about 80 cycles each; K and V have rings of their own because a
 // stage's K is free as soon as its scores are done, its V only after P V) and the Q tile through
-// mbarriers; one thread of warp 1 issues every MMA; warps 4..7 and 8..11 are two softmax groups (one
+// mbarriers; one thread of warp 2 issues every MMA; warps 4..7 and 8..11 are two softmax groups (one
 // thread per row each) that take alternate stages, each with its own score buffer, P buffer, running
 // (max, sum) and O accumulator in tensor memory; the first group combines the two at the end of the
 // item and writes the result.  A group's softmax of a stage (fp32, base 2) therefore has two stage
@@ -34,6 +34,9 @@ constexpr int ATT2_THREADS = 384;
 constexpr int ATT2_ROWS = 128;
 constexpr int ATT2_STAGE_KEYS = 64;
 constexpr float ATT2_RESCALE_GAP = 8.0f;   // log2 units
+// The producer and the MMA issuer sit on the schedulers of the softmax warps that own rows 96..127 and 64..95: with
+// fewer than 128 rows in a tile those are the warps with the least (or nothing) to do.
+constexpr int ATT2_PRODUCER_WARP = 3, ATT2_MMA_WARP = 2;
 
 template <int HD>
 struct Attn2Smem {
@@ -111,7 +114,7 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         mbar_fence_init();
         if (!list_ok) atomicExch(p.status, 2);
     }
-    if (warp == 1) {
+    if (warp == ATT2_MMA_WARP) {
         tmem_alloc(tmem_slot, SM::TMEM_COLS);
         tmem_relinquish();
     }
@@ -122,7 +125,7 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();   // Q and the chunk's K/V come from the preceding projection kernel
 
-    if (warp == 0) {
+    if (warp == ATT2_PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
         // lane -> (page of the stage, K or V): one request each
         const int my_pg = lane >> 1, my_v = lane & 1;
@@ -179,7 +182,7 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == ATT2_MMA_WARP) {
         // ------------------------------------------------------------ MMA issuer (one thread)
         // Two streams of work share the tensor pipe: the scores of stage k (ready when its K has
         // landed and the owning softmax group has read its previous scores) and O += P V of stage k
@@ -286,6 +289,7 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             const int qi = it - it_begin;
             const int rows = item.nj * G;
             const bool live = row < rows;
+            const bool wlive = wq * 32 < rows;   // a warp none of whose rows exist only keeps the barriers' counts
             const int j = row / G, gq = row - j * G;
             const int lim = item.q_pos0 + j;   // last visible key position of this row
             float m_used = -INFINITY, l = 0.f;
@@ -295,7 +299,7 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 const uint32_t us = st >> 1;   // use number of this group's buffers
                 uint32_t s0[32], s1[32];
                 if (ok) ok = wait_all(&s_full[wg], us & 1u);
-                if (ok) {
+                if (ok && wlive) {
                     // the two partial sums of the scores (halves of the head dimension)
                     uint32_t b0[32];
                     tc_fence_after();
@@ -316,6 +320,7 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
                 __syncwarp();
                 if (lane == 0 && ok) mbar_arrive(&s_empty[wg]);
+                if (wlive) {
                 // keys this row sees in the stage: positions < min(kv_end, lim + 1)
                 const int nvalid = min(item.kv_end, lim + 1) - kv0;
                 if (nvalid < ATT2_STAGE_KEYS) {
@@ -368,8 +373,8 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     const float c2 = ex2_approx(fmaf(__uint_as_float(s1[2 * c]), p.scale_log2, -base));
                     const float d = ex2_approx(fmaf(__uint_as_float(s1[2 * c + 1]), p.scale_log2, -base));
                     sum += (a + b) + (c2 + d);
-                    pw[c] = live ? pack_op(a, b) : 0u;
-                    pw[16 + c] = live ? pack_op(c2, d) : 0u;
+                    pw[c] = pack_op(a, b);   // (rows beyond the tile's hold garbage: they only meet themselves in the products)
+                    pw[16 + c] = pack_op(c2, d);
                 }
                 l += sum;
                 if (ok) {
@@ -380,6 +385,10 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                             make_uint4(pw[4 * c16], pw[4 * c16 + 1], pw[4 * c16 + 2], pw[4 * c16 + 3]);
                     fence_proxy_async_smem();
                     tc_fence_before();
+                }
+                } else if (us >= 1 && ok) {
+                    // keeps this warp in step with the others: one arrival per warp and phase on p_full
+                    ok = wait_all(&p_empty[wg], (us - 1) & 1u);
                 }
                 __syncwarp();
                 if (lane == 0 && ok) mbar_arrive(&p_full[wg]);
@@ -487,7 +496,7 @@ attn2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == ATT2_MMA_WARP) {
         tc_fence_after();
         tmem_dealloc(tmem_base, SM::TMEM_COLS);
     }
