@@ -110,6 +110,8 @@ def _judge_batch(syn, synthetic, cfg, wl, shape, model, kv, batch):
     acc, cor, logits = kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens,
                                        n_uncached=batch.n_uncached, want_logits=True)
     assert model.status() == 0
+    # which attention kernel the planner took: the tcgen05 one where a chunk is more than one 64-row tile
+    assert model.last_step_stats().attn_rows == (128 if cfg in (5, 6) else 64)
     # the same step again: bit-identical (static schedules, fixed summation orders, counters back at zero)
     acc2, cor2, logits2 = kv.verify_batch(toks, batch.chunk_offsets, batch.page_tables, batch.ctx_lens,
                                           n_uncached=batch.n_uncached, want_logits=True)
