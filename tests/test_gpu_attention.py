@@ -83,3 +83,54 @@ def _run(hd, Hq, Hkv, ctx, chunk):
     st = plan.stats()
     if max(ctx) > 1000:
         assert st.attn_split_items > 0
+
+
+@pytest.mark.parametrize("kind", [1, 2], ids=["warp_mma", "tcgen05"])
+@pytest.mark.parametrize("hd,Hq,Hkv", [(128, 8, 2), (64, 8, 2)])
+def test_scores_that_keep_growing_along_the_keys(hd, Hq, Hkv, kind):
+    """Keys whose scores rise steadily with the position (about 13 in log2 units per 64 keys, in one half of the
+    query heads; falling in the other half): the running maximum moves in every stage, so the tcgen05 kernel
+    rescales its accumulator in tensor memory every time instead of about once in a thousand stages, and the last
+    keys carry almost all the weight."""
+    import paper_2511_07423_b200 as syn
+    syn.debug_set_attention(kind)
+    try:
+        shape = ModelShape("att-grow", 1, 256, Hq, Hkv, hd, 256, 512)
+        seed = 9
+        ctx, chunk = [700, 130, 1400], [16, 5, 32]
+        batch = _batch(ctx, chunk, seed=seed)
+        glob, layers = cpu_model(shape, seed)
+        gg, gl = to_cuda(glob, layers)
+        model = syn.Model(shape, gg, gl)
+        kv = syn.KVCache(model, batch.n_pages)
+        orc = Oracle(shape)
+        pools = orc.new_pool(batch.n_pages)
+        T = batch.n_tokens
+        # q: a large component along dimension 0 (sign by head), small noise elsewhere; k: component 0 grows with the position
+        q = 0.05 * rng.normal_f32(rng.stream_key(seed, 77), 0, T * shape.q_dim, 1.0).view(T, Hq, hd)
+        q[:, :, 0] = torch.tensor([31.0 if h % 2 == 0 else -31.0 for h in range(Hq)])
+        q = q.reshape(T, shape.q_dim).to(torch.float16)
+        slope = 0.2 * (hd ** 0.5) / (31.0 * 1.4426950408889634)      # 0.2 log2 units per key
+        for r in range(batch.n_req):
+            tot = int(batch.ctx_lens[r] + batch.chunk_lens[r])
+            pt = batch.page_tables[r]
+            k, v = gen.gen_kv(shape, seed, 0, r, 0, tot)
+            k = (0.05 * k.float())
+            k[:, :, 0] = (slope * torch.arange(1, tot + 1, dtype=torch.float32))[:, None]
+            k = k.to(torch.bfloat16)
+            kv.import_kv(0, pt, 0, k.cuda(), v.cuda())
+            orc.load_kv(pools[0], pt.numpy(), 0, k.float().numpy(), v.float().numpy())
+        plan = syn.Plan(kv, torch.zeros(T, dtype=torch.int32), batch.chunk_offsets, batch.page_tables, batch.ctx_lens)
+        out = plan.attention(0, q.cuda())
+        torch.cuda.synchronize()
+        assert model.status() == 0
+        got = out.float().cpu().numpy()
+        assert np.isfinite(got).all()
+        for r in range(batch.n_req):
+            b, n = int(batch.chunk_offsets[r]), int(batch.chunk_lens[r])
+            ref = orc.attention(q[b:b + n].double().numpy(), pools[0], batch.page_tables[r].numpy(), int(batch.ctx_lens[r]))
+            scale = np.abs(ref).max()
+            err = np.abs(got[b:b + n] - ref).max()
+            assert err <= 2e-3 * scale, (r, err, scale)
+    finally:
+        syn.debug_set_attention(0)
