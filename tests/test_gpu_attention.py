@@ -29,6 +29,8 @@ CASES = [
     (128, 8, 2, [100, 5, 0], [32, 19, 17]),                          # chunks beyond 16: two token groups per request
     (128, 10, 2, [50], [30]),                                        # G=5, three token groups
     (64, 16, 2, [200], [32]),                                        # G=8, four token groups
+    (128, 8, 2, [3000, 40], [32, 32]),                               # 128-row tiles whose key ranges are split over items
+    (128, 10, 2, [2500], [25]),                                      # G=5: 125 rows in one tile of the tcgen05 kernel, split keys
 ]
 
 
