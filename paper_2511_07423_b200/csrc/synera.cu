@@ -1196,6 +1196,8 @@ static int gemm2_plan(int T, int packed_rows, int K, int n_sm, int mode, int for
         if (quad_items >= n_cl_max) kind = PAIR_QUAD;                                   // full waves of 512-feature items
         else if (4 * quad_items >= 3 * n_cl_max) kind = PAIR_QUAD;                      // one wave, at least three quarters full: measured
                                                                                         // 7-9 % ahead of 256-feature items in two rounds
+        else if (!may_split && 8 * quad_items >= 5 * n_cl_max) kind = PAIR_QUAD;        // (without a residual epilogue already from five
+                                                                                        // eighths: qkv at 921 tokens 94 us against 102)
         else if (may_split && g.num_kb >= 96 && n_cl_max / quad_items >= 2) kind = PAIR_QUAD;   // long K: shared between clusters
         else if (2 * duo_items >= n_cl_max) kind = PAIR_DUO;
         else return PAIR_NONE;
