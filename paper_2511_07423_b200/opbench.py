@@ -51,13 +51,14 @@ def _time(fn, iters: int, warmup: int = 3):
 
 
 def bench_linear(a):
+    syn.debug_set_schedule(1 if a.one_cta else 0)
     key = rng.stream_key(0, 1234)
     x = rng.normal_f32(key, 0, a.T * a.K, 1.0, device="cuda").view(a.T, a.K).to(torch.float16)
     w = rng.normal_f32(key, a.T * a.K, a.N * a.K, 0.02, device="cuda").view(a.N, a.K).to(torch.bfloat16)
     syn.syn_op_linear(x, w, schedule_as=a.sched)
     med, best = _time(lambda: syn.syn_op_linear(x, w, schedule_as=a.sched, reuse_pack=True), a.iters)
     fl = 2.0 * a.T * a.N * a.K
-    print(json.dumps({"op": "linear", "sched": a.sched, "T": a.T, "N": a.N, "K": a.K, "ms_median": med, "ms_best": best,
+    print(json.dumps({"op": "linear", "sched": a.sched, "one_cta": bool(a.one_cta), "T": a.T, "N": a.N, "K": a.K, "ms_median": med, "ms_best": best,
                       "tflops": fl / med / 1e9, "weight_gbs": 2.0 * a.N * a.K / med / 1e6,
                       "note": "includes the fp32 [T][N] store of the test epilogue and a stream sync per call"}))
 
@@ -220,6 +221,7 @@ def main():
     l.add_argument("--K", type=int, default=4096)
     l.add_argument("--iters", type=int, default=10)
     l.add_argument("--sched", default="plain", help="schedule: plain, qkv, resid, swiglu, lmhead, pair_quad, pair_duo, pair_quad_resid, pair_duo_resid")
+    l.add_argument("--one-cta", action="store_true", help="keep the projection on the one-CTA kernel whatever its shape")
     t = sub.add_parser("attention")
     t.add_argument("--config", type=int, default=3)
     t.add_argument("--pool-tokens", type=int, default=None)
