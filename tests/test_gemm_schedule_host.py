@@ -161,6 +161,14 @@ def test_pair_schedules_of_the_configurations():
     assert _check2(544, 6144, 4096, "qkv")["kind"] == 2 and _check2(544, 4096, 4096, "resid")["kind"] == 2
     p = _check2(544, 4096, 14336, "resid")
     assert (p["kind"], p["splits"], p["n_clusters"]) == (1, 3, 72)
+    # one wave of 512-feature items at least three quarters full (five eighths without a residual epilogue):
+    # o and down at 2 048 tokens (64 items), the 32B shape's qkv at 1 194 (70), qkv at 921 (48); the 32B shape's
+    # o at 1 194 tokens (50 items, residual epilogue) stays on the one-CTA kernel
+    for T, N, K, epi, want in ((2048, 4096, 4096, "resid", (1, 64)), (2048, 4096, 14336, "resid", (1, 64)),
+                               (1194, 7168, 5120, "qkv", (1, 70)), (921, 6144, 4096, "qkv", (1, 48))):
+        p = _check2(T, N, K, epi)
+        assert (p["kind"], p["n_clusters"]) == want and p["splits"] == 1
+    assert syn.gemm2_plan_host(1194, 5120, 5120, "resid")["kind"] == 0
 
 
 @pytest.mark.parametrize("force", ["quad", "duo"])
